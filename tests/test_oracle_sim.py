@@ -1,0 +1,273 @@
+"""Pins for the oracle's round loop (Algorithm 1, Eq. 3-6) against special
+cases the paper names and closed forms that follow from its rules."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import abs_sim, models, timing
+from oracle.abs_sim import ABSOracle, K_FIXED, BOUND_FIXED
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _lsq_problem(M=512, d=6, seed=0, noise=0.1):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((M, d))
+    w_star = rng.standard_normal(d)
+    y = X @ w_star + noise * rng.standard_normal(M)
+    return X, y, w_star
+
+
+def _check_invariants(o, rows, W, S):
+    jobs_started = 0
+    prev_T, prev_K = 0, 0
+    comm = W
+    for row in rows:
+        assert len(row["sel"]) == row["K"] == len(row["tau"])          # |K^t| = K^t
+        assert len(set(row["sel"])) == row["K"]
+        assert not (set(row["sel"]) & set(row["restart"]))
+        assert row["restart"] == sorted(row["restart"])
+        assert 0 <= row["theta"] <= S
+        assert all(0 <= tau <= S for tau in row["tau"])                # bounded staleness
+        assert row["T_end"] >= prev_T and row["K"] >= prev_K and row["K"] <= W
+        prev_T, prev_K = row["T_end"], row["K"]
+        jobs_started += row["K"] + len(row["restart"])
+        comm += row["K"] + len(row["restart"])
+        assert row["comm"] == comm                                     # +1 per worker that communicates
+    assert sum(o.job) == jobs_started
+    assert all(v <= o.t for v in o.version)
+    assert all(o.t - v <= max(S, 0) for v in o.version) or S == 0
+
+
+# ---------------------------------------------------------------- reductions
+def test_sync_sgd_reduction():
+    """K = N and bound 0 is synchronous minibatch SGD (Sec. II-B): the model
+    follows a plain loop that averages the N minibatch gradients."""
+    X, y, _ = _lsq_problem()
+    W, B, lr, seed = 4, 8, 0.05, 42
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), B, lr, W, W, 0, dist, seed)
+    rows = o.run(25)
+    w = np.zeros(6)
+    for t in range(25):
+        idx = np.concatenate([abs_sim.minibatch_indices(seed, n, t, B, W, X.shape[0])
+                              for n in range(W)])
+        r = X[idx] @ w - y[idx]
+        w = w - lr * (X[idx].T @ r) / (W * B)
+    assert np.allclose(o.w, w, rtol=1e-12, atol=1e-14)
+    for t, row in enumerate(rows):
+        assert sorted(row["sel"]) == list(range(W)) and set(row["tau"]) == {0}
+        assert row["restart"] == []
+    assert o.job == [25] * W
+    _check_invariants(o, rows, W, 0)
+
+
+def test_k_sync_reduction():
+    """Bound 0 with fixed K < N: the stragglers' work is thrown away every
+    round (K-sync SGD, Sec. I): all ages 0, N - K restarts per round."""
+    X, y, _ = _lsq_problem()
+    W, K = 6, 2
+    dist = timing.TimeDist(timing.SHIFTED_EXP, shift=1.0, rate=1.0)
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, W, K, 0, dist, 7, k_mode=K_FIXED)
+    rows = o.run(30)
+    for row in rows:
+        assert row["K"] == K and set(row["tau"]) == {0}
+        assert len(row["restart"]) == W - K and row["theta"] == 0
+    _check_invariants(o, rows, W, 0)
+
+
+def test_asgd_reduction_statistics():
+    """Fixed K = 1 is ASGD (Sec. II-B).  With i.i.d. exponential job times the
+    arriving worker is uniform over the N workers in every round (memoryless),
+    so the age of a consumed gradient is geometric with mean N - 1."""
+    X, y, _ = _lsq_problem(d=3)
+    W, rounds = 5, 6000
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    o = ABSOracle(models.LSQ, [3, 1], X, y, np.zeros(3), 2, 0.01, W, 1, 200, dist, 3,
+                  k_mode=K_FIXED, bound_mode=BOUND_FIXED)
+    rows = o.run(rounds)
+    ids = np.array([row["sel"][0] for row in rows])
+    taus = np.array([row["tau"][0] for row in rows[200:]])
+    assert all(row["K"] == 1 and row["restart"] == [] for row in rows)
+    counts = np.bincount(ids, minlength=W) / rounds
+    assert np.all(np.abs(counts - 1 / W) < 4 * math.sqrt(0.16 / rounds))
+    # geometric(p = 1/W) on {0,1,...}: mean W-1, variance (1-p)/p^2 = W(W-1)
+    assert abs(taus.mean() - (W - 1)) < 5 * math.sqrt(W * (W - 1) / len(taus))
+
+
+def test_lock_step_constant_times():
+    """Equal deterministic times: arrivals go round-robin in id order."""
+    X, y, _ = _lsq_problem()
+    W, K, D = 8, 2, 3.0
+    dist = timing.TimeDist(timing.CONST, shift=D)
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.01, W, K, W // K - 1, dist, 1,
+                  k_mode=K_FIXED, bound_mode=BOUND_FIXED)
+    rows = o.run(40)
+    for t, row in enumerate(rows):
+        first = (t * K) % W
+        assert row["sel"] == list(range(first, first + K))
+        assert row["T_end"] == int(D * 2 ** 20) * ((t * K) // W + 1)
+        assert row["tau"] == [min(t, W // K - 1)] * K
+        assert row["restart"] == []
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.01, W, W, 0, dist, 1)
+    for t, row in enumerate(o.run(10)):
+        assert row["sel"] == list(range(W)) and row["T_end"] == (t + 1) * int(D * 2 ** 20)
+        assert set(row["tau"]) == {0}
+
+
+def test_straggler_is_restarted_every_theta_plus_one_rounds():
+    """One worker whose jobs take 2^40 ticks never arrives; Eq. 6 (in Algorithm
+    1's order) sends it the fresh model whenever its age would exceed theta."""
+    X, y, _ = _lsq_problem()
+    W, K, S = 5, 2, 3
+    dist = timing.TimeDist(timing.CONST, shift=1.0, slow_mod=W, slow_rem=4, slow_factor=2.0 ** 20)
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.01, W, K, S, dist, 1,
+                  k_mode=K_FIXED, bound_mode=BOUND_FIXED)
+    rows = o.run(41)
+    for t, row in enumerate(rows):
+        assert 4 not in row["sel"]
+        assert (4 in row["restart"]) == (t % (S + 1) == S)
+    _check_invariants(o, rows, W, S)
+    # literal reading of Eq. 6 (pre-increment age) fires one round later
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.01, W, K, S, dist, 1,
+                  k_mode=K_FIXED, bound_mode=BOUND_FIXED, literal_eq6=True)
+    for t, row in enumerate(o.run(41)):
+        assert (4 in row["restart"]) == (t % (S + 2) == S + 1)
+
+
+# ------------------------------------------------------------------- rules
+def test_selection_is_the_k_smallest_with_ties_to_lower_id():
+    X, y, _ = _lsq_problem(d=2)
+    dist = timing.TimeDist(timing.CONST, shift=1.0)
+    for ticks in itertools.product([3, 5, 7], repeat=5):
+        for K in (1, 2, 4):
+            o = ABSOracle(models.LSQ, [2, 1], X, y, np.zeros(2), 2, 0.0, 5, K, 9, dist, 0,
+                          k_mode=K_FIXED, bound_mode=BOUND_FIXED)
+            o.c = list(ticks)
+            row = o.round()
+            pending = list(range(5))
+            brute = []
+            for _ in range(K):            # repeated extraction of the minimum
+                best = min(pending, key=lambda n: ticks[n] * 10 + n)
+                brute.append(best)
+                pending.remove(best)
+            assert row["sel"] == brute
+            assert row["T_end"] == ticks[brute[-1]]
+
+
+def test_k_rule_hand_cases():
+    f = np.float32
+    assert abs_sim.next_k(4, 4, 64, f(2.0), f(2.0)) == 4          # same loss -> K0
+    assert abs_sim.next_k(4, 4, 64, f(2.0), f(0.5)) == 8          # loss / 4 -> K doubles
+    assert abs_sim.next_k(4, 4, 64, f(2.0), f(0.5000001)) == 7    # just above the boundary
+    assert abs_sim.next_k(4, 4, 64, f(1.0), f(1.0 / 9.0)) == 11   # 1/9 rounds up in binary32: 144*f(1/9) > 16
+    assert abs_sim.next_k(4, 4, 64, f(1.0), f(0.0625)) == 16
+    assert abs_sim.next_k(9, 4, 64, f(2.0), f(8.0)) == 9          # never decreases
+    assert abs_sim.next_k(4, 4, 10, f(2.0), f(1e-6)) == 10        # capped at N
+    assert abs_sim.next_k(4, 4, 10, f(2.0), f(0.0)) == 10
+    with pytest.raises(abs_sim.Diverged):
+        abs_sim.next_k(4, 4, 10, f(2.0), f(np.inf))
+    # agrees with the real-valued formula K0 sqrt(L0/Lt) away from boundaries
+    rng = np.random.default_rng(1)
+    for _ in range(300):
+        l0, lt = f(rng.uniform(0.5, 3)), f(rng.uniform(0.01, 3))
+        real = 5 * math.sqrt(float(l0) / float(lt))
+        if abs(real - round(real)) > 1e-6:
+            assert abs_sim.next_k(5, 5, 1000, l0, lt) == max(5, min(1000, math.floor(real)))
+
+
+def test_first_round_keeps_k0():
+    X, y, _ = _lsq_problem()
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 8, 3, 4, dist, 5)
+    rows = o.run(2)
+    assert rows[0]["K"] == 3 and rows[1]["K"] == 3     # L_0 / L_0 = 1  ->  K^1 = K^0
+
+
+def test_theta_table():
+    with open(os.path.join(GOLDEN, "theta_table.txt")) as f:
+        rows = [tuple(int(v) for v in line.split()) for line in f
+                if line.strip() and not line.startswith("#")]
+    assert len(rows) >= 20
+    for W, K0, S, K, theta in rows:
+        assert abs_sim.theta_rule(W, K0, S, K) == theta
+    assert abs_sim.theta_rule(8, 8, 0, 8) == 0           # bound 0 overrides the floor of 1
+
+
+def test_loss_estimate_order_and_rounding():
+    assert abs_sim.tree_sum([1.0, 2.0, 3.0]) == 6.0
+    # ((a+b)+(c+0)): with a = 1, b = 2^-53, c = 2^-53 the pairs decide the bits
+    a, b = 1.0, 2.0 ** -53
+    assert abs_sim.tree_sum([a, b, b]) == (a + b) + (b + 0.0) == 1.0
+    assert abs_sim.tree_sum([b, b, a]) == (b + b) + (a + 0.0) == 1.0 + 2.0 ** -52
+    vals = [np.float32(x) for x in (0.1, 0.2, 0.3, 0.4, 0.5)]
+    est = abs_sim.loss_estimate(vals)
+    assert isinstance(est, np.float32)
+    assert abs(float(est) - 0.3) < 1e-7
+
+
+# ---------------------------------------------------------- whole-run behaviour
+def test_lsq_run_reaches_normal_equation_solution():
+    X, y, w_star = _lsq_problem(M=2048, d=8, seed=3, noise=0.1)
+    w_ls = np.linalg.solve(X.T @ X, X.T @ y)
+    dist = timing.TimeDist(timing.SHIFTED_EXP, shift=1.0, rate=1.0)
+    o = ABSOracle(models.LSQ, [8, 1], X, y, np.zeros(8), 32, 0.05, 8, 2, 4, dist, 2001)
+    rows = o.run(400)
+    assert np.linalg.norm(o.w - w_ls) / np.linalg.norm(w_ls) < 0.03
+    assert np.linalg.norm(o.w - w_star) / np.linalg.norm(w_star) < 0.05
+    assert rows[-1]["loss_mean"] < 0.02 and rows[0]["loss_mean"] > 1.0
+    assert rows[-1]["K"] == 8                   # K has grown to N as the loss fell
+    _check_invariants(o, rows, 8, 4)
+
+
+@pytest.mark.parametrize("kind,dims,quant", [(models.SOFTMAX, [12, 4], False),
+                                             (models.MLP, [12, 9, 4], True)])
+def test_invariants_on_classifier_runs(kind, dims, quant):
+    rng = np.random.default_rng(5)
+    means = rng.standard_normal((4, 12))
+    lab = rng.integers(0, 4, size=600)
+    X = models.round_bf16(means[lab] + rng.standard_normal((600, 12)))
+    w0 = rng.standard_normal(models.n_params(kind, dims)) * 0.3
+    dist = timing.TimeDist(timing.PARETO2, scale=1.0)
+    o = ABSOracle(kind, dims, X, lab, w0, 8, 0.1, 12, 3, 6, dist, 77, quant=quant)
+    rows = o.run(120)
+    _check_invariants(o, rows, 12, 6)
+    assert rows[-1]["loss_mean"] < rows[0]["loss_mean"]
+    assert any(row["restart"] for row in rows)
+    assert max(max(row["tau"]) for row in rows) >= 2
+
+
+def test_restarts_do_not_increase_with_the_bound():
+    """Sanity of the qualitative claim of Sec. V-B: a larger threshold offset
+    discards fewer computations."""
+    X, y, _ = _lsq_problem()
+    dist = timing.TimeDist(timing.PARETO2, scale=1.0)
+    totals = []
+    for S in (1, 2, 4, 8):
+        o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.02, 12, 2, S, dist, 9,
+                      k_mode=K_FIXED, bound_mode=BOUND_FIXED)
+        totals.append(sum(len(r["restart"]) for r in o.run(150)))
+    assert totals == sorted(totals, reverse=True) and totals[0] > totals[-1]
+
+
+def test_forced_losses_only_steer_k():
+    X, y, _ = _lsq_problem()
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    a = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 8, 2, 4, dist, 5)
+    rows = a.run(30)
+    b = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 8, 2, 4, dist, 5)
+    rows_b = b.run(30, forced_losses=[r["sel_loss"] for r in rows])
+    assert [r["sel"] for r in rows] == [r["sel"] for r in rows_b]
+    assert np.array_equal(a.w, b.w)
+
+
+def test_divergence_is_reported():
+    X, y, _ = _lsq_problem()
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    o = ABSOracle(models.LSQ, [6, 1], X * 1e3, y, np.zeros(6), 4, 10.0, 4, 4, 0, dist, 5)
+    with pytest.raises(abs_sim.Diverged):
+        o.run(200)
+    assert 0 < len(o.trace) < 200
