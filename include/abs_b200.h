@@ -1,0 +1,170 @@
+/*
+ * abs_b200 -- C ABI of the B200 implementation of the ABS parameter-server
+ * round loop (adaptive bounded staleness, arXiv 2301.08895).
+ *
+ * One context simulates N workers and one server on one GPU.  A round is
+ * Algorithm 1's "server executes" block: wait for the K^t fastest uploads,
+ * apply Eq. 3, adapt K (Eq. 5) and the staleness threshold (Eq. 4), update the
+ * ages and restart over-stale workers (Eq. 6).  Worker uploads are minibatch
+ * gradients (Eq. 2 with U = 1) evaluated at the model version the worker
+ * holds; the bounded staleness lets the library keep only S + 1 model versions
+ * in a ring instead of one model per worker.
+ *
+ * Conventions
+ *  - Every function returns ABS_OK (0) or a negative ABS_E* code; nothing
+ *    throws, aborts or prints.  abs_last_error() gives the text of the last
+ *    failure on the calling thread.
+ *  - "device" pointers are CUDA device addresses of the current device,
+ *    "host" pointers are ordinary memory.  The library allocates no device
+ *    memory: the caller passes one workspace (size from abs_workspace_bytes)
+ *    that must stay valid and untouched until abs_destroy.
+ *  - All work is enqueued on the caller's stream; abs_run_rounds synchronises
+ *    that stream once before it returns.
+ *  - Parameter vector layout (w0 and abs_get_params): for each layer in order
+ *    W[in][out] row-major followed by b[out]; least squares has w[d] only.
+ *  - Times are integer ticks, 2^20 per time unit.
+ */
+#ifndef ABS_B200_H
+#define ABS_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ABS_OK            0
+#define ABS_EINVAL       -1  /* bad argument (text names it) */
+#define ABS_ENOSPACE     -2  /* workspace, trace capacity or round capacity too small */
+#define ABS_EUNSUPPORTED -3  /* local_steps != 1, unknown kind */
+#define ABS_ESTATE       -4  /* call order */
+#define ABS_ECUDA        -5  /* a CUDA call failed; sticky for the context */
+#define ABS_ETIMEOUT     -6  /* a bounded device-side wait expired */
+#define ABS_EDIVERGED    -7  /* a non-finite loss was uploaded; see abs_run_rounds */
+#define ABS_ERANGE       -8  /* simulated time left the 2^53 tick range */
+
+/* model kinds: the sample loss f of Eq. 1 */
+#define ABS_LSQ      0  /* f = 1/2 (x.w - y)^2, dims = {d, 1}, no bias */
+#define ABS_SOFTMAX  1  /* one affine layer + soft-max cross-entropy */
+#define ABS_MLP      2  /* affine layers with ReLU between them + soft-max cross-entropy */
+
+/* storage/arithmetic type */
+#define ABS_FP32             0  /* fp32 data, fp32 models, fp32 FMA */
+#define ABS_BF16_FP32MASTER  1  /* bf16 data, bf16 model versions, activations and deltas;
+                                   fp32 accumulation; fp32 master parameters */
+
+#define ABS_K_ADAPTIVE      0   /* K^{t+1} from Eq. 5 */
+#define ABS_K_FIXED         1   /* K^t = K0 for all t (K-sync / K-async / ASGD baselines, Sec. II-B) */
+#define ABS_BOUND_ADAPTIVE  0   /* threshold from Eq. 4, capped by the staleness bound */
+#define ABS_BOUND_FIXED     1   /* threshold = staleness bound in every round (Fig. 1 setting) */
+
+/* execution-time laws (random execution times with stragglers, Sec. V-A) */
+#define ABS_T_CONST        0    /* shift */
+#define ABS_T_EXP          1    /* Exp(rate) */
+#define ABS_T_SHIFTED_EXP  2    /* shift + Exp(rate) */
+#define ABS_T_PARETO2      3    /* Pareto, shape 2, minimum `scale` */
+
+#define ABS_MAX_LAYERS   7
+#define ABS_MAX_WORKERS  1024
+#define ABS_MAX_BOUND    255
+
+typedef struct abs_ctx abs_ctx;
+
+/* Everything the paper calls f, D, B, eta, w^0 (Sec. II-A). */
+typedef struct {
+  int kind;                 /* ABS_LSQ | ABS_SOFTMAX | ABS_MLP */
+  int n_layers;             /* affine layers; dims has n_layers + 1 entries */
+  int dims[ABS_MAX_LAYERS + 1]; /* e.g. {3072,1024,512,10}; LSQ: {d,1}; last dim = classes (<= 64) */
+  int batch;                /* B of Eq. 2, 1..1024 */
+  float lr;                 /* eta, constant */
+  int dtype;                /* ABS_FP32 | ABS_BF16_FP32MASTER */
+  int local_steps;          /* U of Eq. 2; must be 1 */
+  int k_mode;               /* ABS_K_* */
+  int bound_mode;           /* ABS_BOUND_* */
+  int max_rounds;           /* trace capacity: total rounds this context may run */
+  int data_on_host;         /* 0: X, y are device pointers owned by the caller and must outlive
+                               the context.  1: X, y are host pointers; abs_init copies them into
+                               the workspace (abs_workspace_bytes accounts for the room) */
+  const void* X;            /* [n_samples][dims[0]] row-major; float (FP32) or bf16 bits (BF16) */
+  const void* y;            /* float targets (LSQ) or int32 labels in [0, classes) */
+  long long n_samples;      /* M of Eq. 1; worker n owns samples [n*M/N, (n+1)*M/N) */
+  const float* w0;          /* host, n_params floats, copied by abs_init */
+  void* workspace;          /* device, 256-byte aligned */
+  size_t workspace_bytes;
+  void* stream;             /* cudaStream_t (0 = default stream) */
+} abs_model_desc;
+
+typedef struct {
+  int kind;                 /* ABS_T_* */
+  double shift, rate, scale;
+  int slow_mod, slow_rem;   /* workers with n % slow_mod == slow_rem are slow (slow_mod 0: none) */
+  double slow_factor;       /* their durations are multiplied by this */
+} abs_time_dist;
+
+/* Caller-owned host arrays receiving rounds [first_round, first_round + n_rounds).
+ * Per-round arrays need n_rounds entries (sel_off/rst_off: n_rounds + 1, offsets into the flat
+ * arrays relative to the first returned round).  Flat arrays need cap_sel / cap_rst entries.
+ * Any pointer may be NULL to skip that field. */
+typedef struct {
+  int32_t*  K;          /* K^t */
+  int32_t*  n_restart;  /* workers restarted by Eq. 6 after round t */
+  int32_t*  theta;      /* threshold used by that restart test (Eq. 4 at K^{t+1}) */
+  uint64_t* T_end;      /* tick at which the K^t-th upload arrived */
+  float*    loss_mean;  /* estimate of f(w^t): mean uploaded loss */
+  uint64_t* comm;       /* cumulative communication rounds (Sec. V-B) after round t */
+  int64_t*  sel_off;    /* [n_rounds + 1] */
+  int64_t*  rst_off;    /* [n_rounds + 1] */
+  int32_t*  sel_id;     /* selected worker ids, arrival order */
+  int32_t*  sel_tau;    /* staleness of each consumed gradient */
+  float*    sel_loss;   /* each upload's mean minibatch loss */
+  int32_t*  rst_id;     /* restarted worker ids, ascending */
+  size_t    cap_sel, cap_rst;
+} abs_trace;
+
+/* Bytes of device workspace a context needs (Sec. II-A sizes: N workers, ring of S + 1 model
+ * versions, activations for N*B rows, trace for max_rounds).  Only kind, dims, batch, dtype,
+ * max_rounds, data_on_host and n_samples of `model` are read. */
+int abs_workspace_bytes(const abs_model_desc* model, int W, int staleness_bound, size_t* out);
+
+/* Algorithm 1, initialisation: K^0, threshold N/K^0 + a := staleness_bound, w^0 broadcast to all
+ * workers (every worker starts job 0 at tick 0).  Copies w0 (and the dataset if data_on_host)
+ * to the device, enqueues the set-up kernels, synchronises the stream.
+ * W in [1, 1024], K0 in [1, W], staleness_bound in [0, 255].
+ * First call per process should come before any stream capture. */
+int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int staleness_bound,
+             const abs_time_dist* time_dist, unsigned long long seed);
+
+/* Algorithm 1, n iterations of the server loop (Eq. 2-6).  Enqueues n rounds without host
+ * synchronisation between them, then synchronises once.  Returns ABS_EDIVERGED if a non-finite
+ * loss was uploaded: the round in which it happened and all later ones are not applied, the
+ * parameters and the trace stay valid up to the round before.  Errors are sticky. */
+int abs_run_rounds(abs_ctx* ctx, int n);
+
+/* Same as abs_run_rounds but returns after enqueueing; the device status is read by the next
+ * abs_run_rounds / abs_rounds_done / abs_get_* call.  Used to time the loop with CUDA events. */
+int abs_enqueue_rounds(abs_ctx* ctx, int n);
+
+/* Rounds completed so far (synchronises the stream). */
+int abs_rounds_done(abs_ctx* ctx, int* rounds);
+
+/* The global model w^t (Eq. 3) as fp32, layout of w0.  dst_host needs n_params floats
+ * (cap = its capacity in floats); *d_out receives n_params. */
+int abs_get_params(abs_ctx* ctx, float* dst_host, size_t cap, size_t* d_out);
+
+/* Per-round record of Algorithm 1's decisions for rounds [first_round, first_round + n_rounds):
+ * K^t, the arrival-ordered selected workers, each gradient's staleness, the restarted workers. */
+int abs_get_trace(abs_ctx* ctx, int first_round, int n_rounds, abs_trace* out_host);
+
+/* Kernels of ours launched on behalf of this context so far (set-up included). */
+int abs_launch_count(abs_ctx* ctx, long long* launches);
+
+int abs_destroy(abs_ctx* ctx);
+
+/* Text of the last error on this thread ("" if none). */
+const char* abs_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,239 @@
+"""ctypes binding of the C-ABI library `libabs_b200.so` (see include/abs_b200.h).
+
+Argument marshalling only: every step of the round loop runs in the library's
+CUDA kernels.  PyTorch supplies device memory (workspace, dataset) and the
+stream.  There is no CPU fallback: if the library has not been built, or no
+CUDA device is present, the calls raise.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libabs_b200.so")
+
+OK, EINVAL, ENOSPACE, EUNSUPPORTED, ESTATE, ECUDA, ETIMEOUT, EDIVERGED, ERANGE = \
+    0, -1, -2, -3, -4, -5, -6, -7, -8
+LSQ, SOFTMAX, MLP = 0, 1, 2
+FP32, BF16_FP32MASTER = 0, 1
+K_ADAPTIVE, K_FIXED = 0, 1
+BOUND_ADAPTIVE, BOUND_FIXED = 0, 1
+T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2 = 0, 1, 2, 3
+MAX_LAYERS = 7
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [("kind", C.c_int), ("n_layers", C.c_int), ("dims", C.c_int * (MAX_LAYERS + 1)),
+                ("batch", C.c_int), ("lr", C.c_float), ("dtype", C.c_int),
+                ("local_steps", C.c_int), ("k_mode", C.c_int), ("bound_mode", C.c_int),
+                ("max_rounds", C.c_int), ("data_on_host", C.c_int),
+                ("X", C.c_void_p), ("y", C.c_void_p), ("n_samples", C.c_longlong),
+                ("w0", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("stream", C.c_void_p)]
+
+
+class TimeDist(C.Structure):
+    _fields_ = [("kind", C.c_int), ("shift", C.c_double), ("rate", C.c_double),
+                ("scale", C.c_double), ("slow_mod", C.c_int), ("slow_rem", C.c_int),
+                ("slow_factor", C.c_double)]
+
+
+class Trace(C.Structure):
+    _fields_ = [("K", C.c_void_p), ("n_restart", C.c_void_p), ("theta", C.c_void_p),
+                ("T_end", C.c_void_p), ("loss_mean", C.c_void_p), ("comm", C.c_void_p),
+                ("sel_off", C.c_void_p), ("rst_off", C.c_void_p), ("sel_id", C.c_void_p),
+                ("sel_tau", C.c_void_p), ("sel_loss", C.c_void_p), ("rst_id", C.c_void_p),
+                ("cap_sel", C.c_size_t), ("cap_rst", C.c_size_t)]
+
+
+class AbsError(RuntimeError):
+    def __init__(self, code, text):
+        super().__init__("abs_b200 error %d: %s" % (code, text))
+        self.code = code
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("%s is missing: run `python -m paper_2301_08895_b200.build` "
+                               "(there is no CPU fallback)" % LIB_PATH)
+        l = C.CDLL(LIB_PATH)
+        l.abs_last_error.restype = C.c_char_p
+        l.abs_workspace_bytes.argtypes = [C.POINTER(ModelDesc), C.c_int, C.c_int,
+                                          C.POINTER(C.c_size_t)]
+        l.abs_init.argtypes = [C.POINTER(C.c_void_p), C.POINTER(ModelDesc), C.c_int, C.c_int,
+                               C.c_int, C.POINTER(TimeDist), C.c_ulonglong]
+        l.abs_run_rounds.argtypes = [C.c_void_p, C.c_int]
+        l.abs_enqueue_rounds.argtypes = [C.c_void_p, C.c_int]
+        l.abs_rounds_done.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
+        l.abs_get_params.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
+        l.abs_get_trace.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(Trace)]
+        l.abs_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_longlong)]
+        l.abs_destroy.argtypes = [C.c_void_p]
+        _lib = l
+    return _lib
+
+
+def last_error():
+    return lib().abs_last_error().decode()
+
+
+def _check(rc):
+    if rc != OK:
+        raise AbsError(rc, last_error())
+
+
+def n_params(kind, dims):
+    if kind == LSQ:
+        return dims[0]
+    return sum(dims[l] * dims[l + 1] + dims[l + 1] for l in range(len(dims) - 1))
+
+
+def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
+          local_steps=1, data_on_host=0):
+    m = ModelDesc()
+    m.kind, m.n_layers = kind, len(dims) - 1
+    for i, v in enumerate(dims):
+        m.dims[i] = int(v)
+    m.batch, m.lr, m.dtype = int(batch), float(lr), dtype
+    m.local_steps, m.k_mode, m.bound_mode = local_steps, k_mode, bound_mode
+    m.max_rounds, m.data_on_host, m.n_samples = int(max_rounds), data_on_host, int(n_samples)
+    return m
+
+
+def workspace_bytes(kind, dims, batch, dtype, W, S, max_rounds, n_samples, data_on_host=0):
+    m = _desc(kind, dims, batch, 0.0, dtype, max_rounds, n_samples, 0, 0, 1, data_on_host)
+    out = C.c_size_t(0)
+    _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(out)))
+    return out.value
+
+
+class Context:
+    """One ABS run (abs_init .. abs_destroy).
+
+    X, y: torch CUDA tensors (X float32 or bfloat16 [n, in]; y float32 or int32),
+    or, with `data_on_host=True`, numpy arrays (bf16 as uint16 patterns) that the
+    library copies to the device itself.  w0: numpy float32.
+    """
+
+    def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, time, seed, max_rounds,
+                 dtype=FP32, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE, local_steps=1,
+                 data_on_host=False, stream=None, device="cuda:0"):
+        import torch
+        self._torch = torch
+        self.kind, self.dims, self.W, self.S = kind, list(dims), W, S
+        self.max_rounds = max_rounds
+        n_samples = X.shape[0]
+        m = _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
+                  local_steps, 1 if data_on_host else 0)
+        need = C.c_size_t(0)
+        _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(need)))
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.workspace = torch.empty(need.value, dtype=torch.uint8, device=self.device)
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        self._keep = (X, y)
+        if data_on_host:
+            X = np.ascontiguousarray(X)
+            y = np.ascontiguousarray(y)
+            m.X, m.y = X.ctypes.data, y.ctypes.data
+            self._keep = (X, y)
+        else:
+            assert X.is_cuda and y.is_cuda and X.is_contiguous() and y.is_contiguous()
+            m.X, m.y = X.data_ptr(), y.data_ptr()
+        w0 = np.ascontiguousarray(w0, dtype=np.float32)
+        assert w0.shape[0] == n_params(kind, dims)
+        m.w0 = w0.ctypes.data
+        m.workspace, m.workspace_bytes = self.workspace.data_ptr(), need.value
+        m.stream = self.stream.cuda_stream
+        td = TimeDist(time.kind, time.shift, time.rate, time.scale, time.slow_mod, time.slow_rem,
+                      time.slow_factor)
+        self._ctx = C.c_void_p(None)
+        self._desc = m
+        _check(lib().abs_init(C.byref(self._ctx), C.byref(m), W, K0, S, C.byref(td),
+                              C.c_ulonglong(seed)))
+
+    def run_rounds(self, n):
+        _check(lib().abs_run_rounds(self._ctx, n))
+
+    def enqueue_rounds(self, n):
+        _check(lib().abs_enqueue_rounds(self._ctx, n))
+
+    def rounds_done(self):
+        """(completed rounds, status code) without raising on a device status."""
+        r = C.c_int(0)
+        rc = lib().abs_rounds_done(self._ctx, C.byref(r))
+        return r.value, rc
+
+    def get_params(self):
+        d = n_params(self.kind, self.dims)
+        out = np.empty(d, dtype=np.float32)
+        got = C.c_size_t(0)
+        _check(lib().abs_get_params(self._ctx, out.ctypes.data, d, C.byref(got)))
+        assert got.value == d
+        return out
+
+    def get_trace(self, first=0, n=None):
+        if n is None:
+            n = self.rounds_done()[0] - first
+        W = self.W
+        a = dict(K=np.zeros(n, np.int32), n_restart=np.zeros(n, np.int32),
+                 theta=np.zeros(n, np.int32), T_end=np.zeros(n, np.uint64),
+                 loss_mean=np.zeros(n, np.float32), comm=np.zeros(n, np.uint64),
+                 sel_off=np.zeros(n + 1, np.int64), rst_off=np.zeros(n + 1, np.int64),
+                 sel_id=np.zeros(n * W, np.int32), sel_tau=np.zeros(n * W, np.int32),
+                 sel_loss=np.zeros(n * W, np.float32), rst_id=np.zeros(n * W, np.int32))
+        t = Trace()
+        for k, v in a.items():
+            setattr(t, k, v.ctypes.data)
+        t.cap_sel = t.cap_rst = n * W
+        _check(lib().abs_get_trace(self._ctx, first, n, C.byref(t)))
+        ns, nr = int(a["sel_off"][n]), int(a["rst_off"][n])
+        for k in ("sel_id", "sel_tau", "sel_loss"):
+            a[k] = a[k][:ns]
+        a["rst_id"] = a["rst_id"][:nr]
+        return a
+
+    def launch_count(self):
+        v = C.c_longlong(0)
+        _check(lib().abs_launch_count(self._ctx, C.byref(v)))
+        return v.value
+
+    def close(self):
+        if self._ctx:
+            lib().abs_destroy(self._ctx)
+            self._ctx = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def trace_rows(tr):
+    """Trace arrays -> list of per-round dicts (K, sel, tau, restart, T_end, theta, ...)."""
+    rows = []
+    for i in range(len(tr["K"])):
+        s0, s1 = int(tr["sel_off"][i]), int(tr["sel_off"][i + 1])
+        r0, r1 = int(tr["rst_off"][i]), int(tr["rst_off"][i + 1])
+        rows.append(dict(K=int(tr["K"][i]), sel=[int(x) for x in tr["sel_id"][s0:s1]],
+                         tau=[int(x) for x in tr["sel_tau"][s0:s1]],
+                         restart=[int(x) for x in tr["rst_id"][r0:r1]],
+                         T_end=int(tr["T_end"][i]), theta=int(tr["theta"][i]),
+                         loss_mean=float(tr["loss_mean"][i]), comm=int(tr["comm"][i]),
+                         sel_loss=[float(x) for x in tr["sel_loss"][s0:s1]]))
+    return rows
+
+
+def context_from_config(cfg, X, y, w0, max_rounds=None, **kw):
+    """Context for an `inputs.Config`; X, y as produced by `inputs.make_data` moved to the
+    device by the caller (or numpy with data_on_host=True)."""
+    return Context(cfg.kind, cfg.dims, X, y, w0, cfg.batch, cfg.lr, cfg.W, cfg.K0, cfg.S, cfg.time,
+                   cfg.run_seed, max_rounds or cfg.rounds, dtype=cfg.dtype, **kw)

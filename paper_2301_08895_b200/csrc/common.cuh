@@ -1,0 +1,81 @@
+// Shared device/host declarations of the ABS round loop.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/abs_b200.h"
+
+namespace absb {
+
+typedef unsigned long long u64;
+typedef long long i64;
+
+// Device status words (DevState::status).  0 = running.
+enum : int {
+  ST_OK = 0,
+  ST_DIVERGED = 1,   // a non-finite loss was uploaded in round `t`
+  ST_RANGE = 2,      // a completion tick left the 2^53 range
+  ST_NOSPACE = 3,    // round index reached the trace capacity
+  ST_INTERNAL = 4,   // an invariant failed (consumed staleness above the bound)
+  ST_TIMEOUT = 5,    // a bounded wait inside a kernel expired
+};
+
+constexpr int MAX_W = ABS_MAX_WORKERS;
+constexpr int MAX_TAU = ABS_MAX_BOUND + 1;
+
+struct TimeDist {
+  int kind;
+  double shift, rate, scale;
+  int slow_mod, slow_rem;
+  double slow_factor;
+};
+
+// Scalars of Algorithm 1 that live on the device between rounds.
+struct DevState {
+  // constants of the run
+  int W, K0, S, B, RB;            // RB: every version group's rows are padded to a multiple of RB
+  int k_mode, bound_mode, max_rounds;
+  i64 n_samples;
+  uint32_t key0, key1;            // Philox key = (seed low, seed high)
+  TimeDist dist;
+  // server state
+  int t;                          // round index of the next round to select
+  int K;                          // K^t
+  int theta;                      // threshold of the last restart test
+  int status;                     // ST_*
+  int diverged;                   // set by the loss kernels of the open round
+  int open;                       // 1 between selection and completion of a round
+  float L0;                       // loss estimate of round 0, f(w^0) in Eq. 5
+  u64 T_end;                      // end tick of the open round
+  int n_rows;                     // padded gradient rows of the open round
+  int n_row_tiles;                // n_rows / RB
+  int n_groups;
+  i64 sel_total, rst_total;       // flat trace fill
+  u64 comm;                       // communication-round counter (Sec. V-B)
+  int timeout_where;
+};
+
+// Pointers the control kernel works on (all device memory inside the workspace).
+struct CtlArgs {
+  DevState* st;
+  u64* c;              // [W] completion tick of each worker's job in flight
+  int* version;        // [W] round index of the model the worker holds
+  int* job;            // [W] index of the job in flight
+  int* sel;            // [W] selected worker ids of the open round, arrival order
+  int* sel_tau;        // [W]
+  int* sel_row0;       // [W] first gradient row of each selected worker
+  float* loss;         // [W] mean minibatch loss of each selected worker
+  float* row_loss;     // [rows_cap] per-sample losses (network models), else null
+  int* row_idx;        // [rows_cap] sample index of each gradient row, -1 for padding
+  int* tile_slot;      // [rows_cap / RB] ring slot of each row tile
+  // trace
+  int* tr_K; int* tr_R; int* tr_theta; u64* tr_T; float* tr_loss; u64* tr_comm;
+  i64* tr_sel_off; i64* tr_rst_off;
+  int* tr_sel_id; int* tr_sel_tau; float* tr_sel_loss; int* tr_rst_id;
+};
+
+__host__ __device__ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+__host__ __device__ inline size_t round_up_sz(size_t a, size_t b) { return (a + b - 1) / b * b; }
+
+}  // namespace absb

@@ -1,0 +1,341 @@
+// Server-side integer engine of Algorithm 1: arrival selection, Eq. 4-6 bookkeeping,
+// Philox job durations and minibatch indices.  One CTA of 1024 threads; every result is an
+// integer decided by exact arithmetic, so the trace is reproducible bit for bit.
+#pragma once
+#include "common.cuh"
+
+namespace absb {
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies, with the key
+// advanced by Weyl constants between rounds.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t out[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi_a = __umulhi(0xD2511F53u, c0), lo_a = 0xD2511F53u * c0;
+    const uint32_t hi_b = __umulhi(0xCD9E8D57u, c2), lo_b = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi_b ^ c1 ^ k0, n2 = hi_a ^ c3 ^ k1;
+    c0 = n0; c1 = lo_b; c2 = n2; c3 = lo_a;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Series logarithm that defines the exponential job times: u = m 2^e with m in [sqrt(1/2),
+// sqrt(2)), s = (m-1)/(m+1), ln u = e ln2 + 2s(1 + s^2/3 + ... + s^22/23).  Each step is one
+// binary64 operation rounded to nearest (the _rn intrinsics are never contracted into FMAs).
+__device__ __forceinline__ double ln_series(double u) {
+  const u64 bits = (u64)__double_as_longlong(u);
+  int e = (int)((bits >> 52) & 0x7FF) - 1023;
+  double m = __longlong_as_double((i64)((bits & 0x000FFFFFFFFFFFFFull) | 0x3FF0000000000000ull));
+  if (m >= 1.4142135623730951) { m = __dmul_rn(m, 0.5); e += 1; }
+  const double s = __ddiv_rn(__dadd_rn(m, -1.0), __dadd_rn(m, 1.0));
+  const double s2 = __dmul_rn(s, s);
+  double p = __ddiv_rn(1.0, 23.0);
+#pragma unroll
+  for (int k = 10; k >= 0; --k) {
+    p = __dmul_rn(p, s2);
+    p = __dadd_rn(p, __ddiv_rn(1.0, (double)(2 * k + 1)));
+  }
+  const double head = __dmul_rn((double)e, 0.6931471805599453);
+  const double tail = __dmul_rn(__dmul_rn(2.0, s), p);
+  return __dadd_rn(head, tail);
+}
+
+// Duration of job j of worker n in ticks (2^20 per time unit); 0 signals "out of range".
+__device__ __forceinline__ u64 job_ticks(const TimeDist& d, uint32_t k0, uint32_t k1, int n, int j) {
+  uint32_t w[4];
+  philox4x32_10((uint32_t)n, (uint32_t)j, 0u, 0u, k0, k1, w);
+  const double u = __dmul_rn(__dadd_rn((double)w[0], 0.5), 2.3283064365386963e-10);  // 2^-32
+  double dur;
+  if (d.kind == ABS_T_CONST) dur = d.shift;
+  else if (d.kind == ABS_T_EXP) dur = __ddiv_rn(-ln_series(u), d.rate);
+  else if (d.kind == ABS_T_SHIFTED_EXP) dur = __dadd_rn(d.shift, __ddiv_rn(-ln_series(u), d.rate));
+  else dur = __ddiv_rn(d.scale, __dsqrt_rn(u));
+  if (d.slow_mod > 0 && n % d.slow_mod == d.slow_rem) dur = __dmul_rn(dur, d.slow_factor);
+  const double scaled = __dmul_rn(dur, 1048576.0);
+  if (!(scaled < 9007199254740992.0)) return 0ull;
+  const u64 ticks = __double2ull_rd(scaled);
+  return ticks < 1ull ? 1ull : ticks;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Bitonic sort of 1024 64-bit keys, one per thread, ascending by thread index.
+// Exchange distances below 32 use shuffles, the others go through shared memory.
+__device__ __forceinline__ u64 bitonic_sort_1024(u64 key, u64* smem, int n_pow2) {
+  const int tid = threadIdx.x;
+  for (int k = 2; k <= n_pow2; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      u64 other;
+      if (j >= 32) {
+        smem[tid] = key;
+        __syncthreads();
+        other = smem[tid ^ j];
+        __syncthreads();
+      } else {
+        other = __shfl_xor_sync(0xffffffffu, key, j);
+      }
+      const bool up = ((tid & k) == 0);
+      const bool lower = ((tid & j) == 0);
+      const u64 mn = key < other ? key : other;
+      const u64 mx = key < other ? other : key;
+      key = (lower == up) ? mn : mx;
+    }
+  }
+  return key;
+}
+
+__device__ __forceinline__ i64 floor_div(i64 a, i64 b) {  // b > 0
+  i64 q = a / b;
+  if ((a % b != 0) && (a < 0)) --q;
+  return q;
+}
+
+struct CtlShared {
+  u64 keys[1024];
+  double red[32];
+  unsigned short wcnt[32][MAX_TAU];   // per-warp count of selected workers per staleness
+  int cnt[MAX_TAU];                    // selected workers per staleness
+  int grow0[MAX_TAU];                  // first row of each staleness group
+  unsigned char flag[1024];            // selected marker per worker id
+  int warp_tot[32];
+  int scalar[8];
+};
+
+// Completes the open round (Eq. 5, Eq. 4, Eq. 6, trace row), then selects the arrivals of the
+// next round and lays out its gradient rows.
+//   do_finish: complete the open round if there is one
+//   do_select: open the next round
+__global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select) {
+  __shared__ CtlShared sh;
+  DevState* st = a.st;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int W = st->W, S = st->S, B = st->B, RB = st->RB;
+  const int status0 = st->status;
+  const int open0 = st->open;
+  int t = st->t, K = st->K;
+  __syncthreads();
+  if (status0 != ST_OK) return;
+
+  // ------------------------------------------------------------------ finish round t
+  if (do_finish && open0) {
+    const u64 T_end = st->T_end;
+    // per-worker mean loss of network models: fixed-order sum of the per-sample losses
+    if (a.row_loss != nullptr) {
+      for (int i = warp; i < K; i += 32) {
+        const int r0 = a.sel_row0[i];
+        float acc = 0.f;
+        for (int b = lane; b < B; b += 32) acc += a.row_loss[r0 + b];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) a.loss[i] = __fdiv_rn(acc, (float)B);
+      }
+      __syncthreads();
+    }
+    const float my_loss = (tid < K) ? a.loss[tid] : 0.f;
+    const int bad = __syncthreads_or((tid < K) && !isfinite(my_loss)) || st->diverged;
+    if (bad) {
+      if (tid == 0) { st->status = ST_DIVERGED; st->open = 0; }
+      return;
+    }
+    // loss estimate: adjacent-pair tree sum in binary64 over 1024 leaves, /K, rounded to binary32
+    double v = (double)my_loss;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) v = __dadd_rn(v, __shfl_down_sync(0xffffffffu, v, o));
+    if (lane == 0) sh.red[warp] = v;
+    sh.flag[tid] = 0;
+    __syncthreads();
+    if (warp == 0) {
+      double x = sh.red[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) x = __dadd_rn(x, __shfl_down_sync(0xffffffffu, x, o));
+      if (lane == 0) sh.red[0] = x;
+    }
+    if (tid < K) sh.flag[a.sel[tid]] = 1;
+    __syncthreads();
+    const float Lt = __double2float_rn(__ddiv_rn(sh.red[0], (double)K));
+    const float L0 = (t == 0) ? Lt : st->L0;
+    // Eq. 5 as an exact integer rule: largest k with k^2 Lt <= K0^2 L0
+    int K_next = K;
+    if (st->k_mode == ABS_K_ADAPTIVE) {
+      int ok = 0;
+      if (Lt <= 0.f) {
+        ok = (tid == 0) ? W : 0;
+      } else if (tid < W) {
+        const int k = tid + 1;
+        const double lhs = __dmul_rn((double)(k * k), (double)Lt);
+        const double rhs = __dmul_rn((double)(st->K0 * st->K0), (double)L0);
+        ok = (lhs <= rhs) ? k : 0;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ok = max(ok, __shfl_xor_sync(0xffffffffu, ok, o));
+      if (lane == 0) sh.warp_tot[warp] = ok;
+      __syncthreads();
+      int kr = sh.warp_tot[lane];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) kr = max(kr, __shfl_xor_sync(0xffffffffu, kr, o));
+      K_next = min(W, max(K, kr));
+      __syncthreads();
+    }
+    // Eq. 4 with a = S - N/K0, in integers
+    int theta = S;
+    if (st->bound_mode == ABS_BOUND_ADAPTIVE) {
+      const i64 fl = floor_div((i64)W * (i64)(st->K0 - K_next), (i64)K_next * (i64)st->K0);
+      i64 th = (i64)S + fl;
+      if (th < 1) th = 1;
+      if (th > S) th = S;
+      theta = (int)th;
+    }
+    // Eq. 6 in Algorithm 1's order: arrivals and over-stale workers get w^{t+1}
+    int restart = 0, renew = 0;
+    if (tid < W) {
+      const int sel_me = sh.flag[tid];
+      restart = (!sel_me) && ((t + 1 - a.version[tid]) > theta);
+      renew = sel_me || restart;
+    }
+    int range_err = 0;
+    if (renew) {
+      const int j = a.job[tid] + 1;
+      const u64 dt = job_ticks(st->dist, st->key0, st->key1, tid, j);
+      const u64 cn = T_end + dt;
+      if (dt == 0ull || cn >= (1ull << 53)) range_err = 1;
+      a.job[tid] = j;
+      a.version[tid] = t + 1;
+      a.c[tid] = cn;
+    }
+    // ascending list of restarted ids
+    const unsigned rb = __ballot_sync(0xffffffffu, restart);
+    if (lane == 0) sh.warp_tot[warp] = __popc(rb);
+    range_err = __syncthreads_or(range_err);
+    int base = 0, R = 0;
+    for (int w = 0; w < 32; ++w) { const int c = sh.warp_tot[w]; if (w < warp) base += c; R += c; }
+    const i64 sel_off = st->sel_total, rst_off = st->rst_total;
+    if (restart) a.tr_rst_id[rst_off + base + __popc(rb & ((1u << lane) - 1u))] = tid;
+    if (tid < K) {
+      a.tr_sel_id[sel_off + tid] = a.sel[tid];
+      a.tr_sel_tau[sel_off + tid] = a.sel_tau[tid];
+      a.tr_sel_loss[sel_off + tid] = my_loss;
+    }
+    const u64 comm = st->comm + (u64)(K + R);
+    __syncthreads();
+    if (tid == 0) {
+      a.tr_K[t] = K; a.tr_R[t] = R; a.tr_theta[t] = theta; a.tr_T[t] = T_end;
+      a.tr_loss[t] = Lt; a.tr_comm[t] = comm;
+      a.tr_sel_off[t] = sel_off; a.tr_rst_off[t] = rst_off;
+      a.tr_sel_off[t + 1] = sel_off + K; a.tr_rst_off[t + 1] = rst_off + R;
+      st->sel_total = sel_off + K; st->rst_total = rst_off + R; st->comm = comm;
+      st->L0 = L0; st->theta = theta; st->K = K_next; st->t = t + 1; st->open = 0;
+      if (range_err) st->status = ST_RANGE;
+    }
+    if (range_err) return;
+    t = t + 1;
+    K = K_next;
+    __syncthreads();
+  }
+
+  // ------------------------------------------------------------------ select round t
+  if (!do_select) return;
+  if (t >= st->max_rounds) {
+    if (tid == 0) st->status = ST_NOSPACE;
+    return;
+  }
+  {
+    // arrivals: the K smallest (completion tick, worker id) keys
+    int n_pow2 = 32;
+    while (n_pow2 < W) n_pow2 <<= 1;
+    u64 key = (tid < W) ? ((a.c[tid] << 10) | (u64)tid) : ~0ull;
+    key = bitonic_sort_1024(key, sh.keys, n_pow2);
+    sh.keys[tid] = key;
+    for (int i = tid; i < 32 * MAX_TAU; i += 1024) (&sh.wcnt[0][0])[i] = 0;
+    __syncthreads();
+    const u64 T_end = sh.keys[K - 1] >> 10;
+    int n = -1, tau = -1;
+    if (tid < K) {
+      n = (int)(key & 1023ull);
+      tau = t - a.version[n];
+    }
+    const int tau_bad = __syncthreads_or(tid < K && (tau < 0 || tau > S));
+    if (tau_bad) {
+      if (tid == 0) st->status = ST_INTERNAL;
+      return;
+    }
+    // group the arrivals by staleness (all members of a group read the same ring slot);
+    // inside a group keep arrival order
+    const unsigned peers = __match_any_sync(0xffffffffu, tau);
+    const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+    if (tau >= 0 && rank_in_warp == 0) sh.wcnt[warp][tau] = (unsigned short)__popc(peers);
+    __syncthreads();
+    if (tid <= S) {
+      int c = 0;
+      for (int w = 0; w < 32; ++w) { const int x = sh.wcnt[w][tid]; sh.wcnt[w][tid] = (unsigned short)c; c += x; }
+      sh.cnt[tid] = c;
+    }
+    __syncthreads();
+    if (tid <= S) {
+      int r0 = 0, g = 0;
+      for (int q = 0; q < tid; ++q) { r0 += round_up(sh.cnt[q] * B, RB); g += sh.cnt[q] > 0; }
+      sh.grow0[tid] = r0;
+      if (tid == S) {
+        sh.scalar[0] = r0 + round_up(sh.cnt[S] * B, RB);
+        sh.scalar[1] = g + (sh.cnt[S] > 0);
+      }
+    }
+    __syncthreads();
+    const int n_rows = sh.scalar[0];
+    if (tid < K) {
+      const int row0 = sh.grow0[tau] + ((int)sh.wcnt[warp][tau] + rank_in_warp) * B;
+      a.sel[tid] = n;
+      a.sel_tau[tid] = tau;
+      a.sel_row0[tid] = row0;
+      sh.keys[tid] = ((u64)(unsigned)row0 << 32) | (u64)(unsigned)n;   // reuse as (row0, n)
+    }
+    // ring slot of every row tile, and padding rows
+    if (tid <= S && sh.cnt[tid] > 0) {
+      const int slot = (t - tid) % (S + 1);
+      const int r0 = sh.grow0[tid], r1 = r0 + round_up(sh.cnt[tid] * B, RB);
+      for (int r = r0; r < r1; r += RB) a.tile_slot[r / RB] = slot;
+      for (int r = r0 + sh.cnt[tid] * B; r < r1; ++r) a.row_idx[r] = -1;
+    }
+    __syncthreads();
+    // minibatch draws: sample b of job (n, j) = word b%4 of Philox block (n, j, 1, b/4),
+    // mapped into the worker's shard [n M / N, (n+1) M / N)
+    const int blocks_per = (B + 3) >> 2;
+    const i64 M = st->n_samples;
+    for (int item = tid; item < K * blocks_per; item += 1024) {
+      const int i = item / blocks_per, blk = item - i * blocks_per;
+      const int wn = (int)(sh.keys[i] & 0xffffffffull), row0 = (int)(sh.keys[i] >> 32);
+      const i64 lo = ((i64)wn * M) / W, hi = ((i64)(wn + 1) * M) / W;
+      uint32_t w4[4];
+      philox4x32_10((uint32_t)wn, (uint32_t)a.job[wn], 1u, (uint32_t)blk, st->key0, st->key1, w4);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int b = blk * 4 + q;
+        if (b < B) a.row_idx[row0 + b] = (int)(lo + (i64)(((u64)w4[q] * (u64)(hi - lo)) >> 32));
+      }
+    }
+    if (tid == 0) {
+      st->T_end = T_end;
+      st->n_rows = n_rows;
+      st->n_row_tiles = n_rows / RB;
+      st->n_groups = sh.scalar[1];
+      st->diverged = 0;
+      st->open = 1;
+    }
+  }
+}
+
+// Algorithm 1, initialisation: every worker holds w^0 and starts job 0 at tick 0.
+__global__ void abs_init_state_kernel(CtlArgs a) {
+  DevState* st = a.st;
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (tid < st->W) {
+    const u64 dt = job_ticks(st->dist, st->key0, st->key1, tid, 0);
+    if (dt == 0ull) st->status = ST_RANGE;
+    a.c[tid] = dt;
+    a.version[tid] = 0;
+    a.job[tid] = 0;
+  }
+}
+
+}  // namespace absb

@@ -1,0 +1,66 @@
+"""Shared helpers of the parity tests: run the CUDA library and the oracle on
+the same seeded inputs and compare."""
+import numpy as np
+
+from conftest import make_oracle
+from paper_2301_08895_b200 import abs as gpu
+from paper_2301_08895_b200 import inputs
+
+INT_FIELDS = ("K", "sel", "tau", "restart", "T_end", "theta", "comm")
+
+
+def to_device(cfg, X, y):
+    import torch
+    if cfg.dtype == inputs.BF16:
+        Xd = torch.from_numpy(X.view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        Xd = torch.from_numpy(X).cuda()
+    return Xd, torch.from_numpy(y).cuda()
+
+
+def gpu_run(cfg, X, y, w0, rounds, **kw):
+    Xd, yd = to_device(cfg, X, y)
+    ctx = gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=rounds, **kw)
+    ctx.run_rounds(rounds)
+    rows = gpu.trace_rows(ctx.get_trace())
+    params = ctx.get_params()
+    ctx.close()
+    return rows, params
+
+
+def first_integer_mismatch(rows_a, rows_b):
+    for t, (a, b) in enumerate(zip(rows_a, rows_b)):
+        for f in INT_FIELDS:
+            if a[f] != b[f]:
+                return t, f, a[f], b[f]
+    if len(rows_a) != len(rows_b):
+        return min(len(rows_a), len(rows_b)), "length", len(rows_a), len(rows_b)
+    return None
+
+
+def rel_l2(a, b):
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def compare_with_oracle(cfg, X, y, w0, rounds, tol, forced=False, loss_tol=None, **kw):
+    """GPU run vs oracle run.  forced=False: both run freely and the integer
+    traces must be identical.  forced=True: the oracle's K rule is fed the
+    GPU's uploaded losses (its own losses and parameters are still its own),
+    which separates the integer machinery from last-bit loss differences."""
+    gkw = {k: v for k, v in kw.items() if k in ("k_mode", "bound_mode")}
+    rows, params = gpu_run(cfg, X, y, w0, rounds, **gkw)
+    assert len(rows) == rounds
+    o = make_oracle(cfg, X, y, w0, **gkw)
+    orows = o.run(rounds, forced_losses=[r["sel_loss"] for r in rows] if forced else None)
+    mm = first_integer_mismatch(rows, orows)
+    assert mm is None, "integer trace differs at round %s field %s: gpu %s oracle %s (oracle " \
+        "decision margin %.3g)" % (mm + (o.min_margin,))
+    err = rel_l2(params, o.w)
+    assert err <= tol, "parameters differ: rel L2 %.3g > %.3g" % (err, tol)
+    lt = loss_tol if loss_tol is not None else tol * 10
+    for t, (a, b) in enumerate(zip(rows, orows)):
+        la, lb = np.array(a["sel_loss"]), np.array(b["sel_loss"])
+        assert np.all(np.abs(la - lb) <= lt * np.maximum(1.0, np.abs(lb))), \
+            "uploaded losses differ in round %d" % t
+    return rows, orows, err, o

@@ -1,0 +1,214 @@
+"""Parity of the CUDA round loop (through the C ABI) with the CPU oracle.
+
+Integer trace (K, selected ids in arrival order, staleness, restarts, end tick,
+threshold, communication counter): bit-exact.  Parameters: relative L2 within
+1e-5 for fp32 storage and 2e-2 for bf16 storage with fp32 master.
+"""
+import numpy as np
+import pytest
+
+from helpers import compare_with_oracle, gpu_run, rel_l2
+from conftest import make_oracle
+from paper_2301_08895_b200 import abs as gpu
+from paper_2301_08895_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32, TOL_BF16 = 1e-5, 2e-2
+
+
+def _problem(cfg):
+    X, y, _ = inputs.make_data(cfg)
+    return X, y, inputs.make_w0(cfg)
+
+
+# ------------------------------------------------------------------ the benchmark configurations
+def test_config1_lsq_fp32_full():
+    cfg = inputs.config(1)
+    X, y, w0 = _problem(cfg)
+    rows, orows, err, o = compare_with_oracle(cfg, X, y, w0, cfg.rounds, TOL_FP32)
+    assert rows[-1]["K"] == cfg.W and rows[0]["K"] == cfg.K0
+    assert any(r["restart"] for r in rows)
+
+
+def test_config2_softmax_fp32_full():
+    cfg = inputs.config(2)
+    X, y, w0 = _problem(cfg)
+    rows, orows, err, o = compare_with_oracle(cfg, X, y, w0, cfg.rounds, TOL_FP32)
+    assert rows[-1]["K"] == cfg.W
+
+
+def test_config3_mlp_bf16_prefix():
+    cfg = inputs.config(3).scaled(n_samples=16384)
+    X, y, w0 = _problem(cfg)
+    # forced: the oracle's K rule reads the GPU's uploaded losses (bf16 activations make the two
+    # loss streams differ in the 3rd digit, enough to move an Eq. 5 decision by a round)
+    compare_with_oracle(cfg, X, y, w0, 100, TOL_BF16, forced=True, loss_tol=5e-2)
+
+
+def test_config3_free_running_prefix():
+    cfg = inputs.config(3).scaled(n_samples=16384)
+    X, y, w0 = _problem(cfg)
+    compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, loss_tol=5e-2)
+
+
+def test_config4_mlp_bf16_prefix():
+    cfg = inputs.config(4).scaled(n_samples=8192)
+    X, y, w0 = _problem(cfg)
+    compare_with_oracle(cfg, X, y, w0, 10, TOL_BF16, forced=True, loss_tol=5e-2)
+
+
+@pytest.mark.parametrize("W", [256, 1024])
+def test_config5_lsq_bf16_reduced(W):
+    cfg = inputs.config(5, W).scaled(n_samples=32768)
+    X, y, w0 = _problem(cfg)
+    compare_with_oracle(cfg, X, y, w0, 40 if W == 256 else 12, TOL_BF16, forced=True, loss_tol=1e-3)
+
+
+# ------------------------------------------------------------------ ragged shapes and modes
+def _small_cfg(kind, dims, dtype, W, B, K0, S, time, n=3000, lr=0.05, seed=5):
+    data = "lsq" if kind == inputs.LSQ else "mixture"
+    c = inputs.Config("small", kind, tuple(dims), dtype, W, B, K0, S, 60, lr, n, time, data,
+                      sigma=1.0, w0="he" if kind == inputs.MLP else "zeros")
+    c.data_seed, c.run_seed, c.w0_seed = seed, seed + 1, seed + 2
+    return c
+
+
+EXP = inputs.TimeSpec(inputs.T_EXP, rate=1.0)
+SEXP = inputs.TimeSpec(inputs.T_SHIFTED_EXP, shift=0.5, rate=2.0)
+PARETO = inputs.TimeSpec(inputs.T_PARETO2, scale=1.0)
+
+
+@pytest.mark.parametrize("dtype,tol", [(inputs.FP32, TOL_FP32), (inputs.BF16, TOL_BF16)])
+@pytest.mark.parametrize("kind,dims,B", [
+    (inputs.LSQ, (77, 1), 19),
+    (inputs.SOFTMAX, (131, 7), 24),
+    (inputs.MLP, (50, 37, 5), 24),
+    (inputs.MLP, (200, 136, 72, 10), 40),
+])
+def test_ragged_shapes(kind, dims, B, dtype, tol):
+    cfg = _small_cfg(kind, dims, dtype, 13, B, 3, 5, PARETO)
+    X, y, w0 = _problem(cfg)
+    forced = dtype == inputs.BF16
+    compare_with_oracle(cfg, X, y, w0, 60, tol, forced=forced, loss_tol=5e-2 if forced else None)
+
+
+@pytest.mark.parametrize("k_mode,bound_mode,K0,S", [
+    (gpu.K_FIXED, gpu.BOUND_FIXED, 1, 40),      # ASGD
+    (gpu.K_FIXED, gpu.BOUND_ADAPTIVE, 4, 0),    # K-sync: everything restarts
+    (gpu.K_FIXED, gpu.BOUND_FIXED, 3, 2),       # K-async with a tight fixed bound
+    (gpu.K_ADAPTIVE, gpu.BOUND_FIXED, 2, 3),
+    (gpu.K_ADAPTIVE, gpu.BOUND_ADAPTIVE, 11, 0),  # K = N, bound 0: synchronous SGD
+])
+def test_modes_fixed_k_traces_are_pure_integer(k_mode, bound_mode, K0, S):
+    cfg = _small_cfg(inputs.SOFTMAX, (40, 6), inputs.FP32, 11, 16, K0, S, SEXP)
+    X, y, w0 = _problem(cfg)
+    rows, orows, err, o = compare_with_oracle(cfg, X, y, w0, 80, TOL_FP32, k_mode=k_mode,
+                                              bound_mode=bound_mode)
+    if S == 0 and k_mode == gpu.K_FIXED:
+        assert all(len(r["restart"]) == 11 - K0 and set(r["tau"]) == {0} for r in rows)
+    if K0 == 1:
+        assert max(max(r["tau"]) for r in rows) > 11
+
+
+def test_lock_step_constant_times():
+    cfg = _small_cfg(inputs.LSQ, (16, 1), inputs.FP32, 8, 4, 2, 3,
+                     inputs.TimeSpec(inputs.T_CONST, shift=3.0))
+    X, y, w0 = _problem(cfg)
+    rows, params = gpu_run(cfg, X, y, w0, 40, k_mode=gpu.K_FIXED, bound_mode=gpu.BOUND_FIXED)
+    for t, r in enumerate(rows):
+        assert r["sel"] == [(t * 2) % 8, (t * 2) % 8 + 1]
+        assert r["T_end"] == 3 * 2 ** 20 * ((t * 2) // 8 + 1)
+        assert r["tau"] == [min(t, 3)] * 2 and r["restart"] == []
+
+
+def test_straggler_restarts_every_theta_plus_one_rounds():
+    time = inputs.TimeSpec(inputs.T_CONST, shift=1.0, slow_mod=5, slow_rem=4, slow_factor=2.0 ** 20)
+    cfg = _small_cfg(inputs.LSQ, (16, 1), inputs.FP32, 5, 4, 2, 3, time)
+    X, y, w0 = _problem(cfg)
+    rows, _ = gpu_run(cfg, X, y, w0, 41, k_mode=gpu.K_FIXED, bound_mode=gpu.BOUND_FIXED)
+    for t, r in enumerate(rows):
+        assert 4 not in r["sel"] and (4 in r["restart"]) == (t % 4 == 3)
+    compare_with_oracle(cfg, X, y, w0, 41, TOL_FP32, k_mode=gpu.K_FIXED, bound_mode=gpu.BOUND_FIXED)
+
+
+@pytest.mark.parametrize("W,B,K0,S", [(1, 1, 1, 0), (2, 1, 1, 1), (1024, 2, 128, 32), (33, 64, 5, 255)])
+def test_edge_sizes(W, B, K0, S):
+    cfg = _small_cfg(inputs.LSQ, (24, 1), inputs.FP32, W, B, K0, S, EXP, n=4096, lr=0.02)
+    X, y, w0 = _problem(cfg)
+    compare_with_oracle(cfg, X, y, w0, 30, TOL_FP32)
+
+
+def test_many_workers_network():
+    cfg = _small_cfg(inputs.SOFTMAX, (32, 4), inputs.FP32, 300, 3, 20, 12, PARETO, n=6000)
+    X, y, w0 = _problem(cfg)
+    compare_with_oracle(cfg, X, y, w0, 40, TOL_FP32)
+
+
+# ------------------------------------------------------------------ API behaviour
+def test_rounds_in_several_calls_equal_one_call():
+    cfg = inputs.config(1)
+    X, y, w0 = _problem(cfg)
+    rows_a, params_a = gpu_run(cfg, X, y, w0, 50)
+    from helpers import to_device
+    Xd, yd = to_device(cfg, X, y)
+    ctx = gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=50)
+    for n in (1, 0, 7, 42):
+        ctx.run_rounds(n)
+    rows_b = gpu.trace_rows(ctx.get_trace())
+    assert rows_a == rows_b and np.array_equal(params_a, ctx.get_params())
+    part = gpu.trace_rows(ctx.get_trace(10, 5))
+    assert part == rows_a[10:15]
+    with pytest.raises(gpu.AbsError) as e:
+        ctx.run_rounds(1)
+    assert e.value.code == gpu.ENOSPACE
+    with pytest.raises(gpu.AbsError) as e:
+        ctx.get_trace(45, 10)
+    assert e.value.code == gpu.EINVAL
+    assert ctx.launch_count() > 150
+    ctx.close()
+
+
+def test_host_dataset_entry_gives_same_result():
+    cfg = inputs.config(1)
+    X, y, w0 = _problem(cfg)
+    rows_a, params_a = gpu_run(cfg, X, y, w0, 30)
+    ctx = gpu.context_from_config(cfg, X, y, w0, max_rounds=30, data_on_host=True)
+    ctx.run_rounds(30)
+    assert gpu.trace_rows(ctx.get_trace()) == rows_a
+    assert np.array_equal(ctx.get_params(), params_a)
+    ctx.close()
+
+
+def test_divergence_is_reported_and_state_stays_readable():
+    cfg = _small_cfg(inputs.LSQ, (16, 1), inputs.FP32, 4, 8, 4, 0, EXP, lr=1e4)
+    X, y, w0 = _problem(cfg)
+    from helpers import to_device
+    Xd, yd = to_device(cfg, X, y)
+    ctx = gpu.context_from_config(cfg, Xd * 100, yd, w0, max_rounds=200)
+    with pytest.raises(gpu.AbsError) as e:
+        ctx.run_rounds(200)
+    assert e.value.code == gpu.EDIVERGED
+    done, rc = ctx.rounds_done()
+    assert rc == gpu.EDIVERGED and 0 < done < 200
+    rows = gpu.trace_rows(ctx.get_trace(0, done))
+    assert len(rows) == done and np.all(np.isfinite(ctx.get_params()))
+    o = make_oracle(cfg, X * 100, y, w0)
+    from oracle import abs_sim
+    with pytest.raises(abs_sim.Diverged):
+        o.run(200)
+    assert abs(len(o.trace) - done) <= 1
+    ctx.close()
+
+
+def test_tick_range_error():
+    time = inputs.TimeSpec(inputs.T_CONST, shift=2.0 ** 31)
+    cfg = _small_cfg(inputs.LSQ, (16, 1), inputs.FP32, 4, 8, 2, 2, time)
+    X, y, w0 = _problem(cfg)
+    from helpers import to_device
+    Xd, yd = to_device(cfg, X, y)
+    ctx = gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=20)
+    with pytest.raises(gpu.AbsError) as e:
+        ctx.run_rounds(20)
+    assert e.value.code == gpu.ERANGE
+    ctx.close()
