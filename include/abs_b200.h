@@ -65,6 +65,20 @@ extern "C" {
 #define ABS_T_SHIFTED_EXP  2    /* shift + Exp(rate) */
 #define ABS_T_PARETO2      3    /* Pareto, shape 2, minimum `scale` */
 
+#define ABS_FLAG_NO_TENSOR_CORES 1  /* run the hidden-layer contractions on the FP32-FMA kernels */
+
+/* kernel classes reported by abs_profile_read */
+#define ABS_KC_CTL     0  /* arrival selection + Eq. 4-6 bookkeeping */
+#define ABS_KC_GATHER  1  /* minibatch row gather */
+#define ABS_KC_FWD     2  /* hidden-layer forward contraction (Eq. 2) */
+#define ABS_KC_DGRAD   3  /* hidden-layer delta back-propagation */
+#define ABS_KC_WGRAD   4  /* weight gradient summed over the selected workers (Eq. 3) */
+#define ABS_KC_OUTPUT  5  /* output layer: forward + loss, its back-propagation and gradient */
+#define ABS_KC_BIAS    6  /* bias gradients */
+#define ABS_KC_LSQ     7  /* least-squares residual + gradient */
+#define ABS_KC_UPDATE  8  /* Eq. 3 step + ring write */
+#define ABS_KC_COUNT   9
+
 #define ABS_MAX_LAYERS   7
 #define ABS_MAX_WORKERS  1024
 #define ABS_MAX_BOUND    255
@@ -83,6 +97,7 @@ typedef struct {
   int k_mode;               /* ABS_K_* */
   int bound_mode;           /* ABS_BOUND_* */
   int max_rounds;           /* trace capacity: total rounds this context may run */
+  int flags;                /* ABS_FLAG_* bits */
   int data_on_host;         /* 0: X, y are device pointers owned by the caller and must outlive
                                the context.  1: X, y are host pointers; abs_init copies them into
                                the workspace (abs_workspace_bytes accounts for the room) */
@@ -158,6 +173,13 @@ int abs_get_trace(abs_ctx* ctx, int first_round, int n_rounds, abs_trace* out_ho
 
 /* Kernels of ours launched on behalf of this context so far (set-up included). */
 int abs_launch_count(abs_ctx* ctx, long long* launches);
+
+/* Measurement aid (the paper has no counterpart).  After abs_profile_start, every kernel launch
+ * of this context is bracketed by a pair of CUDA events on the context's stream until
+ * max_launches pairs are used.  abs_profile_read synchronises, adds the elapsed times up per
+ * kernel class (ABS_KC_*; both arrays need ABS_KC_COUNT entries), and ends profiling. */
+int abs_profile_start(abs_ctx* ctx, int max_launches);
+int abs_profile_read(abs_ctx* ctx, long long* launches, double* total_ms);
 
 int abs_destroy(abs_ctx* ctx);
 

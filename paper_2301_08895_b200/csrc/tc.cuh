@@ -1,0 +1,396 @@
+// Grouped bf16 GEMMs of the hidden layers on the 5th-generation tensor cores (tcgen05, accumulators
+// in tensor memory, operands staged by TMA into 128-byte-swizzled shared memory).
+//
+// One persistent, warp-specialised kernel serves the three contractions of Eq. 2 / Eq. 3:
+//   FWD    H[r][n]  = relu( sum_k A[r][k] W_s[k][n] + b_s[n] )          rows grouped by model version
+//   DGRAD  D[r][m]  = ( sum_n Dl[r][n] W_s[m][n] ) * [H[r][m] > 0]
+//   WGRAD  G_p[m][n] = sum_{r in chunk p} A[r][m] Dl[r][n]               summed over ALL selected workers
+// "s" is the ring slot of the row tile's model version (all rows of a 128-row tile share it).
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the tensor-memory allocation),
+// warps 2..5 = epilogue (tensor memory -> registers -> global).  Two accumulators alternate so the
+// epilogue of one tile overlaps the main loop of the next.  Every mbarrier wait is bounded; on
+// expiry the CTA raises ST_TIMEOUT, drains its own copies, frees tensor memory and returns.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace absb {
+namespace tc {
+
+constexpr int BM = 128;      // tile rows (UMMA M)
+constexpr int BK = 64;       // k elements per stage = one 128-byte swizzle row of bf16
+constexpr int UK = 16;       // k per tcgen05.mma of kind::f16
+constexpr int THREADS = 192;
+
+enum Mode : int { FWD = 0, DGRAD = 1, WGRAD = 2 };
+
+struct Params {
+  DevState* st;
+  const int* tile_slot;
+  int mode;
+  int M_total;             // WGRAD: in (rows of G); FWD/DGRAD: unused
+  int N_total;             // FWD: out, DGRAD: in, WGRAD: out
+  int K_total;             // FWD: in,  DGRAD: out, WGRAD: unused (rows come from the device state)
+  int P;                   // WGRAD split count
+  const __nv_bfloat16* ring; size_t slot_stride; size_t b_off;   // FWD bias: ring + slot*stride + b_off
+  const __nv_bfloat16* mask_src;   // DGRAD: H[r][N_total]
+  __nv_bfloat16* out_bf16;         // FWD/DGRAD result [rows][N_total]
+  float* out_f32;                  // WGRAD: G + w_off, partial p at + p*slot_stride, row pitch N_total
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait (about two seconds, and never more than 2^28 polls).  False = gave up, or another
+// role of this CTA already gave up; *abort is the CTA-wide flag.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+  if (mbar_test(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t i = 1; i < (1u << 28); ++i) {
+    if (mbar_test(bar, parity)) return true;
+    if ((i & 63u) == 0u) {
+      if (*abort) return false;
+      if (global_ns() - t0 > 2000000000ull) break;
+    }
+  }
+  *abort = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor of a 128-byte-swizzled bf16 operand tile:
+// bits [0,14) start >> 4, [16,30) leading byte offset >> 4, [32,46) stride byte offset >> 4,
+// [46,48) descriptor version 1, [61,64) layout 2 = 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, majors, N >> 3, M >> 4.
+__host__ __device__ constexpr uint32_t instr_desc(int a_mn_major, int b_mn_major, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+template <int BN> struct Cfg {
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct TileCoord { int a_row, b_col, slot, k_begin, n_kb, split; };
+
+template <int BN>
+__global__ void __launch_bounds__(THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params p) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  DevState* st = p.st;
+  if (st->status != ST_OK) return;
+  const int n_rows = st->n_rows;
+  const int n_row_tiles = n_rows / BM;
+  const int mode = p.mode;
+  const int n_ct = (p.N_total + BN - 1) / BN;
+  const int n_mt = (mode == WGRAD) ? (p.M_total + BM - 1) / BM : n_row_tiles;
+  const int n_tiles = (mode == WGRAD) ? n_mt * n_ct * p.P : n_row_tiles * n_ct;
+  if ((int)blockIdx.x >= n_tiles) return;
+  const int chunk = (mode == WGRAD) ? round_up((n_rows + p.P - 1) / p.P, BK) : 0;
+  const int RB = st->RB;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)C::STAGES * C::STAGE_BYTES);
+  uint64_t* full = bars;                     // [STAGES] TMA bytes landed
+  uint64_t* empty = bars + C::STAGES;        // [STAGES] MMAs that read the stage are done
+  uint64_t* acc_full = bars + 2 * C::STAGES; // [2] accumulator complete
+  uint64_t* acc_empty = acc_full + 2;        // [2] accumulator drained by the epilogue
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+    *abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  auto tile_coord = [&](int tile) -> TileCoord {
+    TileCoord c;
+    if (mode == WGRAD) {
+      const int per_split = n_mt * n_ct;
+      c.split = tile / per_split;
+      const int rem = tile - c.split * per_split;
+      c.a_row = (rem / n_ct) * BM;           // m0
+      c.b_col = (rem % n_ct) * BN;           // n0
+      c.slot = 0;
+      c.k_begin = min(n_rows, c.split * chunk);
+      const int k_end = min(n_rows, (c.split + 1) * chunk);
+      c.n_kb = (k_end - c.k_begin) / BK;
+    } else {
+      const int rt = tile / n_ct;
+      c.split = 0;
+      c.a_row = rt * BM;
+      c.b_col = (tile - rt * n_ct) * BN;
+      c.slot = p.tile_slot[c.a_row / RB];
+      c.k_begin = 0;
+      c.n_kb = (p.K_total + BK - 1) / BK;
+    }
+    return c;
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int armed[C::STAGES];
+      for (int s = 0; s < C::STAGES; ++s) armed[s] = -1;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const TileCoord c = tile_coord(tile);
+        for (int kb = 0; kb < c.n_kb; ++kb) {
+          if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) { ok = false; break; }
+          uint8_t* sa = smem + (size_t)stage * C::STAGE_BYTES;
+          uint8_t* sb = sa + C::A_BYTES;
+          mbar_expect_tx(&full[stage], C::STAGE_BYTES);
+          armed[stage] = (int)phase;
+          const int k0 = c.k_begin + kb * BK;
+          if (mode == FWD) {
+            tma_load_2d(sa, &map_a, &full[stage], k0, c.a_row);
+            for (int j = 0; j < BN / 64; ++j) tma_load_3d(sb + j * 8192, &map_b, &full[stage], c.b_col + 64 * j, k0, c.slot);
+          } else if (mode == DGRAD) {
+            tma_load_2d(sa, &map_a, &full[stage], k0, c.a_row);
+            tma_load_3d(sb, &map_b, &full[stage], k0, c.b_col, c.slot);
+          } else {
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * 8192, &map_a, &full[stage], c.a_row + 64 * j, k0);
+            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, &map_b, &full[stage], c.b_col + 64 * j, k0);
+          }
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      // tail: every stage's release (an asynchronous arrive from the tensor core) must have landed
+      // before this CTA's shared memory goes away
+      for (int s = 0; s < C::STAGES && ok; ++s) {
+        if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) ok = false;
+        if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        // let this CTA's copies in flight land before the shared memory is released
+        for (int s = 0; s < C::STAGES; ++s)
+          if (armed[s] >= 0) {
+            const unsigned long long t0 = global_ns();
+            while (!mbar_test(&full[s], (uint32_t)armed[s]) && global_ns() - t0 < 100000000ull) {}
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const bool a_mn = (mode == WGRAD), b_mn = (mode != DGRAD);
+      const uint32_t idesc = instr_desc(a_mn ? 1 : 0, b_mn ? 1 : 0, BN);
+      // K-major tile: rows of 128 B, 8-row groups 1024 B apart; a k step of 16 elements is 32 B.
+      // MN-major tile: 64-wide boxes 8192 B apart (leading offset), 8-k groups 1024 B apart;
+      // a k step of 16 rows is 2048 B.
+      const uint32_t a_lbo = a_mn ? 8192u : 16u, b_lbo = b_mn ? 8192u : 16u;
+      const uint32_t a_kstep = a_mn ? 2048u : 32u, b_kstep = b_mn ? 2048u : 32u;
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const TileCoord c = tile_coord(tile);
+        if (c.n_kb == 0) continue;
+        if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < c.n_kb; ++kb) {
+          if (!mbar_wait(&full[stage], phase, abort)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + (uint32_t)stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < BK / UK; ++kk) {
+            const uint64_t da = smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
+            const uint64_t db = smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
+            umma(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(&empty[stage]);
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(&acc_full[acc]);
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps)
+    const int q = warp & 3;                    // tensor-memory lane quarter this warp may read
+    const int row_in_tile = q * 32 + lane;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+      const TileCoord c = tile_coord(tile);
+      const bool have = c.n_kb > 0;
+      if (have) {
+        if (!mbar_wait(&acc_full[acc], acc_phase, abort)) break;
+        tc_fence_after();
+      }
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+      const int r = c.a_row + row_in_tile;     // output row (FWD/DGRAD) or m (WGRAD)
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        const int n0 = c.b_col + c0;
+        if (n0 >= p.N_total) break;            // uniform in the warp
+        uint32_t v[32];
+        if (have) tmem_ld32(t_row + (uint32_t)c0, v);
+        else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = 0u;
+        }
+        if (mode == WGRAD) {
+          if (r < p.M_total) {
+            float* dst = p.out_f32 + (size_t)c.split * p.slot_stride + (size_t)r * p.N_total + n0;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              if (n0 + i < p.N_total)
+                *reinterpret_cast<uint4*>(dst + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+          }
+        } else {
+          __nv_bfloat16* dst = p.out_bf16 + (size_t)r * p.N_total + n0;
+          if (mode == FWD) {
+            const __nv_bfloat16* bias = p.ring + (size_t)c.slot * p.slot_stride + p.b_off + n0;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              if (n0 + i < p.N_total) {
+                const uint4 bb = *reinterpret_cast<const uint4*>(bias + i);
+                const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&bb);
+                uint4 o;
+                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const float2 bf = __bfloat1622float2(b2[j]);
+                  const float x = fmaxf(__uint_as_float(v[i + 2 * j]) + bf.x, 0.f);
+                  const float y = fmaxf(__uint_as_float(v[i + 2 * j + 1]) + bf.y, 0.f);
+                  o2[j] = __floats2bfloat162_rn(x, y);
+                }
+                *reinterpret_cast<uint4*>(dst + i) = o;
+              }
+            }
+          } else {
+            const __nv_bfloat16* h = p.mask_src + (size_t)r * p.N_total + n0;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              if (n0 + i < p.N_total) {
+                const uint4 hh = *reinterpret_cast<const uint4*>(h + i);
+                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&hh);
+                uint4 o;
+                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const float2 hf = __bfloat1622float2(h2[j]);
+                  const float x = hf.x > 0.f ? __uint_as_float(v[i + 2 * j]) : 0.f;
+                  const float y = hf.y > 0.f ? __uint_as_float(v[i + 2 * j + 1]) : 0.f;
+                  o2[j] = __floats2bfloat162_rn(x, y);
+                }
+                *reinterpret_cast<uint4*>(dst + i) = o;
+              }
+            }
+          }
+        }
+      }
+      if (have) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
+  }
+  if (threadIdx.x == 0 && *abort) {
+    st->timeout_where = 100 + mode;
+    st->status = ST_TIMEOUT;
+  }
+}
+
+}  // namespace tc
+}  // namespace absb
