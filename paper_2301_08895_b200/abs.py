@@ -21,13 +21,15 @@ K_ADAPTIVE, K_FIXED = 0, 1
 BOUND_ADAPTIVE, BOUND_FIXED = 0, 1
 T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2 = 0, 1, 2, 3
 MAX_LAYERS = 7
+FLAG_NO_TENSOR_CORES = 1
+KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update")
 
 
 class ModelDesc(C.Structure):
     _fields_ = [("kind", C.c_int), ("n_layers", C.c_int), ("dims", C.c_int * (MAX_LAYERS + 1)),
                 ("batch", C.c_int), ("lr", C.c_float), ("dtype", C.c_int),
                 ("local_steps", C.c_int), ("k_mode", C.c_int), ("bound_mode", C.c_int),
-                ("max_rounds", C.c_int), ("data_on_host", C.c_int),
+                ("max_rounds", C.c_int), ("flags", C.c_int), ("data_on_host", C.c_int),
                 ("X", C.c_void_p), ("y", C.c_void_p), ("n_samples", C.c_longlong),
                 ("w0", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("stream", C.c_void_p)]
@@ -75,6 +77,8 @@ def lib():
         l.abs_get_params.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
         l.abs_get_trace.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(Trace)]
         l.abs_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_longlong)]
+        l.abs_profile_start.argtypes = [C.c_void_p, C.c_int]
+        l.abs_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
         l.abs_destroy.argtypes = [C.c_void_p]
         _lib = l
     return _lib
@@ -96,7 +100,7 @@ def n_params(kind, dims):
 
 
 def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-          local_steps=1, data_on_host=0):
+          local_steps=1, data_on_host=0, flags=0):
     m = ModelDesc()
     m.kind, m.n_layers = kind, len(dims) - 1
     for i, v in enumerate(dims):
@@ -104,11 +108,13 @@ def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mod
     m.batch, m.lr, m.dtype = int(batch), float(lr), dtype
     m.local_steps, m.k_mode, m.bound_mode = local_steps, k_mode, bound_mode
     m.max_rounds, m.data_on_host, m.n_samples = int(max_rounds), data_on_host, int(n_samples)
+    m.flags = int(flags)
     return m
 
 
-def workspace_bytes(kind, dims, batch, dtype, W, S, max_rounds, n_samples, data_on_host=0):
-    m = _desc(kind, dims, batch, 0.0, dtype, max_rounds, n_samples, 0, 0, 1, data_on_host)
+def workspace_bytes(kind, dims, batch, dtype, W, S, max_rounds, n_samples, data_on_host=0,
+                    flags=0):
+    m = _desc(kind, dims, batch, 0.0, dtype, max_rounds, n_samples, 0, 0, 1, data_on_host, flags)
     out = C.c_size_t(0)
     _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(out)))
     return out.value
@@ -124,14 +130,14 @@ class Context:
 
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, time, seed, max_rounds,
                  dtype=FP32, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE, local_steps=1,
-                 data_on_host=False, stream=None, device="cuda:0"):
+                 data_on_host=False, stream=None, device="cuda:0", flags=0):
         import torch
         self._torch = torch
         self.kind, self.dims, self.W, self.S = kind, list(dims), W, S
         self.max_rounds = max_rounds
         n_samples = X.shape[0]
         m = _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-                  local_steps, 1 if data_on_host else 0)
+                  local_steps, 1 if data_on_host else 0, flags)
         need = C.c_size_t(0)
         _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(need)))
         self.device = torch.device(device)
@@ -204,6 +210,16 @@ class Context:
         v = C.c_longlong(0)
         _check(lib().abs_launch_count(self._ctx, C.byref(v)))
         return v.value
+
+    def profile_start(self, max_launches):
+        _check(lib().abs_profile_start(self._ctx, int(max_launches)))
+
+    def profile_read(self):
+        """{class name: (launches, total ms)} of the launches recorded since profile_start."""
+        n = (C.c_longlong * len(KC_NAMES))()
+        ms = (C.c_double * len(KC_NAMES))()
+        _check(lib().abs_profile_read(self._ctx, n, ms))
+        return {KC_NAMES[i]: (int(n[i]), float(ms[i])) for i in range(len(KC_NAMES))}
 
     def close(self):
         if self._ctx:

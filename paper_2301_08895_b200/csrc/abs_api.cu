@@ -11,6 +11,8 @@
 #include "common.cuh"
 #include "ctl.cuh"
 #include "simt.cuh"
+#include "narrow.cuh"
+#include "tc.cuh"
 
 using namespace absb;
 
@@ -38,8 +40,13 @@ struct Carver {
 };
 
 // Byte offsets of everything inside the workspace.
+enum LayerPath : int { PATH_SIMT = 0, PATH_TC = 1, PATH_NARROW = 2 };
+
 struct Layout {
   int n_layers = 0, RB = 0, rows_cap = 0, P = 0, n_tiles_cap = 0;
+  int path[ABS_MAX_LAYERS] = {};        // how each layer's contractions run
+  int bn_fwd[ABS_MAX_LAYERS] = {}, bn_dg[ABS_MAX_LAYERS] = {}, bn_wg[ABS_MAX_LAYERS] = {};
+  bool any_tc = false;
   size_t esz = 4;                       // bytes per stored element (4 or 2)
   size_t d = 0, d_pad = 0;
   size_t w_off[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the padded vector
@@ -92,12 +99,45 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   }
   L->d = src;
   L->d_pad = round_up_sz(off, 256);
-  L->RB = lsq ? m->batch : 64;
+  // per-layer path: tensor cores for bf16 hidden layers whose sizes TMA can address, the
+  // narrow-output kernels for a last layer of at most 16 classes, FP32-FMA tiles otherwise
+  const bool tc_ok = m->dtype == ABS_BF16_FP32MASTER && !(m->flags & ABS_FLAG_NO_TENSOR_CORES);
+  L->any_tc = false;
+  for (int l = 0; l < m->n_layers && !lsq; ++l) {
+    const int in = m->dims[l], out = m->dims[l + 1];
+    const bool last = l == m->n_layers - 1;
+    if (last && out <= NARROW_MAX_C && (size_t)in * out <= 10240) L->path[l] = PATH_NARROW;
+    else if (!last && tc_ok && in % 8 == 0 && out % 8 == 0 && in >= 64 && out >= 64) {
+      L->path[l] = PATH_TC;
+      L->any_tc = true;
+    } else L->path[l] = PATH_SIMT;
+  }
+  L->RB = lsq ? m->batch : (L->any_tc ? 128 : 64);
   const int groups = (W < S + 1) ? W : S + 1;
   L->rows_cap = round_up(W * m->batch, L->RB) + groups * L->RB;
   L->n_tiles_cap = L->rows_cap / L->RB;
   if (lsq) {
     L->P = 0;
+  } else if (L->any_tc) {
+    // tile widths: widest tile that still gives every SM work; split count of the row reduction
+    // sized so the largest weight gradient fills about two waves of 148 CTAs
+    const int row_tiles = L->rows_cap / 128;
+    auto pick = [](int n, int other_tiles) {
+      for (int bn : {256, 128}) if (n >= bn && other_tiles * ((n + bn - 1) / bn) >= 120) return bn;
+      return n >= 128 ? 128 : 64;
+    };
+    size_t biggest = 1;
+    for (int l = 0; l < m->n_layers; ++l) {
+      if (L->path[l] != PATH_TC) continue;
+      const int in = m->dims[l], out = m->dims[l + 1];
+      L->bn_fwd[l] = pick(out, row_tiles);
+      L->bn_dg[l] = pick(in, row_tiles);
+      L->bn_wg[l] = pick(out, ((in + 127) / 128) * 3);
+      biggest = std::max(biggest, (size_t)((in + 127) / 128) * ((out + L->bn_wg[l] - 1) / L->bn_wg[l]));
+    }
+    int P = (int)((296 + biggest / 2) / biggest);
+    P = std::min(P, std::max(1, W * m->batch / 512));
+    L->P = std::max(1, std::min(P, 8));
   } else {
     // split count of the row reduction in the weight-gradient kernels
     size_t tiles = 0;
@@ -125,6 +165,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   if (!lsq) {
     const int C = m->dims[m->n_layers];
     L->logits = cv.take(4 * (size_t)L->rows_cap * C);
+    L->act[0] = (L->path[0] == PATH_TC) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     for (int l = 1; l <= m->n_layers; ++l) {
       L->act[l] = (l < m->n_layers) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]) : 0;
       L->delta[l] = cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]);
@@ -152,10 +193,15 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
 
 }  // namespace
 
+struct TcLayer {
+  CUtensorMap fwd_a, fwd_b, dg_a, dg_b, wg_a, wg_b;
+};
+
 struct abs_ctx {
   abs_model_desc m;
   Layout L;
   int W, K0, S;
+  int sm_count = 148;
   cudaStream_t stream;
   char* ws;
   const void* X;
@@ -164,6 +210,11 @@ struct abs_ctx {
   int sticky = ABS_OK;
   long long launches = 0;
   CtlArgs ctl;
+  TcLayer tcl[ABS_MAX_LAYERS];
+  // profiling: event pairs around launches
+  std::vector<cudaEvent_t> ev;       // 2 per recorded launch
+  std::vector<int> ev_class;
+  int ev_cap = 0;                    // launches that may still be recorded
   template <typename U> U* at(size_t off) const { return reinterpret_cast<U*>(ws + off); }
 };
 
@@ -180,6 +231,104 @@ int cuda_fail(abs_ctx* ctx, cudaError_t e, const char* what) {
     if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);       \
   } while (0)
 
+// Runs `launch` (one kernel launch on ctx->stream), counted and, while profiling, bracketed by events.
+template <class F>
+void launch_k(abs_ctx* ctx, int cls, F launch) {
+  const bool rec = (int)ctx->ev_class.size() < ctx->ev_cap;
+  if (rec) cudaEventRecord(ctx->ev[2 * ctx->ev_class.size()], ctx->stream);
+  launch();
+  if (rec) {
+    cudaEventRecord(ctx->ev[2 * ctx->ev_class.size() + 1], ctx->stream);
+    ctx->ev_class.push_back(cls);
+  }
+  ctx->launches += 1;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// bf16 tensor map with 128-byte swizzle; dims/strides innermost first, strides in bytes for dims 1...
+bool make_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
+              const cuuint32_t* box) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_act_map(CUtensorMap* map, const void* base, int dim, int rows, int box_rows) {
+  const cuuint64_t dims[2] = {(cuuint64_t)dim, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)dim * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  return make_map(map, base, 2, dims, strides, box);
+}
+
+bool make_w_map(CUtensorMap* map, const void* base, int in, int out, int slots, size_t slot_stride, int box_rows) {
+  const cuuint64_t dims[3] = {(cuuint64_t)out, (cuuint64_t)in, (cuuint64_t)slots};
+  const cuuint64_t strides[2] = {(cuuint64_t)out * 2, (cuuint64_t)slot_stride * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  return make_map(map, base, 3, dims, strides, box);
+}
+
+template <int BN>
+void launch_tc(abs_ctx* ctx, int cls, const CUtensorMap& a, const CUtensorMap& b, const tc::Params& p, int max_tiles) {
+  const int grid = std::max(1, std::min(ctx->sm_count, max_tiles));
+  launch_k(ctx, cls, [&] {
+    tc::tc_gemm_kernel<BN><<<grid, tc::THREADS, tc::Cfg<BN>::SMEM_BYTES, ctx->stream>>>(a, b, p);
+  });
+}
+
+void launch_tc_bn(abs_ctx* ctx, int bn, int cls, const CUtensorMap& a, const CUtensorMap& b, const tc::Params& p,
+                  int max_tiles) {
+  if (bn == 256) launch_tc<256>(ctx, cls, a, b, p, max_tiles);
+  else if (bn == 128) launch_tc<128>(ctx, cls, a, b, p, max_tiles);
+  else launch_tc<64>(ctx, cls, a, b, p, max_tiles);
+}
+
+int setup_tc(abs_ctx* ctx) {
+  const abs_model_desc& m = ctx->m;
+  const Layout& L = ctx->L;
+  if (!L.any_tc) return ABS_OK;
+  cudaError_t e;
+  e = cudaFuncSetAttribute(tc::tc_gemm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<256>::SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<128>::SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<64>::SMEM_BYTES);
+  if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaFuncSetAttribute(tc_gemm_kernel)");
+  const char* ring = ctx->at<char>(L.ring);
+  for (int l = 0; l < m.n_layers; ++l) {
+    if (L.path[l] != PATH_TC) continue;
+    const int in = m.dims[l], out = m.dims[l + 1];
+    TcLayer& t = ctx->tcl[l];
+    const void* act_in = ctx->at<void>(L.act[l]);
+    const void* delta_out = ctx->at<void>(L.delta[l + 1]);
+    const void* wbase = ring + 2 * L.w_off[l];
+    bool ok = make_act_map(&t.fwd_a, act_in, in, L.rows_cap, 128) &&
+              make_w_map(&t.fwd_b, wbase, in, out, ctx->S + 1, L.d_pad, 64) &&
+              make_act_map(&t.wg_a, act_in, in, L.rows_cap, 64) &&
+              make_act_map(&t.wg_b, delta_out, out, L.rows_cap, 64);
+    if (ok && l > 0)
+      ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
+           make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l]);
+    if (!ok) return fail(ABS_ECUDA, "cuTensorMapEncodeTiled failed for layer %d", l);
+  }
+  return ABS_OK;
+}
+
 template <typename T>
 void enqueue_gradient(abs_ctx* ctx) {
   const abs_model_desc& m = ctx->m;
@@ -192,44 +341,120 @@ void enqueue_gradient(abs_ctx* ctx) {
     a.X = ctx->X; a.y = (const float*)ctx->y;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad;
     a.loss = ctx->ctl.loss; a.G = ctx->at<float>(L.G); a.d = m.dims[0];
-    lsq_grad_kernel<T><<<ctx->W, 256, 0, s>>>(a);
-    ctx->launches += 1;
+    launch_k(ctx, ABS_KC_LSQ, [&] { lsq_grad_kernel<T><<<ctx->W, 256, 0, s>>>(a); });
     return;
   }
   const int nl = m.n_layers;
   const int row_tiles = L.rows_cap / TM;
+  const int row_tiles128 = L.rows_cap / 128;
+  const bool gathered = L.path[0] == PATH_TC;     // layer 0 reads the gathered copy act[0]
   LayerArgs la[ABS_MAX_LAYERS];
   for (int l = 0; l < nl; ++l) {
     LayerArgs& a = la[l];
     a.st = st; a.tile_slot = ctx->ctl.tile_slot; a.row_idx = ctx->ctl.row_idx;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad; a.w_off = L.w_off[l];
     a.in = m.dims[l]; a.out = m.dims[l + 1];
-    a.gather = (l == 0);
-    a.act_in = (l == 0) ? ctx->X : ctx->at<void>(L.act[l]);
+    a.gather = (l == 0 && !gathered);
+    a.act_in = (l == 0 && !gathered) ? ctx->X : ctx->at<void>(L.act[l]);
     a.act_out = (l == nl - 1) ? ctx->at<void>(L.logits) : ctx->at<void>(L.act[l + 1]);
     a.delta_out = ctx->at<void>(L.delta[l + 1]);
     a.delta_in = (l == 0) ? nullptr : ctx->at<void>(L.delta[l]);
     a.G = ctx->at<float>(L.G); a.P = L.P;
   }
+  auto tc_params = [&](int l, int mode) {
+    tc::Params p;
+    memset(&p, 0, sizeof p);
+    p.st = st; p.tile_slot = ctx->ctl.tile_slot; p.mode = mode; p.P = L.P;
+    p.ring = ctx->at<__nv_bfloat16>(L.ring); p.slot_stride = L.d_pad;
+    p.b_off = L.w_off[l] + (size_t)m.dims[l] * m.dims[l + 1];
+    return p;
+  };
+  auto narrow_args = [&](int l) {
+    NarrowArgs a;
+    a.st = st; a.tile_slot = ctx->ctl.tile_slot; a.row_idx = ctx->ctl.row_idx; a.labels = (const int*)ctx->y;
+    a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad; a.w_off = L.w_off[l];
+    a.in = m.dims[l]; a.C = m.dims[l + 1];
+    a.gather = la[l].gather; a.act_in = la[l].act_in;
+    a.delta_out = ctx->at<void>(L.delta[l + 1]);
+    a.delta_in = (l == 0) ? nullptr : ctx->at<void>(L.delta[l]);
+    a.row_loss = ctx->ctl.row_loss; a.G = ctx->at<float>(L.G); a.P = L.P;
+    return a;
+  };
+  if (gathered) {
+    launch_k(ctx, ABS_KC_GATHER, [&] {
+      gather_rows_kernel<<<ctx->sm_count * 8, 256, 0, s>>>(st, ctx->ctl.row_idx, (const __nv_bfloat16*)ctx->X,
+                                                           ctx->at<__nv_bfloat16>(L.act[0]), m.dims[0]);
+    });
+  }
+  // ---- forward (Eq. 2 at the model version each worker holds)
   for (int l = 0; l < nl; ++l) {
-    dim3 grid((la[l].out + TN - 1) / TN, row_tiles);
-    if (l == nl - 1) simt_fwd_kernel<T, true><<<grid, 256, 0, s>>>(la[l]);
-    else simt_fwd_kernel<T, false><<<grid, 256, 0, s>>>(la[l]);
-  }
-  LossArgs lo;
-  lo.st = st; lo.row_idx = ctx->ctl.row_idx; lo.labels = (const int*)ctx->y;
-  lo.logits = ctx->at<float>(L.logits); lo.delta = ctx->at<void>(L.delta[nl]);
-  lo.row_loss = ctx->ctl.row_loss; lo.C = m.dims[nl];
-  net_loss_kernel<T><<<(L.rows_cap + 255) / 256, 256, 0, s>>>(lo);
-  for (int l = nl - 1; l >= 0; --l) {
-    if (l > 0) {
-      dim3 grid((la[l].in + TN - 1) / TN, row_tiles);
-      simt_dgrad_kernel<T><<<grid, 256, 0, s>>>(la[l]);
+    const bool last = l == nl - 1;
+    if (L.path[l] == PATH_TC) {
+      tc::Params p = tc_params(l, tc::FWD);
+      p.N_total = la[l].out; p.K_total = la[l].in;
+      p.out_bf16 = (__nv_bfloat16*)la[l].act_out;
+      const int bn = L.bn_fwd[l];
+      launch_tc_bn(ctx, bn, ABS_KC_FWD, ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
+    } else if (L.path[l] == PATH_NARROW) {
+      NarrowArgs a = narrow_args(l);
+      const size_t sm = sizeof(float) * ((size_t)a.in * a.C + a.C);
+      launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_fwd_loss_kernel<T><<<row_tiles, 256, sm, s>>>(a); });
+    } else {
+      dim3 grid((la[l].out + TN - 1) / TN, row_tiles);
+      const int cls = last ? ABS_KC_OUTPUT : ABS_KC_FWD;
+      if (last) launch_k(ctx, cls, [&] { simt_fwd_kernel<T, true><<<grid, 256, 0, s>>>(la[l]); });
+      else launch_k(ctx, cls, [&] { simt_fwd_kernel<T, false><<<grid, 256, 0, s>>>(la[l]); });
+      if (last) {
+        LossArgs lo;
+        lo.st = st; lo.row_idx = ctx->ctl.row_idx; lo.labels = (const int*)ctx->y;
+        lo.logits = ctx->at<float>(L.logits); lo.delta = ctx->at<void>(L.delta[nl]);
+        lo.row_loss = ctx->ctl.row_loss; lo.C = m.dims[nl];
+        launch_k(ctx, ABS_KC_OUTPUT, [&] { net_loss_kernel<T><<<(L.rows_cap + 255) / 256, 256, 0, s>>>(lo); });
+      }
     }
-    dim3 gridw((la[l].out + TN - 1) / TN, (la[l].in + 1 + TM - 1) / TM, L.P);
-    simt_wgrad_kernel<T><<<gridw, 256, 0, s>>>(la[l]);
   }
-  ctx->launches += 3 * nl;
+  // ---- backward: deltas, then the weight gradients summed over all selected workers (Eq. 3)
+  for (int l = nl - 1; l >= 0; --l) {
+    if (L.path[l] == PATH_TC) {
+      if (l > 0) {
+        tc::Params p = tc_params(l, tc::DGRAD);
+        p.N_total = la[l].in; p.K_total = la[l].out;
+        p.mask_src = (const __nv_bfloat16*)la[l].act_in;
+        p.out_bf16 = (__nv_bfloat16*)la[l].delta_in;
+        const int bn = L.bn_dg[l];
+        launch_tc_bn(ctx, bn, ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, p, row_tiles128 * ((la[l].in + bn - 1) / bn));
+      }
+      tc::Params p = tc_params(l, tc::WGRAD);
+      p.M_total = la[l].in; p.N_total = la[l].out;
+      p.out_f32 = ctx->at<float>(L.G) + L.w_off[l];
+      const int bn = L.bn_wg[l];
+      launch_tc_bn(ctx, bn, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, p,
+                   ((la[l].in + 127) / 128) * ((la[l].out + bn - 1) / bn) * L.P);
+      dim3 gridb((la[l].out + 31) / 32, L.P);
+      const T* dl = (const T*)la[l].delta_out;
+      float* G = ctx->at<float>(L.G);
+      const size_t b_off = L.w_off[l] + (size_t)la[l].in * la[l].out;
+      const int out = la[l].out, P = L.P;
+      const size_t stride = L.d_pad;
+      launch_k(ctx, ABS_KC_BIAS, [&] { colsum_kernel<T><<<gridb, 1024, 0, s>>>(st, dl, G, stride, b_off, out, P); });
+    } else if (L.path[l] == PATH_NARROW) {
+      NarrowArgs a = narrow_args(l);
+      if (l > 0) {
+        const size_t sm = sizeof(float) * ((size_t)a.in * a.C + 64 * a.C);
+        launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_dgrad_kernel<T><<<row_tiles, 256, sm, s>>>(a); });
+      }
+      dim3 gridw((a.in + 1 + 31) / 32, L.P);
+      launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_wgrad_kernel<T><<<gridw, 1024, 0, s>>>(a); });
+    } else {
+      const bool last = l == nl - 1;
+      if (l > 0) {
+        dim3 grid((la[l].in + TN - 1) / TN, row_tiles);
+        launch_k(ctx, last ? ABS_KC_OUTPUT : ABS_KC_DGRAD, [&] { simt_dgrad_kernel<T><<<grid, 256, 0, s>>>(la[l]); });
+      }
+      dim3 gridw((la[l].out + TN - 1) / TN, (la[l].in + 1 + TM - 1) / TM, L.P);
+      launch_k(ctx, last ? ABS_KC_OUTPUT : ABS_KC_WGRAD, [&] { simt_wgrad_kernel<T><<<gridw, 256, 0, s>>>(la[l]); });
+    }
+  }
 }
 
 template <typename T>
@@ -239,9 +464,8 @@ void enqueue_update(abs_ctx* ctx) {
   u.st = ctx->at<DevState>(L.st); u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
   u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
   const size_t n4 = L.d_pad / 4;
-  const int blocks = (int)std::min<size_t>((n4 + 255) / 256, 148 * 8);
-  update_kernel<T><<<blocks, 256, 0, ctx->stream>>>(u);
-  ctx->launches += 1;
+  const int blocks = (int)std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * 8);
+  launch_k(ctx, ABS_KC_UPDATE, [&] { update_kernel<T><<<blocks, 256, 0, ctx->stream>>>(u); });
 }
 
 int read_status(abs_ctx* ctx, DevState* host) {
@@ -365,6 +589,14 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   c.tr_sel_id = ctx->at<int>(L.tr_sel_id); c.tr_sel_tau = ctx->at<int>(L.tr_sel_tau);
   c.tr_sel_loss = ctx->at<float>(L.tr_sel_loss); c.tr_rst_id = ctx->at<int>(L.tr_rst_id);
 
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      ctx->sm_count = sms;
+  }
+  rc = setup_tc(ctx);
+  if (rc != ABS_OK) return bail(rc);
   abs_init_state_kernel<<<(W + 255) / 256, 256, 0, s>>>(c);
   if (model->dtype == ABS_FP32) ring_init_kernel<float><<<148, 256, 0, s>>>(ctx->at<float>(L.master), ctx->at<void>(L.ring), L.d_pad);
   else ring_init_kernel<__nv_bfloat16><<<148, 256, 0, s>>>(ctx->at<float>(L.master), ctx->at<void>(L.ring), L.d_pad);
@@ -390,14 +622,12 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
   const bool f32 = ctx->m.dtype == ABS_FP32;
   for (int r = 0; r < n; ++r) {
     // the control kernel completes the previous round (if any) and selects this round's arrivals
-    abs_ctl_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->ctl, 1, 1);
-    ctx->launches += 1;
+    launch_k(ctx, ABS_KC_CTL, [&] { abs_ctl_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->ctl, 1, 1); });
     if (f32) { enqueue_gradient<float>(ctx); enqueue_update<float>(ctx); }
     else { enqueue_gradient<__nv_bfloat16>(ctx); enqueue_update<__nv_bfloat16>(ctx); }
   }
   if (n > 0) {
-    abs_ctl_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->ctl, 1, 0);
-    ctx->launches += 1;
+    launch_k(ctx, ABS_KC_CTL, [&] { abs_ctl_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->ctl, 1, 0); });
   }
   CU(cudaGetLastError());
   ctx->rounds_enqueued += n;
@@ -481,9 +711,37 @@ int abs_launch_count(abs_ctx* ctx, long long* launches) {
   return ABS_OK;
 }
 
+int abs_profile_start(abs_ctx* ctx, int max_launches) {
+  if (!ctx || max_launches < 0) return fail(ABS_EINVAL, "bad argument");
+  ctx->ev_class.clear();
+  while ((int)ctx->ev.size() < 2 * max_launches) {
+    cudaEvent_t e;
+    CU(cudaEventCreate(&e));
+    ctx->ev.push_back(e);
+  }
+  ctx->ev_cap = max_launches;
+  return ABS_OK;
+}
+
+int abs_profile_read(abs_ctx* ctx, long long* launches, double* total_ms) {
+  if (!ctx || !launches || !total_ms) return fail(ABS_EINVAL, "null argument");
+  CU(cudaStreamSynchronize(ctx->stream));
+  for (int c = 0; c < ABS_KC_COUNT; ++c) { launches[c] = 0; total_ms[c] = 0.0; }
+  for (size_t i = 0; i < ctx->ev_class.size(); ++i) {
+    float ms = 0.f;
+    CU(cudaEventElapsedTime(&ms, ctx->ev[2 * i], ctx->ev[2 * i + 1]));
+    launches[ctx->ev_class[i]] += 1;
+    total_ms[ctx->ev_class[i]] += ms;
+  }
+  ctx->ev_cap = 0;
+  ctx->ev_class.clear();
+  return ABS_OK;
+}
+
 int abs_destroy(abs_ctx* ctx) {
   if (!ctx) return ABS_OK;
   cudaStreamSynchronize(ctx->stream);
+  for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
   delete ctx;
   return ABS_OK;
 }

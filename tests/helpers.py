@@ -49,7 +49,7 @@ def compare_with_oracle(cfg, X, y, w0, rounds, tol, forced=False, loss_tol=None,
     GPU's uploaded losses (its own losses and parameters are still its own),
     which separates the integer machinery from last-bit loss differences."""
     gkw = {k: v for k, v in kw.items() if k in ("k_mode", "bound_mode")}
-    rows, params = gpu_run(cfg, X, y, w0, rounds, **gkw)
+    rows, params = gpu_run(cfg, X, y, w0, rounds, flags=kw.get("flags", 0), **gkw)
     assert len(rows) == rounds
     o = make_oracle(cfg, X, y, w0, **gkw)
     orows = o.run(rounds, forced_losses=[r["sel_loss"] for r in rows] if forced else None)
