@@ -174,6 +174,13 @@ int abs_get_trace(abs_ctx* ctx, int first_round, int n_rounds, abs_trace* out_ho
 /* Kernels of ours launched on behalf of this context so far (set-up included). */
 int abs_launch_count(abs_ctx* ctx, long long* launches);
 
+/* How the context runs (the paper has no counterpart): *partials = number of fp32 partial sums
+ * the Eq. 3 step adds up per parameter (0: one per selected worker), *row_block = padding unit of
+ * a version group's gradient rows, *rows_cap = row capacity of the activation buffers,
+ * path[l] (n_layers entries) = 0 FP32-FMA tiles, 1 tensor cores, 2 narrow output layer.
+ * Any pointer may be NULL. */
+int abs_get_plan(abs_ctx* ctx, int* partials, int* row_block, int* rows_cap, int* path);
+
 /* Measurement aid (the paper has no counterpart).  After abs_profile_start, every kernel launch
  * of this context is bracketed by a pair of CUDA events on the context's stream until
  * max_launches pairs are used.  abs_profile_read synchronises, adds the elapsed times up per

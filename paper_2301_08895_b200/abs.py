@@ -77,6 +77,8 @@ def lib():
         l.abs_get_params.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
         l.abs_get_trace.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(Trace)]
         l.abs_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_longlong)]
+        l.abs_get_plan.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int),
+                                   C.POINTER(C.c_int), C.POINTER(C.c_int)]
         l.abs_profile_start.argtypes = [C.c_void_p, C.c_int]
         l.abs_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
         l.abs_destroy.argtypes = [C.c_void_p]
@@ -210,6 +212,14 @@ class Context:
         v = C.c_longlong(0)
         _check(lib().abs_launch_count(self._ctx, C.byref(v)))
         return v.value
+
+    def plan(self):
+        """dict(partials, row_block, rows_cap, path) describing how the context runs."""
+        P, rb, rc = C.c_int(0), C.c_int(0), C.c_int(0)
+        path = (C.c_int * MAX_LAYERS)()
+        _check(lib().abs_get_plan(self._ctx, C.byref(P), C.byref(rb), C.byref(rc), path))
+        return dict(partials=P.value, row_block=rb.value, rows_cap=rc.value,
+                    path=[path[i] for i in range(len(self.dims) - 1)])
 
     def profile_start(self, max_launches):
         _check(lib().abs_profile_start(self._ctx, int(max_launches)))

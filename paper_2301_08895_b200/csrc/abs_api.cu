@@ -711,6 +711,15 @@ int abs_launch_count(abs_ctx* ctx, long long* launches) {
   return ABS_OK;
 }
 
+int abs_get_plan(abs_ctx* ctx, int* partials, int* row_block, int* rows_cap, int* path) {
+  if (!ctx) return fail(ABS_EINVAL, "ctx is null");
+  if (partials) *partials = ctx->L.P;
+  if (row_block) *row_block = ctx->L.RB;
+  if (rows_cap) *rows_cap = ctx->L.rows_cap;
+  if (path) for (int l = 0; l < ctx->m.n_layers; ++l) path[l] = ctx->L.path[l];
+  return ABS_OK;
+}
+
 int abs_profile_start(abs_ctx* ctx, int max_launches) {
   if (!ctx || max_launches < 0) return fail(ABS_EINVAL, "bad argument");
   ctx->ev_class.clear();
