@@ -174,6 +174,19 @@ int abs_get_trace(abs_ctx* ctx, int first_round, int n_rounds, abs_trace* out_ho
 /* Kernels of ours launched on behalf of this context so far (set-up included). */
 int abs_launch_count(abs_ctx* ctx, long long* launches);
 
+/* Stand-alone operation: Eq. 2 with U = 1 for n workers of the least-squares model at one model w,
+ * and the mean of their uploads (the sum of Eq. 3 divided by n).  Worker i's minibatch is the B
+ * sample indices idx[i*B .. i*B+B).  Results: loss_out[i] = mean_b 1/2 (x_b.w - y_b)^2 and
+ * g_out[j] = 1/(n B) sum_i sum_b (x_b.w - y_b) x_b[j].
+ * All pointers are device memory: X [n_samples][d] and w [d] in the storage type of `dtype`
+ * (float, or bf16 for ABS_BF16_FP32MASTER), y float, idx int32 [n*B], g_out float [d], loss_out
+ * float [n], scratch float [scratch_floats] with scratch_floats >= n*d (per-worker partial sums,
+ * contents undefined afterwards).  n in [1, 1024], B in [1, 1024], d in [1, 2^20].
+ * Enqueues on `stream` and returns without synchronising. */
+int abs_lsq_gradient(const void* X, const float* y, const void* w, const int* idx, int n, int B, int d,
+                     int dtype, float* scratch, size_t scratch_floats, float* g_out, float* loss_out,
+                     void* stream);
+
 /* How the context runs (the paper has no counterpart): *partials = number of fp32 partial sums
  * the Eq. 3 step adds up per parameter (0: one per selected worker), *row_block = padding unit of
  * a version group's gradient rows, *rows_cap = row capacity of the activation buffers,

@@ -77,6 +77,9 @@ def lib():
         l.abs_get_params.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
         l.abs_get_trace.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(Trace)]
         l.abs_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_longlong)]
+        l.abs_lsq_gradient.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                       C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t,
+                                       C.c_void_p, C.c_void_p, C.c_void_p]
         l.abs_get_plan.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int),
                                    C.POINTER(C.c_int), C.POINTER(C.c_int)]
         l.abs_profile_start.argtypes = [C.c_void_p, C.c_int]
@@ -241,6 +244,19 @@ class Context:
             self.close()
         except Exception:
             pass
+
+
+def lsq_gradient(X, y, w, idx, g_out, loss_out, scratch, stream=None):
+    """abs_lsq_gradient on torch CUDA tensors: X [M, d] and w [d] float32 or bfloat16, y float32,
+    idx int32 [n, B], g_out float32 [d], loss_out float32 [n], scratch float32 (>= n*d)."""
+    import torch
+    n, B = idx.shape
+    d = X.shape[1]
+    dtype = BF16_FP32MASTER if X.dtype == torch.bfloat16 else FP32
+    s = stream if stream is not None else torch.cuda.current_stream(X.device)
+    _check(lib().abs_lsq_gradient(X.data_ptr(), y.data_ptr(), w.data_ptr(), idx.data_ptr(), n, B, d,
+                                  dtype, scratch.data_ptr(), scratch.numel(), g_out.data_ptr(),
+                                  loss_out.data_ptr(), s.cuda_stream))
 
 
 def trace_rows(tr):

@@ -9,7 +9,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libabs_b200.so")
 STAMP = os.path.join(HERE, "libabs_b200.so.stamp")
-SOURCES = ["abs_api.cu"]
+SOURCES = ["abs_api.cu", "ops.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--expt-relaxed-constexpr", "--expt-extended-lambda",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]

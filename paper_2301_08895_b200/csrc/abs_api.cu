@@ -20,6 +20,14 @@ namespace {
 
 thread_local std::string g_err;
 
+}  // namespace
+
+namespace absb {
+void set_last_error(const char* text) { g_err = text; }
+}
+
+namespace {
+
 int fail(int code, const char* fmt, ...) {
   char buf[512];
   va_list ap;
