@@ -187,6 +187,23 @@ int abs_lsq_gradient(const void* X, const float* y, const void* w, const int* id
                      int dtype, float* scratch, size_t scratch_floats, float* g_out, float* loss_out,
                      void* stream);
 
+/* abs_lsq_gradient for callers that must not allocate (the paper has no counterpart; this is a
+ * packaging variant of the operation above).  Meant for code that runs where cudaMalloc is off
+ * limits: inside a pre-sized memory plan, in a process whose device memory is entirely owned by
+ * another component, or on a path where an allocation's implicit synchronisation is not allowed.
+ * Same arguments and results as abs_lsq_gradient without the scratch pair: the per-worker
+ * partial sums go to a fixed 4 MiB array built into the library (every GPU that loads the
+ * library holds it until the process exits), so n*d must not exceed 1048576 floats -- larger
+ * requests fail with ABS_ENOSPACE and change nothing.  The function calls no allocator of any
+ * kind.  The first call on each device looks up the array's device address (that device must be
+ * current); make that first call outside any stream capture.  All calls on a device share the
+ * one array and it keeps the previous call's contents (each call overwrites what it reads, so
+ * nothing has to be cleared), which means two calls that may overlap on the GPU -- different
+ * streams, or different host threads -- race on it: run them on one stream or order them with
+ * events. */
+int abs_lsq_gradient_noalloc(const void* X, const float* y, const void* w, const int* idx, int n, int B,
+                             int d, int dtype, float* g_out, float* loss_out, void* stream);
+
 /* How the context runs (the paper has no counterpart): *partials = number of fp32 partial sums
  * the Eq. 3 step adds up per parameter (0: one per selected worker), *row_block = padding unit of
  * a version group's gradient rows, *rows_cap = row capacity of the activation buffers,

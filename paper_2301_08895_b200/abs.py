@@ -80,6 +80,9 @@ def lib():
         l.abs_lsq_gradient.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                        C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t,
                                        C.c_void_p, C.c_void_p, C.c_void_p]
+        l.abs_lsq_gradient_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                               C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                               C.c_void_p, C.c_void_p]
         l.abs_get_plan.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int),
                                    C.POINTER(C.c_int), C.POINTER(C.c_int)]
         l.abs_profile_start.argtypes = [C.c_void_p, C.c_int]
@@ -257,6 +260,20 @@ def lsq_gradient(X, y, w, idx, g_out, loss_out, scratch, stream=None):
     _check(lib().abs_lsq_gradient(X.data_ptr(), y.data_ptr(), w.data_ptr(), idx.data_ptr(), n, B, d,
                                   dtype, scratch.data_ptr(), scratch.numel(), g_out.data_ptr(),
                                   loss_out.data_ptr(), s.cuda_stream))
+
+
+def lsq_gradient_noalloc(X, y, w, idx, g_out, loss_out, stream=None):
+    """abs_lsq_gradient_noalloc: same operation as `lsq_gradient`, for callers that may not
+    allocate device memory; partial sums use the library's built-in 4 MiB array, so n*d must be
+    at most 1048576.  Calls sharing a device must not overlap on the GPU."""
+    import torch
+    n, B = idx.shape
+    d = X.shape[1]
+    dtype = BF16_FP32MASTER if X.dtype == torch.bfloat16 else FP32
+    s = stream if stream is not None else torch.cuda.current_stream(X.device)
+    _check(lib().abs_lsq_gradient_noalloc(X.data_ptr(), y.data_ptr(), w.data_ptr(), idx.data_ptr(),
+                                          n, B, d, dtype, g_out.data_ptr(), loss_out.data_ptr(),
+                                          s.cuda_stream))
 
 
 def trace_rows(tr):

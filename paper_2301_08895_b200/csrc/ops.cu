@@ -2,6 +2,7 @@
 // several workers at one model, and their mean (Eq. 2 with U = 1, then the sum of Eq. 3).
 #include <cstdarg>
 #include <cstdio>
+#include <mutex>
 #include <string>
 
 #include "common.cuh"
@@ -106,5 +107,53 @@ extern "C" int abs_lsq_gradient(const void* X, const float* y, const void* w, co
   if (!scratch) return op_fail(ABS_EINVAL, "scratch is null");
   if (scratch_floats < (size_t)n * d)
     return op_fail(ABS_ENOSPACE, "scratch holds %zu floats, n*d = %zu needed", scratch_floats, (size_t)n * d);
+  return run(X, y, w, idx, n, B, d, dtype, scratch, g_out, loss_out, (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Variant for callers that cannot allocate device memory.  The per-worker partial sums live in a
+// fixed array that is part of the loaded library image on every GPU (4 MiB, held until exit).
+namespace {
+
+constexpr size_t NOALLOC_MAX_FLOATS = 1u << 20;          // n * d limit of the no-allocation variant
+static __device__ __align__(256) float g_noalloc_partials[NOALLOC_MAX_FLOATS];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_noalloc_mutex;
+float* g_noalloc_ptr[MAX_DEVICES] = {};                  // device address of the array, per device
+
+// Device address of the array on the current device.  In host code the array's name is only a
+// handle; the address a kernel can use comes from cudaGetSymbolAddress, looked up once per device.
+int noalloc_scratch(float** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return op_fail(ABS_ECUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= MAX_DEVICES) return op_fail(ABS_EUNSUPPORTED, "device index %d not supported", dev);
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_ptr[dev]) {
+    float* p = nullptr;
+    e = cudaGetSymbolAddress((void**)&p, g_noalloc_partials);
+    if (e != cudaSuccess || !p)
+      return op_fail(ABS_ECUDA, "cudaGetSymbolAddress(partials): %s", cudaGetErrorString(e));
+    g_noalloc_ptr[dev] = p;
+  }
+  *out = g_noalloc_ptr[dev];
+  return ABS_OK;
+}
+
+}  // namespace
+
+extern "C" int abs_lsq_gradient_noalloc(const void* X, const float* y, const void* w, const int* idx, int n, int B,
+                                        int d, int dtype, float* g_out, float* loss_out, void* stream) {
+  const int rc = check_args(X, y, w, idx, n, B, d, dtype, g_out, loss_out);
+  if (rc != ABS_OK) return rc;
+  if ((size_t)n * (size_t)d > NOALLOC_MAX_FLOATS)
+    return op_fail(ABS_ENOSPACE, "n*d = %zu exceeds the built-in limit of %zu floats; use abs_lsq_gradient with "
+                   "caller scratch", (size_t)n * d, NOALLOC_MAX_FLOATS);
+  float* scratch = nullptr;
+  const int rs = noalloc_scratch(&scratch);
+  if (rs != ABS_OK) return rs;
+  // every partial that the reduction reads is written by the first kernel of this call, so the
+  // previous call's leftovers in the shared array never need clearing
   return run(X, y, w, idx, n, B, d, dtype, scratch, g_out, loss_out, (cudaStream_t)stream);
 }
