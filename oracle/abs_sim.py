@@ -58,24 +58,25 @@ def minibatch_indices(seed, n, j, batch, W, M):
 
 
 def tree_sum(values):
-    """Sum of binary64 numbers by adjacent pairs, level by level, after padding
-    with zeros to a power of two.  The order is part of the loss-estimate
-    definition so that a parallel implementation gets the same bits."""
-    v = [float(x) for x in values]
+    """Sum of binary32 numbers by adjacent pairs, level by level, after padding
+    with zeros to a power of two; every addition is rounded to binary32.  The
+    order and precision are part of the loss-estimate definition so that a
+    parallel implementation gets the same bits."""
+    v = [np.float32(x) for x in values]
     size = 1
     while size < len(v):
         size *= 2
-    v += [0.0] * (size - len(v))
+    v += [np.float32(0.0)] * (size - len(v))
     while len(v) > 1:
-        v = [v[2 * i] + v[2 * i + 1] for i in range(len(v) // 2)]
+        v = [np.float32(v[2 * i] + v[2 * i + 1]) for i in range(len(v) // 2)]
     return v[0]
 
 
 def loss_estimate(upload_losses):
-    """Estimate of f(w^t): mean of the uploaded binary32 losses, rounded to
-    binary32 (the stored precision of every loss that decides an integer)."""
+    """Estimate of f(w^t): mean of the uploaded binary32 losses, in binary32
+    (the stored precision of every loss that decides an integer)."""
     k = len(upload_losses)
-    return np.float32(tree_sum(upload_losses) / float(k))
+    return np.float32(tree_sum(upload_losses) / np.float32(k))
 
 
 def next_k(k_now, k0, W, l0, lt):

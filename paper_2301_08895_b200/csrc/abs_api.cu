@@ -59,8 +59,8 @@ struct Layout {
   size_t d = 0, d_pad = 0;
   size_t w_off[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the padded vector
   size_t w_src[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the caller's vector
-  size_t st, c, version, job, sel, sel_tau, sel_row0, loss, row_loss, row_idx, tile_slot;
-  size_t master, ring, G, logits;
+  size_t st, c, version, job, next_dur, dur_job, sel, sel_tau, sel_row0, loss, row_loss, row_idx, tile_slot;
+  size_t master, ring, G, logits, red;
   size_t act[ABS_MAX_LAYERS + 1], delta[ABS_MAX_LAYERS + 1];
   size_t tr_K, tr_R, tr_theta, tr_T, tr_loss, tr_comm, tr_sel_off, tr_rst_off;
   size_t tr_sel_id, tr_sel_tau, tr_sel_loss, tr_rst_id;
@@ -160,6 +160,8 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   L->c = cv.take(sizeof(u64) * W);
   L->version = cv.take(4 * W);
   L->job = cv.take(4 * W);
+  L->next_dur = cv.take(8 * W);
+  L->dur_job = cv.take(4 * W);
   L->sel = cv.take(4 * W);
   L->sel_tau = cv.take(4 * W);
   L->sel_row0 = cv.take(4 * W);
@@ -173,6 +175,12 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   if (!lsq) {
     const int C = m->dims[m->n_layers];
     L->logits = cv.take(4 * (size_t)L->rows_cap * C);
+    {
+      // chunk partials of the two-stage column reductions (bias sums, output-layer gradient)
+      size_t len = (size_t)(m->dims[m->n_layers - 1] + 1) * C;
+      for (int l = 0; l < m->n_layers; ++l) len = std::max(len, (size_t)m->dims[l + 1]);
+      L->red = cv.take(4 * len * (size_t)(L->rows_cap / 64));
+    }
     L->act[0] = (L->path[0] == PATH_TC) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     for (int l = 1; l <= m->n_layers; ++l) {
       L->act[l] = (l < m->n_layers) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]) : 0;
@@ -345,7 +353,7 @@ void enqueue_gradient(abs_ctx* ctx) {
   DevState* st = ctx->at<DevState>(L.st);
   if (m.kind == ABS_LSQ) {
     LsqArgs a;
-    a.st = st; a.sel_tau = ctx->ctl.sel_tau; a.sel_row0 = ctx->ctl.sel_row0; a.row_idx = ctx->ctl.row_idx;
+    a.st = st; a.sel = ctx->ctl.sel; a.job = ctx->ctl.job; a.sel_tau = ctx->ctl.sel_tau; a.sel_row0 = ctx->ctl.sel_row0; a.row_idx = ctx->ctl.row_idx;
     a.X = ctx->X; a.y = (const float*)ctx->y;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad;
     a.loss = ctx->ctl.loss; a.G = ctx->at<float>(L.G); a.d = m.dims[0];
@@ -405,8 +413,15 @@ void enqueue_gradient(abs_ctx* ctx) {
       launch_tc_bn(ctx, bn, ABS_KC_FWD, ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
-      const size_t sm = sizeof(float) * ((size_t)a.in * a.C + a.C);
-      launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_fwd_loss_kernel<T><<<row_tiles, 256, sm, s>>>(a); });
+      if (a.in % 8 == 0) {
+        const size_t sm = sizeof(T) * (size_t)a.in * a.C + sizeof(float) * a.C;
+        launch_k(ctx, ABS_KC_OUTPUT, [&] {
+          narrow_fwd_loss_v8_kernel<T><<<L.rows_cap / NARROW_ROWS, 256, sm, s>>>(a);
+        });
+      } else {
+        const size_t sm = sizeof(float) * ((size_t)a.in * a.C + a.C);
+        launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_fwd_loss_kernel<T><<<row_tiles, 256, sm, s>>>(a); });
+      }
     } else {
       dim3 grid((la[l].out + TN - 1) / TN, row_tiles);
       const int cls = last ? ABS_KC_OUTPUT : ABS_KC_FWD;
@@ -438,21 +453,35 @@ void enqueue_gradient(abs_ctx* ctx) {
       const int bn = L.bn_wg[l];
       launch_tc_bn(ctx, bn, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, p,
                    ((la[l].in + 127) / 128) * ((la[l].out + bn - 1) / bn) * L.P);
-      dim3 gridb((la[l].out + 31) / 32, L.P);
+      // bias gradient: per-chunk column sums, then one ordered sum over the chunks into partial 0
       const T* dl = (const T*)la[l].delta_out;
-      float* G = ctx->at<float>(L.G);
       const size_t b_off = L.w_off[l] + (size_t)la[l].in * la[l].out;
-      const int out = la[l].out, P = L.P;
-      const size_t stride = L.d_pad;
-      launch_k(ctx, ABS_KC_BIAS, [&] { colsum_kernel<T><<<gridb, 1024, 0, s>>>(st, dl, G, stride, b_off, out, P); });
+      const int out = la[l].out;
+      float* part = ctx->at<float>(L.red);
+      float* dstb = ctx->at<float>(L.G) + b_off;
+      const int per = std::min(out / 8, 256), lanes = 256 / per;
+      const size_t smb = lanes > 1 ? sizeof(float) * (size_t)lanes * out : 0;
+      launch_k(ctx, ABS_KC_BIAS, [&] { colsum_chunk_kernel<T><<<L.rows_cap / 64, 256, smb, s>>>(st, dl, out, part); });
+      launch_k(ctx, ABS_KC_BIAS, [&] { chunk_reduce_kernel<<<(out + 31) / 32, 256, 0, s>>>(st, part, out, dstb); });
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (l > 0) {
-        const size_t sm = sizeof(float) * ((size_t)a.in * a.C + 64 * a.C);
-        launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_dgrad_kernel<T><<<row_tiles, 256, sm, s>>>(a); });
+        if (a.in % 8 == 0) {
+          const size_t sm = sizeof(T) * (size_t)a.in * a.C + sizeof(float) * NARROW_ROWS * a.C;
+          launch_k(ctx, ABS_KC_OUTPUT, [&] {
+            narrow_dgrad_v8_kernel<T><<<L.rows_cap / NARROW_ROWS, 256, sm, s>>>(a);
+          });
+        } else {
+          const size_t sm = sizeof(float) * ((size_t)a.in * a.C + 64 * a.C);
+          launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_dgrad_kernel<T><<<row_tiles, 256, sm, s>>>(a); });
+        }
       }
-      dim3 gridw((a.in + 1 + 31) / 32, L.P);
-      launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_wgrad_kernel<T><<<gridw, 1024, 0, s>>>(a); });
+      // weight gradient: per-chunk partial sums, then one ordered sum over the chunks into partial 0
+      float* part = ctx->at<float>(L.red);
+      float* dstw = ctx->at<float>(L.G) + L.w_off[l];
+      const int len = (a.in + 1) * a.C;
+      launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_wgrad_chunk_kernel<T><<<L.rows_cap / 64, 256, 0, s>>>(a, part); });
+      launch_k(ctx, ABS_KC_OUTPUT, [&] { chunk_reduce_kernel<<<(len + 31) / 32, 256, 0, s>>>(st, part, len, dstw); });
     } else {
       const bool last = l == nl - 1;
       if (l > 0) {
@@ -471,8 +500,9 @@ void enqueue_update(abs_ctx* ctx) {
   UpdateArgs u;
   u.st = ctx->at<DevState>(L.st); u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
   u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
+  u.job = ctx->ctl.job; u.next_dur = ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
   const size_t n4 = L.d_pad / 4;
-  const int blocks = (int)std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * 8);
+  const int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * 8), (size_t)(ctx->W + 31) / 32);
   launch_k(ctx, ABS_KC_UPDATE, [&] { update_kernel<T><<<blocks, 256, 0, ctx->stream>>>(u); });
 }
 
@@ -587,6 +617,7 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   CtlArgs& c = ctx->ctl;
   c.st = ctx->at<DevState>(L.st);
   c.c = ctx->at<u64>(L.c); c.version = ctx->at<int>(L.version); c.job = ctx->at<int>(L.job);
+  c.next_dur = ctx->at<u64>(L.next_dur); c.dur_job = ctx->at<int>(L.dur_job);
   c.sel = ctx->at<int>(L.sel); c.sel_tau = ctx->at<int>(L.sel_tau); c.sel_row0 = ctx->at<int>(L.sel_row0);
   c.loss = ctx->at<float>(L.loss);
   c.row_loss = model->kind == ABS_LSQ ? nullptr : ctx->at<float>(L.row_loss);
@@ -605,7 +636,7 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);
-  abs_init_state_kernel<<<(W + 255) / 256, 256, 0, s>>>(c);
+  abs_init_state_kernel<<<(W + 31) / 32, 32, 0, s>>>(c);
   if (model->dtype == ABS_FP32) ring_init_kernel<float><<<148, 256, 0, s>>>(ctx->at<float>(L.master), ctx->at<void>(L.ring), L.d_pad);
   else ring_init_kernel<__nv_bfloat16><<<148, 256, 0, s>>>(ctx->at<float>(L.master), ctx->at<void>(L.ring), L.d_pad);
   ctx->launches += 2;

@@ -69,11 +69,18 @@ struct CtlArgs {
   float* row_loss;     // [rows_cap] per-sample losses (network models), else null
   int* row_idx;        // [rows_cap] sample index of each gradient row, -1 for padding
   int* tile_slot;      // [rows_cap / RB] ring slot of each row tile
+  u64* next_dur;       // [W] duration of the job each worker starts next, computed ahead of time
+  int* dur_job;        // [W] job index next_dur[n] belongs to
   // trace
   int* tr_K; int* tr_R; int* tr_theta; u64* tr_T; float* tr_loss; u64* tr_comm;
   i64* tr_sel_off; i64* tr_rst_off;
   int* tr_sel_id; int* tr_sel_tau; float* tr_sel_loss; int* tr_rst_id;
 };
+
+__device__ __forceinline__ float ldf(const float* p, size_t i) { return p[i]; }
+__device__ __forceinline__ float ldf(const __nv_bfloat16* p, size_t i) { return __bfloat162float(p[i]); }
+__device__ __forceinline__ void stf(float* p, size_t i, float v) { p[i] = v; }
+__device__ __forceinline__ void stf(__nv_bfloat16* p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
 
 __host__ __device__ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 __host__ __device__ inline size_t round_up_sz(size_t a, size_t b) { return (a + b - 1) / b * b; }

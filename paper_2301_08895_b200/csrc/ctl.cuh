@@ -60,27 +60,44 @@ __device__ __forceinline__ u64 job_ticks(const TimeDist& d, uint32_t k0, uint32_
   return ticks < 1ull ? 1ull : ticks;
 }
 
+// The double-precision pipe of one SM is narrow, so the control CTA does not compute durations
+// itself: the duration of the job a worker will start NEXT depends only on (worker, job index)
+// and is prepared ahead of time by one warp of each of the first ceil(N/32) CTAs of a wide
+// kernel that runs between two control kernels.  Only workers whose job index moved are redone.
+__device__ __forceinline__ void refresh_next_durations(const DevState* st, const int* job, u64* next_dur,
+                                                       int* dur_job, int n) {
+  if (n >= st->W) return;
+  const int j = job[n] + 1;
+  if (dur_job[n] != j) {
+    next_dur[n] = job_ticks(st->dist, st->key0, st->key1, n, j);
+    dur_job[n] = j;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Bitonic sort of 1024 64-bit keys, one per thread, ascending by thread index.
 // Exchange distances below 32 use shuffles, the others go through shared memory.
 __device__ __forceinline__ u64 bitonic_sort_1024(u64 key, u64* smem, int n_pow2) {
   const int tid = threadIdx.x;
+  const bool active = tid < n_pow2;          // whole warps: n_pow2 is a multiple of 32
   for (int k = 2; k <= n_pow2; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
-      u64 other;
+      u64 other = key;
       if (j >= 32) {
-        smem[tid] = key;
+        if (active) smem[tid] = key;
         __syncthreads();
-        other = smem[tid ^ j];
+        if (active) other = smem[tid ^ j];
         __syncthreads();
-      } else {
+      } else if (active) {
         other = __shfl_xor_sync(0xffffffffu, key, j);
       }
-      const bool up = ((tid & k) == 0);
-      const bool lower = ((tid & j) == 0);
-      const u64 mn = key < other ? key : other;
-      const u64 mx = key < other ? other : key;
-      key = (lower == up) ? mn : mx;
+      if (active) {
+        const bool up = ((tid & k) == 0);
+        const bool lower = ((tid & j) == 0);
+        const u64 mn = key < other ? key : other;
+        const u64 mx = key < other ? other : key;
+        key = (lower == up) ? mn : mx;
+      }
     }
   }
   return key;
@@ -94,12 +111,16 @@ __device__ __forceinline__ i64 floor_div(i64 a, i64 b) {  // b > 0
 
 struct CtlShared {
   u64 keys[1024];
-  double red[32];
+  float redf[32];
   unsigned short wcnt[32][MAX_TAU];   // per-warp count of selected workers per staleness
   int cnt[MAX_TAU];                    // selected workers per staleness
   int grow0[MAX_TAU];                  // first row of each staleness group
   unsigned char flag[1024];            // selected marker per worker id
+  int cnt_or_row0[1024];               // first gradient row of each selected worker
+  float lossv[1024];                   // mean minibatch loss of each selected worker
   int warp_tot[32];
+  int shard_lo[1024];
+  unsigned shard_len[1024];
   int scalar[8];
 };
 
@@ -123,61 +144,70 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     const u64 T_end = st->T_end;
     // per-worker mean loss of network models: fixed-order sum of the per-sample losses
     if (a.row_loss != nullptr) {
+      if (tid < K) sh.cnt_or_row0[tid] = a.sel_row0[tid];
+      __syncthreads();
+#pragma unroll 4
       for (int i = warp; i < K; i += 32) {
-        const int r0 = a.sel_row0[i];
+        const int r0 = sh.cnt_or_row0[i];
         float acc = 0.f;
         for (int b = lane; b < B; b += 32) acc += a.row_loss[r0 + b];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == 0) a.loss[i] = __fdiv_rn(acc, (float)B);
+        if (lane == 0) sh.lossv[i] = __fdiv_rn(acc, (float)B);
       }
       __syncthreads();
+    } else if (tid < K) {
+      sh.lossv[tid] = a.loss[tid];
     }
-    const float my_loss = (tid < K) ? a.loss[tid] : 0.f;
+    if (a.row_loss == nullptr) __syncthreads();
+    const float my_loss = (tid < K) ? sh.lossv[tid] : 0.f;
     const int bad = __syncthreads_or((tid < K) && !isfinite(my_loss)) || st->diverged;
     if (bad) {
       if (tid == 0) { st->status = ST_DIVERGED; st->open = 0; }
       return;
     }
-    // loss estimate: adjacent-pair tree sum in binary64 over 1024 leaves, /K, rounded to binary32
-    double v = (double)my_loss;
+    // loss estimate: adjacent-pair tree sum in binary32 over 1024 leaves, /K in binary32
+    float v = my_loss;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) v = __dadd_rn(v, __shfl_down_sync(0xffffffffu, v, o));
-    if (lane == 0) sh.red[warp] = v;
+    for (int o = 1; o < 32; o <<= 1) v = __fadd_rn(v, __shfl_down_sync(0xffffffffu, v, o));
+    if (lane == 0) sh.redf[warp] = v;
     sh.flag[tid] = 0;
     __syncthreads();
     if (warp == 0) {
-      double x = sh.red[lane];
+      float x = sh.redf[lane];
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) x = __dadd_rn(x, __shfl_down_sync(0xffffffffu, x, o));
-      if (lane == 0) sh.red[0] = x;
+      for (int o = 1; o < 32; o <<= 1) x = __fadd_rn(x, __shfl_down_sync(0xffffffffu, x, o));
+      if (lane == 0) {
+        const float Lt0 = __fdiv_rn(x, (float)K);
+        const float L00 = (t == 0) ? Lt0 : st->L0;
+        // Eq. 5 as an exact integer rule: largest k with k^2 Lt <= K0^2 L0 (binary64 products of a
+        // 20-bit integer and a binary32 value are exact).  A binary32 estimate of K0 sqrt(L0/Lt)
+        // is corrected with the exact test, so only a handful of double operations are issued.
+        int kr = 0;
+        if (st->k_mode == ABS_K_ADAPTIVE) {
+          if (Lt0 <= 0.f) {
+            kr = W;
+          } else {
+            const double rhs = __dmul_rn((double)(st->K0 * st->K0), (double)L00);
+            const double lt = (double)Lt0;
+            const float est = (float)st->K0 * sqrtf(L00 / Lt0);
+            int k = (est >= (float)W) ? W : ((est >= 1.f) ? (int)est : 1);
+            while (k < W && __dmul_rn((double)((k + 1) * (k + 1)), lt) <= rhs) ++k;
+            while (k >= 1 && !(__dmul_rn((double)(k * k), lt) <= rhs)) --k;
+            kr = k;
+          }
+        }
+        sh.redf[0] = Lt0;
+        sh.redf[1] = L00;
+        sh.scalar[2] = kr;
+      }
     }
     if (tid < K) sh.flag[a.sel[tid]] = 1;
     __syncthreads();
-    const float Lt = __double2float_rn(__ddiv_rn(sh.red[0], (double)K));
-    const float L0 = (t == 0) ? Lt : st->L0;
-    // Eq. 5 as an exact integer rule: largest k with k^2 Lt <= K0^2 L0
+    const float Lt = sh.redf[0];
+    const float L0 = sh.redf[1];
     int K_next = K;
-    if (st->k_mode == ABS_K_ADAPTIVE) {
-      int ok = 0;
-      if (Lt <= 0.f) {
-        ok = (tid == 0) ? W : 0;
-      } else if (tid < W) {
-        const int k = tid + 1;
-        const double lhs = __dmul_rn((double)(k * k), (double)Lt);
-        const double rhs = __dmul_rn((double)(st->K0 * st->K0), (double)L0);
-        ok = (lhs <= rhs) ? k : 0;
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ok = max(ok, __shfl_xor_sync(0xffffffffu, ok, o));
-      if (lane == 0) sh.warp_tot[warp] = ok;
-      __syncthreads();
-      int kr = sh.warp_tot[lane];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) kr = max(kr, __shfl_xor_sync(0xffffffffu, kr, o));
-      K_next = min(W, max(K, kr));
-      __syncthreads();
-    }
+    if (st->k_mode == ABS_K_ADAPTIVE) K_next = min(W, max(K, sh.scalar[2]));
     // Eq. 4 with a = S - N/K0, in integers
     int theta = S;
     if (st->bound_mode == ABS_BOUND_ADAPTIVE) {
@@ -197,7 +227,7 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     int range_err = 0;
     if (renew) {
       const int j = a.job[tid] + 1;
-      const u64 dt = job_ticks(st->dist, st->key0, st->key1, tid, j);
+      const u64 dt = (a.dur_job[tid] == j) ? a.next_dur[tid] : job_ticks(st->dist, st->key0, st->key1, tid, j);
       const u64 cn = T_end + dt;
       if (dt == 0ull || cn >= (1ull << 53)) range_err = 1;
       a.job[tid] = j;
@@ -290,28 +320,49 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
       a.sel_row0[tid] = row0;
       sh.keys[tid] = ((u64)(unsigned)row0 << 32) | (u64)(unsigned)n;   // reuse as (row0, n)
     }
-    // ring slot of every row tile, and padding rows
-    if (tid <= S && sh.cnt[tid] > 0) {
-      const int slot = (t - tid) % (S + 1);
-      const int r0 = sh.grow0[tid], r1 = r0 + round_up(sh.cnt[tid] * B, RB);
-      for (int r = r0; r < r1; r += RB) a.tile_slot[r / RB] = slot;
-      for (int r = r0 + sh.cnt[tid] * B; r < r1; ++r) a.row_idx[r] = -1;
+    // ring slot of every row tile and padding rows, all threads; least squares reads neither
+    if (a.row_loss != nullptr) {
+      const int n_tiles = n_rows / RB;
+      for (int q = tid; q < n_tiles; q += 1024) {
+        const int r = q * RB;
+        int g = 0;                                  // last non-empty group starting at or before r
+        for (int u = 0; u <= S; ++u) if (sh.cnt[u] > 0 && sh.grow0[u] <= r) g = u;
+        a.tile_slot[q] = (t - g) % (S + 1);
+      }
+      for (int g = 0; g <= S; ++g) {
+        const int c = sh.cnt[g];
+        if (c == 0) continue;
+        const int p0 = sh.grow0[g] + c * B, p1 = sh.grow0[g] + round_up(c * B, RB);
+        for (int r = p0 + tid; r < p1; r += 1024) a.row_idx[r] = -1;
+      }
     }
     __syncthreads();
     // minibatch draws: sample b of job (n, j) = word b%4 of Philox block (n, j, 1, b/4),
-    // mapped into the worker's shard [n M / N, (n+1) M / N)
-    const int blocks_per = (B + 3) >> 2;
-    const i64 M = st->n_samples;
-    for (int item = tid; item < K * blocks_per; item += 1024) {
-      const int i = item / blocks_per, blk = item - i * blocks_per;
-      const int wn = (int)(sh.keys[i] & 0xffffffffull), row0 = (int)(sh.keys[i] >> 32);
-      const i64 lo = ((i64)wn * M) / W, hi = ((i64)(wn + 1) * M) / W;
-      uint32_t w4[4];
-      philox4x32_10((uint32_t)wn, (uint32_t)a.job[wn], 1u, (uint32_t)blk, st->key0, st->key1, w4);
+    // mapped into the worker's shard [n M / N, (n+1) M / N).  Least squares draws them in its
+    // own gradient kernel (one CTA per worker), so the control CTA skips them.
+    if (a.row_loss != nullptr) {
+      const int blocks_per = (B + 3) >> 2;
+      const i64 M = st->n_samples;
+      if (tid < K) {
+        const int wn = (int)(sh.keys[tid] & 0xffffffffull);
+        const i64 lo = ((i64)wn * M) / W, hi = ((i64)(wn + 1) * M) / W;
+        sh.shard_lo[tid] = (int)lo;
+        sh.shard_len[tid] = (unsigned)(hi - lo);
+        sh.cnt_or_row0[tid] = a.job[wn];
+      }
+      __syncthreads();
+      for (int item = tid; item < K * blocks_per; item += 1024) {
+        const int i = item / blocks_per, blk = item - i * blocks_per;
+        const int wn = (int)(sh.keys[i] & 0xffffffffull), row0 = (int)(sh.keys[i] >> 32);
+        uint32_t w4[4];
+        philox4x32_10((uint32_t)wn, (uint32_t)sh.cnt_or_row0[i], 1u, (uint32_t)blk, st->key0, st->key1, w4);
+        const int lo = sh.shard_lo[i];
+        const u64 len = (u64)sh.shard_len[i];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int b = blk * 4 + q;
-        if (b < B) a.row_idx[row0 + b] = (int)(lo + (i64)(((u64)w4[q] * (u64)(hi - lo)) >> 32));
+        for (int q = 0; q < 4; ++q) {
+          const int b = blk * 4 + q;
+          if (b < B) a.row_idx[row0 + b] = lo + (int)(((u64)w4[q] * len) >> 32);
+        }
       }
     }
     if (tid == 0) {
@@ -335,6 +386,8 @@ __global__ void abs_init_state_kernel(CtlArgs a) {
     a.c[tid] = dt;
     a.version[tid] = 0;
     a.job[tid] = 0;
+    a.next_dur[tid] = job_ticks(st->dist, st->key0, st->key1, tid, 1);
+    a.dur_job[tid] = 1;
   }
 }
 

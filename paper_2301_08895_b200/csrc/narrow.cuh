@@ -219,4 +219,305 @@ __global__ void __launch_bounds__(1024) narrow_wgrad_kernel(NarrowArgs a) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Vectorised variants (feature counts that are multiples of 8): 16-byte loads, weights kept in
+// shared memory transposed ([class][feature], storage type) so that a lane's 8 consecutive
+// features of one class are one conflict-free 16-byte read.
+
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 u = *reinterpret_cast<const uint4*>(p);
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) { const float2 f = __bfloat1622float2(h[j]); v[2 * j] = f.x; v[2 * j + 1] = f.y; }
+}
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+  const float4 a = reinterpret_cast<const float4*>(p)[0], b = reinterpret_cast<const float4*>(p)[1];
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8]) {
+  uint4 u;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) h[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+  *reinterpret_cast<uint4*>(p) = u;
+}
+__device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
+  reinterpret_cast<float4*>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
+  reinterpret_cast<float4*>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+
+constexpr int NARROW_ROWS = 16;   // rows per block of the vectorised forward / dgrad kernels
+
+// Output layer forward + soft-max cross-entropy + delta, 16 rows per block, one warp per row pair.
+template <typename T>
+__global__ void __launch_bounds__(256) narrow_fwd_loss_v8_kernel(NarrowArgs a) {
+  extern __shared__ __align__(16) unsigned char nsm_raw[];
+  T* wT = reinterpret_cast<T*>(nsm_raw);                 // [C][in]
+  DevState* st = a.st;
+  if (st->status != ST_OK) return;
+  const int r0 = blockIdx.x * NARROW_ROWS;
+  if (r0 >= st->n_rows) return;
+  const int in = a.in, C = a.C;
+  float* bias = reinterpret_cast<float*>(wT + (size_t)C * in);
+  const int slot = a.tile_slot[r0 / st->RB];
+  const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
+#pragma unroll 8
+  for (int i = threadIdx.x; i < in * C; i += 256) {
+    const int k = i / C, c = i - k * C;
+    wT[(size_t)c * in + k] = Wm[i];
+  }
+  if (threadIdx.x < C) bias[threadIdx.x] = ldf(Wm, (size_t)in * C + threadIdx.x);
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const T* src = (const T*)a.act_in;
+  const int nvec = in >> 3;
+  bool bad = false;
+  for (int rr = warp; rr < NARROW_ROWS; rr += 8) {
+    const int r = r0 + rr;
+    const int s = a.row_idx[r];
+    T* d = (T*)a.delta_out + (size_t)r * C;
+    if (s < 0) {
+      if (lane < C) stf(d, lane, 0.f);
+      if (lane == 0) a.row_loss[r] = 0.f;
+      continue;
+    }
+    const T* x = a.gather ? src + (size_t)s * in : src + (size_t)r * in;
+    float acc[NARROW_MAX_C];
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c) acc[c] = 0.f;
+#pragma unroll 2
+    for (int v = lane; v < nvec; v += 32) {
+      float xv[8];
+      load8(x + v * 8, xv);
+#pragma unroll
+      for (int c = 0; c < NARROW_MAX_C; ++c)
+        if (c < C) {
+          float wv[8];
+          load8(wT + (size_t)c * in + v * 8, wv);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[c] = fmaf(xv[j], wv[j], acc[c]);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+        acc[c] += bias[c];
+      }
+    const int y = a.labels[s];
+    float zmax = acc[0], zy = 0.f;
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) { zmax = fmaxf(zmax, acc[c]); if (c == y) zy = acc[c]; }
+    float se = 0.f;
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) { acc[c] = expf(acc[c] - zmax); se += acc[c]; }
+    const float inv = 1.f / se;
+    float mine = 0.f;
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c == lane) mine = acc[c] * inv - (c == y ? 1.f : 0.f);
+    if (lane < C) stf(d, lane, mine);
+    const float loss = logf(se) - (zy - zmax);
+    if (lane == 0) a.row_loss[r] = loss;
+    bad |= !isfinite(loss);
+  }
+  if (bad && lane == 0) st->diverged = 1;
+}
+
+// Back-propagation through the output layer and the ReLU before it, 16 rows per block; a work
+// item is (row, 8 consecutive features).
+template <typename T>
+__global__ void __launch_bounds__(256) narrow_dgrad_v8_kernel(NarrowArgs a) {
+  extern __shared__ __align__(16) unsigned char nsm_raw[];
+  T* wT = reinterpret_cast<T*>(nsm_raw);                 // [C][in]
+  DevState* st = a.st;
+  if (st->status != ST_OK) return;
+  const int r0 = blockIdx.x * NARROW_ROWS;
+  if (r0 >= st->n_rows) return;
+  const int in = a.in, C = a.C;
+  float* dsm = reinterpret_cast<float*>(wT + (size_t)C * in);   // [16][C]
+  const int slot = a.tile_slot[r0 / st->RB];
+  const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
+#pragma unroll 8
+  for (int i = threadIdx.x; i < in * C; i += 256) {
+    const int k = i / C, c = i - k * C;
+    wT[(size_t)c * in + k] = Wm[i];
+  }
+  const T* dl = (const T*)a.delta_out + (size_t)r0 * C;
+  for (int i = threadIdx.x; i < NARROW_ROWS * C; i += 256) dsm[i] = ldf(dl, i);
+  __syncthreads();
+  const T* h = (const T*)a.act_in;
+  T* out = (T*)a.delta_in;
+  const int nvec = in >> 3;
+  for (int item = threadIdx.x; item < NARROW_ROWS * nvec; item += 256) {
+    const int rr = item / nvec, v = item - rr * nvec;
+    const size_t o = (size_t)(r0 + rr) * in + (size_t)v * 8;
+    float hv[8], acc[8];
+    load8(h + o, hv);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) {
+        float wv[8];
+        load8(wT + (size_t)c * in + v * 8, wv);
+        const float dv = dsm[rr * C + c];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = fmaf(dv, wv[j], acc[j]);
+      }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = hv[j] > 0.f ? acc[j] : 0.f;
+    store8(out + o, acc);
+  }
+}
+
+__device__ __forceinline__ void load2(const __nv_bfloat16* p, float& x, float& y) {
+  const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+  x = f.x; y = f.y;
+}
+__device__ __forceinline__ void load2(const float* p, float& x, float& y) {
+  const float2 f = *reinterpret_cast<const float2*>(p);
+  x = f.x; y = f.y;
+}
+
+// Stage 1 of the output layer's weight gradient: per 64-row chunk q,
+// part[q][m][c] = sum_{r in chunk} act_in[r][m] delta_out[r][c], with row m = `in` the bias sums.
+// A thread owns two neighbouring features (one 4/8-byte load per row), rows are fetched eight
+// at a time so the loads overlap.  Padding rows have zero deltas, so whatever finite input they
+// point at adds nothing.
+template <typename T>
+__global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, float* part) {
+  __shared__ float dsm[64][NARROW_MAX_C];
+  __shared__ long long rowoff[64];
+  DevState* st = a.st;
+  if (st->status != ST_OK) return;
+  const int r0 = blockIdx.x * 64;
+  if (r0 >= st->n_rows) return;
+  const int in = a.in, C = a.C;
+  const T* dl = (const T*)a.delta_out + (size_t)r0 * C;
+  for (int i = threadIdx.x; i < 64 * C; i += 256) dsm[i / C][i % C] = ldf(dl, i);
+  if (threadIdx.x < 64) {
+    const int r = r0 + threadIdx.x;
+    long long off = (long long)r * in;
+    if (a.gather) { const int s = a.row_idx[r]; off = s < 0 ? 0 : (long long)s * in; }
+    rowoff[threadIdx.x] = off;
+  }
+  __syncthreads();
+  const T* src = (const T*)a.act_in;
+  float* dst = part + (size_t)blockIdx.x * (size_t)(in + 1) * C;
+  const bool pairs = (in & 1) == 0;
+  const int n_items = pairs ? in / 2 : in;
+  for (int it = threadIdx.x; it < n_items; it += 256) {
+    const int m = pairs ? 2 * it : it;
+    float acc0[NARROW_MAX_C], acc1[NARROW_MAX_C];
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c) { acc0[c] = 0.f; acc1[c] = 0.f; }
+    for (int rb = 0; rb < 64; rb += 8) {
+      float x0[8], x1[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const T* px = src + (size_t)rowoff[rb + j] + m;
+        if (pairs) load2(px, x0[j], x1[j]);
+        else { x0[j] = ldf(px, 0); x1[j] = 0.f; }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int c = 0; c < NARROW_MAX_C; ++c)
+          if (c < C) {
+            const float dv = dsm[rb + j][c];
+            acc0[c] = fmaf(x0[j], dv, acc0[c]);
+            acc1[c] = fmaf(x1[j], dv, acc1[c]);
+          }
+    }
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) {
+        dst[(size_t)m * C + c] = acc0[c];
+        if (pairs) dst[(size_t)(m + 1) * C + c] = acc1[c];
+      }
+  }
+  if (threadIdx.x < C) {                       // bias row: column sums of the deltas
+    float tot = 0.f;
+    for (int rr = 0; rr < 64; ++rr) tot += dsm[rr][threadIdx.x];
+    dst[(size_t)in * C + threadIdx.x] = tot;
+  }
+}
+
+// Stage 1 of a hidden layer's bias gradient: part[q][n] = sum over the 64 rows of chunk q of
+// delta[r][n]; `out` a multiple of 8.
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_chunk_kernel(const DevState* st, const T* delta, int out, float* part) {
+  extern __shared__ __align__(16) unsigned char nsm_raw[];
+  float* red = reinterpret_cast<float*>(nsm_raw);        // [row lanes][out]
+  if (st->status != ST_OK) return;
+  const int r0 = blockIdx.x * 64;
+  if (r0 >= st->n_rows) return;
+  const int nvec = out >> 3;
+  const int per = min(nvec, 256);                         // threads along a row
+  const int lanes = 256 / per;                            // rows worked on side by side
+  for (int v0 = 0; v0 < nvec; v0 += 256) {
+    const int v = v0 + (int)threadIdx.x % per;
+    const int rl = (int)threadIdx.x / per;
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    const bool active = rl < lanes && v < nvec;
+    if (active)
+      for (int rr = rl; rr < 64; rr += lanes) {
+        float dv[8];
+        load8(delta + (size_t)(r0 + rr) * out + (size_t)v * 8, dv);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] += dv[j];
+      }
+    if (lanes == 1) {
+      if (active) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) part[(size_t)blockIdx.x * out + v * 8 + j] = acc[j];
+      }
+      continue;
+    }
+    if (active) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) red[(size_t)rl * out + v * 8 + j] = acc[j];
+    }
+    __syncthreads();
+    if (active && rl == 0) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float tot = 0.f;
+        for (int q = 0; q < lanes; ++q) tot += red[(size_t)q * out + v * 8 + j];
+        part[(size_t)blockIdx.x * out + v * 8 + j] = tot;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// Stage 2: dst[i] = sum over the active chunks q of part[q][i], i < len.  Block = 32 outputs x 8
+// chunk lanes; lane w adds chunks w, w+8, ... in order, then the 8 lanes are added in order.
+__global__ void __launch_bounds__(256) chunk_reduce_kernel(const DevState* st, const float* part, int len, float* dst) {
+  __shared__ float red[8][33];
+  if (st->status != ST_OK) return;
+  const int n_chunks = st->n_rows / 64;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int i = blockIdx.x * 32 + lane;
+  float acc = 0.f;
+  if (i < len) {
+#pragma unroll 8
+    for (int q = w; q < n_chunks; q += 8) acc += part[(size_t)q * len + i];
+  }
+  red[w][lane] = acc;
+  __syncthreads();
+  if (w == 0 && i < len) {
+    float tot = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) tot += red[q][lane];
+    dst[i] = tot;
+  }
+}
+
 }  // namespace absb

@@ -6,7 +6,6 @@
 #include <string>
 
 #include "common.cuh"
-#include "simt.cuh"
 
 using namespace absb;
 

@@ -5,13 +5,10 @@
 // reduced over all gradient rows of the round and never stored per worker.
 #pragma once
 #include "common.cuh"
+#include "ctl.cuh"
 
 namespace absb {
 
-__device__ __forceinline__ float ldf(const float* p, size_t i) { return p[i]; }
-__device__ __forceinline__ float ldf(const __nv_bfloat16* p, size_t i) { return __bfloat162float(p[i]); }
-__device__ __forceinline__ void stf(float* p, size_t i, float v) { p[i] = v; }
-__device__ __forceinline__ void stf(__nv_bfloat16* p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
 
 constexpr int TM = 64, TN = 64, TK = 16;
 
@@ -236,6 +233,7 @@ __global__ void __launch_bounds__(256) net_loss_kernel(LossArgs a) {
 
 struct LsqArgs {
   DevState* st;
+  const int* sel; const int* job;
   const int* sel_tau; const int* sel_row0; const int* row_idx;
   const void* X; const float* y;
   const void* ring; size_t slot_stride;
@@ -260,8 +258,21 @@ __global__ void __launch_bounds__(256) lsq_grad_kernel(LsqArgs a) {
   const int slot = (st->t - a.sel_tau[i]) % (st->S + 1);
   const T* w = (const T*)a.ring + (size_t)slot * a.slot_stride;
   const T* X = (const T*)a.X;
-  const int row0 = a.sel_row0[i];
-  for (int b = tid; b < B; b += 256) sidx[b] = a.row_idx[row0 + b];
+  {
+    // minibatch of the worker's job in flight: draw b = word b%4 of Philox block (n, j, 1, b/4),
+    // mapped into the worker's shard [n M / N, (n+1) M / N)
+    const int wn = a.sel[i], j = a.job[wn], W = st->W;
+    const i64 M = st->n_samples;
+    const i64 lo = ((i64)wn * M) / W, hi = ((i64)(wn + 1) * M) / W;
+    const u64 len = (u64)(hi - lo);
+    for (int blk = tid; blk < ((B + 3) >> 2); blk += 256) {
+      uint32_t w4[4];
+      philox4x32_10((uint32_t)wn, (uint32_t)j, 1u, (uint32_t)blk, st->key0, st->key1, w4);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (blk * 4 + q < B) sidx[blk * 4 + q] = (int)lo + (int)(((u64)w4[q] * len) >> 32);
+    }
+  }
   __syncthreads();
   for (int b = warp; b < B; b += 8) {
     const T* x = X + (size_t)sidx[b] * d;
@@ -295,6 +306,7 @@ __global__ void __launch_bounds__(256) lsq_grad_kernel(LsqArgs a) {
 
 struct UpdateArgs {
   const DevState* st;
+  const int* job; u64* next_dur; int* dur_job;   // duration look-ahead (see refresh_next_durations)
   float* master;          // [d_pad]
   void* ring;             // [S+1][d_pad] storage type
   const float* G;         // [P][d_pad]
@@ -308,7 +320,9 @@ struct UpdateArgs {
 template <typename T>
 __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
   const DevState* st = a.st;
-  if (st->status != ST_OK || st->diverged) return;
+  if (st->status != ST_OK) return;
+  if (threadIdx.x < 32) refresh_next_durations(st, a.job, a.next_dur, a.dur_job, blockIdx.x * 32 + threadIdx.x);
+  if (st->diverged) return;
   const int K = st->K;
   const int P = a.P > 0 ? a.P : K;
   const float step = __fdiv_rn(a.lr, (float)(K * st->B));

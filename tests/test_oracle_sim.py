@@ -198,15 +198,19 @@ def test_theta_table():
 
 
 def test_loss_estimate_order_and_rounding():
+    f = np.float32
     assert abs_sim.tree_sum([1.0, 2.0, 3.0]) == 6.0
-    # ((a+b)+(c+0)): with a = 1, b = 2^-53, c = 2^-53 the pairs decide the bits
-    a, b = 1.0, 2.0 ** -53
-    assert abs_sim.tree_sum([a, b, b]) == (a + b) + (b + 0.0) == 1.0
-    assert abs_sim.tree_sum([b, b, a]) == (b + b) + (a + 0.0) == 1.0 + 2.0 ** -52
-    vals = [np.float32(x) for x in (0.1, 0.2, 0.3, 0.4, 0.5)]
+    # ((a+b)+(c+0)) in binary32: with a = 1, b = c = 2^-24 the pairing decides the bits
+    a, b = f(1.0), f(2.0 ** -24)
+    assert abs_sim.tree_sum([a, b, b]) == f(f(a + b) + f(b + f(0))) == f(1.0)
+    assert abs_sim.tree_sum([b, b, a]) == f(f(b + b) + f(a + f(0))) == f(1.0 + 2.0 ** -23)
+    vals = [f(x) for x in (0.1, 0.2, 0.3, 0.4, 0.5)]
     est = abs_sim.loss_estimate(vals)
     assert isinstance(est, np.float32)
     assert abs(float(est) - 0.3) < 1e-7
+    # every intermediate is a binary32 value: a sum that binary64 would keep exact gets rounded
+    assert abs_sim.tree_sum([f(16777216.0), f(1.0)]) == f(16777216.0)
+    assert float(abs_sim.loss_estimate([f(1.0), f(2.0)])) == 1.5
 
 
 # ---------------------------------------------------------- whole-run behaviour
