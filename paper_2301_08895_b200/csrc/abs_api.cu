@@ -634,6 +634,11 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
       ctx->sm_count = sms;
   }
+  {
+    const cudaError_t ea = cudaFuncSetAttribute(abs_ctl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)sizeof(CtlShared));
+    if (ea != cudaSuccess) return bail(cuda_fail(nullptr, ea, "cudaFuncSetAttribute(abs_ctl_kernel)"));
+  }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);
   abs_init_state_kernel<<<(W + 31) / 32, 32, 0, s>>>(c);
@@ -661,12 +666,12 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
   const bool f32 = ctx->m.dtype == ABS_FP32;
   for (int r = 0; r < n; ++r) {
     // the control kernel completes the previous round (if any) and selects this round's arrivals
-    launch_k(ctx, ABS_KC_CTL, [&] { abs_ctl_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->ctl, 1, 1); });
+    launch_k(ctx, ABS_KC_CTL, [&] { abs_ctl_kernel<<<1, 1024, sizeof(CtlShared), ctx->stream>>>(ctx->ctl, 1, 1); });
     if (f32) { enqueue_gradient<float>(ctx); enqueue_update<float>(ctx); }
     else { enqueue_gradient<__nv_bfloat16>(ctx); enqueue_update<__nv_bfloat16>(ctx); }
   }
   if (n > 0) {
-    launch_k(ctx, ABS_KC_CTL, [&] { abs_ctl_kernel<<<1, 1024, 0, ctx->stream>>>(ctx->ctl, 1, 0); });
+    launch_k(ctx, ABS_KC_CTL, [&] { abs_ctl_kernel<<<1, 1024, sizeof(CtlShared), ctx->stream>>>(ctx->ctl, 1, 0); });
   }
   CU(cudaGetLastError());
   ctx->rounds_enqueued += n;

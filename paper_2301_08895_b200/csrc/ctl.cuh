@@ -75,32 +75,41 @@ __device__ __forceinline__ void refresh_next_durations(const DevState* st, const
 }
 
 // ---------------------------------------------------------------------------------------------
-// Bitonic sort of 1024 64-bit keys, one per thread, ascending by thread index.
-// Exchange distances below 32 use shuffles, the others go through shared memory.
-__device__ __forceinline__ u64 bitonic_sort_1024(u64 key, u64* smem, int n_pow2) {
-  const int tid = threadIdx.x;
-  const bool active = tid < n_pow2;          // whole warps: n_pow2 is a multiple of 32
-  for (int k = 2; k <= n_pow2; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      u64 other = key;
-      if (j >= 32) {
-        if (active) smem[tid] = key;
-        __syncthreads();
-        if (active) other = smem[tid ^ j];
-        __syncthreads();
-      } else if (active) {
-        other = __shfl_xor_sync(0xffffffffu, key, j);
-      }
-      if (active) {
-        const bool up = ((tid & k) == 0);
-        const bool lower = ((tid & j) == 0);
-        const u64 mn = key < other ? key : other;
-        const u64 mx = key < other ? other : key;
-        key = (lower == up) ? mn : mx;
-      }
-    }
+// Sort of up to 1024 distinct 64-bit keys, one per thread, by ranking: inside a warp every key
+// counts the smaller keys of its warp (31 shuffles, no dependent chain); sorted runs are then
+// merged pairwise, each key finding its place in the sibling run by binary search.  All steps
+// are short and independent per thread, which matters because one CTA does this alone.
+// Returns the buffer (A or B) that holds the sorted keys.
+__device__ __forceinline__ u64* rank_merge_sort(u64 key, u64* A, u64* B, int n_pow2) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const bool active = tid < n_pow2;            // whole warps: n_pow2 is a multiple of 32
+  if (active) {
+    int rank = 0;
+#pragma unroll
+    for (int l = 0; l < 32; ++l) rank += (__shfl_sync(0xffffffffu, key, l) < key) ? 1 : 0;
+    A[(tid - lane) + rank] = key;
   }
-  return key;
+  __syncthreads();
+  u64* src = A;
+  u64* dst = B;
+  for (int L = 32; L < n_pow2; L <<= 1) {
+    if (active) {
+      const u64 k = src[tid];
+      const int pair_base = tid & ~(2 * L - 1);
+      const int idx = tid - pair_base;
+      const int own = idx & (L - 1);
+      const u64* other = src + pair_base + ((idx < L) ? L : 0);
+      int lo = 0, hi = L;
+      while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (other[mid] < k) lo = mid + 1; else hi = mid;
+      }
+      dst[pair_base + own + lo] = k;
+    }
+    __syncthreads();
+    u64* tmp = src; src = dst; dst = tmp;
+  }
+  return src;
 }
 
 __device__ __forceinline__ i64 floor_div(i64 a, i64 b) {  // b > 0
@@ -110,17 +119,18 @@ __device__ __forceinline__ i64 floor_div(i64 a, i64 b) {  // b > 0
 }
 
 struct CtlShared {
-  u64 keys[1024];
-  float redf[32];
+  u64 keysA[1024], keysB[1024];
   unsigned short wcnt[32][MAX_TAU];   // per-warp count of selected workers per staleness
   int cnt[MAX_TAU];                    // selected workers per staleness
   int grow0[MAX_TAU];                  // first row of each staleness group
   unsigned char flag[1024];            // selected marker per worker id
-  int cnt_or_row0[1024];               // first gradient row of each selected worker
+  int row0[1024];                      // first gradient row of each selected worker
   float lossv[1024];                   // mean minibatch loss of each selected worker
-  int warp_tot[32];
+  int version[1024], job[1024];        // per-worker state after the round's bookkeeping
   int shard_lo[1024];
   unsigned shard_len[1024];
+  float redf[32];
+  int warp_tot[32];
   int scalar[8];
 };
 
@@ -128,46 +138,72 @@ struct CtlShared {
 // next round and lays out its gradient rows.
 //   do_finish: complete the open round if there is one
 //   do_select: open the next round
+// A dependent global-memory access costs this lone CTA close to a microsecond, so everything it
+// needs is loaded up front in one wave and later phases work from registers and shared memory.
 __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select) {
-  __shared__ CtlShared sh;
+  extern __shared__ __align__(16) unsigned char ctl_smem[];
+  CtlShared& sh = *reinterpret_cast<CtlShared*>(ctl_smem);
   DevState* st = a.st;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int W = st->W, S = st->S, B = st->B, RB = st->RB;
-  const int status0 = st->status;
-  const int open0 = st->open;
+  // ---- one wave of loads
+  const int W = st->W, S = st->S, B = st->B, RB = st->RB, K0 = st->K0;
+  const int status0 = st->status, open0 = st->open, diverged0 = st->diverged;
+  const int k_mode = st->k_mode, bound_mode = st->bound_mode, max_rounds = st->max_rounds;
+  const uint32_t key0 = st->key0, key1 = st->key1;
+  const i64 n_samples = st->n_samples;
+  const u64 T_end0 = st->T_end;
+  const float L0_prev = st->L0;
+  const i64 sel_off = st->sel_total, rst_off = st->rst_total;
+  const u64 comm0 = st->comm;
   int t = st->t, K = st->K;
-  __syncthreads();
+  const bool net = a.row_loss != nullptr;
+  const bool fin = do_finish && open0;
+  u64 my_c = 0;
+  int my_version = 0, my_job = 0, my_dur_job = -1;
+  u64 my_next_dur = 0;
+  if (tid < W) {
+    my_c = a.c[tid]; my_version = a.version[tid]; my_job = a.job[tid];
+    my_dur_job = a.dur_job[tid]; my_next_dur = a.next_dur[tid];
+  }
+  int my_sel = 0, my_tau = 0, my_row0 = 0;
+  float my_loss = 0.f;
+  if (fin && tid < K) {
+    my_sel = a.sel[tid]; my_tau = a.sel_tau[tid]; my_row0 = a.sel_row0[tid];
+    if (!net) my_loss = a.loss[tid];
+  }
   if (status0 != ST_OK) return;
 
   // ------------------------------------------------------------------ finish round t
-  if (do_finish && open0) {
-    const u64 T_end = st->T_end;
-    // per-worker mean loss of network models: fixed-order sum of the per-sample losses
-    if (a.row_loss != nullptr) {
-      if (tid < K) sh.cnt_or_row0[tid] = a.sel_row0[tid];
+  if (fin) {
+    const u64 T_end = T_end0;
+    if (net) {
+      // per-worker mean of the per-sample losses: TPW neighbouring threads share a worker, each
+      // adds every TPW-th row (independent loads), then the TPW partial sums are added by a
+      // fixed shuffle tree
+      sh.row0[tid] = my_row0;
       __syncthreads();
-#pragma unroll 4
-      for (int i = warp; i < K; i += 32) {
-        const int r0 = sh.cnt_or_row0[i];
-        float acc = 0.f;
-        for (int b = lane; b < B; b += 32) acc += a.row_loss[r0 + b];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == 0) sh.lossv[i] = __fdiv_rn(acc, (float)B);
+      int kp = 32;
+      while (kp < K) kp <<= 1;
+      const int tpw = min(32, 1024 / kp);
+      const int i = tid / tpw, sub = tid - i * tpw;
+      float acc = 0.f;
+      if (i < K) {
+        const float* rl = a.row_loss + sh.row0[i];
+#pragma unroll 8
+        for (int b = sub; b < B; b += tpw) acc += rl[b];
       }
+      for (int o = tpw >> 1; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (i < K && sub == 0) sh.lossv[i] = __fdiv_rn(acc, (float)B);
       __syncthreads();
-    } else if (tid < K) {
-      sh.lossv[tid] = a.loss[tid];
+      if (tid < K) my_loss = sh.lossv[tid];
     }
-    if (a.row_loss == nullptr) __syncthreads();
-    const float my_loss = (tid < K) ? sh.lossv[tid] : 0.f;
-    const int bad = __syncthreads_or((tid < K) && !isfinite(my_loss)) || st->diverged;
+    const int bad = __syncthreads_or((tid < K) && !isfinite(my_loss)) || diverged0;
     if (bad) {
       if (tid == 0) { st->status = ST_DIVERGED; st->open = 0; }
       return;
     }
     // loss estimate: adjacent-pair tree sum in binary32 over 1024 leaves, /K in binary32
-    float v = my_loss;
+    float v = (tid < K) ? my_loss : 0.f;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) v = __fadd_rn(v, __shfl_down_sync(0xffffffffu, v, o));
     if (lane == 0) sh.redf[warp] = v;
@@ -179,18 +215,18 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
       for (int o = 1; o < 32; o <<= 1) x = __fadd_rn(x, __shfl_down_sync(0xffffffffu, x, o));
       if (lane == 0) {
         const float Lt0 = __fdiv_rn(x, (float)K);
-        const float L00 = (t == 0) ? Lt0 : st->L0;
+        const float L00 = (t == 0) ? Lt0 : L0_prev;
         // Eq. 5 as an exact integer rule: largest k with k^2 Lt <= K0^2 L0 (binary64 products of a
         // 20-bit integer and a binary32 value are exact).  A binary32 estimate of K0 sqrt(L0/Lt)
         // is corrected with the exact test, so only a handful of double operations are issued.
         int kr = 0;
-        if (st->k_mode == ABS_K_ADAPTIVE) {
+        if (k_mode == ABS_K_ADAPTIVE) {
           if (Lt0 <= 0.f) {
             kr = W;
           } else {
-            const double rhs = __dmul_rn((double)(st->K0 * st->K0), (double)L00);
+            const double rhs = __dmul_rn((double)(K0 * K0), (double)L00);
             const double lt = (double)Lt0;
-            const float est = (float)st->K0 * sqrtf(L00 / Lt0);
+            const float est = (float)K0 * sqrtf(L00 / Lt0);
             int k = (est >= (float)W) ? W : ((est >= 1.f) ? (int)est : 1);
             while (k < W && __dmul_rn((double)((k + 1) * (k + 1)), lt) <= rhs) ++k;
             while (k >= 1 && !(__dmul_rn((double)(k * k), lt) <= rhs)) --k;
@@ -202,16 +238,16 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
         sh.scalar[2] = kr;
       }
     }
-    if (tid < K) sh.flag[a.sel[tid]] = 1;
+    if (tid < K) sh.flag[my_sel] = 1;
     __syncthreads();
     const float Lt = sh.redf[0];
     const float L0 = sh.redf[1];
     int K_next = K;
-    if (st->k_mode == ABS_K_ADAPTIVE) K_next = min(W, max(K, sh.scalar[2]));
+    if (k_mode == ABS_K_ADAPTIVE) K_next = min(W, max(K, sh.scalar[2]));
     // Eq. 4 with a = S - N/K0, in integers
     int theta = S;
-    if (st->bound_mode == ABS_BOUND_ADAPTIVE) {
-      const i64 fl = floor_div((i64)W * (i64)(st->K0 - K_next), (i64)K_next * (i64)st->K0);
+    if (bound_mode == ABS_BOUND_ADAPTIVE) {
+      const i64 fl = floor_div((i64)W * (i64)(K0 - K_next), (i64)K_next * (i64)K0);
       i64 th = (i64)S + fl;
       if (th < 1) th = 1;
       if (th > S) th = S;
@@ -221,15 +257,16 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     int restart = 0, renew = 0;
     if (tid < W) {
       const int sel_me = sh.flag[tid];
-      restart = (!sel_me) && ((t + 1 - a.version[tid]) > theta);
+      restart = (!sel_me) && ((t + 1 - my_version) > theta);
       renew = sel_me || restart;
     }
     int range_err = 0;
     if (renew) {
-      const int j = a.job[tid] + 1;
-      const u64 dt = (a.dur_job[tid] == j) ? a.next_dur[tid] : job_ticks(st->dist, st->key0, st->key1, tid, j);
+      const int j = my_job + 1;
+      const u64 dt = (my_dur_job == j) ? my_next_dur : job_ticks(st->dist, key0, key1, tid, j);
       const u64 cn = T_end + dt;
       if (dt == 0ull || cn >= (1ull << 53)) range_err = 1;
+      my_job = j; my_version = t + 1; my_c = cn;
       a.job[tid] = j;
       a.version[tid] = t + 1;
       a.c[tid] = cn;
@@ -240,15 +277,13 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     range_err = __syncthreads_or(range_err);
     int base = 0, R = 0;
     for (int w = 0; w < 32; ++w) { const int c = sh.warp_tot[w]; if (w < warp) base += c; R += c; }
-    const i64 sel_off = st->sel_total, rst_off = st->rst_total;
     if (restart) a.tr_rst_id[rst_off + base + __popc(rb & ((1u << lane) - 1u))] = tid;
     if (tid < K) {
-      a.tr_sel_id[sel_off + tid] = a.sel[tid];
-      a.tr_sel_tau[sel_off + tid] = a.sel_tau[tid];
+      a.tr_sel_id[sel_off + tid] = my_sel;
+      a.tr_sel_tau[sel_off + tid] = my_tau;
       a.tr_sel_loss[sel_off + tid] = my_loss;
     }
-    const u64 comm = st->comm + (u64)(K + R);
-    __syncthreads();
+    const u64 comm = comm0 + (u64)(K + R);
     if (tid == 0) {
       a.tr_K[t] = K; a.tr_R[t] = R; a.tr_theta[t] = theta; a.tr_T[t] = T_end;
       a.tr_loss[t] = Lt; a.tr_comm[t] = comm;
@@ -266,24 +301,25 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
 
   // ------------------------------------------------------------------ select round t
   if (!do_select) return;
-  if (t >= st->max_rounds) {
+  if (t >= max_rounds) {
     if (tid == 0) st->status = ST_NOSPACE;
     return;
   }
   {
-    // arrivals: the K smallest (completion tick, worker id) keys
+    sh.version[tid] = my_version;
+    sh.job[tid] = my_job;
+    for (int i = tid; i < 32 * MAX_TAU; i += 1024) (&sh.wcnt[0][0])[i] = 0;
+    // arrivals: the K smallest (completion tick, worker id) keys; unused slots get distinct
+    // keys above every real one
     int n_pow2 = 32;
     while (n_pow2 < W) n_pow2 <<= 1;
-    u64 key = (tid < W) ? ((a.c[tid] << 10) | (u64)tid) : ~0ull;
-    key = bitonic_sort_1024(key, sh.keys, n_pow2);
-    sh.keys[tid] = key;
-    for (int i = tid; i < 32 * MAX_TAU; i += 1024) (&sh.wcnt[0][0])[i] = 0;
-    __syncthreads();
-    const u64 T_end = sh.keys[K - 1] >> 10;
+    const u64 key_in = (tid < W) ? ((my_c << 10) | (u64)tid) : (0xFFFFFFFFFFFFFC00ull | (u64)tid);
+    const u64* sorted = rank_merge_sort(key_in, sh.keysA, sh.keysB, n_pow2);
+    const u64 T_end = sorted[K - 1] >> 10;
     int n = -1, tau = -1;
     if (tid < K) {
-      n = (int)(key & 1023ull);
-      tau = t - a.version[n];
+      n = (int)(sorted[tid] & 1023ull);
+      tau = t - sh.version[n];
     }
     const int tau_bad = __syncthreads_or(tid < K && (tau < 0 || tau > S));
     if (tau_bad) {
@@ -318,10 +354,26 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
       a.sel[tid] = n;
       a.sel_tau[tid] = tau;
       a.sel_row0[tid] = row0;
-      sh.keys[tid] = ((u64)(unsigned)row0 << 32) | (u64)(unsigned)n;   // reuse as (row0, n)
+      sh.row0[tid] = row0;
+      sh.flag[tid] = 0;
+      if (net) {
+        const i64 lo = ((i64)n * n_samples) / W, hi = ((i64)(n + 1) * n_samples) / W;
+        sh.shard_lo[tid] = (int)lo;
+        sh.shard_len[tid] = (unsigned)(hi - lo);
+      }
     }
-    // ring slot of every row tile and padding rows, all threads; least squares reads neither
-    if (a.row_loss != nullptr) {
+    if (tid == 0) {
+      st->T_end = T_end;
+      st->n_rows = n_rows;
+      st->n_row_tiles = n_rows / RB;
+      st->n_groups = sh.scalar[1];
+      st->diverged = 0;
+      st->open = 1;
+    }
+    if (!net) return;             // least squares: no row tiles, minibatches drawn by its own kernel
+    __syncthreads();
+    // ring slot of every row tile and padding rows
+    {
       const int n_tiles = n_rows / RB;
       for (int q = tid; q < n_tiles; q += 1024) {
         const int r = q * RB;
@@ -336,42 +388,21 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
         for (int r = p0 + tid; r < p1; r += 1024) a.row_idx[r] = -1;
       }
     }
-    __syncthreads();
     // minibatch draws: sample b of job (n, j) = word b%4 of Philox block (n, j, 1, b/4),
-    // mapped into the worker's shard [n M / N, (n+1) M / N).  Least squares draws them in its
-    // own gradient kernel (one CTA per worker), so the control CTA skips them.
-    if (a.row_loss != nullptr) {
-      const int blocks_per = (B + 3) >> 2;
-      const i64 M = st->n_samples;
-      if (tid < K) {
-        const int wn = (int)(sh.keys[tid] & 0xffffffffull);
-        const i64 lo = ((i64)wn * M) / W, hi = ((i64)(wn + 1) * M) / W;
-        sh.shard_lo[tid] = (int)lo;
-        sh.shard_len[tid] = (unsigned)(hi - lo);
-        sh.cnt_or_row0[tid] = a.job[wn];
-      }
-      __syncthreads();
-      for (int item = tid; item < K * blocks_per; item += 1024) {
-        const int i = item / blocks_per, blk = item - i * blocks_per;
-        const int wn = (int)(sh.keys[i] & 0xffffffffull), row0 = (int)(sh.keys[i] >> 32);
-        uint32_t w4[4];
-        philox4x32_10((uint32_t)wn, (uint32_t)sh.cnt_or_row0[i], 1u, (uint32_t)blk, st->key0, st->key1, w4);
-        const int lo = sh.shard_lo[i];
-        const u64 len = (u64)sh.shard_len[i];
+    // mapped into the worker's shard [n M / N, (n+1) M / N)
+    const int blocks_per = (B + 3) >> 2;
+    for (int item = tid; item < K * blocks_per; item += 1024) {
+      const int i = item / blocks_per, blk = item - i * blocks_per;
+      const int wn = (int)(sorted[i] & 1023ull);
+      uint32_t w4[4];
+      philox4x32_10((uint32_t)wn, (uint32_t)sh.job[wn], 1u, (uint32_t)blk, key0, key1, w4);
+      const int lo = sh.shard_lo[i], row0 = sh.row0[i];
+      const u64 len = (u64)sh.shard_len[i];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int b = blk * 4 + q;
-          if (b < B) a.row_idx[row0 + b] = lo + (int)(((u64)w4[q] * len) >> 32);
-        }
+      for (int q = 0; q < 4; ++q) {
+        const int b = blk * 4 + q;
+        if (b < B) a.row_idx[row0 + b] = lo + (int)(((u64)w4[q] * len) >> 32);
       }
-    }
-    if (tid == 0) {
-      st->T_end = T_end;
-      st->n_rows = n_rows;
-      st->n_row_tiles = n_rows / RB;
-      st->n_groups = sh.scalar[1];
-      st->diverged = 0;
-      st->open = 1;
     }
   }
 }
