@@ -60,7 +60,8 @@ struct Layout {
   size_t w_off[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the padded vector
   size_t w_src[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the caller's vector
   size_t st, c, version, job, next_dur, dur_job, sel, sel_tau, sel_row0, loss, row_loss, row_idx, tile_slot;
-  size_t master, ring, G, logits, red;
+  size_t master, ring, G, logits, red, ones;
+  size_t bits[ABS_MAX_LAYERS + 1];      // ReLU sign bits of act[l] (tensor-core layers)
   size_t act[ABS_MAX_LAYERS + 1], delta[ABS_MAX_LAYERS + 1];
   size_t tr_K, tr_R, tr_theta, tr_T, tr_loss, tr_comm, tr_sel_off, tr_rst_off;
   size_t tr_sel_id, tr_sel_tau, tr_sel_loss, tr_rst_id;
@@ -181,6 +182,10 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       for (int l = 0; l < m->n_layers; ++l) len = std::max(len, (size_t)m->dims[l + 1]);
       L->red = cv.take(4 * len * (size_t)(L->rows_cap / 64));
     }
+    L->ones = L->any_tc ? cv.take(2 * 64 * (size_t)L->rows_cap) : 0;
+    for (int l = 0; l <= m->n_layers; ++l) L->bits[l] = 0;
+    for (int l = 0; l + 1 < m->n_layers; ++l)
+      if (L->path[l] == PATH_TC) L->bits[l + 1] = cv.take(4 * (size_t)L->rows_cap * ((m->dims[l + 1] + 31) / 32));
     L->act[0] = (L->path[0] == PATH_TC) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     for (int l = 1; l <= m->n_layers; ++l) {
       L->act[l] = (l < m->n_layers) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]) : 0;
@@ -213,6 +218,13 @@ struct TcLayer {
   CUtensorMap fwd_a, fwd_b, dg_a, dg_b, wg_a, wg_b;
 };
 
+// ones[r][0] = 1 (bf16), the rest of the 64-wide rows stays zero: the extra operand row that turns
+// the weight-gradient GEMM into weight + bias gradient
+__global__ void ones_init_kernel(__nv_bfloat16* ones, int rows) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r < rows) ones[(size_t)r * 64] = __float2bfloat16_rn(1.f);
+}
+
 struct abs_ctx {
   abs_model_desc m;
   Layout L;
@@ -227,6 +239,7 @@ struct abs_ctx {
   long long launches = 0;
   CtlArgs ctl;
   TcLayer tcl[ABS_MAX_LAYERS];
+  CUtensorMap ones_map;
   // profiling: event pairs around launches
   std::vector<cudaEvent_t> ev;       // 2 per recorded launch
   std::vector<int> ev_class;
@@ -305,7 +318,7 @@ template <int BN>
 void launch_tc(abs_ctx* ctx, int cls, const CUtensorMap& a, const CUtensorMap& b, const tc::Params& p, int max_tiles) {
   const int grid = std::max(1, std::min(ctx->sm_count, max_tiles));
   launch_k(ctx, cls, [&] {
-    tc::tc_gemm_kernel<BN><<<grid, tc::THREADS, tc::Cfg<BN>::SMEM_BYTES, ctx->stream>>>(a, b, p);
+    tc::tc_gemm_kernel<BN><<<grid, tc::THREADS, tc::Cfg<BN>::SMEM_BYTES, ctx->stream>>>(a, b, ctx->ones_map, p);
   });
 }
 
@@ -326,6 +339,10 @@ int setup_tc(abs_ctx* ctx) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<64>::SMEM_BYTES);
   if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaFuncSetAttribute(tc_gemm_kernel)");
   const char* ring = ctx->at<char>(L.ring);
+  if (!make_act_map(&ctx->ones_map, ctx->at<void>(L.ones), 64, L.rows_cap, 64))
+    return fail(ABS_ECUDA, "cuTensorMapEncodeTiled failed for the ones matrix");
+  ones_init_kernel<<<(L.rows_cap + 255) / 256, 256, 0, ctx->stream>>>(ctx->at<__nv_bfloat16>(L.ones), L.rows_cap);
+  ctx->launches += 1;
   for (int l = 0; l < m.n_layers; ++l) {
     if (L.path[l] != PATH_TC) continue;
     const int in = m.dims[l], out = m.dims[l + 1];
@@ -409,6 +426,8 @@ void enqueue_gradient(abs_ctx* ctx) {
       tc::Params p = tc_params(l, tc::FWD);
       p.N_total = la[l].out; p.K_total = la[l].in;
       p.out_bf16 = (__nv_bfloat16*)la[l].act_out;
+      p.relu_bits = L.bits[l + 1] ? ctx->at<uint32_t>(L.bits[l + 1]) : nullptr;
+      p.mask_words = (la[l].out + 31) / 32;
       const int bn = L.bn_fwd[l];
       launch_tc_bn(ctx, bn, ABS_KC_FWD, ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
     } else if (L.path[l] == PATH_NARROW) {
@@ -443,26 +462,18 @@ void enqueue_gradient(abs_ctx* ctx) {
         tc::Params p = tc_params(l, tc::DGRAD);
         p.N_total = la[l].in; p.K_total = la[l].out;
         p.mask_src = (const __nv_bfloat16*)la[l].act_in;
+        p.mask_bits = L.bits[l] ? ctx->at<uint32_t>(L.bits[l]) : nullptr;
+        p.mask_words = (la[l].in + 31) / 32;
         p.out_bf16 = (__nv_bfloat16*)la[l].delta_in;
         const int bn = L.bn_dg[l];
         launch_tc_bn(ctx, bn, ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, p, row_tiles128 * ((la[l].in + bn - 1) / bn));
       }
       tc::Params p = tc_params(l, tc::WGRAD);
-      p.M_total = la[l].in; p.N_total = la[l].out;
+      p.M_total = la[l].in + 1; p.N_total = la[l].out;     // row `in` of the result is the bias gradient
       p.out_f32 = ctx->at<float>(L.G) + L.w_off[l];
       const int bn = L.bn_wg[l];
       launch_tc_bn(ctx, bn, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, p,
-                   ((la[l].in + 127) / 128) * ((la[l].out + bn - 1) / bn) * L.P);
-      // bias gradient: per-chunk column sums, then one ordered sum over the chunks into partial 0
-      const T* dl = (const T*)la[l].delta_out;
-      const size_t b_off = L.w_off[l] + (size_t)la[l].in * la[l].out;
-      const int out = la[l].out;
-      float* part = ctx->at<float>(L.red);
-      float* dstb = ctx->at<float>(L.G) + b_off;
-      const int per = std::min(out / 8, 256), lanes = 256 / per;
-      const size_t smb = lanes > 1 ? sizeof(float) * (size_t)lanes * out : 0;
-      launch_k(ctx, ABS_KC_BIAS, [&] { colsum_chunk_kernel<T><<<L.rows_cap / 64, 256, smb, s>>>(st, dl, out, part); });
-      launch_k(ctx, ABS_KC_BIAS, [&] { chunk_reduce_kernel<<<(out + 31) / 32, 256, 0, s>>>(st, part, out, dstb); });
+                   ((la[l].in + 127) / 128 + 1) * ((la[l].out + bn - 1) / bn) * L.P);
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (l > 0) {

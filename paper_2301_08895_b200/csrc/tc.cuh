@@ -30,12 +30,15 @@ struct Params {
   DevState* st;
   const int* tile_slot;
   int mode;
-  int M_total;             // WGRAD: in (rows of G); FWD/DGRAD: unused
+  int M_total;             // WGRAD: in + 1 (weight rows and the bias row of G); FWD/DGRAD: unused
   int N_total;             // FWD: out, DGRAD: in, WGRAD: out
   int K_total;             // FWD: in,  DGRAD: out, WGRAD: unused (rows come from the device state)
   int P;                   // WGRAD split count
   const __nv_bfloat16* ring; size_t slot_stride; size_t b_off;   // FWD bias: ring + slot*stride + b_off
-  const __nv_bfloat16* mask_src;   // DGRAD: H[r][N_total]
+  const __nv_bfloat16* mask_src;   // DGRAD: H[r][N_total] (used when mask_bits is null)
+  const uint32_t* mask_bits;       // DGRAD: bit n%32 of word [r][n/32] = (H[r][n] > 0)
+  uint32_t* relu_bits;             // FWD: the same bits for this layer's output (may be null)
+  int mask_words;                  // words per row of mask_bits / relu_bits = ceil(N_total / 32)
   __nv_bfloat16* out_bf16;         // FWD/DGRAD result [rows][N_total]
   float* out_f32;                  // WGRAD: G + w_off, partial p at + p*slot_stride, row pitch N_total
 };
@@ -138,14 +141,16 @@ template <int BN> struct Cfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr size_t SMEM_BYTES =
+      (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 2 * BN * 4 /*bias*/;
 };
 
-struct TileCoord { int a_row, b_col, slot, k_begin, n_kb, split; };
+struct TileCoord { int a_row, b_col, slot, k_begin, n_kb, split, bias_tile; };
 
 template <int BN>
 __global__ void __launch_bounds__(THREADS, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params p) {
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_ones, const Params p) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   DevState* st = p.st;
@@ -154,7 +159,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int n_row_tiles = n_rows / BM;
   const int mode = p.mode;
   const int n_ct = (p.N_total + BN - 1) / BN;
-  const int n_mt = (mode == WGRAD) ? (p.M_total + BM - 1) / BM : n_row_tiles;
+  // WGRAD: one extra row tile multiplies a column of ones with the deltas, which yields the bias
+  // gradient (row `in` of the [in + 1][out] gradient block) on the tensor cores for free
+  const int n_mt_w = (p.M_total - 1 + BM - 1) / BM;
+  const int n_mt = (mode == WGRAD) ? n_mt_w + 1 : n_row_tiles;
   const int n_tiles = (mode == WGRAD) ? n_mt * n_ct * p.P : n_row_tiles * n_ct;
   if ((int)blockIdx.x >= n_tiles) return;
   const int chunk = (mode == WGRAD) ? round_up((n_rows + p.P - 1) / p.P, BK) : 0;
@@ -169,6 +177,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   uint64_t* acc_empty = acc_full + 2;        // [2] accumulator drained by the epilogue
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* bias_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [2][BN]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -192,7 +201,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int per_split = n_mt * n_ct;
       c.split = tile / per_split;
       const int rem = tile - c.split * per_split;
-      c.a_row = (rem / n_ct) * BM;           // m0
+      const int mt = rem / n_ct;
+      c.bias_tile = (mt == n_mt_w);
+      c.a_row = mt * BM;                     // m0
       c.b_col = (rem % n_ct) * BN;           // n0
       c.slot = 0;
       c.k_begin = min(n_rows, c.split * chunk);
@@ -201,6 +212,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
       const int rt = tile / n_ct;
       c.split = 0;
+      c.bias_tile = 0;
       c.a_row = rt * BM;
       c.b_col = (tile - rt * n_ct) * BN;
       c.slot = p.tile_slot[c.a_row / RB];
@@ -234,7 +246,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             tma_load_2d(sa, &map_a, &full[stage], k0, c.a_row);
             tma_load_3d(sb, &map_b, &full[stage], k0, c.b_col, c.slot);
           } else {
-            for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * 8192, &map_a, &full[stage], c.a_row + 64 * j, k0);
+            if (c.bias_tile) {   // second box lies outside the 64-wide ones matrix: zero fill
+              for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * 8192, &map_ones, &full[stage], 64 * j, k0);
+            } else {
+              for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * 8192, &map_a, &full[stage], c.a_row + 64 * j, k0);
+            }
             for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, &map_b, &full[stage], c.b_col + 64 * j, k0);
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -302,12 +318,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       const TileCoord c = tile_coord(tile);
       const bool have = c.n_kb > 0;
+      // output row (FWD/DGRAD) or gradient row m (WGRAD; the bias tile's row 0 is row `in`)
+      const int r = (mode == WGRAD && c.bias_tile) ? (p.M_total - 1) + row_in_tile : c.a_row + row_in_tile;
+      // fetch what the epilogue needs from global memory before waiting for the accumulator
+      uint32_t mw[BN / 32];
+      float* bias_t = bias_s + acc * BN;
+      if (mode == FWD) {
+        const __nv_bfloat16* bias = p.ring + (size_t)c.slot * p.slot_stride + p.b_off;
+        for (int i = (int)threadIdx.x - 64; i < BN; i += 128) {
+          const int n = c.b_col + i;
+          bias_t[i] = n < p.N_total ? __bfloat162float(bias[n]) : 0.f;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      } else if (mode == DGRAD && p.mask_bits != nullptr) {
+#pragma unroll
+        for (int i = 0; i < BN / 32; ++i) {
+          const int w = c.b_col / 32 + i;
+          mw[i] = w < p.mask_words ? p.mask_bits[(size_t)r * p.mask_words + w] : 0u;
+        }
+      }
       if (have) {
         if (!mbar_wait(&acc_full[acc], acc_phase, abort)) break;
         tc_fence_after();
       }
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-      const int r = c.a_row + row_in_tile;     // output row (FWD/DGRAD) or m (WGRAD)
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         const int n0 = c.b_col + c0;
@@ -319,7 +353,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int i = 0; i < 32; ++i) v[i] = 0u;
         }
         if (mode == WGRAD) {
-          if (r < p.M_total) {
+          if (r < (c.bias_tile ? p.M_total : p.M_total - 1)) {
             float* dst = p.out_f32 + (size_t)c.split * p.slot_stride + (size_t)r * p.N_total + n0;
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
@@ -329,19 +363,38 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         } else {
           __nv_bfloat16* dst = p.out_bf16 + (size_t)r * p.N_total + n0;
           if (mode == FWD) {
-            const __nv_bfloat16* bias = p.ring + (size_t)c.slot * p.slot_stride + p.b_off + n0;
+            uint32_t bits = 0u;
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
               if (n0 + i < p.N_total) {
-                const uint4 bb = *reinterpret_cast<const uint4*>(bias + i);
-                const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&bb);
                 uint4 o;
                 __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                  const float2 bf = __bfloat1622float2(b2[j]);
-                  const float x = fmaxf(__uint_as_float(v[i + 2 * j]) + bf.x, 0.f);
-                  const float y = fmaxf(__uint_as_float(v[i + 2 * j + 1]) + bf.y, 0.f);
+                  const float x = fmaxf(__uint_as_float(v[i + 2 * j]) + bias_t[c0 + i + 2 * j], 0.f);
+                  const float y = fmaxf(__uint_as_float(v[i + 2 * j + 1]) + bias_t[c0 + i + 2 * j + 1], 0.f);
+                  o2[j] = __floats2bfloat162_rn(x, y);
+                  // the bit records the sign of the STORED (bf16-rounded) activation
+                  bits |= (__low2float(o2[j]) > 0.f ? 1u : 0u) << (i + 2 * j);
+                  bits |= (__high2float(o2[j]) > 0.f ? 1u : 0u) << (i + 2 * j + 1);
+                }
+                *reinterpret_cast<uint4*>(dst + i) = o;
+              }
+            }
+            if (p.relu_bits != nullptr) p.relu_bits[(size_t)r * p.mask_words + (n0 >> 5)] = bits;
+          } else if (p.mask_bits != nullptr) {
+            uint32_t bits = 0u;
+#pragma unroll
+            for (int i = 0; i < BN / 32; ++i) bits = (i == (c0 >> 5)) ? mw[i] : bits;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              if (n0 + i < p.N_total) {
+                uint4 o;
+                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const float x = ((bits >> (i + 2 * j)) & 1u) ? __uint_as_float(v[i + 2 * j]) : 0.f;
+                  const float y = ((bits >> (i + 2 * j + 1)) & 1u) ? __uint_as_float(v[i + 2 * j + 1]) : 0.f;
                   o2[j] = __floats2bfloat162_rn(x, y);
                 }
                 *reinterpret_cast<uint4*>(dst + i) = o;
