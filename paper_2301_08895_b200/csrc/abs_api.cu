@@ -216,6 +216,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
 
 struct TcLayer {
   CUtensorMap fwd_a, fwd_b, dg_a, dg_b, wg_a, wg_b;
+  CUtensorMap fwd_out, dg_out, wg_out;     // result tensors written by bulk tensor stores
 };
 
 // ones[r][0] = 1 (bf16), the rest of the 64-wide rows stays zero: the extra operand row that turns
@@ -291,11 +292,11 @@ EncodeTiledFn encode_fn() {
 
 // bf16 tensor map with 128-byte swizzle; dims/strides innermost first, strides in bytes for dims 1...
 bool make_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
-              const cuuint32_t* box) {
+              const cuuint32_t* box, CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, dt, (cuuint32_t)rank, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -314,19 +315,28 @@ bool make_w_map(CUtensorMap* map, const void* base, int in, int out, int slots, 
   return make_map(map, base, 3, dims, strides, box);
 }
 
+// fp32 gradient block of one layer inside the partial-sum buffers: (out, in, P), 32 x 128 boxes
+bool make_g_map(CUtensorMap* map, const void* base, int in, int out, int P, size_t slot_stride) {
+  const cuuint64_t dims[3] = {(cuuint64_t)out, (cuuint64_t)in, (cuuint64_t)P};
+  const cuuint64_t strides[2] = {(cuuint64_t)out * 4, (cuuint64_t)slot_stride * 4};
+  const cuuint32_t box[3] = {32, 128, 1};
+  return make_map(map, base, 3, dims, strides, box, CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
+}
+
 template <int BN>
-void launch_tc(abs_ctx* ctx, int cls, const CUtensorMap& a, const CUtensorMap& b, const tc::Params& p, int max_tiles) {
+void launch_tc(abs_ctx* ctx, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
+               const tc::Params& p, int max_tiles) {
   const int grid = std::max(1, std::min(ctx->sm_count, max_tiles));
   launch_k(ctx, cls, [&] {
-    tc::tc_gemm_kernel<BN><<<grid, tc::THREADS, tc::Cfg<BN>::SMEM_BYTES, ctx->stream>>>(a, b, ctx->ones_map, p);
+    tc::tc_gemm_kernel<BN><<<grid, tc::THREADS, tc::Cfg<BN>::SMEM_BYTES, ctx->stream>>>(a, b, ctx->ones_map, o, p);
   });
 }
 
-void launch_tc_bn(abs_ctx* ctx, int bn, int cls, const CUtensorMap& a, const CUtensorMap& b, const tc::Params& p,
-                  int max_tiles) {
-  if (bn == 256) launch_tc<256>(ctx, cls, a, b, p, max_tiles);
-  else if (bn == 128) launch_tc<128>(ctx, cls, a, b, p, max_tiles);
-  else launch_tc<64>(ctx, cls, a, b, p, max_tiles);
+void launch_tc_bn(abs_ctx* ctx, int bn, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
+                  const tc::Params& p, int max_tiles) {
+  if (bn == 256) launch_tc<256>(ctx, cls, a, b, o, p, max_tiles);
+  else if (bn == 128) launch_tc<128>(ctx, cls, a, b, o, p, max_tiles);
+  else launch_tc<64>(ctx, cls, a, b, o, p, max_tiles);
 }
 
 int setup_tc(abs_ctx* ctx) {
@@ -353,10 +363,13 @@ int setup_tc(abs_ctx* ctx) {
     bool ok = make_act_map(&t.fwd_a, act_in, in, L.rows_cap, 128) &&
               make_w_map(&t.fwd_b, wbase, in, out, ctx->S + 1, L.d_pad, 64) &&
               make_act_map(&t.wg_a, act_in, in, L.rows_cap, 64) &&
-              make_act_map(&t.wg_b, delta_out, out, L.rows_cap, 64);
+              make_act_map(&t.wg_b, delta_out, out, L.rows_cap, 64) &&
+              make_act_map(&t.fwd_out, ctx->at<void>(L.act[l + 1]), out, L.rows_cap, 128) &&
+              make_g_map(&t.wg_out, ctx->at<float>(L.G) + L.w_off[l], in, out, L.P, L.d_pad);
     if (ok && l > 0)
       ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
-           make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l]);
+           make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l]) &&
+           make_act_map(&t.dg_out, ctx->at<void>(L.delta[l]), in, L.rows_cap, 128);
     if (!ok) return fail(ABS_ECUDA, "cuTensorMapEncodeTiled failed for layer %d", l);
   }
   return ABS_OK;
@@ -429,7 +442,7 @@ void enqueue_gradient(abs_ctx* ctx) {
       p.relu_bits = L.bits[l + 1] ? ctx->at<uint32_t>(L.bits[l + 1]) : nullptr;
       p.mask_words = (la[l].out + 31) / 32;
       const int bn = L.bn_fwd[l];
-      launch_tc_bn(ctx, bn, ABS_KC_FWD, ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
+      launch_tc_bn(ctx, bn, ABS_KC_FWD, ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (a.in % 8 == 0) {
@@ -466,13 +479,13 @@ void enqueue_gradient(abs_ctx* ctx) {
         p.mask_words = (la[l].in + 31) / 32;
         p.out_bf16 = (__nv_bfloat16*)la[l].delta_in;
         const int bn = L.bn_dg[l];
-        launch_tc_bn(ctx, bn, ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, p, row_tiles128 * ((la[l].in + bn - 1) / bn));
+        launch_tc_bn(ctx, bn, ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, ctx->tcl[l].dg_out, p, row_tiles128 * ((la[l].in + bn - 1) / bn));
       }
       tc::Params p = tc_params(l, tc::WGRAD);
       p.M_total = la[l].in + 1; p.N_total = la[l].out;     // row `in` of the result is the bias gradient
       p.out_f32 = ctx->at<float>(L.G) + L.w_off[l];
       const int bn = L.bn_wg[l];
-      launch_tc_bn(ctx, bn, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, p,
+      launch_tc_bn(ctx, bn, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
                    ((la[l].in + 127) / 128 + 1) * ((la[l].out + bn - 1) / bn) * L.P);
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);

@@ -141,8 +141,9 @@ template <int BN> struct Cfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;
+  static constexpr int OUT_BYTES = 128 * 128;          // staging box of the epilogue
   static constexpr size_t SMEM_BYTES =
-      (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 2 * BN * 4 /*bias*/;
+      (size_t)STAGES * STAGE_BYTES + OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 2 * BN * 4 /*bias*/;
 };
 
 struct TileCoord { int a_row, b_col, slot, k_begin, n_kb, split, bias_tile; };
@@ -150,7 +151,8 @@ struct TileCoord { int a_row, b_col, slot, k_begin, n_kb, split, bias_tile; };
 template <int BN>
 __global__ void __launch_bounds__(THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_ones, const Params p) {
+               const __grid_constant__ CUtensorMap map_ones, const __grid_constant__ CUtensorMap map_out,
+               const Params p) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   DevState* st = p.st;
@@ -170,7 +172,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)C::STAGES * C::STAGE_BYTES);
+  uint8_t* stage_out = smem + (size_t)C::STAGES * C::STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stage_out + C::OUT_BYTES);
   uint64_t* full = bars;                     // [STAGES] TMA bytes landed
   uint64_t* empty = bars + C::STAGES;        // [STAGES] MMAs that read the stage are done
   uint64_t* acc_full = bars + 2 * C::STAGES; // [2] accumulator complete
@@ -311,8 +314,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else {
     // ------------------------------------------------------------------ epilogue (4 warps)
+    // Results leave through a 16 KB staging box (128 rows x 128 bytes, 128-byte swizzle) and one
+    // bulk tensor store per box, so global memory sees whole rows instead of 32 scattered 16-byte
+    // pieces per store instruction.
     const int q = warp & 3;                    // tensor-memory lane quarter this warp may read
     const int row_in_tile = q * 32 + lane;
+    const bool issuer = threadIdx.x == 64;     // the thread that issues and tracks the bulk stores
+    uint8_t* my_row = stage_out + row_in_tile * 128;
+    const int sw = row_in_tile & 7;
+    const int box_cols = (mode == WGRAD) ? 32 : 64;
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -330,11 +340,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           bias_t[i] = n < p.N_total ? __bfloat162float(bias[n]) : 0.f;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-      } else if (mode == DGRAD && p.mask_bits != nullptr) {
+      } else if (mode == DGRAD) {
 #pragma unroll
         for (int i = 0; i < BN / 32; ++i) {
           const int w = c.b_col / 32 + i;
-          mw[i] = w < p.mask_words ? p.mask_bits[(size_t)r * p.mask_words + w] : 0u;
+          if (p.mask_bits != nullptr) {
+            mw[i] = w < p.mask_words ? p.mask_bits[(size_t)r * p.mask_words + w] : 0u;
+          } else {                               // no stored sign bits: derive them from the activations
+            uint32_t bits = 0u;
+            for (int j = 0; j < 32; ++j) {
+              const int n = w * 32 + j;
+              if (n < p.N_total && __bfloat162float(p.mask_src[(size_t)r * p.N_total + n]) > 0.f) bits |= 1u << j;
+            }
+            mw[i] = bits;
+          }
         }
       }
       if (have) {
@@ -343,83 +362,87 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = 0; c0 < BN; c0 += box_cols) {
         const int n0 = c.b_col + c0;
-        if (n0 >= p.N_total) break;            // uniform in the warp
+        if (n0 >= p.N_total) break;            // uniform in the CTA
+        // the staging box is free once the previous bulk store has read it
+        if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        asm volatile("bar.sync 1, 128;" ::: "memory");
         uint32_t v[32];
-        if (have) tmem_ld32(t_row + (uint32_t)c0, v);
-        else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = 0u;
-        }
         if (mode == WGRAD) {
-          if (r < (c.bias_tile ? p.M_total : p.M_total - 1)) {
-            float* dst = p.out_f32 + (size_t)c.split * p.slot_stride + (size_t)r * p.N_total + n0;
+          if (have) tmem_ld32(t_row + (uint32_t)c0, v);
+          else {
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              if (n0 + i < p.N_total)
-                *reinterpret_cast<uint4*>(dst + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+            for (int i = 0; i < 32; ++i) v[i] = 0u;
           }
-        } else {
-          __nv_bfloat16* dst = p.out_bf16 + (size_t)r * p.N_total + n0;
-          if (mode == FWD) {
-            uint32_t bits = 0u;
+          if (c.bias_tile) {                   // a single useful row: plain stores
+            if (row_in_tile == 0) {
+              float* dst = p.out_f32 + (size_t)c.split * p.slot_stride + (size_t)r * p.N_total + n0;
 #pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              if (n0 + i < p.N_total) {
-                uint4 o;
-                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const float x = fmaxf(__uint_as_float(v[i + 2 * j]) + bias_t[c0 + i + 2 * j], 0.f);
-                  const float y = fmaxf(__uint_as_float(v[i + 2 * j + 1]) + bias_t[c0 + i + 2 * j + 1], 0.f);
-                  o2[j] = __floats2bfloat162_rn(x, y);
-                  // the bit records the sign of the STORED (bf16-rounded) activation
-                  bits |= (__low2float(o2[j]) > 0.f ? 1u : 0u) << (i + 2 * j);
-                  bits |= (__high2float(o2[j]) > 0.f ? 1u : 0u) << (i + 2 * j + 1);
-                }
-                *reinterpret_cast<uint4*>(dst + i) = o;
-              }
-            }
-            if (p.relu_bits != nullptr) p.relu_bits[(size_t)r * p.mask_words + (n0 >> 5)] = bits;
-          } else if (p.mask_bits != nullptr) {
-            uint32_t bits = 0u;
-#pragma unroll
-            for (int i = 0; i < BN / 32; ++i) bits = (i == (c0 >> 5)) ? mw[i] : bits;
-#pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              if (n0 + i < p.N_total) {
-                uint4 o;
-                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const float x = ((bits >> (i + 2 * j)) & 1u) ? __uint_as_float(v[i + 2 * j]) : 0.f;
-                  const float y = ((bits >> (i + 2 * j + 1)) & 1u) ? __uint_as_float(v[i + 2 * j + 1]) : 0.f;
-                  o2[j] = __floats2bfloat162_rn(x, y);
-                }
-                *reinterpret_cast<uint4*>(dst + i) = o;
-              }
+              for (int i = 0; i < 32; i += 4)
+                if (n0 + i < p.N_total)
+                  *reinterpret_cast<uint4*>(dst + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
             }
           } else {
-            const __nv_bfloat16* h = p.mask_src + (size_t)r * p.N_total + n0;
 #pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              if (n0 + i < p.N_total) {
-                const uint4 hh = *reinterpret_cast<const uint4*>(h + i);
-                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&hh);
-                uint4 o;
-                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const float2 hf = __bfloat1622float2(h2[j]);
-                  const float x = hf.x > 0.f ? __uint_as_float(v[i + 2 * j]) : 0.f;
-                  const float y = hf.y > 0.f ? __uint_as_float(v[i + 2 * j + 1]) : 0.f;
-                  o2[j] = __floats2bfloat162_rn(x, y);
-                }
-                *reinterpret_cast<uint4*>(dst + i) = o;
-              }
-            }
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<uint4*>(my_row + ((j ^ sw) << 4)) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
           }
+        } else {
+#pragma unroll
+          for (int hlf = 0; hlf < 2; ++hlf) {
+            const int cc = c0 + 32 * hlf;       // column offset inside the tile
+            if (c.b_col + cc >= p.N_total) break;
+            if (have) tmem_ld32(t_row + (uint32_t)cc, v);
+            else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) v[i] = 0u;
+            }
+            uint32_t bits = 0u;
+            if (mode == DGRAD) {
+#pragma unroll
+              for (int i = 0; i < BN / 32; ++i) bits = (i == (cc >> 5)) ? mw[i] : bits;
+            }
+            uint32_t relu = 0u;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint4 o;
+              __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int i = 8 * j + 2 * e;
+                float x = __uint_as_float(v[i]), y = __uint_as_float(v[i + 1]);
+                if (mode == FWD) {
+                  x = fmaxf(x + bias_t[cc + i], 0.f);
+                  y = fmaxf(y + bias_t[cc + i + 1], 0.f);
+                } else {
+                  x = ((bits >> i) & 1u) ? x : 0.f;
+                  y = ((bits >> (i + 1)) & 1u) ? y : 0.f;
+                }
+                o2[e] = __floats2bfloat162_rn(x, y);
+                if (mode == FWD) {             // the bit records the sign of the STORED activation
+                  relu |= (__low2float(o2[e]) > 0.f ? 1u : 0u) << i;
+                  relu |= (__high2float(o2[e]) > 0.f ? 1u : 0u) << (i + 1);
+                }
+              }
+              *reinterpret_cast<uint4*>(my_row + (((4 * hlf + j) ^ sw) << 4)) = o;
+            }
+            if (mode == FWD && p.relu_bits != nullptr)
+              p.relu_bits[(size_t)r * p.mask_words + ((c.b_col + cc) >> 5)] = relu;
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (issuer && !(mode == WGRAD && c.bias_tile)) {
+          if (mode == WGRAD)
+            asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                         ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(smem_u32(stage_out)), "r"(n0), "r"(c.a_row), "r"(c.split)
+                         : "memory");
+          else
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                         ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(smem_u32(stage_out)), "r"(n0), "r"(c.a_row)
+                         : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       }
       if (have) {
@@ -430,6 +453,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (acc == 0) acc_phase ^= 1u;
       }
     }
+    if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   // ------------------------------------------------------------------ teardown
