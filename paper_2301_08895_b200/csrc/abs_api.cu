@@ -55,6 +55,7 @@ struct Layout {
   int path[ABS_MAX_LAYERS] = {};        // how each layer's contractions run
   int bn_fwd[ABS_MAX_LAYERS] = {}, bn_dg[ABS_MAX_LAYERS] = {}, bn_wg[ABS_MAX_LAYERS] = {};
   bool any_tc = false;
+  int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
   size_t esz = 4;                       // bytes per stored element (4 or 2)
   size_t d = 0, d_pad = 0;
   size_t w_off[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the padded vector
@@ -135,18 +136,31 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       for (int bn : {256, 128}) if (n >= bn && other_tiles * ((n + bn - 1) / bn) >= 120) return bn;
       return n >= 128 ? 128 : 64;
     };
-    size_t biggest = 1;
     for (int l = 0; l < m->n_layers; ++l) {
       if (L->path[l] != PATH_TC) continue;
       const int in = m->dims[l], out = m->dims[l + 1];
       L->bn_fwd[l] = pick(out, row_tiles);
       L->bn_dg[l] = pick(in, row_tiles);
-      L->bn_wg[l] = pick(out, ((in + 127) / 128) * 3);
-      biggest = std::max(biggest, (size_t)((in + 127) / 128) * ((out + L->bn_wg[l] - 1) / L->bn_wg[l]));
+      L->bn_wg[l] = pick(out, ((in + 127) / 128 + 1) * 3);
     }
-    int P = (int)((296 + biggest / 2) / biggest);
-    P = std::min(P, std::max(1, W * m->batch / 512));
-    L->P = std::max(1, std::min(P, 8));
+    // split count P of the row reduction: the one that minimises the modelled time of all weight
+    // gradients (whole waves of 148 CTAs, one tile = 128 x BN x rows/P) plus the extra partial
+    // sums the Eq. 3 step then has to read
+    double best = 1e30;
+    int bestP = 1;
+    const int maxP = std::max(1, std::min(8, W * m->batch / 512));
+    for (int P = 1; P <= maxP; ++P) {
+      double t = 4.0 * (double)L->d_pad * P / 5e12;
+      for (int l = 0; l < m->n_layers; ++l) {
+        if (L->path[l] != PATH_TC) continue;
+        const int in = m->dims[l], out = m->dims[l + 1], bn = L->bn_wg[l];
+        const long tiles = (long)((in + 127) / 128 + 1) * ((out + bn - 1) / bn) * P;
+        const long waves = (tiles + 147) / 148;
+        t += (double)waves * 2.0 * 128.0 * bn * ((double)L->rows_cap / P) / 9e12;
+      }
+      if (t < best * 0.999) { best = t; bestP = P; }
+    }
+    L->P = bestP;
   } else {
     // split count of the row reduction in the weight-gradient kernels
     size_t tiles = 0;
@@ -180,7 +194,14 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       // chunk partials of the two-stage column reductions (bias sums, output-layer gradient)
       size_t len = (size_t)(m->dims[m->n_layers - 1] + 1) * C;
       for (int l = 0; l < m->n_layers; ++l) len = std::max(len, (size_t)m->dims[l + 1]);
-      L->red = cv.take(4 * len * (size_t)(L->rows_cap / 64));
+      // the fused output-layer kernel keeps R input rows in shared memory
+      const int inl = m->dims[m->n_layers - 1];
+      L->fused_R = 0;
+      if (L->path[m->n_layers - 1] == PATH_NARROW && inl % 8 == 0)
+        for (int R : {32, 16, 8})     // (rows, transposed weights in fp32 or storage type, stored weights, deltas)
+          if ((size_t)R * inl * L->esz + (size_t)C * (inl + 8) * 4 + (size_t)(inl + 1) * C * L->esz + 64 +
+                  (size_t)R * 64 <= 100 * 1024) { L->fused_R = R; break; }
+      L->red = cv.take(4 * len * (size_t)(L->rows_cap / (L->fused_R ? L->fused_R : 64)));
     }
     L->ones = L->any_tc ? cv.take(2 * 64 * (size_t)L->rows_cap) : 0;
     for (int l = 0; l <= m->n_layers; ++l) L->bits[l] = 0;
@@ -315,11 +336,11 @@ bool make_w_map(CUtensorMap* map, const void* base, int in, int out, int slots, 
   return make_map(map, base, 3, dims, strides, box);
 }
 
-// fp32 gradient block of one layer inside the partial-sum buffers: (out, in, P), 32 x 128 boxes
+// fp32 gradient block of one layer inside the partial-sum buffers: (out, in, P), 32 x 32 boxes
 bool make_g_map(CUtensorMap* map, const void* base, int in, int out, int P, size_t slot_stride) {
   const cuuint64_t dims[3] = {(cuuint64_t)out, (cuuint64_t)in, (cuuint64_t)P};
   const cuuint64_t strides[2] = {(cuuint64_t)out * 4, (cuuint64_t)slot_stride * 4};
-  const cuuint32_t box[3] = {32, 128, 1};
+  const cuuint32_t box[3] = {32, 32, 1};
   return make_map(map, base, 3, dims, strides, box, CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
 }
 
@@ -364,12 +385,12 @@ int setup_tc(abs_ctx* ctx) {
               make_w_map(&t.fwd_b, wbase, in, out, ctx->S + 1, L.d_pad, 64) &&
               make_act_map(&t.wg_a, act_in, in, L.rows_cap, 64) &&
               make_act_map(&t.wg_b, delta_out, out, L.rows_cap, 64) &&
-              make_act_map(&t.fwd_out, ctx->at<void>(L.act[l + 1]), out, L.rows_cap, 128) &&
+              make_act_map(&t.fwd_out, ctx->at<void>(L.act[l + 1]), out, L.rows_cap, 32) &&
               make_g_map(&t.wg_out, ctx->at<float>(L.G) + L.w_off[l], in, out, L.P, L.d_pad);
     if (ok && l > 0)
       ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
            make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l]) &&
-           make_act_map(&t.dg_out, ctx->at<void>(L.delta[l]), in, L.rows_cap, 128);
+           make_act_map(&t.dg_out, ctx->at<void>(L.delta[l]), in, L.rows_cap, 32);
     if (!ok) return fail(ABS_ECUDA, "cuTensorMapEncodeTiled failed for layer %d", l);
   }
   return ABS_OK;
@@ -445,7 +466,26 @@ void enqueue_gradient(abs_ctx* ctx) {
       launch_tc_bn(ctx, bn, ABS_KC_FWD, ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
-      if (a.in % 8 == 0) {
+      if (L.fused_R) {
+        const int R = L.fused_R;
+        const size_t sm = sizeof(T) * ((size_t)R * a.in + (size_t)a.C * (a.in + 8) + (size_t)(a.in + 1) * a.C) + 64 +
+                          sizeof(float) * (size_t)R * NARROW_MAX_C;
+        float* part = ctx->at<float>(L.red);
+        float* dstw = ctx->at<float>(L.G) + L.w_off[l];
+        const int len = (a.in + 1) * a.C, has_dgrad = l > 0 ? 1 : 0;
+        if (a.C == 10) {
+          const size_t smc = sizeof(T) * ((size_t)R * a.in + (size_t)(a.in + 1) * 10) + 32 +
+                             sizeof(float) * ((size_t)10 * (a.in + 4) + (size_t)R * 10);
+          launch_k(ctx, ABS_KC_OUTPUT, [&] {
+            narrow_fused_cc_kernel<T, 10><<<L.rows_cap / R, 256, smc, s>>>(a, part, R, has_dgrad);
+          });
+        } else {
+          launch_k(ctx, ABS_KC_OUTPUT, [&] {
+            narrow_fused_kernel<T><<<L.rows_cap / R, 256, sm, s>>>(a, part, R, has_dgrad);
+          });
+        }
+        launch_k(ctx, ABS_KC_OUTPUT, [&] { chunk_reduce_kernel<<<(len + 31) / 32, 256, 0, s>>>(st, part, len, dstw, R); });
+      } else if (a.in % 8 == 0) {
         const size_t sm = sizeof(T) * (size_t)a.in * a.C + sizeof(float) * a.C;
         launch_k(ctx, ABS_KC_OUTPUT, [&] {
           narrow_fwd_loss_v8_kernel<T><<<L.rows_cap / NARROW_ROWS, 256, sm, s>>>(a);
@@ -487,6 +527,8 @@ void enqueue_gradient(abs_ctx* ctx) {
       const int bn = L.bn_wg[l];
       launch_tc_bn(ctx, bn, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
                    ((la[l].in + 127) / 128 + 1) * ((la[l].out + bn - 1) / bn) * L.P);
+    } else if (L.path[l] == PATH_NARROW && L.fused_R) {
+      // forward, loss, delta of the layer below and the gradient were all done by the fused kernel
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (l > 0) {
@@ -505,7 +547,7 @@ void enqueue_gradient(abs_ctx* ctx) {
       float* dstw = ctx->at<float>(L.G) + L.w_off[l];
       const int len = (a.in + 1) * a.C;
       launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_wgrad_chunk_kernel<T><<<L.rows_cap / 64, 256, 0, s>>>(a, part); });
-      launch_k(ctx, ABS_KC_OUTPUT, [&] { chunk_reduce_kernel<<<(len + 31) / 32, 256, 0, s>>>(st, part, len, dstw); });
+      launch_k(ctx, ABS_KC_OUTPUT, [&] { chunk_reduce_kernel<<<(len + 31) / 32, 256, 0, s>>>(st, part, len, dstw, 64); });
     } else {
       const bool last = l == nl - 1;
       if (l > 0) {
@@ -662,6 +704,16 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     const cudaError_t ea = cudaFuncSetAttribute(abs_ctl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 (int)sizeof(CtlShared));
     if (ea != cudaSuccess) return bail(cuda_fail(nullptr, ea, "cudaFuncSetAttribute(abs_ctl_kernel)"));
+  }
+  if (L.fused_R) {
+    cudaError_t ef = cudaFuncSetAttribute(narrow_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (ef == cudaSuccess)
+      ef = cudaFuncSetAttribute(narrow_fused_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (ef == cudaSuccess)
+      ef = cudaFuncSetAttribute(narrow_fused_cc_kernel<float, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (ef == cudaSuccess)
+      ef = cudaFuncSetAttribute(narrow_fused_cc_kernel<__nv_bfloat16, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (ef != cudaSuccess) return bail(cuda_fail(nullptr, ef, "cudaFuncSetAttribute(narrow_fused_kernel)"));
   }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);

@@ -499,10 +499,11 @@ __global__ void __launch_bounds__(256) colsum_chunk_kernel(const DevState* st, c
 
 // Stage 2: dst[i] = sum over the active chunks q of part[q][i], i < len.  Block = 32 outputs x 8
 // chunk lanes; lane w adds chunks w, w+8, ... in order, then the 8 lanes are added in order.
-__global__ void __launch_bounds__(256) chunk_reduce_kernel(const DevState* st, const float* part, int len, float* dst) {
+__global__ void __launch_bounds__(256) chunk_reduce_kernel(const DevState* st, const float* part, int len, float* dst,
+                                                           int chunk_rows) {
   __shared__ float red[8][33];
   if (st->status != ST_OK) return;
-  const int n_chunks = st->n_rows / 64;
+  const int n_chunks = st->n_rows / chunk_rows;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int i = blockIdx.x * 32 + lane;
   float acc = 0.f;
@@ -517,6 +518,351 @@ __global__ void __launch_bounds__(256) chunk_reduce_kernel(const DevState* st, c
 #pragma unroll
     for (int q = 0; q < 8; ++q) tot += red[q][lane];
     dst[i] = tot;
+  }
+}
+
+__device__ __forceinline__ void copy8(__nv_bfloat16* dst, const __nv_bfloat16* src) {
+  *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+}
+__device__ __forceinline__ void copy8(float* dst, const float* src) {
+  reinterpret_cast<float4*>(dst)[0] = reinterpret_cast<const float4*>(src)[0];
+  reinterpret_cast<float4*>(dst)[1] = reinterpret_cast<const float4*>(src)[1];
+}
+__device__ __forceinline__ void zero8(__nv_bfloat16* dst) { *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u); }
+__device__ __forceinline__ void zero8(float* dst) {
+  reinterpret_cast<float4*>(dst)[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+  reinterpret_cast<float4*>(dst)[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+__device__ __forceinline__ float round_store(float x, const __nv_bfloat16*) { return __bfloat162float(__float2bfloat16_rn(x)); }
+__device__ __forceinline__ float round_store(float x, const float*) { return x; }
+
+// The whole output layer in one pass over R rows per block (R rows of the layer's input stay in
+// shared memory): logits, soft-max cross-entropy loss and delta (Eq. 2 at the rows' model
+// version), the back-propagated delta of the layer below, and this block's share of the layer's
+// weight and bias gradient (part[block][m][c], row m = `in` the bias sums; stage 2 adds the blocks
+// up in order).  Feature count a multiple of 8, at most 16 classes.
+template <typename T>
+__global__ void __launch_bounds__(256) narrow_fused_kernel(NarrowArgs a, float* part, int R, int has_dgrad) {
+  extern __shared__ __align__(16) unsigned char nsm_raw[];
+  DevState* st = a.st;
+  if (st->status != ST_OK) return;
+  const int r0 = blockIdx.x * R;
+  if (r0 >= st->n_rows) return;
+  const int in = a.in, C = a.C, nvec = in >> 3;
+  const int wld = in + 8;                                      // padded row of the transposed weights
+  T* hs = reinterpret_cast<T*>(nsm_raw);                       // [R][in] input rows
+  T* wT = hs + (size_t)R * in;                                 // [C][in + 8] weights, transposed
+  T* wraw = wT + (size_t)C * wld;                              // [in][C] + bias[C] as stored
+  float* d3 = reinterpret_cast<float*>(wraw + (size_t)(in + 1) * C + 8);  // [R][16] deltas of this layer's output
+  d3 = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(d3) + 15) & ~(uintptr_t)15);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const T* src = (const T*)a.act_in;
+  // asynchronous 16-byte copies: every thread issues all of its copies before anyone waits
+  constexpr int PIECES = sizeof(T) * 8 / 16;                   // 16-byte pieces per 8 elements
+  for (int item = tid; item < R * nvec; item += 256) {
+    const int rr = item / nvec, v = item - rr * nvec;
+    long long row = r0 + rr;
+    if (a.gather) row = a.row_idx[r0 + rr];
+    T* d = hs + (size_t)rr * in + v * 8;
+    if (row < 0) zero8(d);
+    else {
+      const T* g = src + (size_t)row * in + v * 8;
+#pragma unroll
+      for (int q = 0; q < PIECES; ++q)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(
+                         reinterpret_cast<unsigned char*>(d) + 16 * q)), "l"(reinterpret_cast<const unsigned char*>(g) + 16 * q) : "memory");
+    }
+  }
+  const int slot = a.tile_slot[r0 / st->RB];
+  const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
+  {
+    // weights + bias are contiguous and start on a 128-byte boundary; copy whole 16-byte pieces
+    const int n16 = (int)(((size_t)(in + 1) * C * sizeof(T) + 15) / 16);
+    for (int i = tid; i < n16; i += 256)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(
+                       reinterpret_cast<unsigned char*>(wraw) + 16 * i)), "l"(reinterpret_cast<const unsigned char*>(Wm) + 16 * i) : "memory");
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  for (int i = tid; i < in * C; i += 256) {
+    const int k = i / C, c = i - k * C;
+    wT[(size_t)c * wld + k] = wraw[i];
+  }
+  const T* bias = wraw + (size_t)in * C;
+  __syncthreads();
+  // ---- logits, loss, delta: one warp per row
+  bool bad = false;
+  for (int rr = warp; rr < R; rr += 8) {
+    const int r = r0 + rr;
+    const int s = a.row_idx[r];
+    if (s < 0) {                                // padding row: contributes nothing to Eq. 3
+      if (lane < NARROW_MAX_C) d3[rr * NARROW_MAX_C + lane] = 0.f;
+      if (lane == 0) a.row_loss[r] = 0.f;
+      continue;
+    }
+    const T* x = hs + (size_t)rr * in;
+    float acc[NARROW_MAX_C];
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c) acc[c] = 0.f;
+    for (int v = lane; v < nvec; v += 32) {
+      float xv[8];
+      load8(x + v * 8, xv);
+#pragma unroll
+      for (int c = 0; c < NARROW_MAX_C; ++c)
+        if (c < C) {
+          float wv[8];
+          load8(wT + (size_t)c * wld + v * 8, wv);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[c] = fmaf(xv[j], wv[j], acc[c]);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+        acc[c] += ldf(bias, c);
+      }
+    const int y = a.labels[s];
+    float zmax = acc[0], zy = 0.f;
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) { zmax = fmaxf(zmax, acc[c]); if (c == y) zy = acc[c]; }
+    float se = 0.f;
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) { acc[c] = expf(acc[c] - zmax); se += acc[c]; }
+    const float inv = 1.f / se;
+    float mine = 0.f;
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c == lane) mine = acc[c] * inv - (c == y ? 1.f : 0.f);
+    // the delta is a stored quantity: round it to the storage type like every other delta
+    if (lane < NARROW_MAX_C) d3[rr * NARROW_MAX_C + lane] = lane < C ? round_store(mine, (const T*)nullptr) : 0.f;
+    const float loss = logf(se) - (zy - zmax);
+    if (lane == 0) a.row_loss[r] = loss;
+    bad |= !isfinite(loss);
+  }
+  if (bad && lane == 0) st->diverged = 1;
+  __syncthreads();
+  // ---- delta of the layer below: (delta W^T) masked by the ReLU of the input rows
+  if (has_dgrad) {
+    T* out = (T*)a.delta_in;
+    for (int item = tid; item < R * nvec; item += 256) {
+      const int rr = item / nvec, v = item - rr * nvec;
+      float hv[8], acc[8];
+      load8(hs + (size_t)rr * in + v * 8, hv);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+#pragma unroll
+      for (int c = 0; c < NARROW_MAX_C; ++c)
+        if (c < C) {
+          float wv[8];
+          load8(wT + (size_t)c * wld + v * 8, wv);
+          const float dv = d3[rr * NARROW_MAX_C + c];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[j] = fmaf(dv, wv[j], acc[j]);
+        }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] = hv[j] > 0.f ? acc[j] : 0.f;
+      store8(out + (size_t)(r0 + rr) * in + (size_t)v * 8, acc);
+    }
+  }
+  // ---- this block's share of the weight and bias gradient
+  float* dst = part + (size_t)blockIdx.x * (size_t)(in + 1) * C;
+  for (int it = tid; it < in / 2; it += 256) {
+    const int m = 2 * it;
+    float acc0[NARROW_MAX_C], acc1[NARROW_MAX_C];
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c) { acc0[c] = 0.f; acc1[c] = 0.f; }
+    for (int rr = 0; rr < R; ++rr) {
+      float x0, x1;
+      load2(hs + (size_t)rr * in + m, x0, x1);
+#pragma unroll
+      for (int c = 0; c < NARROW_MAX_C; ++c)
+        if (c < C) {
+          const float dv = d3[rr * NARROW_MAX_C + c];
+          acc0[c] = fmaf(x0, dv, acc0[c]);
+          acc1[c] = fmaf(x1, dv, acc1[c]);
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < NARROW_MAX_C; ++c)
+      if (c < C) { dst[(size_t)m * C + c] = acc0[c]; dst[(size_t)(m + 1) * C + c] = acc1[c]; }
+  }
+  if (tid < C) {
+    float tot = 0.f;
+    for (int rr = 0; rr < R; ++rr) tot += d3[rr * NARROW_MAX_C + tid];
+    dst[(size_t)in * C + tid] = tot;
+  }
+}
+
+// Same operation as narrow_fused_kernel with the class count CC known at compile time: weights are
+// kept as fp32 in shared memory, every weight fetched from shared memory is used for four rows
+// (forward) or stays in registers for all rows of the block (delta of the layer below).
+template <typename T, int CC>
+__global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, float* part, int R, int has_dgrad) {
+  extern __shared__ __align__(16) unsigned char nsm_raw[];
+  DevState* st = a.st;
+  if (st->status != ST_OK) return;
+  const int r0 = blockIdx.x * R;
+  if (r0 >= st->n_rows) return;
+  const int in = a.in, nvec = in >> 3;
+  const int wld = in + 4;                                      // padded row of the transposed fp32 weights
+  T* hs = reinterpret_cast<T*>(nsm_raw);                       // [R][in] input rows
+  float* wf = reinterpret_cast<float*>(hs + (size_t)R * in);   // [CC][in + 4]
+  float* d3 = wf + (size_t)CC * wld;                           // [R][CC] deltas of this layer's output
+  T* wraw = reinterpret_cast<T*>(d3 + (size_t)R * CC);         // [in][CC] + bias[CC] as stored (16-byte aligned)
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const T* src = (const T*)a.act_in;
+  constexpr int PIECES = sizeof(T) * 8 / 16;
+  for (int item = tid; item < R * nvec; item += 256) {
+    const int rr = item / nvec, v = item - rr * nvec;
+    long long row = r0 + rr;
+    if (a.gather) row = a.row_idx[r0 + rr];
+    T* d = hs + (size_t)rr * in + v * 8;
+    if (row < 0) zero8(d);
+    else {
+      const T* g = src + (size_t)row * in + v * 8;
+#pragma unroll
+      for (int q = 0; q < PIECES; ++q)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(
+                         reinterpret_cast<unsigned char*>(d) + 16 * q)), "l"(reinterpret_cast<const unsigned char*>(g) + 16 * q) : "memory");
+    }
+  }
+  const int slot = a.tile_slot[r0 / st->RB];
+  const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
+  {
+    const int n16 = (int)(((size_t)(in + 1) * CC * sizeof(T) + 15) / 16);
+    for (int i = tid; i < n16; i += 256)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(
+                       reinterpret_cast<unsigned char*>(wraw) + 16 * i)), "l"(reinterpret_cast<const unsigned char*>(Wm) + 16 * i) : "memory");
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  for (int i = tid; i < in * CC; i += 256) {
+    const int k = i / CC, c = i - k * CC;
+    wf[(size_t)c * wld + k] = ldf(wraw, i);
+  }
+  __syncthreads();
+  // ---- logits, loss, delta: a warp takes four rows at a time
+  bool bad = false;
+  for (int rb = warp * 4; rb < R; rb += 32) {
+    float acc[4][CC];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+      for (int c = 0; c < CC; ++c) acc[q][c] = 0.f;
+    for (int v = lane; v < nvec; v += 32) {
+      float xv[4][8];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) load8(hs + (size_t)(rb + q) * in + v * 8, xv[q]);
+#pragma unroll
+      for (int c = 0; c < CC; ++c) {
+        float wv[8];
+        load8(wf + (size_t)c * wld + v * 8, wv);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[q][c] = fmaf(xv[q][j], wv[j], acc[q][c]);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+      for (int c = 0; c < CC; ++c)
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc[q][c] += __shfl_xor_sync(0xffffffffu, acc[q][c], o);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int rr = rb + q, r = r0 + rr;
+      const int s = a.row_idx[r];
+      if (s < 0) {                              // padding row: contributes nothing to Eq. 3
+        if (lane < CC) d3[rr * CC + lane] = 0.f;
+        if (lane == 0) a.row_loss[r] = 0.f;
+        continue;
+      }
+      const int y = a.labels[s];
+      float z[CC];
+      float zmax = -3.0e38f, zy = 0.f;
+#pragma unroll
+      for (int c = 0; c < CC; ++c) {
+        z[c] = acc[q][c] + ldf(wraw, (size_t)in * CC + c);
+        zmax = fmaxf(zmax, z[c]);
+        if (c == y) zy = z[c];
+      }
+      float se = 0.f;
+#pragma unroll
+      for (int c = 0; c < CC; ++c) { z[c] = expf(z[c] - zmax); se += z[c]; }
+      const float inv = 1.f / se;
+      float mine = 0.f;
+#pragma unroll
+      for (int c = 0; c < CC; ++c)
+        if (c == lane) mine = z[c] * inv - (c == y ? 1.f : 0.f);
+      // the delta is a stored quantity: round it to the storage type like every other delta
+      if (lane < CC) d3[rr * CC + lane] = round_store(mine, (const T*)nullptr);
+      const float loss = logf(se) - (zy - zmax);
+      if (lane == 0) a.row_loss[r] = loss;
+      bad |= !isfinite(loss);
+    }
+  }
+  if (bad && lane == 0) st->diverged = 1;
+  __syncthreads();
+  // ---- delta of the layer below: a thread keeps the weights of 8 features in registers
+  if (has_dgrad) {
+    T* out = (T*)a.delta_in;
+    int per = 1;
+    while (per < nvec && per < 256) per <<= 1;
+    const int nrl = 256 / per, rl = tid / per;
+    for (int v0 = 0; v0 < nvec; v0 += per) {
+      const int v = v0 + tid % per;
+      if (v < nvec) {
+        float wr[CC][8];
+#pragma unroll
+        for (int c = 0; c < CC; ++c) load8(wf + (size_t)c * wld + v * 8, wr[c]);
+        for (int rr = rl; rr < R; rr += nrl) {
+          float hv[8], acc8[8];
+          load8(hs + (size_t)rr * in + v * 8, hv);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc8[j] = 0.f;
+#pragma unroll
+          for (int c = 0; c < CC; ++c) {
+            const float dv = d3[rr * CC + c];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc8[j] = fmaf(dv, wr[c][j], acc8[j]);
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc8[j] = hv[j] > 0.f ? acc8[j] : 0.f;
+          store8(out + (size_t)(r0 + rr) * in + (size_t)v * 8, acc8);
+        }
+      }
+    }
+  }
+  // ---- this block's share of the weight and bias gradient
+  float* dst = part + (size_t)blockIdx.x * (size_t)(in + 1) * CC;
+  for (int it = tid; it < in / 2; it += 256) {
+    const int m = 2 * it;
+    float acc0[CC], acc1[CC];
+#pragma unroll
+    for (int c = 0; c < CC; ++c) { acc0[c] = 0.f; acc1[c] = 0.f; }
+#pragma unroll 4
+    for (int rr = 0; rr < R; ++rr) {
+      float x0, x1;
+      load2(hs + (size_t)rr * in + m, x0, x1);
+#pragma unroll
+      for (int c = 0; c < CC; ++c) {
+        const float dv = d3[rr * CC + c];
+        acc0[c] = fmaf(x0, dv, acc0[c]);
+        acc1[c] = fmaf(x1, dv, acc1[c]);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < CC; ++c) { dst[(size_t)m * CC + c] = acc0[c]; dst[(size_t)(m + 1) * CC + c] = acc1[c]; }
+  }
+  if (tid < CC) {
+    float tot = 0.f;
+    for (int rr = 0; rr < R; ++rr) tot += d3[rr * CC + tid];
+    dst[(size_t)in * CC + tid] = tot;
   }
 }
 

@@ -141,9 +141,9 @@ template <int BN> struct Cfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int OUT_BYTES = 128 * 128;          // staging box of the epilogue
+  static constexpr int OUT_BYTES = 2 * 4 * 4096;       // epilogue staging: 2 buffers x 4 warps x (32 rows x 128 B)
   static constexpr size_t SMEM_BYTES =
-      (size_t)STAGES * STAGE_BYTES + OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 2 * BN * 4 /*bias*/;
+      (size_t)STAGES * STAGE_BYTES + OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 2 * BN * 2 /*bias*/;
 };
 
 struct TileCoord { int a_row, b_col, slot, k_begin, n_kb, split, bias_tile; };
@@ -180,7 +180,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   uint64_t* acc_empty = acc_full + 2;        // [2] accumulator drained by the epilogue
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* bias_s = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [2][BN]
+  __nv_bfloat16* bias_s = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [2][BN]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -314,14 +314,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else {
     // ------------------------------------------------------------------ epilogue (4 warps)
-    // Results leave through a 16 KB staging box (128 rows x 128 bytes, 128-byte swizzle) and one
-    // bulk tensor store per box, so global memory sees whole rows instead of 32 scattered 16-byte
-    // pieces per store instruction.
+    // Results leave through per-warp staging boxes (32 rows x 128 bytes, 128-byte swizzle, two
+    // per warp) and one bulk tensor store per box, so global memory sees whole rows instead of 32
+    // scattered 16-byte pieces per store instruction and a warp never waits for another warp.
     const int q = warp & 3;                    // tensor-memory lane quarter this warp may read
     const int row_in_tile = q * 32 + lane;
-    const bool issuer = threadIdx.x == 64;     // the thread that issues and tracks the bulk stores
-    uint8_t* my_row = stage_out + row_in_tile * 128;
-    const int sw = row_in_tile & 7;
+    const bool issuer = lane == 0;             // issues and tracks this warp's bulk stores
+    const int sw = lane & 7;
+    int box_no = 0;
     const int box_cols = (mode == WGRAD) ? 32 : 64;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -332,12 +332,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int r = (mode == WGRAD && c.bias_tile) ? (p.M_total - 1) + row_in_tile : c.a_row + row_in_tile;
       // fetch what the epilogue needs from global memory before waiting for the accumulator
       uint32_t mw[BN / 32];
-      float* bias_t = bias_s + acc * BN;
+      __nv_bfloat16* bias_t = bias_s + acc * BN;
       if (mode == FWD) {
         const __nv_bfloat16* bias = p.ring + (size_t)c.slot * p.slot_stride + p.b_off;
         for (int i = (int)threadIdx.x - 64; i < BN; i += 128) {
           const int n = c.b_col + i;
-          bias_t[i] = n < p.N_total ? __bfloat162float(bias[n]) : 0.f;
+          bias_t[i] = n < p.N_total ? bias[n] : __float2bfloat16_rn(0.f);
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
       } else if (mode == DGRAD) {
@@ -365,9 +365,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int c0 = 0; c0 < BN; c0 += box_cols) {
         const int n0 = c.b_col + c0;
         if (n0 >= p.N_total) break;            // uniform in the CTA
-        // the staging box is free once the previous bulk store has read it
-        if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        // this warp's staging box is free once its store before the previous one has been read
+        uint8_t* my_box = stage_out + (((box_no & 1) * 4 + q) << 12);
+        uint8_t* my_row = my_box + lane * 128;
+        ++box_no;
+        if (issuer) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        __syncwarp();
         uint32_t v[32];
         if (mode == WGRAD) {
           if (have) tmem_ld32(t_row + (uint32_t)c0, v);
@@ -413,8 +416,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int i = 8 * j + 2 * e;
                 float x = __uint_as_float(v[i]), y = __uint_as_float(v[i + 1]);
                 if (mode == FWD) {
-                  x = fmaxf(x + bias_t[cc + i], 0.f);
-                  y = fmaxf(y + bias_t[cc + i + 1], 0.f);
+                  const float2 bf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(bias_t + cc + i));
+                  x = fmaxf(x + bf.x, 0.f);
+                  y = fmaxf(y + bf.y, 0.f);
                 } else {
                   x = ((bits >> i) & 1u) ? x : 0.f;
                   y = ((bits >> (i + 1)) & 1u) ? y : 0.f;
@@ -432,15 +436,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        __syncwarp();
         if (issuer && !(mode == WGRAD && c.bias_tile)) {
           if (mode == WGRAD)
             asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
-                         ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(smem_u32(stage_out)), "r"(n0), "r"(c.a_row), "r"(c.split)
+                         ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(smem_u32(my_box)), "r"(n0), "r"(c.a_row + q * 32), "r"(c.split)
                          : "memory");
           else
             asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                         ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(smem_u32(stage_out)), "r"(n0), "r"(c.a_row)
+                         ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(smem_u32(my_box)), "r"(n0), "r"(c.a_row + q * 32)
                          : "memory");
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
