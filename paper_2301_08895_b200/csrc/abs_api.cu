@@ -259,6 +259,7 @@ struct abs_ctx {
   int rounds_enqueued = 0;
   int sticky = ABS_OK;
   long long launches = 0;
+  cudaError_t launch_error = cudaSuccess;
   CtlArgs ctl;
   TcLayer tcl[ABS_MAX_LAYERS];
   CUtensorMap ones_map;
@@ -282,12 +283,26 @@ int cuda_fail(abs_ctx* ctx, cudaError_t e, const char* what) {
     if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);       \
   } while (0)
 
-// Runs `launch` (one kernel launch on ctx->stream), counted and, while profiling, bracketed by events.
-template <class F>
-void launch_k(abs_ctx* ctx, int cls, F launch) {
+// One kernel launch on ctx->stream, counted and, while profiling, bracketed by events.  Launches
+// carry the programmatic-stream-serialization attribute: the next kernel's CTAs may be scheduled
+// while this one drains; every kernel of the round loop starts with griddepcontrol.wait, which
+// returns once the kernel before it has completed and its writes are visible.
+template <typename... KArgs, typename... Args>
+void launch_ex(abs_ctx* ctx, int cls, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
   const bool rec = (int)ctx->ev_class.size() < ctx->ev_cap;
   if (rec) cudaEventRecord(ctx->ev[2 * ctx->ev_class.size()], ctx->stream);
-  launch();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = ctx->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+  if (e != cudaSuccess && ctx->launch_error == cudaSuccess) ctx->launch_error = e;
   if (rec) {
     cudaEventRecord(ctx->ev[2 * ctx->ev_class.size() + 1], ctx->stream);
     ctx->ev_class.push_back(cls);
@@ -348,9 +363,7 @@ template <int BN>
 void launch_tc(abs_ctx* ctx, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
                const tc::Params& p, int max_tiles) {
   const int grid = std::max(1, std::min(ctx->sm_count, max_tiles));
-  launch_k(ctx, cls, [&] {
-    tc::tc_gemm_kernel<BN><<<grid, tc::THREADS, tc::Cfg<BN>::SMEM_BYTES, ctx->stream>>>(a, b, ctx->ones_map, o, p);
-  });
+  launch_ex(ctx, cls, tc::tc_gemm_kernel<BN>, dim3(grid), dim3(tc::THREADS), tc::Cfg<BN>::SMEM_BYTES, a, b, ctx->ones_map, o, p);
 }
 
 void launch_tc_bn(abs_ctx* ctx, int bn, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
@@ -408,7 +421,7 @@ void enqueue_gradient(abs_ctx* ctx) {
     a.X = ctx->X; a.y = (const float*)ctx->y;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad;
     a.loss = ctx->ctl.loss; a.G = ctx->at<float>(L.G); a.d = m.dims[0];
-    launch_k(ctx, ABS_KC_LSQ, [&] { lsq_grad_kernel<T><<<ctx->W, 256, 0, s>>>(a); });
+    launch_ex(ctx, ABS_KC_LSQ, lsq_grad_kernel<T>, dim3(ctx->W), dim3(256), 0, a);
     return;
   }
   const int nl = m.n_layers;
@@ -448,10 +461,7 @@ void enqueue_gradient(abs_ctx* ctx) {
     return a;
   };
   if (gathered) {
-    launch_k(ctx, ABS_KC_GATHER, [&] {
-      gather_rows_kernel<<<ctx->sm_count * 8, 256, 0, s>>>(st, ctx->ctl.row_idx, (const __nv_bfloat16*)ctx->X,
-                                                           ctx->at<__nv_bfloat16>(L.act[0]), m.dims[0]);
-    });
+    launch_ex(ctx, ABS_KC_GATHER, gather_rows_kernel, dim3(ctx->sm_count * 8), dim3(256), 0, st, ctx->ctl.row_idx, (const __nv_bfloat16*)ctx->X, ctx->at<__nv_bfloat16>(L.act[0]), m.dims[0]);
   }
   // ---- forward (Eq. 2 at the model version each worker holds)
   for (int l = 0; l < nl; ++l) {
@@ -476,35 +486,29 @@ void enqueue_gradient(abs_ctx* ctx) {
         if (a.C == 10) {
           const size_t smc = sizeof(T) * ((size_t)R * a.in + (size_t)(a.in + 1) * 10) + 32 +
                              sizeof(float) * ((size_t)10 * (a.in + 4) + (size_t)R * 10);
-          launch_k(ctx, ABS_KC_OUTPUT, [&] {
-            narrow_fused_cc_kernel<T, 10><<<L.rows_cap / R, 256, smc, s>>>(a, part, R, has_dgrad);
-          });
+          launch_ex(ctx, ABS_KC_OUTPUT, narrow_fused_cc_kernel<T, 10>, dim3(L.rows_cap / R), dim3(256), smc, a, part, R, has_dgrad);
         } else {
-          launch_k(ctx, ABS_KC_OUTPUT, [&] {
-            narrow_fused_kernel<T><<<L.rows_cap / R, 256, sm, s>>>(a, part, R, has_dgrad);
-          });
+          launch_ex(ctx, ABS_KC_OUTPUT, narrow_fused_kernel<T>, dim3(L.rows_cap / R), dim3(256), sm, a, part, R, has_dgrad);
         }
-        launch_k(ctx, ABS_KC_OUTPUT, [&] { chunk_reduce_kernel<<<(len + 31) / 32, 256, 0, s>>>(st, part, len, dstw, R); });
+        launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, part, len, dstw, R);
       } else if (a.in % 8 == 0) {
         const size_t sm = sizeof(T) * (size_t)a.in * a.C + sizeof(float) * a.C;
-        launch_k(ctx, ABS_KC_OUTPUT, [&] {
-          narrow_fwd_loss_v8_kernel<T><<<L.rows_cap / NARROW_ROWS, 256, sm, s>>>(a);
-        });
+        launch_ex(ctx, ABS_KC_OUTPUT, narrow_fwd_loss_v8_kernel<T>, dim3(L.rows_cap / NARROW_ROWS), dim3(256), sm, a);
       } else {
         const size_t sm = sizeof(float) * ((size_t)a.in * a.C + a.C);
-        launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_fwd_loss_kernel<T><<<row_tiles, 256, sm, s>>>(a); });
+        launch_ex(ctx, ABS_KC_OUTPUT, narrow_fwd_loss_kernel<T>, dim3(row_tiles), dim3(256), sm, a);
       }
     } else {
       dim3 grid((la[l].out + TN - 1) / TN, row_tiles);
       const int cls = last ? ABS_KC_OUTPUT : ABS_KC_FWD;
-      if (last) launch_k(ctx, cls, [&] { simt_fwd_kernel<T, true><<<grid, 256, 0, s>>>(la[l]); });
-      else launch_k(ctx, cls, [&] { simt_fwd_kernel<T, false><<<grid, 256, 0, s>>>(la[l]); });
+      if (last) launch_ex(ctx, cls, simt_fwd_kernel<T, true>, dim3(grid), dim3(256), 0, la[l]);
+      else launch_ex(ctx, cls, simt_fwd_kernel<T, false>, dim3(grid), dim3(256), 0, la[l]);
       if (last) {
         LossArgs lo;
         lo.st = st; lo.row_idx = ctx->ctl.row_idx; lo.labels = (const int*)ctx->y;
         lo.logits = ctx->at<float>(L.logits); lo.delta = ctx->at<void>(L.delta[nl]);
         lo.row_loss = ctx->ctl.row_loss; lo.C = m.dims[nl];
-        launch_k(ctx, ABS_KC_OUTPUT, [&] { net_loss_kernel<T><<<(L.rows_cap + 255) / 256, 256, 0, s>>>(lo); });
+        launch_ex(ctx, ABS_KC_OUTPUT, net_loss_kernel<T>, dim3((L.rows_cap + 255) / 256), dim3(256), 0, lo);
       }
     }
   }
@@ -534,28 +538,26 @@ void enqueue_gradient(abs_ctx* ctx) {
       if (l > 0) {
         if (a.in % 8 == 0) {
           const size_t sm = sizeof(T) * (size_t)a.in * a.C + sizeof(float) * NARROW_ROWS * a.C;
-          launch_k(ctx, ABS_KC_OUTPUT, [&] {
-            narrow_dgrad_v8_kernel<T><<<L.rows_cap / NARROW_ROWS, 256, sm, s>>>(a);
-          });
+          launch_ex(ctx, ABS_KC_OUTPUT, narrow_dgrad_v8_kernel<T>, dim3(L.rows_cap / NARROW_ROWS), dim3(256), sm, a);
         } else {
           const size_t sm = sizeof(float) * ((size_t)a.in * a.C + 64 * a.C);
-          launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_dgrad_kernel<T><<<row_tiles, 256, sm, s>>>(a); });
+          launch_ex(ctx, ABS_KC_OUTPUT, narrow_dgrad_kernel<T>, dim3(row_tiles), dim3(256), sm, a);
         }
       }
       // weight gradient: per-chunk partial sums, then one ordered sum over the chunks into partial 0
       float* part = ctx->at<float>(L.red);
       float* dstw = ctx->at<float>(L.G) + L.w_off[l];
       const int len = (a.in + 1) * a.C;
-      launch_k(ctx, ABS_KC_OUTPUT, [&] { narrow_wgrad_chunk_kernel<T><<<L.rows_cap / 64, 256, 0, s>>>(a, part); });
-      launch_k(ctx, ABS_KC_OUTPUT, [&] { chunk_reduce_kernel<<<(len + 31) / 32, 256, 0, s>>>(st, part, len, dstw, 64); });
+      launch_ex(ctx, ABS_KC_OUTPUT, narrow_wgrad_chunk_kernel<T>, dim3(L.rows_cap / 64), dim3(256), 0, a, part);
+      launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, part, len, dstw, 64);
     } else {
       const bool last = l == nl - 1;
       if (l > 0) {
         dim3 grid((la[l].in + TN - 1) / TN, row_tiles);
-        launch_k(ctx, last ? ABS_KC_OUTPUT : ABS_KC_DGRAD, [&] { simt_dgrad_kernel<T><<<grid, 256, 0, s>>>(la[l]); });
+        launch_ex(ctx, last ? ABS_KC_OUTPUT : ABS_KC_DGRAD, simt_dgrad_kernel<T>, dim3(grid), dim3(256), 0, la[l]);
       }
       dim3 gridw((la[l].out + TN - 1) / TN, (la[l].in + 1 + TM - 1) / TM, L.P);
-      launch_k(ctx, last ? ABS_KC_OUTPUT : ABS_KC_WGRAD, [&] { simt_wgrad_kernel<T><<<gridw, 256, 0, s>>>(la[l]); });
+      launch_ex(ctx, last ? ABS_KC_OUTPUT : ABS_KC_WGRAD, simt_wgrad_kernel<T>, dim3(gridw), dim3(256), 0, la[l]);
     }
   }
 }
@@ -569,7 +571,7 @@ void enqueue_update(abs_ctx* ctx) {
   u.job = ctx->ctl.job; u.next_dur = ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
   const size_t n4 = L.d_pad / 4;
   const int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * 8), (size_t)(ctx->W + 31) / 32);
-  launch_k(ctx, ABS_KC_UPDATE, [&] { update_kernel<T><<<blocks, 256, 0, ctx->stream>>>(u); });
+  launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T>, dim3(blocks), dim3(256), 0, u);
 }
 
 int read_status(abs_ctx* ctx, DevState* host) {
@@ -742,13 +744,14 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
   const bool f32 = ctx->m.dtype == ABS_FP32;
   for (int r = 0; r < n; ++r) {
     // the control kernel completes the previous round (if any) and selects this round's arrivals
-    launch_k(ctx, ABS_KC_CTL, [&] { abs_ctl_kernel<<<1, 1024, sizeof(CtlShared), ctx->stream>>>(ctx->ctl, 1, 1); });
+    launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), sizeof(CtlShared), ctx->ctl, 1, 1);
     if (f32) { enqueue_gradient<float>(ctx); enqueue_update<float>(ctx); }
     else { enqueue_gradient<__nv_bfloat16>(ctx); enqueue_update<__nv_bfloat16>(ctx); }
   }
   if (n > 0) {
-    launch_k(ctx, ABS_KC_CTL, [&] { abs_ctl_kernel<<<1, 1024, sizeof(CtlShared), ctx->stream>>>(ctx->ctl, 1, 0); });
+    launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), sizeof(CtlShared), ctx->ctl, 1, 0);
   }
+  if (ctx->launch_error != cudaSuccess) return cuda_fail(ctx, ctx->launch_error, "kernel launch");
   CU(cudaGetLastError());
   ctx->rounds_enqueued += n;
   return ABS_OK;

@@ -82,6 +82,15 @@ __device__ __forceinline__ float ldf(const __nv_bfloat16* p, size_t i) { return 
 __device__ __forceinline__ void stf(float* p, size_t i, float v) { p[i] = v; }
 __device__ __forceinline__ void stf(__nv_bfloat16* p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
 
+// First statement of every kernel of the round loop.  The kernels are launched with programmatic
+// stream serialization, so a kernel's CTAs may be resident before the kernel in front of it has
+// finished: wait until that kernel has completed (its writes are then visible), then allow the
+// kernel behind this one to be scheduled early in the same way.
+__device__ __forceinline__ void grid_dependency_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __host__ __device__ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 __host__ __device__ inline size_t round_up_sz(size_t a, size_t b) { return (a + b - 1) / b * b; }
 

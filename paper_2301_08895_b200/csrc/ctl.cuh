@@ -141,6 +141,7 @@ struct CtlShared {
 // A dependent global-memory access costs this lone CTA close to a microsecond, so everything it
 // needs is loaded up front in one wave and later phases work from registers and shared memory.
 __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char ctl_smem[];
   CtlShared& sh = *reinterpret_cast<CtlShared*>(ctl_smem);
   DevState* st = a.st;

@@ -13,6 +13,7 @@ constexpr int NARROW_MAX_C = 16;
 // act0[r][:] = X[row_idx[r]][:] (zeros for padding rows); bf16, `in` a multiple of 8.
 __global__ void __launch_bounds__(256) gather_rows_kernel(const DevState* st, const int* row_idx,
                                                           const __nv_bfloat16* X, __nv_bfloat16* act0, int in) {
+  grid_dependency_sync();
   if (st->status != ST_OK) return;
   const int n_rows = st->n_rows;
   const int vec_per_row = in >> 3;
@@ -34,6 +35,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const DevState* st, co
 template <typename T>
 __global__ void __launch_bounds__(1024) colsum_kernel(const DevState* st, const T* delta, float* G, size_t slot_stride,
                                                       size_t b_off, int out, int P) {
+  grid_dependency_sync();
   __shared__ float red[32][33];
   if (st->status != ST_OK) return;
   const int n_rows = st->n_rows;
@@ -73,6 +75,7 @@ struct NarrowArgs {
 // One warp per row: lanes stride over the input features, C accumulators each.
 template <typename T>
 __global__ void __launch_bounds__(256) narrow_fwd_loss_kernel(NarrowArgs a) {
+  grid_dependency_sync();
   extern __shared__ float wsm[];               // [in][C] then bias[C]
   DevState* st = a.st;
   if (st->status != ST_OK) return;
@@ -140,6 +143,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_kernel(NarrowArgs a) {
 // delta_in[r][m] = (sum_c delta_out[r][c] W_s[m][c]) * [act_in[r][m] > 0].
 template <typename T>
 __global__ void __launch_bounds__(256) narrow_dgrad_kernel(NarrowArgs a) {
+  grid_dependency_sync();
   extern __shared__ float wsm[];               // [in][C] then delta tile [64][C]
   DevState* st = a.st;
   if (st->status != ST_OK) return;
@@ -175,6 +179,7 @@ __global__ void __launch_bounds__(256) narrow_dgrad_kernel(NarrowArgs a) {
 // Block = 32 feature lanes x 32 row lanes, fixed-order reduction over the row lanes.
 template <typename T>
 __global__ void __launch_bounds__(1024) narrow_wgrad_kernel(NarrowArgs a) {
+  grid_dependency_sync();
   __shared__ float red[32][33];
   DevState* st = a.st;
   if (st->status != ST_OK) return;
@@ -251,6 +256,7 @@ constexpr int NARROW_ROWS = 16;   // rows per block of the vectorised forward / 
 // Output layer forward + soft-max cross-entropy + delta, 16 rows per block, one warp per row pair.
 template <typename T>
 __global__ void __launch_bounds__(256) narrow_fwd_loss_v8_kernel(NarrowArgs a) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   T* wT = reinterpret_cast<T*>(nsm_raw);                 // [C][in]
   DevState* st = a.st;
@@ -331,6 +337,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_v8_kernel(NarrowArgs a) {
 // item is (row, 8 consecutive features).
 template <typename T>
 __global__ void __launch_bounds__(256) narrow_dgrad_v8_kernel(NarrowArgs a) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   T* wT = reinterpret_cast<T*>(nsm_raw);                 // [C][in]
   DevState* st = a.st;
@@ -390,6 +397,7 @@ __device__ __forceinline__ void load2(const float* p, float& x, float& y) {
 // point at adds nothing.
 template <typename T>
 __global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, float* part) {
+  grid_dependency_sync();
   __shared__ float dsm[64][NARROW_MAX_C];
   __shared__ long long rowoff[64];
   DevState* st = a.st;
@@ -451,6 +459,7 @@ __global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, f
 // delta[r][n]; `out` a multiple of 8.
 template <typename T>
 __global__ void __launch_bounds__(256) colsum_chunk_kernel(const DevState* st, const T* delta, int out, float* part) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   float* red = reinterpret_cast<float*>(nsm_raw);        // [row lanes][out]
   if (st->status != ST_OK) return;
@@ -501,6 +510,7 @@ __global__ void __launch_bounds__(256) colsum_chunk_kernel(const DevState* st, c
 // chunk lanes; lane w adds chunks w, w+8, ... in order, then the 8 lanes are added in order.
 __global__ void __launch_bounds__(256) chunk_reduce_kernel(const DevState* st, const float* part, int len, float* dst,
                                                            int chunk_rows) {
+  grid_dependency_sync();
   __shared__ float red[8][33];
   if (st->status != ST_OK) return;
   const int n_chunks = st->n_rows / chunk_rows;
@@ -543,6 +553,7 @@ __device__ __forceinline__ float round_store(float x, const float*) { return x; 
 // up in order).  Feature count a multiple of 8, at most 16 classes.
 template <typename T>
 __global__ void __launch_bounds__(256) narrow_fused_kernel(NarrowArgs a, float* part, int R, int has_dgrad) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   DevState* st = a.st;
   if (st->status != ST_OK) return;
@@ -702,6 +713,7 @@ __global__ void __launch_bounds__(256) narrow_fused_kernel(NarrowArgs a, float* 
 // (forward) or stays in registers for all rows of the block (delta of the layer below).
 template <typename T, int CC>
 __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, float* part, int R, int has_dgrad) {
+  grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   DevState* st = a.st;
   if (st->status != ST_OK) return;

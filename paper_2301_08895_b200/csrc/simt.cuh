@@ -70,6 +70,7 @@ struct LayerArgs {
 // Forward of one affine layer for all rows of the round: act_out = [relu](act_in W_s + b_s).
 template <typename T, bool LAST>
 __global__ void __launch_bounds__(256) simt_fwd_kernel(LayerArgs a) {
+  grid_dependency_sync();
   __shared__ float As[TK][TM + 4], Bs[TK][TN + 4];
   const DevState* st = a.st;
   if (st->status != ST_OK) return;
@@ -115,6 +116,7 @@ __global__ void __launch_bounds__(256) simt_fwd_kernel(LayerArgs a) {
 // delta_in[r][m] = (sum_n delta_out[r][n] W_s[m][n]) * [act_in[r][m] > 0].
 template <typename T>
 __global__ void __launch_bounds__(256) simt_dgrad_kernel(LayerArgs a) {
+  grid_dependency_sync();
   __shared__ float As[TK][TM + 4], Bs[TK][TN + 4];
   const DevState* st = a.st;
   if (st->status != ST_OK) return;
@@ -152,6 +154,7 @@ __global__ void __launch_bounds__(256) simt_dgrad_kernel(LayerArgs a) {
 // result is the bias gradient (an implicit input of ones).
 template <typename T>
 __global__ void __launch_bounds__(256) simt_wgrad_kernel(LayerArgs a) {
+  grid_dependency_sync();
   __shared__ float As[TK][TM + 4], Bs[TK][TN + 4];
   const DevState* st = a.st;
   if (st->status != ST_OK) return;
@@ -206,6 +209,7 @@ struct LossArgs {
 // delta = softmax(z) - onehot(y).  Padding rows get zero delta so they add nothing to Eq. 3.
 template <typename T>
 __global__ void __launch_bounds__(256) net_loss_kernel(LossArgs a) {
+  grid_dependency_sync();
   DevState* st = a.st;
   if (st->status != ST_OK) return;
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
@@ -246,6 +250,7 @@ struct LsqArgs {
 // model version v, loss = mean 1/2 r^2, partial gradient g = sum_b r_b x_b.
 template <typename T>
 __global__ void __launch_bounds__(256) lsq_grad_kernel(LsqArgs a) {
+  grid_dependency_sync();
   __shared__ float res[1024];
   __shared__ int sidx[1024];
   __shared__ float red[8];
@@ -319,6 +324,7 @@ struct UpdateArgs {
 // master and, in storage type, as ring slot (t+1) mod (S+1).  One pass, 16-byte accesses.
 template <typename T>
 __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
+  grid_dependency_sync();
   const DevState* st = a.st;
   if (st->status != ST_OK) return;
   if (threadIdx.x < 32) refresh_next_durations(st, a.job, a.next_dur, a.dur_job, blockIdx.x * 32 + threadIdx.x);

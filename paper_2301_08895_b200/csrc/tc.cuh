@@ -153,6 +153,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_ones, const __grid_constant__ CUtensorMap map_out,
                const Params p) {
+  grid_dependency_sync();
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   DevState* st = p.st;
