@@ -260,6 +260,8 @@ struct abs_ctx {
   int sticky = ABS_OK;
   long long launches = 0;
   cudaError_t launch_error = cudaSuccess;
+  bool lsq_v2 = false;               // least squares through the persistent 16-byte-load kernel
+  int lsq_grid = 0;                  // its grid = number of partial sums
   CtlArgs ctl;
   TcLayer tcl[ABS_MAX_LAYERS];
   CUtensorMap ones_map;
@@ -421,7 +423,8 @@ void enqueue_gradient(abs_ctx* ctx) {
     a.X = ctx->X; a.y = (const float*)ctx->y;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad;
     a.loss = ctx->ctl.loss; a.G = ctx->at<float>(L.G); a.d = m.dims[0];
-    launch_ex(ctx, ABS_KC_LSQ, lsq_grad_kernel<T>, dim3(ctx->W), dim3(256), 0, a);
+    if (ctx->lsq_v2) launch_ex(ctx, ABS_KC_LSQ, lsq_grad_v2_kernel<T>, dim3(ctx->lsq_grid), dim3(256), 0, a);
+    else launch_ex(ctx, ABS_KC_LSQ, lsq_grad_kernel<T>, dim3(ctx->W), dim3(256), 0, a);
     return;
   }
   const int nl = m.n_layers;
@@ -565,6 +568,15 @@ void enqueue_gradient(abs_ctx* ctx) {
 template <typename T>
 void enqueue_update(abs_ctx* ctx) {
   const Layout& L = ctx->L;
+  if (ctx->lsq_v2) {
+    LsqUpdateArgs q;
+    q.st = ctx->at<DevState>(L.st); q.job = ctx->ctl.job; q.next_dur = ctx->ctl.next_dur; q.dur_job = ctx->ctl.dur_job;
+    q.master = ctx->at<float>(L.master); q.ring = ctx->at<void>(L.ring); q.G = ctx->at<float>(L.G);
+    q.d_pad = L.d_pad; q.d = ctx->m.dims[0]; q.P = ctx->lsq_grid; q.lr = ctx->m.lr;
+    const int blocks = std::max((q.d + 31) / 32, (ctx->W + 31) / 32);
+    launch_ex(ctx, ABS_KC_UPDATE, lsq_update_kernel<T>, dim3(blocks), dim3(256), 0, q);
+    return;
+  }
   UpdateArgs u;
   u.st = ctx->at<DevState>(L.st); u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
   u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
@@ -717,6 +729,10 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
       ef = cudaFuncSetAttribute(narrow_fused_cc_kernel<__nv_bfloat16, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (ef != cudaSuccess) return bail(cuda_fail(nullptr, ef, "cudaFuncSetAttribute(narrow_fused_kernel)"));
   }
+  if (model->kind == ABS_LSQ && model->dims[0] % 8 == 0 && model->dims[0] <= LSQ_MAX_D) {
+    ctx->lsq_v2 = true;
+    ctx->lsq_grid = std::min(W, 2 * ctx->sm_count);
+  }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);
   abs_init_state_kernel<<<(W + 31) / 32, 32, 0, s>>>(c);
@@ -836,7 +852,7 @@ int abs_launch_count(abs_ctx* ctx, long long* launches) {
 
 int abs_get_plan(abs_ctx* ctx, int* partials, int* row_block, int* rows_cap, int* path) {
   if (!ctx) return fail(ABS_EINVAL, "ctx is null");
-  if (partials) *partials = ctx->L.P;
+  if (partials) *partials = ctx->lsq_v2 ? ctx->lsq_grid : ctx->L.P;
   if (row_block) *row_block = ctx->L.RB;
   if (rows_cap) *rows_cap = ctx->L.rows_cap;
   if (path) for (int l = 0; l < ctx->m.n_layers; ++l) path[l] = ctx->L.path[l];

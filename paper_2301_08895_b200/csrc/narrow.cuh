@@ -878,4 +878,156 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Least squares, HBM-bound form (feature count a multiple of 8, at most LSQ_MAX_D).  Persistent
+// CTAs take selected workers i = cta, cta + grid, ...; for each they draw the minibatch, compute
+// the residuals r_b = x_b . w_v - y_b with 16-byte loads (one warp per row) and then add
+// sum_b r_b x_b into register accumulators that persist across the CTA's workers (the second pass
+// over the rows hits L2).  Eq. 3 only needs the sum over workers, so a CTA writes one partial sum.
+constexpr int LSQ_MAX_D = 8192;
+
+template <typename T>
+__global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
+  grid_dependency_sync();
+  __shared__ float wf[LSQ_MAX_D];
+  __shared__ float res[1024];
+  __shared__ int sidx[1024];
+  __shared__ float red[8];
+  DevState* st = a.st;
+  if (st->status != ST_OK) return;
+  const int K = st->K, B = st->B, d = a.d, W = st->W, S = st->S, t = st->t;
+  const i64 M = st->n_samples;
+  const uint32_t key0 = st->key0, key1 = st->key1;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = d >> 3;
+  const T* X = (const T*)a.X;
+  float acc[LSQ_MAX_D / 8 / 256][8];
+#pragma unroll
+  for (int q = 0; q < LSQ_MAX_D / 8 / 256; ++q)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[q][j] = 0.f;
+  int slot_loaded = -1;
+  bool bad = false;
+  for (int i = blockIdx.x; i < K; i += gridDim.x) {
+    const int wn = a.sel[i];
+    const int job = a.job[wn];
+    const int slot = (t - a.sel_tau[i]) % (S + 1);
+    __syncthreads();                           // previous worker's res / sidx / wf are no longer read
+    {
+      const i64 lo = ((i64)wn * M) / W, hi = ((i64)(wn + 1) * M) / W;
+      const u64 len = (u64)(hi - lo);
+      for (int blk = tid; blk < ((B + 3) >> 2); blk += 256) {
+        uint32_t w4[4];
+        philox4x32_10((uint32_t)wn, (uint32_t)job, 1u, (uint32_t)blk, key0, key1, w4);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (blk * 4 + q < B) sidx[blk * 4 + q] = (int)lo + (int)(((u64)w4[q] * len) >> 32);
+      }
+    }
+    if (slot != slot_loaded) {
+      const T* w = (const T*)a.ring + (size_t)slot * a.slot_stride;
+      for (int v = tid; v < nvec; v += 256) {
+        float wv[8];
+        load8(w + v * 8, wv);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) wf[v * 8 + j] = wv[j];
+      }
+      slot_loaded = slot;
+    }
+    __syncthreads();
+    // pass 1: residuals, one warp per row
+    for (int b = warp; b < B; b += 8) {
+      const T* x = X + (size_t)sidx[b] * d;
+      float dot = 0.f;
+#pragma unroll 4
+      for (int v = lane; v < nvec; v += 32) {
+        float xv[8];
+        load8(x + v * 8, xv);
+        const float4 w0 = *reinterpret_cast<const float4*>(wf + v * 8), w1 = *reinterpret_cast<const float4*>(wf + v * 8 + 4);
+        dot = fmaf(xv[0], w0.x, dot); dot = fmaf(xv[1], w0.y, dot); dot = fmaf(xv[2], w0.z, dot); dot = fmaf(xv[3], w0.w, dot);
+        dot = fmaf(xv[4], w1.x, dot); dot = fmaf(xv[5], w1.y, dot); dot = fmaf(xv[6], w1.z, dot); dot = fmaf(xv[7], w1.w, dot);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      if (lane == 0) res[b] = dot - a.y[sidx[b]];
+    }
+    __syncthreads();
+    float part = 0.f;
+    for (int b = tid; b < B; b += 256) part += 0.5f * res[b] * res[b];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if (lane == 0) red[warp] = part;
+    // pass 2: this worker's gradient into the running sums (rows come from L2 now)
+#pragma unroll
+    for (int q = 0; q < LSQ_MAX_D / 8 / 256; ++q) {
+      const int v = tid + q * 256;
+      if (v < nvec) {
+#pragma unroll 8
+        for (int b = 0; b < B; ++b) {
+          float xv[8];
+          load8(X + (size_t)sidx[b] * d + (size_t)v * 8, xv);
+          const float rb = res[b];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[q][j] = fmaf(rb, xv[j], acc[q][j]);
+        }
+      }
+    }
+    __syncthreads();
+    if (tid == 0) {
+      float tot = 0.f;
+      for (int q = 0; q < 8; ++q) tot += red[q];
+      const float loss = __fdiv_rn(tot, (float)B);
+      a.loss[i] = loss;
+      bad |= !isfinite(loss);
+    }
+  }
+  if (bad) st->diverged = 1;
+  float* g = a.G + (size_t)blockIdx.x * a.slot_stride;
+#pragma unroll
+  for (int q = 0; q < LSQ_MAX_D / 8 / 256; ++q) {
+    const int v = tid + q * 256;
+    if (v < nvec) store8(g + (size_t)v * 8, acc[q]);
+  }
+}
+
+struct LsqUpdateArgs {
+  const DevState* st;
+  const int* job; u64* next_dur; int* dur_job;
+  float* master; void* ring; const float* G;
+  size_t d_pad; int d; int P; float lr;
+};
+
+// Eq. 3 for least squares: the P per-CTA partial sums are added in a fixed order (32 parameters x
+// 8 partial lanes per block), then w^{t+1} = w^t - eta/(K B) * sum goes to the fp32 master and to
+// ring slot (t+1) mod (S+1).
+template <typename T>
+__global__ void __launch_bounds__(256) lsq_update_kernel(LsqUpdateArgs a) {
+  grid_dependency_sync();
+  __shared__ float red[8][33];
+  const DevState* st = a.st;
+  if (st->status != ST_OK) return;
+  if (threadIdx.x < 32) refresh_next_durations(st, a.job, a.next_dur, a.dur_job, blockIdx.x * 32 + threadIdx.x);
+  if (st->diverged) return;
+  const int K = st->K;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int j = blockIdx.x * 32 + lane;
+  float acc = 0.f;
+  if (j < a.d) {
+#pragma unroll 8
+    for (int p = w; p < a.P; p += 8) acc += a.G[(size_t)p * a.d_pad + j];
+  }
+  red[w][lane] = acc;
+  __syncthreads();
+  if (w == 0 && j < a.d) {
+    float g = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) g += red[q][lane];
+    const float step = __fdiv_rn(a.lr, (float)(K * st->B));
+    const float m = fmaf(-step, g, a.master[j]);
+    a.master[j] = m;
+    const int slot = (st->t + 1) % (st->S + 1);
+    stf((T*)a.ring + (size_t)slot * a.d_pad, j, m);
+  }
+}
+
 }  // namespace absb
