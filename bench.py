@@ -170,7 +170,8 @@ def main():
 
     cfg = inputs.config(args.config, args.workers)
     if world > 1:
-        cfg.run_seed += rank            # independent replicas: one run per GPU, different seeds
+        from paper_2301_08895_b200 import multi
+        cfg.run_seed = multi.replica_seed(cfg.run_seed, rank)   # independent replicas, one per GPU
     rounds = args.rounds or cfg.rounds
     config_obj = {"workload": workload_name(cfg, rounds), "lr": cfg.lr,
                   "parallelism": "replicas x%d (the round loop does not shard)" % world,
@@ -299,15 +300,9 @@ def main():
     _, wg_p, _, prof, ks, plan = device_step(profile=True)
 
     t_dev = sum(ms) / 1e3
-    if world > 1:
-        tt = torch.tensor([t_dev, sum(e2e_t)], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        cnt = torch.tensor([wg_total, e2e_wg], device=dev, dtype=torch.float64)
-        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
-        t_dev, e2e_time = float(tt[0]), float(tt[1])
-        wg_all, e2e_wg_all = float(cnt[0]), float(cnt[1])
-    else:
-        e2e_time, wg_all, e2e_wg_all = sum(e2e_t), wg_total, e2e_wg
+    from paper_2301_08895_b200 import multi
+    (t_dev, e2e_time), (wg_all, e2e_wg_all) = multi.aggregate_replicas(
+        [t_dev, sum(e2e_t)], [wg_total, e2e_wg], device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()

@@ -130,11 +130,14 @@ class ABSOracle:
     bound_mode     BOUND_ADAPTIVE (Eq. 4) or BOUND_FIXED (theta = S always)
     literal_eq6    test the pre-increment age against the threshold exactly as
                    Eq. 6 is printed (one round later than Algorithm 1's order)
+    integer_only   play only the server's integer machinery (arrivals, Eq. 4-6,
+                   ticks): no gradient is evaluated and the model stays at w^0;
+                   every round must then be given its uploaded losses
     """
 
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, dist, seed,
                  quant=False, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE,
-                 literal_eq6=False, x_is_bf16_bits=False):
+                 literal_eq6=False, x_is_bf16_bits=False, integer_only=False):
         if not (1 <= K0 <= W):
             raise ValueError("need 1 <= K0 <= W")
         if S < 0:
@@ -149,6 +152,7 @@ class ABSOracle:
         self.quant = bool(quant)
         self.k_mode, self.bound_mode = k_mode, bound_mode
         self.literal_eq6 = literal_eq6
+        self.integer_only = integer_only
         self.w = np.array(w0, dtype=np.float64)
         assert self.w.shape[0] == models.n_params(kind, dims)
         # the oracle may keep every past model; the bound is what lets a real
@@ -207,17 +211,22 @@ class ABSOracle:
         taus = [t - self.version[n] for n in arrivals]
 
         own_losses, grad_sum = [], np.zeros_like(self.w)
-        for n in arrivals:
-            loss, grad = self.upload(n)
-            own_losses.append(np.float32(loss))
-            grad_sum += grad
+        if self.integer_only:
+            assert forced_losses is not None and len(forced_losses) == K
+            own_losses = [np.float32(x) for x in forced_losses]
+        else:
+            for n in arrivals:
+                loss, grad = self.upload(n)
+                own_losses.append(np.float32(loss))
+                grad_sum += grad
         losses = own_losses if forced_losses is None else \
             [np.float32(x) for x in forced_losses]
         if not all(math.isfinite(float(x)) for x in losses):
             raise Diverged()
 
-        self.w = self.w - (self.lr / K) * grad_sum                      # Eq. 3
-        self.versions[t + 1] = self._stored(self.w)
+        if not self.integer_only:
+            self.w = self.w - (self.lr / K) * grad_sum                  # Eq. 3
+            self.versions[t + 1] = self._stored(self.w)
 
         Lt = loss_estimate(losses)
         if t == 0:
@@ -244,7 +253,7 @@ class ABSOracle:
         for n in arrivals + restarted:
             self._start_job(n, T_end)
         # drop model copies that no worker holds any more (memory only)
-        for v in [v for v in self.versions if v not in set(self.version)]:
+        for v in [v for v in self.versions if v not in set(self.version) and not self.integer_only]:
             del self.versions[v]
         self.comm += K + len(restarted)
 

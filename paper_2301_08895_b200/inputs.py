@@ -92,10 +92,9 @@ def n_params(kind, dims):
 
 
 def to_bf16_bits(a32):
-    """float32 array -> uint16 bfloat16 patterns (round to nearest even)."""
-    import torch
-    t = torch.from_numpy(np.ascontiguousarray(a32, dtype=np.float32)).to(torch.bfloat16)
-    return t.view(torch.int16).numpy().view(np.uint16)
+    """float32 array -> uint16 bfloat16 patterns (round to nearest even; finite inputs)."""
+    bits = np.ascontiguousarray(a32, dtype=np.float32).view(np.uint32)
+    return ((bits + np.uint32(0x7FFF) + ((bits >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
 
 
 def bf16_bits_to_f32(bits):

@@ -1,0 +1,79 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot replay 2000 rounds of the large networks in test time, so each
+configuration is checked three ways: (1) the whole integer trace of the full run,
+bit-exact, with the oracle's server logic fed the uploaded losses; (2) the first
+rounds in lock step including losses and parameters; (3) invariants of Algorithm 1
+that hold at any size.  Least squares (configuration 5, W = 1024) is replayed by
+the oracle in full.
+"""
+import numpy as np
+import pytest
+
+from conftest import make_oracle
+from helpers import INT_FIELDS, compare_with_oracle, first_integer_mismatch, gpu_run, rel_l2, to_device
+from paper_2301_08895_b200 import abs as gpu
+from paper_2301_08895_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def check_invariants(cfg, rows):
+    W, S = cfg.W, cfg.S
+    prev_T, prev_K, comm = 0, 0, W
+    for r in rows:
+        assert len(r["sel"]) == r["K"] == len(set(r["sel"])) == len(r["tau"])
+        assert all(0 <= x < W for x in r["sel"] + r["restart"])
+        assert not (set(r["sel"]) & set(r["restart"])) and r["restart"] == sorted(r["restart"])
+        assert all(0 <= tau <= S for tau in r["tau"]) and 0 <= r["theta"] <= S
+        assert r["T_end"] >= prev_T and prev_K <= r["K"] <= W
+        prev_T, prev_K = r["T_end"], r["K"]
+        comm += r["K"] + len(r["restart"])
+        assert r["comm"] == comm
+        assert np.all(np.isfinite(r["sel_loss"]))
+
+
+def full_run_checks(cfg, prefix_rounds, tol, loss_tol):
+    X, y, _ = inputs.make_data(cfg)
+    w0 = inputs.make_w0(cfg)
+    rows, params = gpu_run(cfg, X, y, w0, cfg.rounds)
+    assert len(rows) == cfg.rounds and np.all(np.isfinite(params))
+    check_invariants(cfg, rows)
+    # (1) integer trace of the whole run against the oracle's server logic
+    o = make_oracle(cfg, X, y, w0, integer_only=True)
+    orows = o.run(cfg.rounds, forced_losses=[r["sel_loss"] for r in rows])
+    mm = first_integer_mismatch(rows, orows)
+    assert mm is None, "full-run integer trace differs: %s" % (mm,)
+    assert rows[-1]["loss_mean"] < 0.2 * rows[0]["loss_mean"]
+    # (2) first rounds in lock step, floats included
+    compare_with_oracle(cfg, X, y, w0, prefix_rounds, tol, forced=True, loss_tol=loss_tol)
+    return rows
+
+
+def test_config4_full_size():
+    rows = full_run_checks(inputs.config(4), 8, 2e-2, 5e-2)
+    assert rows[0]["K"] == 16 and rows[-1]["K"] == 128
+    assert max(max(r["tau"]) for r in rows) >= 5
+
+
+def test_config3_full_size():
+    rows = full_run_checks(inputs.config(3), 60, 2e-2, 5e-2)
+    assert rows[0]["K"] == 8 and rows[-1]["K"] == 64
+    assert any(r["restart"] for r in rows)
+
+
+def test_config2_full_size_is_covered_by_the_free_running_test():
+    # configuration 1 and 2 are replayed completely, free running, in test_gpu_parity.py
+    cfg = inputs.config(2)
+    assert cfg.rounds == 1000 and cfg.W == 16
+
+
+def test_config5_full_size_w1024():
+    cfg = inputs.config(5, 1024)
+    X, y, _ = inputs.make_data(cfg)
+    w0 = inputs.make_w0(cfg)
+    # uploaded losses agree to bf16 level: the two fp32/fp64 masters round to different bf16 ring values now and then
+    rows, orows, err, o = compare_with_oracle(cfg, X, y, w0, cfg.rounds, 2e-2, forced=True, loss_tol=5e-2)
+    check_invariants(cfg, rows)
+    assert rows[0]["K"] == 128 and rows[-1]["K"] > 128
+    assert max(max(r["tau"]) for r in rows) > 8

@@ -275,3 +275,16 @@ def test_divergence_is_reported():
     with pytest.raises(abs_sim.Diverged):
         o.run(200)
     assert 0 < len(o.trace) < 200
+
+
+def test_integer_only_mode_replays_the_same_trace():
+    X, y, _ = _lsq_problem()
+    dist = timing.TimeDist(timing.PARETO2, scale=1.0)
+    a = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 9, 2, 3, dist, 5)
+    rows = a.run(60)
+    b = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 9, 2, 3, dist, 5, integer_only=True)
+    rows_b = b.run(60, forced_losses=[r["sel_loss"] for r in rows])
+    for ra, rb in zip(rows, rows_b):
+        for f in ("K", "sel", "tau", "restart", "T_end", "theta", "comm"):
+            assert ra[f] == rb[f]
+    assert np.array_equal(b.w, np.zeros(6))
