@@ -27,6 +27,9 @@ sys.path.insert(0, ROOT)
 from paper_2301_08895_b200 import inputs  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes (read + write) per launch of the tensor-core GEMM kernel at K = N on configuration 4, from the ncu
+# capture summarised in profiles/tc_gemm_kernel_cfg4.md; valid only for the kernel source it was taken from.
+GEMM_TRAFFIC = {"config": 4, "bytes_per_launch": 38.6e6, "tc_cuh_sha256_16": "ab2a2a44b30ac923"}
 METRIC = "worker_gradients_per_sec"
 UNIT = "worker-gradients/s"
 
@@ -41,6 +44,16 @@ def load_peaks():
     p = dict(FALLBACK_PEAKS)
     p["source"] = "fallback"
     return p
+
+
+def gemm_traffic(config_index):
+    import hashlib
+    path = os.path.join(ROOT, "paper_2301_08895_b200", "csrc", "tc.cuh")
+    with open(path, "rb") as f:
+        sha = hashlib.sha256(f.read()).hexdigest()[:16]
+    if config_index == GEMM_TRAFFIC["config"] and sha == GEMM_TRAFFIC["tc_cuh_sha256_16"]:
+        return GEMM_TRAFFIC["bytes_per_launch"]
+    return None            # kernel changed since the counters were taken (or another workload)
 
 
 def workload_name(cfg, rounds):
@@ -347,7 +360,7 @@ def main():
         peak = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
         out["roofline"] = {"bound": "tensor", "kernel": "tc_gemm_kernel (fwd+dgrad+wgrad launches)",
                            "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                           "traffic": None, "peak_source": peaks["source"] + " (sustained bf16)",
+                           "traffic": gemm_traffic(args.config), "peak_source": peaks["source"] + " (sustained bf16)",
                            "frac_of_burst_peak": ach / peaks["bf16_tflops"],
                            "share_of_profiled_time": t_g / tot_prof,
                            "per_class_tflops": {c: wg_p * flops[c] / (prof[c][1] * 1e-3) / 1e12
