@@ -174,6 +174,7 @@ def main():
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--workers", type=int, default=None, help="W of configuration 5")
     ap.add_argument("--rounds", type=int, default=None, help="rounds per step (default: the configuration's)")
+    ap.add_argument("--flags", type=int, default=0, help="ABS_FLAG_* bits passed to abs_init")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work")
     args = ap.parse_args()
 
@@ -242,8 +243,8 @@ def main():
     def new_ctx(host=False):
         if host:
             return gpu.context_from_config(cfg, Xh, yh, w0, max_rounds=rounds, data_on_host=True,
-                                           device=str(dev))
-        return gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=rounds, device=str(dev))
+                                           device=str(dev), flags=args.flags)
+        return gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=rounds, device=str(dev), flags=args.flags)
 
     def device_step(profile=False):
         """One run; returns (ms on the stream, worker-gradients, launches, profile dict)."""

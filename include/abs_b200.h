@@ -66,6 +66,8 @@ extern "C" {
 #define ABS_T_PARETO2      3    /* Pareto, shape 2, minimum `scale` */
 
 #define ABS_FLAG_NO_TENSOR_CORES 1  /* run the hidden-layer contractions on the FP32-FMA kernels */
+#define ABS_FLAG_NO_OVERLAP      2  /* enqueue every kernel on the caller's stream (no side stream for the
+                                       server-side kernels of the next round) */
 
 /* kernel classes reported by abs_profile_read */
 #define ABS_KC_CTL     0  /* arrival selection + Eq. 4-6 bookkeeping */

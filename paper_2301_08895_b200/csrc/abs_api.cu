@@ -60,7 +60,9 @@ struct Layout {
   size_t d = 0, d_pad = 0;
   size_t w_off[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the padded vector
   size_t w_src[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the caller's vector
-  size_t st, c, version, job, next_dur, dur_job, sel, sel_tau, sel_row0, loss, row_loss, row_idx, tile_slot;
+  size_t st, ri, c, version, job, next_dur, dur_job, loss, row_loss;
+  size_t sel[2], sel_tau[2], sel_row0[2], row_idx[2], tile_slot[2];   // per-round layout, by round parity
+  size_t act0b;                         // second copy of the gathered input rows (odd rounds)
   size_t master, ring, G, logits, red, ones;
   size_t bits[ABS_MAX_LAYERS + 1];      // ReLU sign bits of act[l] (tensor-core layers)
   size_t act[ABS_MAX_LAYERS + 1], delta[ABS_MAX_LAYERS + 1];
@@ -172,18 +174,21 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   }
   Carver cv;
   L->st = cv.take(sizeof(DevState));
+  L->ri = cv.take(2 * sizeof(RoundInfo));
   L->c = cv.take(sizeof(u64) * W);
   L->version = cv.take(4 * W);
   L->job = cv.take(4 * W);
   L->next_dur = cv.take(8 * W);
   L->dur_job = cv.take(4 * W);
-  L->sel = cv.take(4 * W);
-  L->sel_tau = cv.take(4 * W);
-  L->sel_row0 = cv.take(4 * W);
+  for (int q = 0; q < 2; ++q) {
+    L->sel[q] = cv.take(4 * W);
+    L->sel_tau[q] = cv.take(4 * W);
+    L->sel_row0[q] = cv.take(4 * W);
+    L->row_idx[q] = cv.take(4 * (size_t)L->rows_cap);
+    L->tile_slot[q] = cv.take(4 * (size_t)L->n_tiles_cap);
+  }
   L->loss = cv.take(4 * W);
   L->row_loss = cv.take(4 * (size_t)L->rows_cap);
-  L->row_idx = cv.take(4 * (size_t)L->rows_cap);
-  L->tile_slot = cv.take(4 * (size_t)L->n_tiles_cap);
   L->master = cv.take(4 * L->d_pad);
   L->ring = cv.take(L->esz * L->d_pad * (S + 1));
   L->G = cv.take(4 * L->d_pad * (lsq ? W : L->P));
@@ -208,6 +213,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     for (int l = 0; l + 1 < m->n_layers; ++l)
       if (L->path[l] == PATH_TC) L->bits[l + 1] = cv.take(4 * (size_t)L->rows_cap * ((m->dims[l + 1] + 31) / 32));
     L->act[0] = (L->path[0] == PATH_TC) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
+    L->act0b = (L->path[0] == PATH_TC) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     for (int l = 1; l <= m->n_layers; ++l) {
       L->act[l] = (l < m->n_layers) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]) : 0;
       L->delta[l] = cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]);
@@ -238,6 +244,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
 struct TcLayer {
   CUtensorMap fwd_a, fwd_b, dg_a, dg_b, wg_a, wg_b;
   CUtensorMap fwd_out, dg_out, wg_out;     // result tensors written by bulk tensor stores
+  CUtensorMap fwd_a_odd, wg_a_odd;         // layer 0 only: operand maps over the second gathered copy
 };
 
 // ones[r][0] = 1 (bf16), the rest of the 64-wide rows stays zero: the extra operand row that turns
@@ -253,6 +260,11 @@ struct abs_ctx {
   int W, K0, S;
   int sm_count = 148;
   cudaStream_t stream;
+  // The control kernel (and the row gather) of round t+1 only need the losses of round t, so they
+  // run on a second stream next to the backward kernels of round t.
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_loss = nullptr, ev_ctl = nullptr;
+  bool overlap = false;
   char* ws;
   const void* X;
   const void* y;
@@ -290,14 +302,15 @@ int cuda_fail(abs_ctx* ctx, cudaError_t e, const char* what) {
 // while this one drains; every kernel of the round loop starts with griddepcontrol.wait, which
 // returns once the kernel before it has completed and its writes are visible.
 template <typename... KArgs, typename... Args>
-void launch_ex(abs_ctx* ctx, int cls, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+void launch_on(abs_ctx* ctx, cudaStream_t stream, int cls, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+               Args&&... args) {
   const bool rec = (int)ctx->ev_class.size() < ctx->ev_cap;
-  if (rec) cudaEventRecord(ctx->ev[2 * ctx->ev_class.size()], ctx->stream);
+  if (rec) cudaEventRecord(ctx->ev[2 * ctx->ev_class.size()], stream);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
-  cfg.stream = ctx->stream;
+  cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -306,10 +319,15 @@ void launch_ex(abs_ctx* ctx, int cls, void (*kernel)(KArgs...), dim3 grid, dim3 
   const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
   if (e != cudaSuccess && ctx->launch_error == cudaSuccess) ctx->launch_error = e;
   if (rec) {
-    cudaEventRecord(ctx->ev[2 * ctx->ev_class.size() + 1], ctx->stream);
+    cudaEventRecord(ctx->ev[2 * ctx->ev_class.size() + 1], stream);
     ctx->ev_class.push_back(cls);
   }
   ctx->launches += 1;
+}
+
+template <typename... KArgs, typename... Args>
+void launch_ex(abs_ctx* ctx, int cls, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+  launch_on(ctx, ctx->stream, cls, kernel, grid, block, smem, static_cast<Args&&>(args)...);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -402,6 +420,9 @@ int setup_tc(abs_ctx* ctx) {
               make_act_map(&t.wg_b, delta_out, out, L.rows_cap, 64) &&
               make_act_map(&t.fwd_out, ctx->at<void>(L.act[l + 1]), out, L.rows_cap, 32) &&
               make_g_map(&t.wg_out, ctx->at<float>(L.G) + L.w_off[l], in, out, L.P, L.d_pad);
+    if (ok && l == 0)
+      ok = make_act_map(&t.fwd_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 128) &&
+           make_act_map(&t.wg_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 64);
     if (ok && l > 0)
       ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
            make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l]) &&
@@ -411,15 +432,22 @@ int setup_tc(abs_ctx* ctx) {
   return ABS_OK;
 }
 
+enum Phase : int { PH_GATHER = 0, PH_FORWARD = 1, PH_BACKWARD = 2 };
+
+// Kernels of one round, `par` = round parity (layout copy).  PH_GATHER: minibatch row copy (runs on
+// the side stream when rounds overlap).  PH_FORWARD: everything up to the uploaded losses.
+// PH_BACKWARD: the rest of the gradient.
 template <typename T>
-void enqueue_gradient(abs_ctx* ctx) {
+void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
   const abs_model_desc& m = ctx->m;
   const Layout& L = ctx->L;
   cudaStream_t s = ctx->stream;
   DevState* st = ctx->at<DevState>(L.st);
+  RoundInfo* ri = ctx->at<RoundInfo>(L.ri) + par;
   if (m.kind == ABS_LSQ) {
+    if (phase != PH_FORWARD) return;
     LsqArgs a;
-    a.st = st; a.sel = ctx->ctl.sel; a.job = ctx->ctl.job; a.sel_tau = ctx->ctl.sel_tau; a.sel_row0 = ctx->ctl.sel_row0; a.row_idx = ctx->ctl.row_idx;
+    a.st = st; a.ri = ri; a.sel = ctx->ctl.sel[par]; a.job = ctx->ctl.job; a.sel_tau = ctx->ctl.sel_tau[par]; a.sel_row0 = ctx->ctl.sel_row0[par]; a.row_idx = ctx->ctl.row_idx[par];
     a.X = ctx->X; a.y = (const float*)ctx->y;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad;
     a.loss = ctx->ctl.loss; a.G = ctx->at<float>(L.G); a.d = m.dims[0];
@@ -434,11 +462,11 @@ void enqueue_gradient(abs_ctx* ctx) {
   LayerArgs la[ABS_MAX_LAYERS];
   for (int l = 0; l < nl; ++l) {
     LayerArgs& a = la[l];
-    a.st = st; a.tile_slot = ctx->ctl.tile_slot; a.row_idx = ctx->ctl.row_idx;
+    a.st = st; a.ri = ri; a.tile_slot = ctx->ctl.tile_slot[par]; a.row_idx = ctx->ctl.row_idx[par];
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad; a.w_off = L.w_off[l];
     a.in = m.dims[l]; a.out = m.dims[l + 1];
     a.gather = (l == 0 && !gathered);
-    a.act_in = (l == 0 && !gathered) ? ctx->X : ctx->at<void>(L.act[l]);
+    a.act_in = (l == 0 && !gathered) ? ctx->X : ctx->at<void>((l == 0 && par) ? L.act0b : L.act[l]);
     a.act_out = (l == nl - 1) ? ctx->at<void>(L.logits) : ctx->at<void>(L.act[l + 1]);
     a.delta_out = ctx->at<void>(L.delta[l + 1]);
     a.delta_in = (l == 0) ? nullptr : ctx->at<void>(L.delta[l]);
@@ -447,14 +475,14 @@ void enqueue_gradient(abs_ctx* ctx) {
   auto tc_params = [&](int l, int mode) {
     tc::Params p;
     memset(&p, 0, sizeof p);
-    p.st = st; p.tile_slot = ctx->ctl.tile_slot; p.mode = mode; p.P = L.P;
+    p.st = st; p.ri = ri; p.tile_slot = ctx->ctl.tile_slot[par]; p.mode = mode; p.P = L.P;
     p.ring = ctx->at<__nv_bfloat16>(L.ring); p.slot_stride = L.d_pad;
     p.b_off = L.w_off[l] + (size_t)m.dims[l] * m.dims[l + 1];
     return p;
   };
   auto narrow_args = [&](int l) {
     NarrowArgs a;
-    a.st = st; a.tile_slot = ctx->ctl.tile_slot; a.row_idx = ctx->ctl.row_idx; a.labels = (const int*)ctx->y;
+    a.st = st; a.ri = ri; a.tile_slot = ctx->ctl.tile_slot[par]; a.row_idx = ctx->ctl.row_idx[par]; a.labels = (const int*)ctx->y;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad; a.w_off = L.w_off[l];
     a.in = m.dims[l]; a.C = m.dims[l + 1];
     a.gather = la[l].gather; a.act_in = la[l].act_in;
@@ -463,11 +491,14 @@ void enqueue_gradient(abs_ctx* ctx) {
     a.row_loss = ctx->ctl.row_loss; a.G = ctx->at<float>(L.G); a.P = L.P;
     return a;
   };
-  if (gathered) {
-    launch_ex(ctx, ABS_KC_GATHER, gather_rows_kernel, dim3(ctx->sm_count * 8), dim3(256), 0, st, ctx->ctl.row_idx, (const __nv_bfloat16*)ctx->X, ctx->at<__nv_bfloat16>(L.act[0]), m.dims[0]);
+  if (phase == PH_GATHER) {
+    if (gathered)
+      launch_on(ctx, ctx->overlap ? ctx->side : s, ABS_KC_GATHER, gather_rows_kernel, dim3(ctx->sm_count * 8), dim3(256), 0,
+                st, ri, ctx->ctl.row_idx[par], (const __nv_bfloat16*)ctx->X, ctx->at<__nv_bfloat16>(par ? L.act0b : L.act[0]), m.dims[0]);
+    return;
   }
   // ---- forward (Eq. 2 at the model version each worker holds)
-  for (int l = 0; l < nl; ++l) {
+  for (int l = 0; l < nl && phase == PH_FORWARD; ++l) {
     const bool last = l == nl - 1;
     if (L.path[l] == PATH_TC) {
       tc::Params p = tc_params(l, tc::FWD);
@@ -476,7 +507,7 @@ void enqueue_gradient(abs_ctx* ctx) {
       p.relu_bits = L.bits[l + 1] ? ctx->at<uint32_t>(L.bits[l + 1]) : nullptr;
       p.mask_words = (la[l].out + 31) / 32;
       const int bn = L.bn_fwd[l];
-      launch_tc_bn(ctx, bn, ABS_KC_FWD, ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
+      launch_tc_bn(ctx, bn, ABS_KC_FWD, (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (L.fused_R) {
@@ -493,7 +524,7 @@ void enqueue_gradient(abs_ctx* ctx) {
         } else {
           launch_ex(ctx, ABS_KC_OUTPUT, narrow_fused_kernel<T>, dim3(L.rows_cap / R), dim3(256), sm, a, part, R, has_dgrad);
         }
-        launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, part, len, dstw, R);
+        launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, R);
       } else if (a.in % 8 == 0) {
         const size_t sm = sizeof(T) * (size_t)a.in * a.C + sizeof(float) * a.C;
         launch_ex(ctx, ABS_KC_OUTPUT, narrow_fwd_loss_v8_kernel<T>, dim3(L.rows_cap / NARROW_ROWS), dim3(256), sm, a);
@@ -508,7 +539,7 @@ void enqueue_gradient(abs_ctx* ctx) {
       else launch_ex(ctx, cls, simt_fwd_kernel<T, false>, dim3(grid), dim3(256), 0, la[l]);
       if (last) {
         LossArgs lo;
-        lo.st = st; lo.row_idx = ctx->ctl.row_idx; lo.labels = (const int*)ctx->y;
+        lo.st = st; lo.ri = ri; lo.row_idx = ctx->ctl.row_idx[par]; lo.labels = (const int*)ctx->y;
         lo.logits = ctx->at<float>(L.logits); lo.delta = ctx->at<void>(L.delta[nl]);
         lo.row_loss = ctx->ctl.row_loss; lo.C = m.dims[nl];
         launch_ex(ctx, ABS_KC_OUTPUT, net_loss_kernel<T>, dim3((L.rows_cap + 255) / 256), dim3(256), 0, lo);
@@ -516,7 +547,7 @@ void enqueue_gradient(abs_ctx* ctx) {
     }
   }
   // ---- backward: deltas, then the weight gradients summed over all selected workers (Eq. 3)
-  for (int l = nl - 1; l >= 0; --l) {
+  for (int l = nl - 1; l >= 0 && phase == PH_BACKWARD; --l) {
     if (L.path[l] == PATH_TC) {
       if (l > 0) {
         tc::Params p = tc_params(l, tc::DGRAD);
@@ -532,7 +563,7 @@ void enqueue_gradient(abs_ctx* ctx) {
       p.M_total = la[l].in + 1; p.N_total = la[l].out;     // row `in` of the result is the bias gradient
       p.out_f32 = ctx->at<float>(L.G) + L.w_off[l];
       const int bn = L.bn_wg[l];
-      launch_tc_bn(ctx, bn, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
+      launch_tc_bn(ctx, bn, ABS_KC_WGRAD, (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
                    ((la[l].in + 127) / 128 + 1) * ((la[l].out + bn - 1) / bn) * L.P);
     } else if (L.path[l] == PATH_NARROW && L.fused_R) {
       // forward, loss, delta of the layer below and the gradient were all done by the fused kernel
@@ -552,7 +583,7 @@ void enqueue_gradient(abs_ctx* ctx) {
       float* dstw = ctx->at<float>(L.G) + L.w_off[l];
       const int len = (a.in + 1) * a.C;
       launch_ex(ctx, ABS_KC_OUTPUT, narrow_wgrad_chunk_kernel<T>, dim3(L.rows_cap / 64), dim3(256), 0, a, part);
-      launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, part, len, dstw, 64);
+      launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, 64);
     } else {
       const bool last = l == nl - 1;
       if (l > 0) {
@@ -566,11 +597,12 @@ void enqueue_gradient(abs_ctx* ctx) {
 }
 
 template <typename T>
-void enqueue_update(abs_ctx* ctx) {
+void enqueue_update(abs_ctx* ctx, int par) {
   const Layout& L = ctx->L;
+  RoundInfo* ri = ctx->at<RoundInfo>(L.ri) + par;
   if (ctx->lsq_v2) {
     LsqUpdateArgs q;
-    q.st = ctx->at<DevState>(L.st); q.job = ctx->ctl.job; q.next_dur = ctx->ctl.next_dur; q.dur_job = ctx->ctl.dur_job;
+    q.st = ctx->at<DevState>(L.st); q.ri = ri; q.job = ctx->ctl.job; q.next_dur = ctx->ctl.next_dur; q.dur_job = ctx->ctl.dur_job;
     q.master = ctx->at<float>(L.master); q.ring = ctx->at<void>(L.ring); q.G = ctx->at<float>(L.G);
     q.d_pad = L.d_pad; q.d = ctx->m.dims[0]; q.P = ctx->lsq_grid; q.lr = ctx->m.lr;
     const int blocks = std::max((q.d + 31) / 32, (ctx->W + 31) / 32);
@@ -578,7 +610,7 @@ void enqueue_update(abs_ctx* ctx) {
     return;
   }
   UpdateArgs u;
-  u.st = ctx->at<DevState>(L.st); u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
+  u.st = ctx->at<DevState>(L.st); u.ri = ri; u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
   u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
   u.job = ctx->ctl.job; u.next_dur = ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
   const size_t n4 = L.d_pad / 4;
@@ -698,10 +730,13 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   c.st = ctx->at<DevState>(L.st);
   c.c = ctx->at<u64>(L.c); c.version = ctx->at<int>(L.version); c.job = ctx->at<int>(L.job);
   c.next_dur = ctx->at<u64>(L.next_dur); c.dur_job = ctx->at<int>(L.dur_job);
-  c.sel = ctx->at<int>(L.sel); c.sel_tau = ctx->at<int>(L.sel_tau); c.sel_row0 = ctx->at<int>(L.sel_row0);
+  c.ri = ctx->at<RoundInfo>(L.ri);
+  for (int q = 0; q < 2; ++q) {
+    c.sel[q] = ctx->at<int>(L.sel[q]); c.sel_tau[q] = ctx->at<int>(L.sel_tau[q]); c.sel_row0[q] = ctx->at<int>(L.sel_row0[q]);
+    c.row_idx[q] = ctx->at<int>(L.row_idx[q]); c.tile_slot[q] = ctx->at<int>(L.tile_slot[q]);
+  }
   c.loss = ctx->at<float>(L.loss);
   c.row_loss = model->kind == ABS_LSQ ? nullptr : ctx->at<float>(L.row_loss);
-  c.row_idx = ctx->at<int>(L.row_idx); c.tile_slot = ctx->at<int>(L.tile_slot);
   c.tr_K = ctx->at<int>(L.tr_K); c.tr_R = ctx->at<int>(L.tr_R); c.tr_theta = ctx->at<int>(L.tr_theta);
   c.tr_T = ctx->at<u64>(L.tr_T); c.tr_loss = ctx->at<float>(L.tr_loss); c.tr_comm = ctx->at<u64>(L.tr_comm);
   c.tr_sel_off = ctx->at<i64>(L.tr_sel_off); c.tr_rst_off = ctx->at<i64>(L.tr_rst_off);
@@ -735,6 +770,13 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);
+  if (!(model->flags & ABS_FLAG_NO_OVERLAP)) {
+    cudaError_t es = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
+    if (es == cudaSuccess) es = cudaEventCreateWithFlags(&ctx->ev_loss, cudaEventDisableTiming);
+    if (es == cudaSuccess) es = cudaEventCreateWithFlags(&ctx->ev_ctl, cudaEventDisableTiming);
+    if (es != cudaSuccess) return bail(cuda_fail(nullptr, es, "side stream / events"));
+    ctx->overlap = true;
+  }
   abs_init_state_kernel<<<(W + 31) / 32, 32, 0, s>>>(c);
   if (model->dtype == ABS_FP32) ring_init_kernel<float><<<148, 256, 0, s>>>(ctx->at<float>(L.master), ctx->at<void>(L.ring), L.d_pad);
   else ring_init_kernel<__nv_bfloat16><<<148, 256, 0, s>>>(ctx->at<float>(L.master), ctx->at<void>(L.ring), L.d_pad);
@@ -758,14 +800,53 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
   if (ctx->rounds_enqueued + n > ctx->m.max_rounds)
     return fail(ABS_ENOSPACE, "%d rounds requested, %d of capacity %d already used", n, ctx->rounds_enqueued, ctx->m.max_rounds);
   const bool f32 = ctx->m.dtype == ABS_FP32;
-  for (int r = 0; r < n; ++r) {
-    // the control kernel completes the previous round (if any) and selects this round's arrivals
-    launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), sizeof(CtlShared), ctx->ctl, 1, 1);
-    if (f32) { enqueue_gradient<float>(ctx); enqueue_update<float>(ctx); }
-    else { enqueue_gradient<__nv_bfloat16>(ctx); enqueue_update<__nv_bfloat16>(ctx); }
-  }
-  if (n > 0) {
-    launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), sizeof(CtlShared), ctx->ctl, 1, 0);
+  const size_t csm = sizeof(CtlShared);
+  const int times_blocks = (ctx->W + 31) / 32;
+  const DevState* stc = ctx->at<DevState>(ctx->L.st);
+  auto gradient = [&](int par, int phase) {
+    if (f32) enqueue_gradient<float>(ctx, par, phase);
+    else enqueue_gradient<__nv_bfloat16>(ctx, par, phase);
+  };
+  auto update = [&](int par) {
+    if (f32) enqueue_update<float>(ctx, par);
+    else enqueue_update<__nv_bfloat16>(ctx, par);
+  };
+  if (n > 0 && !ctx->overlap) {
+    for (int r = 0; r < n; ++r) {
+      const int t = ctx->rounds_enqueued + r, par = t & 1;
+      // the control kernel completes the previous round (if any) and selects this round's arrivals
+      launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
+      launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
+      gradient(par, PH_GATHER);
+      gradient(par, PH_FORWARD);
+      gradient(par, PH_BACKWARD);
+      update(par);
+    }
+    launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+  } else if (n > 0) {
+    // Two streams.  Side stream per round t: control kernel (finish t-1, select t), row gather,
+    // [event ctl], duration look-ahead.  Main stream: wait ctl, forward kernels, [event loss],
+    // backward kernels and the Eq. 3 step.  The side stream's next control kernel waits for the
+    // loss event only, so it overlaps the backward pass; layouts alternate by round parity.
+    cudaStream_t A = ctx->stream, B = ctx->side;
+    CU(cudaEventRecord(ctx->ev_loss, A));             // everything enqueued so far precedes the side work
+    CU(cudaStreamWaitEvent(B, ctx->ev_loss, 0));
+    for (int r = 0; r < n; ++r) {
+      const int t = ctx->rounds_enqueued + r, par = t & 1;
+      launch_on(ctx, B, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
+      gradient(par, PH_GATHER);
+      CU(cudaEventRecord(ctx->ev_ctl, B));
+      launch_on(ctx, B, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
+      CU(cudaStreamWaitEvent(A, ctx->ev_ctl, 0));
+      gradient(par, PH_FORWARD);
+      CU(cudaEventRecord(ctx->ev_loss, A));
+      CU(cudaStreamWaitEvent(B, ctx->ev_loss, 0));
+      gradient(par, PH_BACKWARD);
+      update(par);
+    }
+    launch_on(ctx, B, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+    CU(cudaEventRecord(ctx->ev_ctl, B));
+    CU(cudaStreamWaitEvent(A, ctx->ev_ctl, 0));       // the caller's stream covers all of it
   }
   if (ctx->launch_error != cudaSuccess) return cuda_fail(ctx, ctx->launch_error, "kernel launch");
   CU(cudaGetLastError());
@@ -890,6 +971,9 @@ int abs_destroy(abs_ctx* ctx) {
   if (!ctx) return ABS_OK;
   cudaStreamSynchronize(ctx->stream);
   for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
+  if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
+  if (ctx->ev_loss) cudaEventDestroy(ctx->ev_loss);
+  if (ctx->ev_ctl) cudaEventDestroy(ctx->ev_ctl);
   delete ctx;
   return ABS_OK;
 }

@@ -56,19 +56,30 @@ struct DevState {
   int timeout_where;
 };
 
+// What the gradient kernels of one round need to know about it.  Two copies alternate by round
+// parity: the control kernel lays out round t+1 while the backward kernels of round t still run.
+struct RoundInfo {
+  int n_rows;       // padded gradient rows
+  int K;            // K^t
+  int t;            // round index
+  int diverged;     // set by the loss kernels of the round
+};
+
 // Pointers the control kernel works on (all device memory inside the workspace).
 struct CtlArgs {
   DevState* st;
+  RoundInfo* ri;       // [2] by round parity
   u64* c;              // [W] completion tick of each worker's job in flight
   int* version;        // [W] round index of the model the worker holds
   int* job;            // [W] index of the job in flight
-  int* sel;            // [W] selected worker ids of the open round, arrival order
-  int* sel_tau;        // [W]
-  int* sel_row0;       // [W] first gradient row of each selected worker
+  // per-round layout, two copies by round parity
+  int* sel[2];         // [W] selected worker ids of the round, arrival order
+  int* sel_tau[2];     // [W]
+  int* sel_row0[2];    // [W] first gradient row of each selected worker
   float* loss;         // [W] mean minibatch loss of each selected worker
   float* row_loss;     // [rows_cap] per-sample losses (network models), else null
-  int* row_idx;        // [rows_cap] sample index of each gradient row, -1 for padding
-  int* tile_slot;      // [rows_cap / RB] ring slot of each row tile
+  int* row_idx[2];     // [rows_cap] sample index of each gradient row, -1 for padding
+  int* tile_slot[2];   // [rows_cap / RB] ring slot of each row tile
   u64* next_dur;       // [W] duration of the job each worker starts next, computed ahead of time
   int* dur_job;        // [W] job index next_dur[n] belongs to
   // trace

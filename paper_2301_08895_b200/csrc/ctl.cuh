@@ -140,7 +140,9 @@ struct CtlShared {
 //   do_select: open the next round
 // A dependent global-memory access costs this lone CTA close to a microsecond, so everything it
 // needs is loaded up front in one wave and later phases work from registers and shared memory.
-__global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select) {
+//   t_sel:     index of the round that follows the open one (the host counts rounds; parity of
+//              t_sel - 1 / t_sel picks the layout copy of the open / the new round)
+__global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select, int t_sel) {
   grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char ctl_smem[];
   CtlShared& sh = *reinterpret_cast<CtlShared*>(ctl_smem);
@@ -148,7 +150,8 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // ---- one wave of loads
   const int W = st->W, S = st->S, B = st->B, RB = st->RB, K0 = st->K0;
-  const int status0 = st->status, open0 = st->open, diverged0 = st->diverged;
+  const int po = (t_sel - 1) & 1, pn = t_sel & 1;     // layout copy of the open / of the new round
+  const int status0 = st->status, open0 = st->open, diverged0 = a.ri[po].diverged;
   const int k_mode = st->k_mode, bound_mode = st->bound_mode, max_rounds = st->max_rounds;
   const uint32_t key0 = st->key0, key1 = st->key1;
   const i64 n_samples = st->n_samples;
@@ -169,7 +172,7 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
   int my_sel = 0, my_tau = 0, my_row0 = 0;
   float my_loss = 0.f;
   if (fin && tid < K) {
-    my_sel = a.sel[tid]; my_tau = a.sel_tau[tid]; my_row0 = a.sel_row0[tid];
+    my_sel = a.sel[po][tid]; my_tau = a.sel_tau[po][tid]; my_row0 = a.sel_row0[po][tid];
     if (!net) my_loss = a.loss[tid];
   }
   if (status0 != ST_OK) return;
@@ -302,6 +305,10 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
 
   // ------------------------------------------------------------------ select round t
   if (!do_select) return;
+  if (t != t_sel) {                      // host and device disagree on the round index
+    if (tid == 0) st->status = ST_INTERNAL;
+    return;
+  }
   if (t >= max_rounds) {
     if (tid == 0) st->status = ST_NOSPACE;
     return;
@@ -352,9 +359,9 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     const int n_rows = sh.scalar[0];
     if (tid < K) {
       const int row0 = sh.grow0[tau] + ((int)sh.wcnt[warp][tau] + rank_in_warp) * B;
-      a.sel[tid] = n;
-      a.sel_tau[tid] = tau;
-      a.sel_row0[tid] = row0;
+      a.sel[pn][tid] = n;
+      a.sel_tau[pn][tid] = tau;
+      a.sel_row0[pn][tid] = row0;
       sh.row0[tid] = row0;
       sh.flag[tid] = 0;
       if (net) {
@@ -368,8 +375,10 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
       st->n_rows = n_rows;
       st->n_row_tiles = n_rows / RB;
       st->n_groups = sh.scalar[1];
-      st->diverged = 0;
       st->open = 1;
+      RoundInfo info;
+      info.n_rows = n_rows; info.K = K; info.t = t; info.diverged = 0;
+      a.ri[pn] = info;
     }
     if (!net) return;             // least squares: no row tiles, minibatches drawn by its own kernel
     __syncthreads();
@@ -380,13 +389,13 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
         const int r = q * RB;
         int g = 0;                                  // last non-empty group starting at or before r
         for (int u = 0; u <= S; ++u) if (sh.cnt[u] > 0 && sh.grow0[u] <= r) g = u;
-        a.tile_slot[q] = (t - g) % (S + 1);
+        a.tile_slot[pn][q] = (t - g) % (S + 1);
       }
       for (int g = 0; g <= S; ++g) {
         const int c = sh.cnt[g];
         if (c == 0) continue;
         const int p0 = sh.grow0[g] + c * B, p1 = sh.grow0[g] + round_up(c * B, RB);
-        for (int r = p0 + tid; r < p1; r += 1024) a.row_idx[r] = -1;
+        for (int r = p0 + tid; r < p1; r += 1024) a.row_idx[pn][r] = -1;
       }
     }
     // minibatch draws: sample b of job (n, j) = word b%4 of Philox block (n, j, 1, b/4),
@@ -402,10 +411,17 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int b = blk * 4 + q;
-        if (b < B) a.row_idx[row0 + b] = lo + (int)(((u64)w4[q] * len) >> 32);
+        if (b < B) a.row_idx[pn][row0 + b] = lo + (int)(((u64)w4[q] * len) >> 32);
       }
     }
   }
+}
+
+// Duration look-ahead (see refresh_next_durations): one warp per 32 workers.
+__global__ void abs_times_kernel(const DevState* st, const int* job, u64* next_dur, int* dur_job) {
+  grid_dependency_sync();
+  if (st->status != ST_OK) return;
+  refresh_next_durations(st, job, next_dur, dur_job, blockIdx.x * 32 + threadIdx.x);
 }
 
 // Algorithm 1, initialisation: every worker holds w^0 and starts job 0 at tick 0.

@@ -11,11 +11,11 @@ namespace absb {
 constexpr int NARROW_MAX_C = 16;
 
 // act0[r][:] = X[row_idx[r]][:] (zeros for padding rows); bf16, `in` a multiple of 8.
-__global__ void __launch_bounds__(256) gather_rows_kernel(const DevState* st, const int* row_idx,
+__global__ void __launch_bounds__(256) gather_rows_kernel(const DevState* st, const RoundInfo* ri, const int* row_idx,
                                                           const __nv_bfloat16* X, __nv_bfloat16* act0, int in) {
   grid_dependency_sync();
   if (st->status != ST_OK) return;
-  const int n_rows = st->n_rows;
+  const int n_rows = ri->n_rows;
   const int vec_per_row = in >> 3;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int r = blockIdx.x * 8 + warp; r < n_rows; r += gridDim.x * 8) {
@@ -33,12 +33,12 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const DevState* st, co
 // Bias gradient of a hidden layer: G_p[b_off + n] = sum over the rows of chunk p of delta[r][n].
 // Block = 32 column lanes x 32 row lanes; fixed-order reduction.
 template <typename T>
-__global__ void __launch_bounds__(1024) colsum_kernel(const DevState* st, const T* delta, float* G, size_t slot_stride,
+__global__ void __launch_bounds__(1024) colsum_kernel(const DevState* st, const RoundInfo* ri, const T* delta, float* G, size_t slot_stride,
                                                       size_t b_off, int out, int P) {
   grid_dependency_sync();
   __shared__ float red[32][33];
   if (st->status != ST_OK) return;
-  const int n_rows = st->n_rows;
+  const int n_rows = ri->n_rows;
   const int chunk = round_up((n_rows + P - 1) / P, 64);
   const int p = blockIdx.y;
   const int k_begin = min(n_rows, p * chunk), k_end = min(n_rows, (p + 1) * chunk);
@@ -58,6 +58,7 @@ __global__ void __launch_bounds__(1024) colsum_kernel(const DevState* st, const 
 
 struct NarrowArgs {
   DevState* st;
+  RoundInfo* ri;
   const int* tile_slot;
   const int* row_idx;
   const int* labels;
@@ -78,9 +79,10 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_kernel(NarrowArgs a) {
   grid_dependency_sync();
   extern __shared__ float wsm[];               // [in][C] then bias[C]
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.x * 64;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   const int slot = a.tile_slot[r0 / st->RB];
   const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
@@ -136,7 +138,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_kernel(NarrowArgs a) {
     if (lane == 0) a.row_loss[r] = loss;
     bad |= !isfinite(loss);
   }
-  if (bad && lane == 0) st->diverged = 1;
+  if (bad && lane == 0) ri->diverged = 1;
 }
 
 // Back-propagation through the output layer and the ReLU before it, 64 rows per block:
@@ -146,9 +148,10 @@ __global__ void __launch_bounds__(256) narrow_dgrad_kernel(NarrowArgs a) {
   grid_dependency_sync();
   extern __shared__ float wsm[];               // [in][C] then delta tile [64][C]
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.x * 64;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   const int slot = a.tile_slot[r0 / st->RB];
   const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
@@ -182,9 +185,10 @@ __global__ void __launch_bounds__(1024) narrow_wgrad_kernel(NarrowArgs a) {
   grid_dependency_sync();
   __shared__ float red[32][33];
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int in = a.in, C = a.C;
-  const int n_rows = st->n_rows;
+  const int n_rows = ri->n_rows;
   const int chunk = round_up((n_rows + a.P - 1) / a.P, 64);
   const int p = blockIdx.y;
   const int k_begin = min(n_rows, p * chunk), k_end = min(n_rows, (p + 1) * chunk);
@@ -260,9 +264,10 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_v8_kernel(NarrowArgs a) {
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   T* wT = reinterpret_cast<T*>(nsm_raw);                 // [C][in]
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.x * NARROW_ROWS;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   float* bias = reinterpret_cast<float*>(wT + (size_t)C * in);
   const int slot = a.tile_slot[r0 / st->RB];
@@ -330,7 +335,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_v8_kernel(NarrowArgs a) {
     if (lane == 0) a.row_loss[r] = loss;
     bad |= !isfinite(loss);
   }
-  if (bad && lane == 0) st->diverged = 1;
+  if (bad && lane == 0) ri->diverged = 1;
 }
 
 // Back-propagation through the output layer and the ReLU before it, 16 rows per block; a work
@@ -341,9 +346,10 @@ __global__ void __launch_bounds__(256) narrow_dgrad_v8_kernel(NarrowArgs a) {
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   T* wT = reinterpret_cast<T*>(nsm_raw);                 // [C][in]
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.x * NARROW_ROWS;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   float* dsm = reinterpret_cast<float*>(wT + (size_t)C * in);   // [16][C]
   const int slot = a.tile_slot[r0 / st->RB];
@@ -401,9 +407,10 @@ __global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, f
   __shared__ float dsm[64][NARROW_MAX_C];
   __shared__ long long rowoff[64];
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.x * 64;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   const T* dl = (const T*)a.delta_out + (size_t)r0 * C;
   for (int i = threadIdx.x; i < 64 * C; i += 256) dsm[i / C][i % C] = ldf(dl, i);
@@ -458,13 +465,13 @@ __global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, f
 // Stage 1 of a hidden layer's bias gradient: part[q][n] = sum over the 64 rows of chunk q of
 // delta[r][n]; `out` a multiple of 8.
 template <typename T>
-__global__ void __launch_bounds__(256) colsum_chunk_kernel(const DevState* st, const T* delta, int out, float* part) {
+__global__ void __launch_bounds__(256) colsum_chunk_kernel(const DevState* st, const RoundInfo* ri, const T* delta, int out, float* part) {
   grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   float* red = reinterpret_cast<float*>(nsm_raw);        // [row lanes][out]
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.x * 64;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int nvec = out >> 3;
   const int per = min(nvec, 256);                         // threads along a row
   const int lanes = 256 / per;                            // rows worked on side by side
@@ -508,12 +515,12 @@ __global__ void __launch_bounds__(256) colsum_chunk_kernel(const DevState* st, c
 
 // Stage 2: dst[i] = sum over the active chunks q of part[q][i], i < len.  Block = 32 outputs x 8
 // chunk lanes; lane w adds chunks w, w+8, ... in order, then the 8 lanes are added in order.
-__global__ void __launch_bounds__(256) chunk_reduce_kernel(const DevState* st, const float* part, int len, float* dst,
+__global__ void __launch_bounds__(256) chunk_reduce_kernel(const DevState* st, const RoundInfo* ri, const float* part, int len, float* dst,
                                                            int chunk_rows) {
   grid_dependency_sync();
   __shared__ float red[8][33];
   if (st->status != ST_OK) return;
-  const int n_chunks = st->n_rows / chunk_rows;
+  const int n_chunks = ri->n_rows / chunk_rows;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int i = blockIdx.x * 32 + lane;
   float acc = 0.f;
@@ -556,9 +563,10 @@ __global__ void __launch_bounds__(256) narrow_fused_kernel(NarrowArgs a, float* 
   grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.x * R;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C, nvec = in >> 3;
   const int wld = in + 8;                                      // padded row of the transposed weights
   T* hs = reinterpret_cast<T*>(nsm_raw);                       // [R][in] input rows
@@ -654,7 +662,7 @@ __global__ void __launch_bounds__(256) narrow_fused_kernel(NarrowArgs a, float* 
     if (lane == 0) a.row_loss[r] = loss;
     bad |= !isfinite(loss);
   }
-  if (bad && lane == 0) st->diverged = 1;
+  if (bad && lane == 0) ri->diverged = 1;
   __syncthreads();
   // ---- delta of the layer below: (delta W^T) masked by the ReLU of the input rows
   if (has_dgrad) {
@@ -716,9 +724,10 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
   grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char nsm_raw[];
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.x * R;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int in = a.in, nvec = in >> 3;
   const int wld = in + 4;                                      // padded row of the transposed fp32 weights
   T* hs = reinterpret_cast<T*>(nsm_raw);                       // [R][in] input rows
@@ -818,7 +827,7 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
       bad |= !isfinite(loss);
     }
   }
-  if (bad && lane == 0) st->diverged = 1;
+  if (bad && lane == 0) ri->diverged = 1;
   __syncthreads();
   // ---- delta of the layer below: a thread keeps the weights of 8 features in registers
   if (has_dgrad) {
@@ -894,8 +903,9 @@ __global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
   __shared__ int sidx[1024];
   __shared__ float red[8];
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
-  const int K = st->K, B = st->B, d = a.d, W = st->W, S = st->S, t = st->t;
+  const int K = ri->K, B = st->B, d = a.d, W = st->W, S = st->S, t = ri->t;
   const i64 M = st->n_samples;
   const uint32_t key0 = st->key0, key1 = st->key1;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -981,7 +991,7 @@ __global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
       bad |= !isfinite(loss);
     }
   }
-  if (bad) st->diverged = 1;
+  if (bad) ri->diverged = 1;
   float* g = a.G + (size_t)blockIdx.x * a.slot_stride;
 #pragma unroll
   for (int q = 0; q < LSQ_MAX_D / 8 / 256; ++q) {
@@ -992,6 +1002,7 @@ __global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
 
 struct LsqUpdateArgs {
   const DevState* st;
+  const RoundInfo* ri;
   const int* job; u64* next_dur; int* dur_job;
   float* master; void* ring; const float* G;
   size_t d_pad; int d; int P; float lr;
@@ -1005,10 +1016,10 @@ __global__ void __launch_bounds__(256) lsq_update_kernel(LsqUpdateArgs a) {
   grid_dependency_sync();
   __shared__ float red[8][33];
   const DevState* st = a.st;
+  const RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
-  if (threadIdx.x < 32) refresh_next_durations(st, a.job, a.next_dur, a.dur_job, blockIdx.x * 32 + threadIdx.x);
-  if (st->diverged) return;
-  const int K = st->K;
+  if (ri->diverged) return;
+  const int K = ri->K;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int j = blockIdx.x * 32 + lane;
   float acc = 0.f;
@@ -1025,7 +1036,7 @@ __global__ void __launch_bounds__(256) lsq_update_kernel(LsqUpdateArgs a) {
     const float step = __fdiv_rn(a.lr, (float)(K * st->B));
     const float m = fmaf(-step, g, a.master[j]);
     a.master[j] = m;
-    const int slot = (st->t + 1) % (st->S + 1);
+    const int slot = (ri->t + 1) % (st->S + 1);
     stf((T*)a.ring + (size_t)slot * a.d_pad, j, m);
   }
 }

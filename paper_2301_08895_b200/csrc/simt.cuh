@@ -52,6 +52,7 @@ __device__ __forceinline__ void tile_fma(float (&acc)[4][4], int k_begin, int k_
 
 struct LayerArgs {
   const DevState* st;
+  const RoundInfo* ri;
   const int* tile_slot;     // ring slot per RB-row tile
   const int* row_idx;       // sample index per row (-1: padding)
   const void* ring;         // model versions, storage type, [S+1][slot_stride]
@@ -73,9 +74,10 @@ __global__ void __launch_bounds__(256) simt_fwd_kernel(LayerArgs a) {
   grid_dependency_sync();
   __shared__ float As[TK][TM + 4], Bs[TK][TN + 4];
   const DevState* st = a.st;
+  const RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int slot = a.tile_slot[r0 / st->RB];
   const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
   const T* bias = Wm + (size_t)a.in * a.out;
@@ -119,9 +121,10 @@ __global__ void __launch_bounds__(256) simt_dgrad_kernel(LayerArgs a) {
   grid_dependency_sync();
   __shared__ float As[TK][TM + 4], Bs[TK][TN + 4];
   const DevState* st = a.st;
+  const RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r0 = blockIdx.y * TM, m0 = blockIdx.x * TN;
-  if (r0 >= st->n_rows) return;
+  if (r0 >= ri->n_rows) return;
   const int slot = a.tile_slot[r0 / st->RB];
   const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
   const T* dl = (const T*)a.delta_out;
@@ -157,9 +160,10 @@ __global__ void __launch_bounds__(256) simt_wgrad_kernel(LayerArgs a) {
   grid_dependency_sync();
   __shared__ float As[TK][TM + 4], Bs[TK][TN + 4];
   const DevState* st = a.st;
+  const RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN, p = blockIdx.z;
-  const int n_rows = st->n_rows;
+  const int n_rows = ri->n_rows;
   const int chunk = round_up((n_rows + a.P - 1) / a.P, TK);
   const int k_begin = min(n_rows, p * chunk), k_end = min(n_rows, (p + 1) * chunk);
   const T* src = (const T*)a.act_in;
@@ -197,6 +201,7 @@ __global__ void __launch_bounds__(256) simt_wgrad_kernel(LayerArgs a) {
 
 struct LossArgs {
   DevState* st;
+  RoundInfo* ri;
   const int* row_idx;
   const int* labels;      // [n_samples]
   const float* logits;    // [rows][C]
@@ -211,9 +216,10 @@ template <typename T>
 __global__ void __launch_bounds__(256) net_loss_kernel(LossArgs a) {
   grid_dependency_sync();
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= st->n_rows) return;
+  if (r >= ri->n_rows) return;
   const int C = a.C;
   T* d = (T*)a.delta + (size_t)r * C;
   const int s = a.row_idx[r];
@@ -232,11 +238,12 @@ __global__ void __launch_bounds__(256) net_loss_kernel(LossArgs a) {
   for (int c = 0; c < C; ++c) stf(d, c, expf(z[c] - zmax) * inv - (c == y ? 1.f : 0.f));
   const float loss = logf(se) - (z[y] - zmax);
   a.row_loss[r] = loss;
-  if (!isfinite(loss)) st->diverged = 1;
+  if (!isfinite(loss)) ri->diverged = 1;
 }
 
 struct LsqArgs {
   DevState* st;
+  RoundInfo* ri;
   const int* sel; const int* job;
   const int* sel_tau; const int* sel_row0; const int* row_idx;
   const void* X; const float* y;
@@ -255,12 +262,13 @@ __global__ void __launch_bounds__(256) lsq_grad_kernel(LsqArgs a) {
   __shared__ int sidx[1024];
   __shared__ float red[8];
   DevState* st = a.st;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   const int i = blockIdx.x;
-  if (i >= st->K) return;
+  if (i >= ri->K) return;
   const int B = st->B, d = a.d;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int slot = (st->t - a.sel_tau[i]) % (st->S + 1);
+  const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
   const T* w = (const T*)a.ring + (size_t)slot * a.slot_stride;
   const T* X = (const T*)a.X;
   {
@@ -299,7 +307,7 @@ __global__ void __launch_bounds__(256) lsq_grad_kernel(LsqArgs a) {
     for (int q = 0; q < 8; ++q) tot += red[q];
     const float loss = __fdiv_rn(tot, (float)B);
     a.loss[i] = loss;
-    if (!isfinite(loss)) st->diverged = 1;
+    if (!isfinite(loss)) ri->diverged = 1;
   }
   float* g = a.G + (size_t)i * a.slot_stride;
   for (int j = tid; j < d; j += 256) {
@@ -311,6 +319,7 @@ __global__ void __launch_bounds__(256) lsq_grad_kernel(LsqArgs a) {
 
 struct UpdateArgs {
   const DevState* st;
+  const RoundInfo* ri;
   const int* job; u64* next_dur; int* dur_job;   // duration look-ahead (see refresh_next_durations)
   float* master;          // [d_pad]
   void* ring;             // [S+1][d_pad] storage type
@@ -326,13 +335,13 @@ template <typename T>
 __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
   grid_dependency_sync();
   const DevState* st = a.st;
+  const RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
-  if (threadIdx.x < 32) refresh_next_durations(st, a.job, a.next_dur, a.dur_job, blockIdx.x * 32 + threadIdx.x);
-  if (st->diverged) return;
-  const int K = st->K;
+  if (ri->diverged) return;
+  const int K = ri->K;
   const int P = a.P > 0 ? a.P : K;
   const float step = __fdiv_rn(a.lr, (float)(K * st->B));
-  const int slot = (st->t + 1) % (st->S + 1);
+  const int slot = (ri->t + 1) % (st->S + 1);
   T* dst = (T*)a.ring + (size_t)slot * a.d_pad;
   const size_t n4 = a.d_pad / 4;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4;

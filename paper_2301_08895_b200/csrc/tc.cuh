@@ -28,6 +28,7 @@ enum Mode : int { FWD = 0, DGRAD = 1, WGRAD = 2 };
 
 struct Params {
   DevState* st;
+  RoundInfo* ri;
   const int* tile_slot;
   int mode;
   int M_total;             // WGRAD: in + 1 (weight rows and the bias row of G); FWD/DGRAD: unused
@@ -157,8 +158,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   DevState* st = p.st;
+  RoundInfo* ri = p.ri;
   if (st->status != ST_OK) return;
-  const int n_rows = st->n_rows;
+  const int n_rows = ri->n_rows;
   const int n_row_tiles = n_rows / BM;
   const int mode = p.mode;
   const int n_ct = (p.N_total + BN - 1) / BN;

@@ -212,3 +212,15 @@ def test_tick_range_error():
         ctx.run_rounds(20)
     assert e.value.code == gpu.ERANGE
     ctx.close()
+
+
+@pytest.mark.parametrize("idx,rounds,n", [(1, 80, 8192), (3, 40, 8192), (5, 30, 16384)])
+def test_side_stream_overlap_changes_nothing(idx, rounds, n):
+    """The server-side kernels of round t+1 run next to the backward pass of round t; switching
+    that off (everything on the caller's stream) must give the same bits."""
+    cfg = inputs.config(idx).scaled(n_samples=n)
+    X, y, w0 = _problem(cfg)
+    rows_a, params_a = gpu_run(cfg, X, y, w0, rounds)
+    rows_b, params_b = gpu_run(cfg, X, y, w0, rounds, flags=gpu.FLAG_NO_OVERLAP)
+    assert rows_a == rows_b
+    assert np.array_equal(params_a, params_b)
