@@ -66,6 +66,8 @@ extern "C" {
 #define ABS_T_PARETO2      3    /* Pareto, shape 2, minimum `scale` */
 
 #define ABS_FLAG_NO_TENSOR_CORES 1  /* run the hidden-layer contractions on the FP32-FMA kernels */
+#define ABS_FLAG_TWO_CTA         4  /* hidden-layer GEMMs with >= 256 output columns run on CTA pairs
+                                       (tcgen05 cta_group::2, tiles of 256 x 256) */
 #define ABS_FLAG_NO_OVERLAP      2  /* enqueue every kernel on the caller's stream (no side stream for the
                                        server-side kernels of the next round) */
 

@@ -23,6 +23,7 @@ T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2 = 0, 1, 2, 3
 MAX_LAYERS = 7
 FLAG_NO_TENSOR_CORES = 1
 FLAG_NO_OVERLAP = 2
+FLAG_TWO_CTA = 4
 KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update")
 
 

@@ -55,6 +55,8 @@ struct Layout {
   int path[ABS_MAX_LAYERS] = {};        // how each layer's contractions run
   int bn_fwd[ABS_MAX_LAYERS] = {}, bn_dg[ABS_MAX_LAYERS] = {}, bn_wg[ABS_MAX_LAYERS] = {};
   bool any_tc = false;
+  bool two_cta = false;                 // GEMMs with N >= 256 run on CTA pairs (tiles of 256 x 256)
+  int cg_fwd[ABS_MAX_LAYERS] = {}, cg_dg[ABS_MAX_LAYERS] = {}, cg_wg[ABS_MAX_LAYERS] = {};
   int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
   size_t esz = 4;                       // bytes per stored element (4 or 2)
   size_t d = 0, d_pad = 0;
@@ -124,7 +126,8 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       L->any_tc = true;
     } else L->path[l] = PATH_SIMT;
   }
-  L->RB = lsq ? m->batch : (L->any_tc ? 128 : 64);
+  L->two_cta = L->any_tc && (m->flags & ABS_FLAG_TWO_CTA);
+  L->RB = lsq ? m->batch : (L->any_tc ? (L->two_cta ? 256 : 128) : 64);
   const int groups = (W < S + 1) ? W : S + 1;
   L->rows_cap = round_up(W * m->batch, L->RB) + groups * L->RB;
   L->n_tiles_cap = L->rows_cap / L->RB;
@@ -144,20 +147,26 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       L->bn_fwd[l] = pick(out, row_tiles);
       L->bn_dg[l] = pick(in, row_tiles);
       L->bn_wg[l] = pick(out, ((in + 127) / 128 + 1) * 3);
+      L->cg_fwd[l] = L->cg_dg[l] = L->cg_wg[l] = 1;
+      if (L->two_cta) {
+        if (out >= 256) { L->cg_fwd[l] = 2; L->bn_fwd[l] = 256; L->cg_wg[l] = 2; L->bn_wg[l] = 256; }
+        if (in >= 256) { L->cg_dg[l] = 2; L->bn_dg[l] = 256; }
+      }
     }
     // split count P of the row reduction: the one that minimises the modelled time of all weight
     // gradients (whole waves of 148 CTAs, one tile = 128 x BN x rows/P) plus the extra partial
     // sums the Eq. 3 step then has to read
     double best = 1e30;
     int bestP = 1;
-    const int maxP = std::max(1, std::min(8, W * m->batch / 512));
+    const int maxP = std::max(1, std::min(4, W * m->batch / 512));   // more partials cost the Eq. 3 step too much
     for (int P = 1; P <= maxP; ++P) {
       double t = 4.0 * (double)L->d_pad * P / 5e12;
       for (int l = 0; l < m->n_layers; ++l) {
         if (L->path[l] != PATH_TC) continue;
         const int in = m->dims[l], out = m->dims[l + 1], bn = L->bn_wg[l];
-        const long tiles = (long)((in + 127) / 128 + 1) * ((out + bn - 1) / bn) * P;
-        const long waves = (tiles + 147) / 148;
+        const int cg = L->cg_wg[l], tm = 128 * cg, units = 148 / cg;
+        const long tiles = (long)((in + tm - 1) / tm + 1) * ((out + bn - 1) / bn) * P;
+        const long waves = (tiles + units - 1) / units;
         t += (double)waves * 2.0 * 128.0 * bn * ((double)L->rows_cap / P) / 9e12;
       }
       if (t < best * 0.999) { best = t; bestP = P; }
@@ -272,6 +281,7 @@ struct abs_ctx {
   int sticky = ABS_OK;
   long long launches = 0;
   cudaError_t launch_error = cudaSuccess;
+  int next_cluster = 1;              // cluster width of the next launch (consumed by launch_on)
   bool lsq_v2 = false;               // least squares through the persistent 16-byte-load kernel
   int lsq_grid = 0;                  // its grid = number of partial sums
   CtlArgs ctl;
@@ -311,11 +321,19 @@ void launch_on(abs_ctx* ctx, cudaStream_t stream, int cls, void (*kernel)(KArgs.
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (ctx->next_cluster > 1) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)ctx->next_cluster;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+    ctx->next_cluster = 1;
+  }
   const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
   if (e != cudaSuccess && ctx->launch_error == cudaSuccess) ctx->launch_error = e;
   if (rec) {
@@ -379,18 +397,23 @@ bool make_g_map(CUtensorMap* map, const void* base, int in, int out, int P, size
   return make_map(map, base, 3, dims, strides, box, CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
 }
 
-template <int BN>
+template <int BN, int CG>
 void launch_tc(abs_ctx* ctx, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
                const tc::Params& p, int max_tiles) {
-  const int grid = std::max(1, std::min(ctx->sm_count, max_tiles));
-  launch_ex(ctx, cls, tc::tc_gemm_kernel<BN>, dim3(grid), dim3(tc::THREADS), tc::Cfg<BN>::SMEM_BYTES, a, b, ctx->ones_map, o, p);
+  const int units = ctx->sm_count / CG;           // CTAs, or CTA pairs
+  const int grid = CG * std::max(1, std::min(units, max_tiles));
+  ctx->next_cluster = CG;
+  launch_ex(ctx, cls, tc::tc_gemm_kernel<BN, CG>, dim3(grid), dim3(tc::THREADS), tc::Cfg<BN, CG>::SMEM_BYTES, a, b,
+            ctx->ones_map, o, p);
 }
 
-void launch_tc_bn(abs_ctx* ctx, int bn, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
+// max_tiles counts tiles of (128 * cg) x bn
+void launch_tc_bn(abs_ctx* ctx, int bn, int cg, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
                   const tc::Params& p, int max_tiles) {
-  if (bn == 256) launch_tc<256>(ctx, cls, a, b, o, p, max_tiles);
-  else if (bn == 128) launch_tc<128>(ctx, cls, a, b, o, p, max_tiles);
-  else launch_tc<64>(ctx, cls, a, b, o, p, max_tiles);
+  if (cg == 2) launch_tc<256, 2>(ctx, cls, a, b, o, p, max_tiles);
+  else if (bn == 256) launch_tc<256, 1>(ctx, cls, a, b, o, p, max_tiles);
+  else if (bn == 128) launch_tc<128, 1>(ctx, cls, a, b, o, p, max_tiles);
+  else launch_tc<64, 1>(ctx, cls, a, b, o, p, max_tiles);
 }
 
 int setup_tc(abs_ctx* ctx) {
@@ -398,9 +421,10 @@ int setup_tc(abs_ctx* ctx) {
   const Layout& L = ctx->L;
   if (!L.any_tc) return ABS_OK;
   cudaError_t e;
-  e = cudaFuncSetAttribute(tc::tc_gemm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<256>::SMEM_BYTES);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<128>::SMEM_BYTES);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<64>::SMEM_BYTES);
+  e = cudaFuncSetAttribute(tc::tc_gemm_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<256, 1>::SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<128, 1>::SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<64, 1>::SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<256, 2>::SMEM_BYTES);
   if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaFuncSetAttribute(tc_gemm_kernel)");
   const char* ring = ctx->at<char>(L.ring);
   if (!make_act_map(&ctx->ones_map, ctx->at<void>(L.ones), 64, L.rows_cap, 64))
@@ -425,7 +449,7 @@ int setup_tc(abs_ctx* ctx) {
            make_act_map(&t.wg_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 64);
     if (ok && l > 0)
       ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
-           make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l]) &&
+           make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l] / L.cg_dg[l]) &&
            make_act_map(&t.dg_out, ctx->at<void>(L.delta[l]), in, L.rows_cap, 32);
     if (!ok) return fail(ABS_ECUDA, "cuTensorMapEncodeTiled failed for layer %d", l);
   }
@@ -507,7 +531,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       p.relu_bits = L.bits[l + 1] ? ctx->at<uint32_t>(L.bits[l + 1]) : nullptr;
       p.mask_words = (la[l].out + 31) / 32;
       const int bn = L.bn_fwd[l];
-      launch_tc_bn(ctx, bn, ABS_KC_FWD, (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, row_tiles128 * ((la[l].out + bn - 1) / bn));
+      launch_tc_bn(ctx, bn, L.cg_fwd[l], ABS_KC_FWD, (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, (row_tiles128 / L.cg_fwd[l]) * ((la[l].out + bn - 1) / bn));
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (L.fused_R) {
@@ -557,14 +581,15 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
         p.mask_words = (la[l].in + 31) / 32;
         p.out_bf16 = (__nv_bfloat16*)la[l].delta_in;
         const int bn = L.bn_dg[l];
-        launch_tc_bn(ctx, bn, ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, ctx->tcl[l].dg_out, p, row_tiles128 * ((la[l].in + bn - 1) / bn));
+        launch_tc_bn(ctx, bn, L.cg_dg[l], ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, ctx->tcl[l].dg_out, p, (row_tiles128 / L.cg_dg[l]) * ((la[l].in + bn - 1) / bn));
       }
       tc::Params p = tc_params(l, tc::WGRAD);
       p.M_total = la[l].in + 1; p.N_total = la[l].out;     // row `in` of the result is the bias gradient
       p.out_f32 = ctx->at<float>(L.G) + L.w_off[l];
       const int bn = L.bn_wg[l];
-      launch_tc_bn(ctx, bn, ABS_KC_WGRAD, (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
-                   ((la[l].in + 127) / 128 + 1) * ((la[l].out + bn - 1) / bn) * L.P);
+      const int tmw = 128 * L.cg_wg[l];
+      launch_tc_bn(ctx, bn, L.cg_wg[l], ABS_KC_WGRAD, (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
+                   ((la[l].in + tmw - 1) / tmw + 1) * ((la[l].out + bn - 1) / bn) * L.P);
     } else if (L.path[l] == PATH_NARROW && L.fused_R) {
       // forward, loss, delta of the layer below and the gradient were all done by the fused kernel
     } else if (L.path[l] == PATH_NARROW) {
@@ -770,7 +795,9 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);
-  if (!(model->flags & ABS_FLAG_NO_OVERLAP)) {
+  // worth it only when a round has a long backward pass to hide behind (tensor-core networks);
+  // for the latency-bound models the cross-stream events cost more than they hide
+  if (!(model->flags & ABS_FLAG_NO_OVERLAP) && L.any_tc) {
     cudaError_t es = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
     if (es == cudaSuccess) es = cudaEventCreateWithFlags(&ctx->ev_loss, cudaEventDisableTiming);
     if (es == cudaSuccess) es = cudaEventCreateWithFlags(&ctx->ev_ctl, cudaEventDisableTiming);

@@ -106,9 +106,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
          (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, majors, N >> 3, M >> 4.
-__host__ __device__ constexpr uint32_t instr_desc(int a_mn_major, int b_mn_major, int n) {
+__host__ __device__ constexpr uint32_t instr_desc(int a_mn_major, int b_mn_major, int n, int m = BM) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
-         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -116,6 +116,49 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// ---- two-CTA form (cta_group::2): one MMA spans the tensor cores of a CTA pair; M = 256 (128 rows
+// per CTA), each CTA supplies its A tile and its half of the B tile from its own shared memory.
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {   // same offset in CTA `rank`
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma2_load_2d(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma2_load_3d(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void umma2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  const uint32_t z = 0u;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(z) : "memory");
+}
+__device__ __forceinline__ void umma2_commit_both(uint64_t* bar) {   // arrives on `bar` in both CTAs of the pair
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -136,10 +179,10 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-template <int BN> struct Cfg {
-  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+template <int BN, int CG = 1> struct Cfg {
+  static constexpr int STAGES = (BN == 256 && CG == 1) ? 4 : 6;
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = (BN / CG) * BK * 2;     // with a CTA pair each CTA holds half of the B tile
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;
   static constexpr int OUT_BYTES = 2 * 4 * 4096;       // epilogue staging: 2 buffers x 4 warps x (32 rows x 128 B)
@@ -149,27 +192,34 @@ template <int BN> struct Cfg {
 
 struct TileCoord { int a_row, b_col, slot, k_begin, n_kb, split, bias_tile; };
 
-template <int BN>
+// CG = 1: one CTA per tile of 128 x BN.  CG = 2: a cluster of two CTAs per tile of 256 x BN; the
+// leader (cluster rank 0) issues the MMAs for both, every CTA loads its own A rows and its half of
+// B and drains its own half of the accumulator.
+template <int BN, int CG>
 __global__ void __launch_bounds__(THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_ones, const __grid_constant__ CUtensorMap map_out,
                const Params p) {
   grid_dependency_sync();
-  using C = Cfg<BN>;
+  using C = Cfg<BN, CG>;
+  constexpr int TM_ROWS = BM * CG;              // rows of one tile
   extern __shared__ uint8_t smem_raw[];
+  const int rank = (CG == 2) ? (int)cluster_rank() : 0;
+  const int unit = (int)blockIdx.x / CG;        // tile-processing unit (CTA or CTA pair)
+  const int n_units = (int)gridDim.x / CG;
   DevState* st = p.st;
   RoundInfo* ri = p.ri;
   if (st->status != ST_OK) return;
   const int n_rows = ri->n_rows;
-  const int n_row_tiles = n_rows / BM;
+  const int n_row_tiles = n_rows / TM_ROWS;
   const int mode = p.mode;
   const int n_ct = (p.N_total + BN - 1) / BN;
   // WGRAD: one extra row tile multiplies a column of ones with the deltas, which yields the bias
   // gradient (row `in` of the [in + 1][out] gradient block) on the tensor cores for free
-  const int n_mt_w = (p.M_total - 1 + BM - 1) / BM;
+  const int n_mt_w = (p.M_total - 1 + TM_ROWS - 1) / TM_ROWS;
   const int n_mt = (mode == WGRAD) ? n_mt_w + 1 : n_row_tiles;
   const int n_tiles = (mode == WGRAD) ? n_mt * n_ct * p.P : n_row_tiles * n_ct;
-  if ((int)blockIdx.x >= n_tiles) return;
+  if (unit >= n_tiles) return;                  // same decision in both CTAs of a pair
   const int chunk = (mode == WGRAD) ? round_up((n_rows + p.P - 1) / p.P, BK) : 0;
   const int RB = st->RB;
 
@@ -188,17 +238,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4 * CG); }
     *abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CG == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();              // the peer's barriers exist before anything signals them
   tc_fence_after();
+  // barriers that live in the leader CTA, as addresses valid from either CTA of the pair
+  const uint32_t full0_addr = (CG == 2) ? map_to_cta(smem_u32(&full[0]), 0) : smem_u32(&full[0]);
+  const uint32_t acc_empty0_addr = (CG == 2) ? map_to_cta(smem_u32(&acc_empty[0]), 0) : smem_u32(&acc_empty[0]);
   const uint32_t tmem_base = *tmem_slot;
 
   auto tile_coord = [&](int tile) -> TileCoord {
@@ -209,7 +268,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int rem = tile - c.split * per_split;
       const int mt = rem / n_ct;
       c.bias_tile = (mt == n_mt_w);
-      c.a_row = mt * BM;                     // m0
+      c.a_row = mt * TM_ROWS + rank * BM;    // m0 of this CTA
       c.b_col = (rem % n_ct) * BN;           // n0
       c.slot = 0;
       c.k_begin = min(n_rows, c.split * chunk);
@@ -219,9 +278,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int rt = tile / n_ct;
       c.split = 0;
       c.bias_tile = 0;
-      c.a_row = rt * BM;
+      c.a_row = rt * TM_ROWS + rank * BM;
       c.b_col = (tile - rt * n_ct) * BN;
-      c.slot = p.tile_slot[c.a_row / RB];
+      c.slot = p.tile_slot[(rt * TM_ROWS) / RB];
       c.k_begin = 0;
       c.n_kb = (p.K_total + BK - 1) / BK;
     }
@@ -236,28 +295,41 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int armed[C::STAGES];
       for (int s = 0; s < C::STAGES; ++s) armed[s] = -1;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      // loads complete on the leader's "full" barrier (own barrier when CG == 1)
+      auto ld2 = [&](void* dst, const CUtensorMap* map, int st_, int x, int y) {
+        if (CG == 2) tma2_load_2d(dst, map, full0_addr + 8u * (uint32_t)st_, x, y);
+        else tma_load_2d(dst, map, &full[st_], x, y);
+      };
+      auto ld3 = [&](void* dst, const CUtensorMap* map, int st_, int x, int y, int z) {
+        if (CG == 2) tma2_load_3d(dst, map, full0_addr + 8u * (uint32_t)st_, x, y, z);
+        else tma_load_3d(dst, map, &full[st_], x, y, z);
+      };
+      constexpr int BH = BN / CG;                // B columns (rows of the B tile) this CTA loads
+      for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
         const TileCoord c = tile_coord(tile);
+        const int b0 = c.b_col + rank * BH;
         for (int kb = 0; kb < c.n_kb; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) { ok = false; break; }
           uint8_t* sa = smem + (size_t)stage * C::STAGE_BYTES;
           uint8_t* sb = sa + C::A_BYTES;
-          mbar_expect_tx(&full[stage], C::STAGE_BYTES);
-          armed[stage] = (int)phase;
+          if (rank == 0) {                       // the leader arms the barrier for the bytes of the whole pair
+            mbar_expect_tx(&full[stage], CG * C::STAGE_BYTES);
+            armed[stage] = (int)phase;
+          }
           const int k0 = c.k_begin + kb * BK;
           if (mode == FWD) {
-            tma_load_2d(sa, &map_a, &full[stage], k0, c.a_row);
-            for (int j = 0; j < BN / 64; ++j) tma_load_3d(sb + j * 8192, &map_b, &full[stage], c.b_col + 64 * j, k0, c.slot);
+            ld2(sa, &map_a, stage, k0, c.a_row);
+            for (int j = 0; j < BH / 64; ++j) ld3(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0, c.slot);
           } else if (mode == DGRAD) {
-            tma_load_2d(sa, &map_a, &full[stage], k0, c.a_row);
-            tma_load_3d(sb, &map_b, &full[stage], k0, c.b_col, c.slot);
+            ld2(sa, &map_a, stage, k0, c.a_row);
+            ld3(sb, &map_b, stage, k0, b0, c.slot);
           } else {
-            if (c.bias_tile) {   // second box lies outside the 64-wide ones matrix: zero fill
-              for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * 8192, &map_ones, &full[stage], 64 * j, k0);
+            if (c.bias_tile) {   // only column 0 of the 64-wide ones matrix is non-zero; the rest is zero fill
+              for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_ones, stage, rank * BM + 64 * j, k0);
             } else {
-              for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * 8192, &map_a, &full[stage], c.a_row + 64 * j, k0);
+              for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_a, stage, c.a_row + 64 * j, k0);
             }
-            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, &map_b, &full[stage], c.b_col + 64 * j, k0);
+            for (int j = 0; j < BH / 64; ++j) ld2(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0);
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -279,9 +351,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {            // with a CTA pair only the leader issues MMAs
       const bool a_mn = (mode == WGRAD), b_mn = (mode != DGRAD);
-      const uint32_t idesc = instr_desc(a_mn ? 1 : 0, b_mn ? 1 : 0, BN);
+      const uint32_t idesc = instr_desc(a_mn ? 1 : 0, b_mn ? 1 : 0, BN, TM_ROWS);
       // K-major tile: rows of 128 B, 8-row groups 1024 B apart; a k step of 16 elements is 32 B.
       // MN-major tile: 64-wide boxes 8192 B apart (leading offset), 8-k groups 1024 B apart;
       // a k step of 16 rows is 2048 B.
@@ -290,7 +362,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
         const TileCoord c = tile_coord(tile);
         if (c.n_kb == 0) continue;
         if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort)) break;
@@ -304,13 +376,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int kk = 0; kk < BK / UK; ++kk) {
             const uint64_t da = smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
             const uint64_t db = smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
-            umma(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+            if (CG == 2) umma2(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+            else umma(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           }
-          umma_commit(&empty[stage]);
+          if (CG == 2) umma2_commit_both(&empty[stage]);      // frees the stage in both CTAs
+          else umma_commit(&empty[stage]);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(&acc_full[acc]);
+        if (CG == 2) umma2_commit_both(&acc_full[acc]);       // wakes both epilogues
+        else umma_commit(&acc_full[acc]);
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -328,11 +403,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int box_cols = (mode == WGRAD) ? 32 : 64;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    for (int tile = unit; tile < n_tiles; tile += n_units) {
       const TileCoord c = tile_coord(tile);
       const bool have = c.n_kb > 0;
       // output row (FWD/DGRAD) or gradient row m (WGRAD; the bias tile's row 0 is row `in`)
-      const int r = (mode == WGRAD && c.bias_tile) ? (p.M_total - 1) + row_in_tile : c.a_row + row_in_tile;
+      const int r = (mode == WGRAD && c.bias_tile) ? (p.M_total - 1) + rank * BM + row_in_tile : c.a_row + row_in_tile;
       // fetch what the epilogue needs from global memory before waiting for the accumulator
       uint32_t mw[BN / 32];
       __nv_bfloat16* bias_t = bias_s + acc * BN;
@@ -382,7 +457,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int i = 0; i < 32; ++i) v[i] = 0u;
           }
           if (c.bias_tile) {                   // a single useful row: plain stores
-            if (row_in_tile == 0) {
+            if (row_in_tile == 0 && rank == 0) {
               float* dst = p.out_f32 + (size_t)c.split * p.slot_stride + (size_t)r * p.N_total + n0;
 #pragma unroll
               for (int i = 0; i < 32; i += 4)
@@ -455,7 +530,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (have) {
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&acc_empty[acc]);
+        if (lane == 0) {                       // the accumulator barrier lives in the leader CTA
+          if (CG == 2) mbar_arrive_cluster(acc_empty0_addr + 8u * (uint32_t)acc);
+          else mbar_arrive(&acc_empty[acc]);
+        }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -466,9 +544,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();              // neither CTA leaves while the pair still uses its memory
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
+    if (CG == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
   }
   if (threadIdx.x == 0 && *abort) {
     st->timeout_where = 100 + mode;
