@@ -475,7 +475,13 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     a.X = ctx->X; a.y = (const float*)ctx->y;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad;
     a.loss = ctx->ctl.loss; a.G = ctx->at<float>(L.G); a.d = m.dims[0];
-    if (ctx->lsq_v2) launch_ex(ctx, ABS_KC_LSQ, lsq_grad_v2_kernel<T>, dim3(ctx->lsq_grid), dim3(256), 0, a);
+    if (ctx->lsq_v2) {
+      const size_t smw = sizeof(float) * (size_t)a.d;
+      const int nv = (a.d + 2047) / 2048;
+      if (nv <= 1) launch_ex(ctx, ABS_KC_LSQ, lsq_grad_v2_kernel<T, 1>, dim3(ctx->lsq_grid), dim3(256), smw, a);
+      else if (nv == 2) launch_ex(ctx, ABS_KC_LSQ, lsq_grad_v2_kernel<T, 2>, dim3(ctx->lsq_grid), dim3(256), smw, a);
+      else launch_ex(ctx, ABS_KC_LSQ, lsq_grad_v2_kernel<T, 4>, dim3(ctx->lsq_grid), dim3(256), smw, a);
+    }
     else launch_ex(ctx, ABS_KC_LSQ, lsq_grad_kernel<T>, dim3(ctx->W), dim3(256), 0, a);
     return;
   }

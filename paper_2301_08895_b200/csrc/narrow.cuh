@@ -895,10 +895,11 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
 // over the rows hits L2).  Eq. 3 only needs the sum over workers, so a CTA writes one partial sum.
 constexpr int LSQ_MAX_D = 8192;
 
-template <typename T>
-__global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
+// NV = 16-byte vectors of the gradient a thread owns (d <= NV * 2048); wf[d] is dynamic shared memory.
+template <typename T, int NV>
+__global__ void __launch_bounds__(256, 2) lsq_grad_v2_kernel(LsqArgs a) {
   grid_dependency_sync();
-  __shared__ float wf[LSQ_MAX_D];
+  extern __shared__ __align__(16) float wf[];
   __shared__ float res[1024];
   __shared__ int sidx[1024];
   __shared__ float red[8];
@@ -911,9 +912,9 @@ __global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = d >> 3;
   const T* X = (const T*)a.X;
-  float acc[LSQ_MAX_D / 8 / 256][8];
+  float acc[NV][8];
 #pragma unroll
-  for (int q = 0; q < LSQ_MAX_D / 8 / 256; ++q)
+  for (int q = 0; q < NV; ++q)
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[q][j] = 0.f;
   int slot_loaded = -1;
@@ -945,21 +946,33 @@ __global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
       slot_loaded = slot;
     }
     __syncthreads();
-    // pass 1: residuals, one warp per row
-    for (int b = warp; b < B; b += 8) {
-      const T* x = X + (size_t)sidx[b] * d;
-      float dot = 0.f;
-#pragma unroll 4
+    // pass 1: residuals; a warp takes two rows at a time and keeps 16 loads in flight per lane
+    for (int b = warp; b < B; b += 16) {
+      const int b2 = b + 8;
+      const bool two = b2 < B;
+      const T* x0 = X + (size_t)sidx[b] * d;
+      const T* x1 = X + (size_t)sidx[two ? b2 : b] * d;
+      float dot0 = 0.f, dot1 = 0.f;
+#pragma unroll 8
       for (int v = lane; v < nvec; v += 32) {
-        float xv[8];
-        load8(x + v * 8, xv);
+        float xa[8], xb[8];
+        load8(x0 + v * 8, xa);
+        load8(x1 + v * 8, xb);
         const float4 w0 = *reinterpret_cast<const float4*>(wf + v * 8), w1 = *reinterpret_cast<const float4*>(wf + v * 8 + 4);
-        dot = fmaf(xv[0], w0.x, dot); dot = fmaf(xv[1], w0.y, dot); dot = fmaf(xv[2], w0.z, dot); dot = fmaf(xv[3], w0.w, dot);
-        dot = fmaf(xv[4], w1.x, dot); dot = fmaf(xv[5], w1.y, dot); dot = fmaf(xv[6], w1.z, dot); dot = fmaf(xv[7], w1.w, dot);
+        dot0 = fmaf(xa[0], w0.x, dot0); dot0 = fmaf(xa[1], w0.y, dot0); dot0 = fmaf(xa[2], w0.z, dot0); dot0 = fmaf(xa[3], w0.w, dot0);
+        dot0 = fmaf(xa[4], w1.x, dot0); dot0 = fmaf(xa[5], w1.y, dot0); dot0 = fmaf(xa[6], w1.z, dot0); dot0 = fmaf(xa[7], w1.w, dot0);
+        dot1 = fmaf(xb[0], w0.x, dot1); dot1 = fmaf(xb[1], w0.y, dot1); dot1 = fmaf(xb[2], w0.z, dot1); dot1 = fmaf(xb[3], w0.w, dot1);
+        dot1 = fmaf(xb[4], w1.x, dot1); dot1 = fmaf(xb[5], w1.y, dot1); dot1 = fmaf(xb[6], w1.z, dot1); dot1 = fmaf(xb[7], w1.w, dot1);
       }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-      if (lane == 0) res[b] = dot - a.y[sidx[b]];
+      for (int o = 16; o > 0; o >>= 1) {
+        dot0 += __shfl_xor_sync(0xffffffffu, dot0, o);
+        dot1 += __shfl_xor_sync(0xffffffffu, dot1, o);
+      }
+      if (lane == 0) {
+        res[b] = dot0 - a.y[sidx[b]];
+        if (two) res[b2] = dot1 - a.y[sidx[b2]];
+      }
     }
     __syncthreads();
     float part = 0.f;
@@ -969,7 +982,7 @@ __global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
     if (lane == 0) red[warp] = part;
     // pass 2: this worker's gradient into the running sums (rows come from L2 now)
 #pragma unroll
-    for (int q = 0; q < LSQ_MAX_D / 8 / 256; ++q) {
+    for (int q = 0; q < NV; ++q) {
       const int v = tid + q * 256;
       if (v < nvec) {
 #pragma unroll 8
@@ -994,7 +1007,7 @@ __global__ void __launch_bounds__(256) lsq_grad_v2_kernel(LsqArgs a) {
   if (bad) ri->diverged = 1;
   float* g = a.G + (size_t)blockIdx.x * a.slot_stride;
 #pragma unroll
-  for (int q = 0; q < LSQ_MAX_D / 8 / 256; ++q) {
+  for (int q = 0; q < NV; ++q) {
     const int v = tid + q * 256;
     if (v < nvec) store8(g + (size_t)v * 8, acc[q]);
   }
