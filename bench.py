@@ -348,9 +348,12 @@ def main():
         # least squares reads each minibatch row once: B*d*esz + B*4 bytes per worker-gradient
         esz = 2 if bf16 else 4
         bytes_wg = cfg.batch * cfg.dims[0] * esz + cfg.batch * 4
-        n_l, t_l = prof["lsq"]
+        persistent = prof.get("rounds", (0, 0.0))[0] > 0
+        n_l, t_l = prof["rounds"] if persistent else prof["lsq"]
         ach = wg_p * bytes_wg / (t_l * 1e-3) / 1e9
-        out["roofline"] = {"bound": "hbm", "kernel": "lsq_grad_kernel", "achieved": ach,
+        out["roofline"] = {"bound": "hbm",
+                           "kernel": "abs_lsq_rounds_kernel (whole rounds, latency-bound)" if persistent
+                           else "lsq_grad_kernel", "achieved": ach,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                            "traffic": None, "peak_source": peaks["source"],
                            "share_of_profiled_time": t_l / tot_prof}

@@ -70,6 +70,8 @@ extern "C" {
                                        (tcgen05 cta_group::2, tiles of 256 x 256) */
 #define ABS_FLAG_NO_OVERLAP      2  /* enqueue every kernel on the caller's stream (no side stream for the
                                        server-side kernels of the next round) */
+#define ABS_FLAG_NO_PERSISTENT   8  /* small least-squares problems: one kernel launch per step of a round
+                                       instead of one persistent kernel that runs all enqueued rounds */
 
 /* kernel classes reported by abs_profile_read */
 #define ABS_KC_CTL     0  /* arrival selection + Eq. 4-6 bookkeeping */
@@ -81,7 +83,9 @@ extern "C" {
 #define ABS_KC_BIAS    6  /* bias gradients */
 #define ABS_KC_LSQ     7  /* least-squares residual + gradient */
 #define ABS_KC_UPDATE  8  /* Eq. 3 step + ring write */
-#define ABS_KC_COUNT   9
+#define ABS_KC_ROUNDS  9  /* whole rounds (control step + Eq. 2 + Eq. 3) of a small least-squares problem
+                             in one persistent kernel; one launch per abs_enqueue_rounds call */
+#define ABS_KC_COUNT   10
 
 #define ABS_MAX_LAYERS   7
 #define ABS_MAX_WORKERS  1024

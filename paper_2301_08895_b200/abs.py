@@ -24,7 +24,8 @@ MAX_LAYERS = 7
 FLAG_NO_TENSOR_CORES = 1
 FLAG_NO_OVERLAP = 2
 FLAG_TWO_CTA = 4
-KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update")
+FLAG_NO_PERSISTENT = 8
+KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update", "rounds")
 
 
 class ModelDesc(C.Structure):

@@ -13,6 +13,7 @@
 #include "simt.cuh"
 #include "narrow.cuh"
 #include "tc.cuh"
+#include "persist.cuh"
 
 using namespace absb;
 
@@ -284,6 +285,7 @@ struct abs_ctx {
   int next_cluster = 1;              // cluster width of the next launch (consumed by launch_on)
   bool lsq_v2 = false;               // least squares through the persistent 16-byte-load kernel
   int lsq_grid = 0;                  // its grid = number of partial sums
+  bool lsq_rounds = false;           // small least squares: all enqueued rounds in one persistent kernel
   CtlArgs ctl;
   TcLayer tcl[ABS_MAX_LAYERS];
   CUtensorMap ones_map;
@@ -799,6 +801,16 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     ctx->lsq_v2 = true;
     ctx->lsq_grid = std::min(W, 2 * ctx->sm_count);
   }
+  if (model->kind == ABS_LSQ && !(model->flags & ABS_FLAG_NO_PERSISTENT) && model->dims[0] % 8 == 0 &&
+      model->dims[0] <= LSQ_ROUNDS_MAX_D && W <= LSQ_ROUNDS_NTG && (size_t)W * model->batch <= LSQ_ROUNDS_MAX_ROWS &&
+      (size_t)(staleness_bound + 1) * model->dims[0] * 4 <= 64 * 1024) {
+    const size_t sm = lsq_rounds_smem(staleness_bound, model->dims[0]);
+    cudaError_t er = cudaFuncSetAttribute(abs_lsq_rounds_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (er == cudaSuccess)
+      er = cudaFuncSetAttribute(abs_lsq_rounds_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (er != cudaSuccess) return bail(cuda_fail(nullptr, er, "cudaFuncSetAttribute(abs_lsq_rounds_kernel)"));
+    ctx->lsq_rounds = true;
+  }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);
   // worth it only when a round has a long backward pass to hide behind (tensor-core networks);
@@ -844,7 +856,15 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     if (f32) enqueue_update<float>(ctx, par);
     else enqueue_update<__nv_bfloat16>(ctx, par);
   };
-  if (n > 0 && !ctx->overlap) {
+  if (n > 0 && ctx->lsq_rounds) {
+    LsqRoundsArgs q;
+    q.X = ctx->X; q.y = (const float*)ctx->y;
+    q.master = ctx->at<float>(ctx->L.master); q.ring = ctx->at<void>(ctx->L.ring);
+    q.d_pad = ctx->L.d_pad; q.d = ctx->m.dims[0]; q.lr = ctx->m.lr;
+    const size_t sm = lsq_rounds_smem(ctx->S, q.d);
+    if (f32) launch_ex(ctx, ABS_KC_ROUNDS, abs_lsq_rounds_kernel<float>, dim3(1), dim3(LSQ_ROUNDS_NT), sm, ctx->ctl, q, ctx->rounds_enqueued, n);
+    else launch_ex(ctx, ABS_KC_ROUNDS, abs_lsq_rounds_kernel<__nv_bfloat16>, dim3(1), dim3(LSQ_ROUNDS_NT), sm, ctx->ctl, q, ctx->rounds_enqueued, n);
+  } else if (n > 0 && !ctx->overlap) {
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
       // the control kernel completes the previous round (if any) and selects this round's arrivals

@@ -127,6 +127,7 @@ struct CtlShared {
   int row0[1024];                      // first gradient row of each selected worker
   float lossv[1024];                   // mean minibatch loss of each selected worker
   int version[1024], job[1024];        // per-worker state after the round's bookkeeping
+  int sel_n[1024];                     // worker id of each arrival, in arrival order
   int shard_lo[1024];
   unsigned shard_len[1024];
   float redf[32];
@@ -142,10 +143,8 @@ struct CtlShared {
 // needs is loaded up front in one wave and later phases work from registers and shared memory.
 //   t_sel:     index of the round that follows the open one (the host counts rounds; parity of
 //              t_sel - 1 / t_sel picks the layout copy of the open / the new round)
-__global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select, int t_sel) {
-  grid_dependency_sync();
-  extern __shared__ __align__(16) unsigned char ctl_smem[];
-  CtlShared& sh = *reinterpret_cast<CtlShared*>(ctl_smem);
+template <int NT>
+__device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do_finish, int do_select, int t_sel) {
   DevState* st = a.st;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // ---- one wave of loads
@@ -175,7 +174,7 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     my_sel = a.sel[po][tid]; my_tau = a.sel_tau[po][tid]; my_row0 = a.sel_row0[po][tid];
     if (!net) my_loss = a.loss[tid];
   }
-  if (status0 != ST_OK) return;
+  if (status0 != ST_OK) return 1;
 
   // ------------------------------------------------------------------ finish round t
   if (fin) {
@@ -188,7 +187,7 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
       __syncthreads();
       int kp = 32;
       while (kp < K) kp <<= 1;
-      const int tpw = min(32, 1024 / kp);
+      const int tpw = min(32, NT / kp);
       const int i = tid / tpw, sub = tid - i * tpw;
       float acc = 0.f;
       if (i < K) {
@@ -204,7 +203,7 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     const int bad = __syncthreads_or((tid < K) && !isfinite(my_loss)) || diverged0;
     if (bad) {
       if (tid == 0) { st->status = ST_DIVERGED; st->open = 0; }
-      return;
+      return 1;
     }
     // loss estimate: adjacent-pair tree sum in binary32 over 1024 leaves, /K in binary32
     float v = (tid < K) ? my_loss : 0.f;
@@ -214,7 +213,7 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     sh.flag[tid] = 0;
     __syncthreads();
     if (warp == 0) {
-      float x = sh.redf[lane];
+      float x = (lane < NT / 32) ? sh.redf[lane] : 0.f;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) x = __fadd_rn(x, __shfl_down_sync(0xffffffffu, x, o));
       if (lane == 0) {
@@ -280,7 +279,7 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     if (lane == 0) sh.warp_tot[warp] = __popc(rb);
     range_err = __syncthreads_or(range_err);
     int base = 0, R = 0;
-    for (int w = 0; w < 32; ++w) { const int c = sh.warp_tot[w]; if (w < warp) base += c; R += c; }
+    for (int w = 0; w < NT / 32; ++w) { const int c = sh.warp_tot[w]; if (w < warp) base += c; R += c; }
     if (restart) a.tr_rst_id[rst_off + base + __popc(rb & ((1u << lane) - 1u))] = tid;
     if (tid < K) {
       a.tr_sel_id[sel_off + tid] = my_sel;
@@ -297,26 +296,26 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
       st->L0 = L0; st->theta = theta; st->K = K_next; st->t = t + 1; st->open = 0;
       if (range_err) st->status = ST_RANGE;
     }
-    if (range_err) return;
+    if (range_err) return 1;
     t = t + 1;
     K = K_next;
     __syncthreads();
   }
 
   // ------------------------------------------------------------------ select round t
-  if (!do_select) return;
+  if (!do_select) return 1;
   if (t != t_sel) {                      // host and device disagree on the round index
     if (tid == 0) st->status = ST_INTERNAL;
-    return;
+    return 1;
   }
   if (t >= max_rounds) {
     if (tid == 0) st->status = ST_NOSPACE;
-    return;
+    return 1;
   }
   {
     sh.version[tid] = my_version;
     sh.job[tid] = my_job;
-    for (int i = tid; i < 32 * MAX_TAU; i += 1024) (&sh.wcnt[0][0])[i] = 0;
+    if (net) for (int i = tid; i < 32 * MAX_TAU; i += NT) (&sh.wcnt[0][0])[i] = 0;
     // arrivals: the K smallest (completion tick, worker id) keys; unused slots get distinct
     // keys above every real one
     int n_pow2 = 32;
@@ -332,37 +331,43 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
     const int tau_bad = __syncthreads_or(tid < K && (tau < 0 || tau > S));
     if (tau_bad) {
       if (tid == 0) st->status = ST_INTERNAL;
-      return;
+      return 1;
     }
-    // group the arrivals by staleness (all members of a group read the same ring slot);
-    // inside a group keep arrival order
-    const unsigned peers = __match_any_sync(0xffffffffu, tau);
-    const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
-    if (tau >= 0 && rank_in_warp == 0) sh.wcnt[warp][tau] = (unsigned short)__popc(peers);
-    __syncthreads();
-    if (tid <= S) {
-      int c = 0;
-      for (int w = 0; w < 32; ++w) { const int x = sh.wcnt[w][tid]; sh.wcnt[w][tid] = (unsigned short)c; c += x; }
-      sh.cnt[tid] = c;
-    }
-    __syncthreads();
-    if (tid <= S) {
-      int r0 = 0, g = 0;
-      for (int q = 0; q < tid; ++q) { r0 += round_up(sh.cnt[q] * B, RB); g += sh.cnt[q] > 0; }
-      sh.grow0[tid] = r0;
-      if (tid == S) {
-        sh.scalar[0] = r0 + round_up(sh.cnt[S] * B, RB);
-        sh.scalar[1] = g + (sh.cnt[S] > 0);
+    // network models: group the arrivals by staleness (all members of a group read the same
+    // ring slot); inside a group keep arrival order.  Least squares needs no row layout.
+    int row0_me = tid * B;
+    if (net) {
+      const unsigned peers = __match_any_sync(0xffffffffu, tau);
+      const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+      if (tau >= 0 && rank_in_warp == 0) sh.wcnt[warp][tau] = (unsigned short)__popc(peers);
+      __syncthreads();
+      if (tid <= S) {
+        int c = 0;
+        for (int w = 0; w < 32; ++w) { const int x = sh.wcnt[w][tid]; sh.wcnt[w][tid] = (unsigned short)c; c += x; }
+        sh.cnt[tid] = c;
       }
+      __syncthreads();
+      if (tid <= S) {
+        int r0 = 0, g = 0;
+        for (int q = 0; q < tid; ++q) { r0 += round_up(sh.cnt[q] * B, RB); g += sh.cnt[q] > 0; }
+        sh.grow0[tid] = r0;
+        if (tid == S) {
+          sh.scalar[0] = r0 + round_up(sh.cnt[S] * B, RB);
+          sh.scalar[1] = g + (sh.cnt[S] > 0);
+        }
+      }
+      __syncthreads();
+      if (tid < K) row0_me = sh.grow0[tau] + ((int)sh.wcnt[warp][tau] + rank_in_warp) * B;
     }
-    __syncthreads();
-    const int n_rows = sh.scalar[0];
+    const int n_rows = net ? sh.scalar[0] : K * B;
+    const int n_groups = net ? sh.scalar[1] : 0;
     if (tid < K) {
-      const int row0 = sh.grow0[tau] + ((int)sh.wcnt[warp][tau] + rank_in_warp) * B;
+      const int row0 = row0_me;
       a.sel[pn][tid] = n;
       a.sel_tau[pn][tid] = tau;
       a.sel_row0[pn][tid] = row0;
       sh.row0[tid] = row0;
+      sh.sel_n[tid] = n;
       sh.flag[tid] = 0;
       if (net) {
         const i64 lo = ((i64)n * n_samples) / W, hi = ((i64)(n + 1) * n_samples) / W;
@@ -374,18 +379,19 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
       st->T_end = T_end;
       st->n_rows = n_rows;
       st->n_row_tiles = n_rows / RB;
-      st->n_groups = sh.scalar[1];
+      st->n_groups = n_groups;
       st->open = 1;
       RoundInfo info;
       info.n_rows = n_rows; info.K = K; info.t = t; info.diverged = 0;
       a.ri[pn] = info;
+      sh.scalar[4] = K; sh.scalar[5] = t;
     }
-    if (!net) return;             // least squares: no row tiles, minibatches drawn by its own kernel
+    if (!net) return 0;           // least squares: no row tiles, minibatches drawn by its own kernel
     __syncthreads();
     // ring slot of every row tile and padding rows
     {
       const int n_tiles = n_rows / RB;
-      for (int q = tid; q < n_tiles; q += 1024) {
+      for (int q = tid; q < n_tiles; q += NT) {
         const int r = q * RB;
         int g = 0;                                  // last non-empty group starting at or before r
         for (int u = 0; u <= S; ++u) if (sh.cnt[u] > 0 && sh.grow0[u] <= r) g = u;
@@ -395,13 +401,13 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
         const int c = sh.cnt[g];
         if (c == 0) continue;
         const int p0 = sh.grow0[g] + c * B, p1 = sh.grow0[g] + round_up(c * B, RB);
-        for (int r = p0 + tid; r < p1; r += 1024) a.row_idx[pn][r] = -1;
+        for (int r = p0 + tid; r < p1; r += NT) a.row_idx[pn][r] = -1;
       }
     }
     // minibatch draws: sample b of job (n, j) = word b%4 of Philox block (n, j, 1, b/4),
     // mapped into the worker's shard [n M / N, (n+1) M / N)
     const int blocks_per = (B + 3) >> 2;
-    for (int item = tid; item < K * blocks_per; item += 1024) {
+    for (int item = tid; item < K * blocks_per; item += NT) {
       const int i = item / blocks_per, blk = item - i * blocks_per;
       const int wn = (int)(sorted[i] & 1023ull);
       uint32_t w4[4];
@@ -415,6 +421,14 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
       }
     }
   }
+  return 0;
+}
+
+__global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select, int t_sel) {
+  grid_dependency_sync();
+  extern __shared__ __align__(16) unsigned char ctl_smem[];
+  CtlShared& sh = *reinterpret_cast<CtlShared*>(ctl_smem);
+  ctl_round<1024>(a, sh, do_finish, do_select, t_sel);
 }
 
 // Duration look-ahead (see refresh_next_durations): one warp per 32 workers.
