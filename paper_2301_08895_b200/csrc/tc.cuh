@@ -8,7 +8,8 @@
 // "s" is the ring slot of the row tile's model version (all rows of a 128-row tile share it).
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the tensor-memory allocation),
-// warps 2..5 = epilogue (tensor memory -> registers -> global).  Two accumulators alternate so the
+// warps 2..9 = epilogue (tensor memory -> registers -> global; two warps per tensor-memory lane
+// quarter, each draining one half of the tile's columns).  Two accumulators alternate so the
 // epilogue of one tile overlaps the main loop of the next.  Every mbarrier wait is bounded; on
 // expiry the CTA raises ST_TIMEOUT, drains its own copies, frees tensor memory and returns.
 #pragma once
@@ -22,7 +23,8 @@ namespace tc {
 constexpr int BM = 128;      // tile rows (UMMA M)
 constexpr int BK = 64;       // k elements per stage = one 128-byte swizzle row of bf16
 constexpr int UK = 16;       // k per tcgen05.mma of kind::f16
-constexpr int THREADS = 192;
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 64 + 32 * EPI_WARPS;
 
 enum Mode : int { FWD = 0, DGRAD = 1, WGRAD = 2 };
 
@@ -185,7 +187,7 @@ template <int BN, int CG = 1> struct Cfg {
   static constexpr int B_BYTES = (BN / CG) * BK * 2;     // with a CTA pair each CTA holds half of the B tile
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int OUT_BYTES = 2 * 4 * 4096;       // epilogue staging: 2 buffers x 4 warps x (32 rows x 128 B)
+  static constexpr int OUT_BYTES = EPI_WARPS * 4096;   // epilogue staging: one box of 32 rows x 128 B per warp
   static constexpr size_t SMEM_BYTES =
       (size_t)STAGES * STAGE_BYTES + OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 2 * BN * 2 /*bias*/;
 };
@@ -238,7 +240,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4 * CG); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS * CG); }
     *abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -391,15 +393,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (4 warps)
-    // Results leave through per-warp staging boxes (32 rows x 128 bytes, 128-byte swizzle, two
-    // per warp) and one bulk tensor store per box, so global memory sees whole rows instead of 32
-    // scattered 16-byte pieces per store instruction and a warp never waits for another warp.
+    // ------------------------------------------------------------------ epilogue (8 warps)
+    // Results leave through per-warp staging boxes (32 rows x 128 bytes, 128-byte swizzle) and one
+    // bulk tensor store per box, so global memory sees whole rows instead of 32 scattered 16-byte
+    // pieces per store instruction and a warp never waits for another warp.
     const int q = warp & 3;                    // tensor-memory lane quarter this warp may read
+    const int half = (warp - 2) >> 2;          // which half of the tile's columns this warp drains
+    constexpr int N_HALF = (BN >= 128) ? 2 : 1;      // a 64-column tile is drained by four warps only
+    constexpr int HALF_COLS = BN / N_HALF;
+    const bool works = half < N_HALF;
     const int row_in_tile = q * 32 + lane;
     const bool issuer = lane == 0;             // issues and tracks this warp's bulk stores
     const int sw = lane & 7;
-    int box_no = 0;
+    uint8_t* my_box = stage_out + ((warp - 2) << 12);
+    uint8_t* my_row = my_box + lane * 128;
     const int box_cols = (mode == WGRAD) ? 32 : 64;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -413,15 +420,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       __nv_bfloat16* bias_t = bias_s + acc * BN;
       if (mode == FWD) {
         const __nv_bfloat16* bias = p.ring + (size_t)c.slot * p.slot_stride + p.b_off;
-        for (int i = (int)threadIdx.x - 64; i < BN; i += 128) {
+        for (int i = (int)threadIdx.x - 64; i < BN; i += 32 * EPI_WARPS) {
           const int n = c.b_col + i;
           bias_t[i] = n < p.N_total ? bias[n] : __float2bfloat16_rn(0.f);
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI_WARPS) : "memory");
       } else if (mode == DGRAD) {
 #pragma unroll
         for (int i = 0; i < BN / 32; ++i) {
           const int w = c.b_col / 32 + i;
+          if (i * 32 / HALF_COLS != half) { mw[i] = 0u; continue; }
           if (p.mask_bits != nullptr) {
             mw[i] = w < p.mask_words ? p.mask_bits[(size_t)r * p.mask_words + w] : 0u;
           } else {                               // no stored sign bits: derive them from the activations
@@ -440,15 +448,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += box_cols) {
+      for (int c0 = half * HALF_COLS; c0 < (half + 1) * HALF_COLS && works; c0 += box_cols) {
         const int n0 = c.b_col + c0;
-        if (n0 >= p.N_total) break;            // uniform in the CTA
-        // this warp's staging box is free once its store before the previous one has been read
-        uint8_t* my_box = stage_out + (((box_no & 1) * 4 + q) << 12);
-        uint8_t* my_row = my_box + lane * 128;
-        ++box_no;
-        if (issuer) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-        __syncwarp();
+        if (n0 >= p.N_total) break;            // uniform in the warp
         uint32_t v[32];
         if (mode == WGRAD) {
           if (have) tmem_ld32(t_row + (uint32_t)c0, v);
@@ -456,6 +458,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0u;
           }
+          // the staging box is free once the bulk store issued from it has read it
+          if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          __syncwarp();
           if (c.bias_tile) {                   // a single useful row: plain stores
             if (row_in_tile == 0 && rank == 0) {
               float* dst = p.out_f32 + (size_t)c.split * p.slot_stride + (size_t)r * p.N_total + n0;
@@ -478,6 +483,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             else {
 #pragma unroll
               for (int i = 0; i < 32; ++i) v[i] = 0u;
+            }
+            if (hlf == 0) {                     // the staging box is free once its last store has read it
+              if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+              __syncwarp();
             }
             uint32_t bits = 0u;
             if (mode == DGRAD) {
@@ -538,7 +547,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (acc == 0) acc_phase ^= 1u;
       }
     }
-    if (issuer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    // shared memory may be released once the stores have read it; their global writes complete
+    // with the grid
+    if (issuer) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
   }
 
   // ------------------------------------------------------------------ teardown
