@@ -13,6 +13,7 @@
 #include "simt.cuh"
 #include "narrow.cuh"
 #include "tc.cuh"
+#include "outlayer.cuh"
 #include "persist.cuh"
 
 using namespace absb;
@@ -59,6 +60,7 @@ struct Layout {
   bool two_cta = false;                 // GEMMs with N >= 256 run on CTA pairs (tiles of 256 x 256)
   int cg_fwd[ABS_MAX_LAYERS] = {}, cg_dg[ABS_MAX_LAYERS] = {}, cg_wg[ABS_MAX_LAYERS] = {};
   int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
+  bool out_mma = false;                 // output layer through the mma.sync kernel (bf16, 64 rows per CTA)
   size_t esz = 4;                       // bytes per stored element (4 or 2)
   size_t d = 0, d_pad = 0;
   size_t w_off[ABS_MAX_LAYERS] = {};    // element offset of W_l inside the padded vector
@@ -152,6 +154,11 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       if (L->two_cta) {
         if (out >= 256) { L->cg_fwd[l] = 2; L->bn_fwd[l] = 256; L->cg_wg[l] = 2; L->bn_wg[l] = 256; }
         if (in >= 256) { L->cg_dg[l] = 2; L->bn_dg[l] = 256; }
+      } else if ((size_t)in * out >= ((size_t)1 << 21) && in >= 256 && out >= 256 && W * m->batch >= 4096) {
+        // a large weight gradient is bound by operand traffic into shared memory: CTA pairs halve
+        // the B operand each CTA has to stage (its tiles are features x outputs, so the row padding
+        // unit of the version groups is not involved)
+        L->cg_wg[l] = 2; L->bn_wg[l] = 256;
       }
     }
     // split count P of the row reduction: the one that minimises the modelled time of all weight
@@ -216,6 +223,8 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
         for (int R : {32, 16, 8})     // (rows, transposed weights in fp32 or storage type, stored weights, deltas)
           if ((size_t)R * inl * L->esz + (size_t)C * (inl + 8) * 4 + (size_t)(inl + 1) * C * L->esz + 64 +
                   (size_t)R * 64 <= 100 * 1024) { L->fused_R = R; break; }
+      L->out_mma = L->fused_R && tc_ok && m->n_layers > 1 &&
+                   (inl == 128 || inl == 256 || inl == 512 || inl == 1024);
       L->red = cv.take(4 * len * (size_t)(L->rows_cap / (L->fused_R ? L->fused_R : 64)));
     }
     L->ones = L->any_tc ? cv.take(2 * 64 * (size_t)L->rows_cap) : 0;
@@ -543,13 +552,21 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (L.fused_R) {
-        const int R = L.fused_R;
+        int R = L.fused_R;
         const size_t sm = sizeof(T) * ((size_t)R * a.in + (size_t)a.C * (a.in + 8) + (size_t)(a.in + 1) * a.C) + 64 +
                           sizeof(float) * (size_t)R * NARROW_MAX_C;
         float* part = ctx->at<float>(L.red);
         float* dstw = ctx->at<float>(L.G) + L.w_off[l];
         const int len = (a.in + 1) * a.C, has_dgrad = l > 0 ? 1 : 0;
-        if (a.C == 10) {
+        if (L.out_mma) {
+          const dim3 og(L.rows_cap / outl::ROWS), ob(outl::THREADS);
+          const size_t osm = outl::smem_bytes(a.in, a.C);
+          if (a.in == 128) launch_ex(ctx, ABS_KC_OUTPUT, outl::out_layer_mma_kernel<1>, og, ob, osm, a, part, has_dgrad);
+          else if (a.in == 256) launch_ex(ctx, ABS_KC_OUTPUT, outl::out_layer_mma_kernel<2>, og, ob, osm, a, part, has_dgrad);
+          else if (a.in == 512) launch_ex(ctx, ABS_KC_OUTPUT, outl::out_layer_mma_kernel<4>, og, ob, osm, a, part, has_dgrad);
+          else launch_ex(ctx, ABS_KC_OUTPUT, outl::out_layer_mma_kernel<8>, og, ob, osm, a, part, has_dgrad);
+          R = outl::ROWS;
+        } else if (a.C == 10) {
           const size_t smc = sizeof(T) * ((size_t)R * a.in + (size_t)(a.in + 1) * 10) + 32 +
                              sizeof(float) * ((size_t)10 * (a.in + 4) + (size_t)R * 10);
           launch_ex(ctx, ABS_KC_OUTPUT, narrow_fused_cc_kernel<T, 10>, dim3(L.rows_cap / R), dim3(256), smc, a, part, R, has_dgrad);
@@ -786,6 +803,14 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     const cudaError_t ea = cudaFuncSetAttribute(abs_ctl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 (int)sizeof(CtlShared));
     if (ea != cudaSuccess) return bail(cuda_fail(nullptr, ea, "cudaFuncSetAttribute(abs_ctl_kernel)"));
+  }
+  if (L.out_mma) {
+    const int osm = (int)outl::smem_bytes(model->dims[model->n_layers - 1], model->dims[model->n_layers]);
+    cudaError_t eo = cudaFuncSetAttribute(outl::out_layer_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, osm);
+    if (eo == cudaSuccess) eo = cudaFuncSetAttribute(outl::out_layer_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, osm);
+    if (eo == cudaSuccess) eo = cudaFuncSetAttribute(outl::out_layer_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, osm);
+    if (eo == cudaSuccess) eo = cudaFuncSetAttribute(outl::out_layer_mma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, osm);
+    if (eo != cudaSuccess) return bail(cuda_fail(nullptr, eo, "cudaFuncSetAttribute(out_layer_mma_kernel)"));
   }
   if (L.fused_R) {
     cudaError_t ef = cudaFuncSetAttribute(narrow_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);

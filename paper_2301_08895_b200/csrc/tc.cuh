@@ -39,7 +39,8 @@ struct Params {
   int P;                   // WGRAD split count
   const __nv_bfloat16* ring; size_t slot_stride; size_t b_off;   // FWD bias: ring + slot*stride + b_off
   const __nv_bfloat16* mask_src;   // DGRAD: H[r][N_total] (used when mask_bits is null)
-  const uint32_t* mask_bits;       // DGRAD: bit n%32 of word [r][n/32] = (H[r][n] > 0)
+  const uint32_t* mask_bits;       // DGRAD: word [r][n/32] holds (H[r][n] > 0) for its 32 columns, column j of
+                                   // the word at bit (j >> 1) + 16 * (j & 1) (even columns low half, odd high)
   uint32_t* relu_bits;             // FWD: the same bits for this layer's output (may be null)
   int mask_words;                  // words per row of mask_bits / relu_bits = ceil(N_total / 32)
   __nv_bfloat16* out_bf16;         // FWD/DGRAD result [rows][N_total]
@@ -436,7 +437,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t bits = 0u;
             for (int j = 0; j < 32; ++j) {
               const int n = w * 32 + j;
-              if (n < p.N_total && __bfloat162float(p.mask_src[(size_t)r * p.N_total + n]) > 0.f) bits |= 1u << j;
+              if (n < p.N_total && __bfloat162float(p.mask_src[(size_t)r * p.N_total + n]) > 0.f)
+                bits |= 1u << ((j >> 1) + 16 * (j & 1));
             }
             mw[i] = bits;
           }
@@ -500,20 +502,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const int i = 8 * j + 2 * e;
+                const int i = 8 * j + 2 * e;    // columns i, i + 1 = pair i / 2 of the 32-column word
                 float x = __uint_as_float(v[i]), y = __uint_as_float(v[i + 1]);
                 if (mode == FWD) {
                   const float2 bf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(bias_t + cc + i));
                   x = fmaxf(x + bf.x, 0.f);
                   y = fmaxf(y + bf.y, 0.f);
-                } else {
-                  x = ((bits >> i) & 1u) ? x : 0.f;
-                  y = ((bits >> (i + 1)) & 1u) ? y : 0.f;
                 }
                 o2[e] = __floats2bfloat162_rn(x, y);
-                if (mode == FWD) {             // the bit records the sign of the STORED activation
-                  relu |= (__low2float(o2[e]) > 0.f ? 1u : 0u) << i;
-                  relu |= (__high2float(o2[e]) > 0.f ? 1u : 0u) << (i + 1);
+                uint32_t& u = *reinterpret_cast<uint32_t*>(&o2[e]);
+                if (mode == FWD) {
+                  // The bit records the sign of the STORED activation.  Stored values are >= 0, so
+                  // "positive" = "magnitude bits non-zero": adding 0x7fff carries into bit 15 of each
+                  // half exactly then.  After 16 pairs the flags of pair q sit at bits q and 16 + q.
+                  relu = (relu >> 1) | (((u & 0x7fff7fffu) + 0x7fff7fffu) & 0x80008000u);
+                } else {
+                  u &= ((bits >> (i >> 1)) & 0x00010001u) * 0xffffu;
                 }
               }
               *reinterpret_cast<uint4*>(my_row + (((4 * hlf + j) ^ sw) << 4)) = o;
