@@ -70,6 +70,10 @@ extern "C" {
                                        (tcgen05 cta_group::2, tiles of 256 x 256) */
 #define ABS_FLAG_NO_OVERLAP      2  /* enqueue every kernel on the caller's stream (no side stream for the
                                        server-side kernels of the next round) */
+#define ABS_FLAG_TMA_GATHER     16  /* tensor-core networks: the first layer's GEMMs fetch the minibatch rows
+                                       from the dataset by row index (TMA four-row gathers) instead of reading
+                                       a dense copy made by a separate kernel; same results, slower when a row
+                                       tile is shared by several column tiles (each re-gathers it) */
 #define ABS_FLAG_NO_PERSISTENT   8  /* small least-squares problems: one kernel launch per step of a round
                                        instead of one persistent kernel that runs all enqueued rounds */
 

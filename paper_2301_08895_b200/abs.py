@@ -25,6 +25,7 @@ FLAG_NO_TENSOR_CORES = 1
 FLAG_NO_OVERLAP = 2
 FLAG_TWO_CTA = 4
 FLAG_NO_PERSISTENT = 8
+FLAG_TMA_GATHER = 16
 KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update", "rounds")
 
 

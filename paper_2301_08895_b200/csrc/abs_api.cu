@@ -57,6 +57,7 @@ struct Layout {
   int path[ABS_MAX_LAYERS] = {};        // how each layer's contractions run
   int bn_fwd[ABS_MAX_LAYERS] = {}, bn_dg[ABS_MAX_LAYERS] = {}, bn_wg[ABS_MAX_LAYERS] = {};
   bool any_tc = false;
+  bool gather_tma = false;              // first-layer GEMMs fetch the minibatch rows from the dataset themselves
   bool two_cta = false;                 // GEMMs with N >= 256 run on CTA pairs (tiles of 256 x 256)
   int cg_fwd[ABS_MAX_LAYERS] = {}, cg_dg[ABS_MAX_LAYERS] = {}, cg_wg[ABS_MAX_LAYERS] = {};
   int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
@@ -130,6 +131,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     } else L->path[l] = PATH_SIMT;
   }
   L->two_cta = L->any_tc && (m->flags & ABS_FLAG_TWO_CTA);
+  L->gather_tma = !lsq && L->path[0] == PATH_TC && (m->flags & ABS_FLAG_TMA_GATHER);
   L->RB = lsq ? m->batch : (L->any_tc ? (L->two_cta ? 256 : 128) : 64);
   const int groups = (W < S + 1) ? W : S + 1;
   L->rows_cap = round_up(W * m->batch, L->RB) + groups * L->RB;
@@ -231,8 +233,9 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     for (int l = 0; l <= m->n_layers; ++l) L->bits[l] = 0;
     for (int l = 0; l + 1 < m->n_layers; ++l)
       if (L->path[l] == PATH_TC) L->bits[l + 1] = cv.take(4 * (size_t)L->rows_cap * ((m->dims[l + 1] + 31) / 32));
-    L->act[0] = (L->path[0] == PATH_TC) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
-    L->act0b = (L->path[0] == PATH_TC) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
+    const bool copy0 = L->path[0] == PATH_TC && !L->gather_tma;     // gathered copies of the input rows
+    L->act[0] = copy0 ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
+    L->act0b = copy0 ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     for (int l = 1; l <= m->n_layers; ++l) {
       L->act[l] = (l < m->n_layers) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]) : 0;
       L->delta[l] = cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]);
@@ -264,6 +267,7 @@ struct TcLayer {
   CUtensorMap fwd_a, fwd_b, dg_a, dg_b, wg_a, wg_b;
   CUtensorMap fwd_out, dg_out, wg_out;     // result tensors written by bulk tensor stores
   CUtensorMap fwd_a_odd, wg_a_odd;         // layer 0 only: operand maps over the second gathered copy
+  CUtensorMap x_rows;                      // layer 0 only: the dataset with a one-row box (row gathers)
 };
 
 // ones[r][0] = 1 (bf16), the rest of the 64-wide rows stays zero: the extra operand row that turns
@@ -446,18 +450,21 @@ int setup_tc(abs_ctx* ctx) {
     if (L.path[l] != PATH_TC) continue;
     const int in = m.dims[l], out = m.dims[l + 1];
     TcLayer& t = ctx->tcl[l];
-    const void* act_in = ctx->at<void>(L.act[l]);
+    const bool from_x = l == 0 && L.gather_tma;      // no gathered copy: fwd_a / wg_a stay unused
+    const void* act_in = from_x ? ctx->X : ctx->at<void>(L.act[l]);
     const void* delta_out = ctx->at<void>(L.delta[l + 1]);
     const void* wbase = ring + 2 * L.w_off[l];
-    bool ok = make_act_map(&t.fwd_a, act_in, in, L.rows_cap, 128) &&
+    bool ok = (from_x || make_act_map(&t.fwd_a, act_in, in, L.rows_cap, 128)) &&
               make_w_map(&t.fwd_b, wbase, in, out, ctx->S + 1, L.d_pad, 64) &&
-              make_act_map(&t.wg_a, act_in, in, L.rows_cap, 64) &&
+              (from_x || make_act_map(&t.wg_a, act_in, in, L.rows_cap, 64)) &&
               make_act_map(&t.wg_b, delta_out, out, L.rows_cap, 64) &&
               make_act_map(&t.fwd_out, ctx->at<void>(L.act[l + 1]), out, L.rows_cap, 32) &&
               make_g_map(&t.wg_out, ctx->at<float>(L.G) + L.w_off[l], in, out, L.P, L.d_pad);
-    if (ok && l == 0)
+    if (ok && l == 0 && !L.gather_tma)
       ok = make_act_map(&t.fwd_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 128) &&
            make_act_map(&t.wg_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 64);
+    if (ok && l == 0 && L.gather_tma)
+      ok = make_act_map(&t.x_rows, ctx->X, in, (int)m.n_samples, 1);
     if (ok && l > 0)
       ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
            make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l] / L.cg_dg[l]) &&
@@ -519,6 +526,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     p.st = st; p.ri = ri; p.tile_slot = ctx->ctl.tile_slot[par]; p.mode = mode; p.P = L.P;
     p.ring = ctx->at<__nv_bfloat16>(L.ring); p.slot_stride = L.d_pad;
     p.b_off = L.w_off[l] + (size_t)m.dims[l] * m.dims[l + 1];
+    if (l == 0 && L.gather_tma && mode != tc::DGRAD) { p.gather_a = 1; p.row_idx = ctx->ctl.row_idx[par]; }
     return p;
   };
   auto narrow_args = [&](int l) {
@@ -533,7 +541,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     return a;
   };
   if (phase == PH_GATHER) {
-    if (gathered)
+    if (gathered && !L.gather_tma)
       launch_on(ctx, ctx->overlap ? ctx->side : s, ABS_KC_GATHER, gather_rows_kernel, dim3(ctx->sm_count * 8), dim3(256), 0,
                 st, ri, ctx->ctl.row_idx[par], (const __nv_bfloat16*)ctx->X, ctx->at<__nv_bfloat16>(par ? L.act0b : L.act[0]), m.dims[0]);
     return;
@@ -548,7 +556,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       p.relu_bits = L.bits[l + 1] ? ctx->at<uint32_t>(L.bits[l + 1]) : nullptr;
       p.mask_words = (la[l].out + 31) / 32;
       const int bn = L.bn_fwd[l];
-      launch_tc_bn(ctx, bn, L.cg_fwd[l], ABS_KC_FWD, (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, (row_tiles128 / L.cg_fwd[l]) * ((la[l].out + bn - 1) / bn));
+      launch_tc_bn(ctx, bn, L.cg_fwd[l], ABS_KC_FWD, (l == 0 && L.gather_tma) ? ctx->tcl[l].x_rows : (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, (row_tiles128 / L.cg_fwd[l]) * ((la[l].out + bn - 1) / bn));
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (L.fused_R) {
@@ -613,7 +621,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       p.out_f32 = ctx->at<float>(L.G) + L.w_off[l];
       const int bn = L.bn_wg[l];
       const int tmw = 128 * L.cg_wg[l];
-      launch_tc_bn(ctx, bn, L.cg_wg[l], ABS_KC_WGRAD, (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
+      launch_tc_bn(ctx, bn, L.cg_wg[l], ABS_KC_WGRAD, (l == 0 && L.gather_tma) ? ctx->tcl[l].x_rows : (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
                    ((la[l].in + tmw - 1) / tmw + 1) * ((la[l].out + bn - 1) / bn) * L.P);
     } else if (L.path[l] == PATH_NARROW && L.fused_R) {
       // forward, loss, delta of the layer below and the gradient were all done by the fused kernel

@@ -43,6 +43,9 @@ struct Params {
                                    // the word at bit (j >> 1) + 16 * (j & 1) (even columns low half, odd high)
   uint32_t* relu_bits;             // FWD: the same bits for this layer's output (may be null)
   int mask_words;                  // words per row of mask_bits / relu_bits = ceil(N_total / 32)
+  const int* row_idx;              // gather_a: sample index of every gradient row (-1 = padding row)
+  int gather_a;                    // FWD/WGRAD: operand A is the dataset, its rows fetched by row_idx
+                                   // (map_a then describes X with a one-row box)
   __nv_bfloat16* out_bf16;         // FWD/DGRAD result [rows][N_total]
   float* out_f32;                  // WGRAD: G + w_off, partial p at + p*slot_stride, row pitch N_total
 };
@@ -149,6 +152,20 @@ __device__ __forceinline__ void tma2_load_3d(void* dst, const CUtensorMap* map, 
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+// Four rows of a 2-D tensor (rows given by index, columns [x, x + box width)) into four consecutive
+// 128-byte rows of a swizzled tile.
+__device__ __forceinline__ void tma_gather4(void* dst, const CUtensorMap* map, uint64_t* bar, int x, const int4& r) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w)
+      : "memory");
+}
+__device__ __forceinline__ void tma2_gather4(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, const int4& r) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w)
       : "memory");
 }
 __device__ __forceinline__ void umma2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -292,53 +309,111 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      int armed[C::STAGES];
-      for (int s = 0; s < C::STAGES; ++s) armed[s] = -1;
-      bool ok = true;
-      // loads complete on the leader's "full" barrier (own barrier when CG == 1)
-      auto ld2 = [&](void* dst, const CUtensorMap* map, int st_, int x, int y) {
-        if (CG == 2) tma2_load_2d(dst, map, full0_addr + 8u * (uint32_t)st_, x, y);
-        else tma_load_2d(dst, map, &full[st_], x, y);
+    int stage = 0;
+    uint32_t phase = 0;
+    int armed[C::STAGES];
+    for (int s = 0; s < C::STAGES; ++s) armed[s] = -1;
+    bool ok = true;
+    // loads complete on the leader's "full" barrier (own barrier when CG == 1)
+    auto ld2 = [&](void* dst, const CUtensorMap* map, int st_, int x, int y) {
+      if (CG == 2) tma2_load_2d(dst, map, full0_addr + 8u * (uint32_t)st_, x, y);
+      else tma_load_2d(dst, map, &full[st_], x, y);
+    };
+    auto ld3 = [&](void* dst, const CUtensorMap* map, int st_, int x, int y, int z) {
+      if (CG == 2) tma2_load_3d(dst, map, full0_addr + 8u * (uint32_t)st_, x, y, z);
+      else tma_load_3d(dst, map, &full[st_], x, y, z);
+    };
+    constexpr int BH = BN / CG;                  // B columns (rows of the B tile) this CTA loads
+    if (p.gather_a == 0) {
+      // one elected lane: the stage ring is shallow, so nothing may sit between a stage being
+      // released and its next loads being issued
+      if (lane == 0) {
+        for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
+          const TileCoord c = tile_coord(tile);
+          const int b0 = c.b_col + rank * BH;
+          for (int kb = 0; kb < c.n_kb; ++kb) {
+            if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) { ok = false; break; }
+            uint8_t* sa = smem + (size_t)stage * C::STAGE_BYTES;
+            uint8_t* sb = sa + C::A_BYTES;
+            if (rank == 0) {                     // the leader arms the barrier for the bytes of the whole pair
+              mbar_expect_tx(&full[stage], CG * C::STAGE_BYTES);
+              armed[stage] = (int)phase;
+            }
+            const int k0 = c.k_begin + kb * BK;
+            if (mode == FWD) {
+              ld2(sa, &map_a, stage, k0, c.a_row);
+              for (int j = 0; j < BH / 64; ++j) ld3(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0, c.slot);
+            } else if (mode == DGRAD) {
+              ld2(sa, &map_a, stage, k0, c.a_row);
+              ld3(sb, &map_b, stage, k0, b0, c.slot);
+            } else {
+              if (c.bias_tile) {   // only column 0 of the 64-wide ones matrix is non-zero; the rest is zero fill
+                for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_ones, stage, rank * BM + 64 * j, k0);
+              } else {
+                for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_a, stage, c.a_row + 64 * j, k0);
+              }
+              for (int j = 0; j < BH / 64; ++j) ld2(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0);
+            }
+            if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    } else {
+      // Operand A is the minibatch itself (first layer, FWD or WGRAD): its rows are fetched straight
+      // from the dataset by row index.  Lane 0 waits, arms the barrier and issues the tiled B loads;
+      // then every lane issues one four-row gather (32 x 4 = the 128 rows of a K-major tile, or
+      // the 64 rows x two 64-feature boxes of an MN-major one).  Rows of padding (index -1) lie
+      // outside the tensor and arrive as zeros.
+      auto ldg4 = [&](void* dst, int st_, int x, const int4& r) {
+        if (CG == 2) tma2_gather4(dst, &map_a, full0_addr + 8u * (uint32_t)st_, x, r);
+        else tma_gather4(dst, &map_a, &full[st_], x, r);
       };
-      auto ld3 = [&](void* dst, const CUtensorMap* map, int st_, int x, int y, int z) {
-        if (CG == 2) tma2_load_3d(dst, map, full0_addr + 8u * (uint32_t)st_, x, y, z);
-        else tma_load_3d(dst, map, &full[st_], x, y, z);
-      };
-      constexpr int BH = BN / CG;                // B columns (rows of the B tile) this CTA loads
       for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
         const TileCoord c = tile_coord(tile);
         const int b0 = c.b_col + rank * BH;
+        const bool g_tile = !(mode == WGRAD && c.bias_tile);
+        // sample indices of the rows this lane gathers: fixed per tile (K-major A: the tile's
+        // rows), or per stage (MN-major A: the stage's 64 reduction rows, fetched one stage ahead)
+        int4 ridx = make_int4(-1, -1, -1, -1);
+        if (g_tile && c.n_kb > 0)
+          ridx = *reinterpret_cast<const int4*>(p.row_idx + (mode == WGRAD ? c.k_begin + 4 * (lane & 15) : c.a_row + 4 * lane));
         for (int kb = 0; kb < c.n_kb; ++kb) {
-          if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) { ok = false; break; }
           uint8_t* sa = smem + (size_t)stage * C::STAGE_BYTES;
           uint8_t* sb = sa + C::A_BYTES;
-          if (rank == 0) {                       // the leader arms the barrier for the bytes of the whole pair
-            mbar_expect_tx(&full[stage], CG * C::STAGE_BYTES);
-            armed[stage] = (int)phase;
-          }
           const int k0 = c.k_begin + kb * BK;
-          if (mode == FWD) {
-            ld2(sa, &map_a, stage, k0, c.a_row);
-            for (int j = 0; j < BH / 64; ++j) ld3(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0, c.slot);
-          } else if (mode == DGRAD) {
-            ld2(sa, &map_a, stage, k0, c.a_row);
-            ld3(sb, &map_b, stage, k0, b0, c.slot);
-          } else {
-            if (c.bias_tile) {   // only column 0 of the 64-wide ones matrix is non-zero; the rest is zero fill
-              for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_ones, stage, rank * BM + 64 * j, k0);
-            } else {
-              for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_a, stage, c.a_row + 64 * j, k0);
+          int4 rnext = ridx;
+          if (g_tile && mode == WGRAD && kb + 1 < c.n_kb)
+            rnext = *reinterpret_cast<const int4*>(p.row_idx + k0 + BK + 4 * (lane & 15));
+          if (lane == 0) {
+            ok = mbar_wait(&empty[stage], phase ^ 1u, abort);
+            if (ok && rank == 0) {
+              mbar_expect_tx(&full[stage], CG * C::STAGE_BYTES);
+              armed[stage] = (int)phase;
             }
-            for (int j = 0; j < BH / 64; ++j) ld2(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0);
+          }
+          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+          if (!ok) break;
+          if (lane == 0) {
+            if (mode == FWD) {
+              for (int j = 0; j < BH / 64; ++j) ld3(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0, c.slot);
+            } else {
+              if (c.bias_tile)
+                for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_ones, stage, rank * BM + 64 * j, k0);
+              for (int j = 0; j < BH / 64; ++j) ld2(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0);
+            }
+          }
+          if (g_tile) {
+            if (mode == WGRAD) ldg4(sa + (lane >> 4) * 8192 + (lane & 15) * 512, stage, c.a_row + 64 * (lane >> 4), ridx);
+            else ldg4(sa + lane * 512, stage, k0, ridx);
+            ridx = rnext;
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      // tail: every stage's release (an asynchronous arrive from the tensor core) must have landed
-      // before this CTA's shared memory goes away
+    }
+    // tail: every stage's release (an asynchronous arrive from the tensor core) must have landed
+    // before this CTA's shared memory goes away
+    if (lane == 0) {
       for (int s = 0; s < C::STAGES && ok; ++s) {
         if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) ok = false;
         if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }

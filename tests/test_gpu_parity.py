@@ -226,6 +226,21 @@ def test_side_stream_overlap_changes_nothing(idx, rounds, n):
     assert np.array_equal(params_a, params_b)
 
 
+@pytest.mark.parametrize("dims,B", [((3072, 1024, 512, 10), 64), ((320, 520, 264, 10), 40), ((784, 256, 10), 128)])
+def test_tma_row_gather_matches_the_copy_kernel(dims, B):
+    """With the flag the first layer's GEMMs fetch the minibatch rows from the dataset by row index
+    (TMA four-row gathers) instead of reading the dense copy made by the gather kernel.  Both feed
+    the tensor cores the same operands, so traces and parameters must be identical bit for bit,
+    and both agree with the oracle."""
+    cfg = _small_cfg(inputs.MLP, dims, inputs.BF16, 13, B, 3, 5, PARETO)
+    X, y, w0 = _problem(cfg)
+    rows_a, params_a = gpu_run(cfg, X, y, w0, 25)
+    rows_b, params_b = gpu_run(cfg, X, y, w0, 25, flags=gpu.FLAG_TMA_GATHER)
+    assert rows_a == rows_b
+    assert np.array_equal(params_a, params_b)
+    compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_TMA_GATHER)
+
+
 def test_cta_pair_gemms_match_single_cta_gemms():
     """Opt-in tcgen05 cta_group::2 tiles (256 x 256 over a CTA pair) against the default tiles."""
     cfg = _small_cfg(inputs.MLP, (320, 520, 264, 10), inputs.BF16, 13, 40, 3, 5, PARETO)
