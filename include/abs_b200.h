@@ -74,6 +74,8 @@ extern "C" {
                                        from the dataset by row index (TMA four-row gathers) instead of reading
                                        a dense copy made by a separate kernel; same results, slower when a row
                                        tile is shared by several column tiles (each re-gathers it) */
+#define ABS_FLAG_NO_BULK_PIPELINE 32 /* bf16 least squares: per-warp 16-byte loads (rows read from HBM, then again
+                                       from L2) instead of the bulk-copy pipeline through shared memory */
 #define ABS_FLAG_NO_PERSISTENT   8  /* small least-squares problems: one kernel launch per step of a round
                                        instead of one persistent kernel that runs all enqueued rounds */
 

@@ -26,6 +26,7 @@ FLAG_NO_OVERLAP = 2
 FLAG_TWO_CTA = 4
 FLAG_NO_PERSISTENT = 8
 FLAG_TMA_GATHER = 16
+FLAG_NO_BULK_PIPELINE = 32
 KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update", "rounds")
 
 

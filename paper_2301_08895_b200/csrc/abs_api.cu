@@ -14,6 +14,7 @@
 #include "narrow.cuh"
 #include "tc.cuh"
 #include "outlayer.cuh"
+#include "lsqpipe.cuh"
 #include "persist.cuh"
 
 using namespace absb;
@@ -296,6 +297,8 @@ struct abs_ctx {
   long long launches = 0;
   cudaError_t launch_error = cudaSuccess;
   int next_cluster = 1;              // cluster width of the next launch (consumed by launch_on)
+  bool lsq_pipe = false;             // bf16 least squares through the bulk-copy pipeline kernel
+  int lsq_stages = 0;
   bool lsq_v2 = false;               // least squares through the persistent 16-byte-load kernel
   int lsq_grid = 0;                  // its grid = number of partial sums
   bool lsq_rounds = false;           // small least squares: all enqueued rounds in one persistent kernel
@@ -493,7 +496,15 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     a.X = ctx->X; a.y = (const float*)ctx->y;
     a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad;
     a.loss = ctx->ctl.loss; a.G = ctx->at<float>(L.G); a.d = m.dims[0];
-    if (ctx->lsq_v2) {
+    if (ctx->lsq_pipe) {
+      lsqp::Args q;
+      q.st = st; q.ri = ri; q.sel = a.sel; q.job = a.job; q.sel_tau = a.sel_tau;
+      q.X = (const __nv_bfloat16*)ctx->X; q.y = a.y; q.ring = (const __nv_bfloat16*)a.ring; q.slot_stride = a.slot_stride;
+      q.loss_part = ctx->at<float>(L.row_loss); q.G = a.G; q.d = a.d; q.stages = ctx->lsq_stages;
+      q.groups = (m.batch + lsqp::GROUP - 1) / lsqp::GROUP;
+      const size_t sm = lsqp::smem_bytes(a.d, ctx->lsq_stages);
+      launch_ex(ctx, ABS_KC_LSQ, lsqp::lsq_pipe_kernel, dim3(ctx->lsq_grid), dim3(lsqp::THREADS), sm, q);
+    } else if (ctx->lsq_v2) {
       const size_t smw = sizeof(float) * (size_t)a.d;
       const int nv = (a.d + 2047) / 2048;
       if (nv <= 1) launch_ex(ctx, ABS_KC_LSQ, lsq_grad_v2_kernel<T, 1>, dim3(ctx->lsq_grid), dim3(256), smw, a);
@@ -663,6 +674,8 @@ void enqueue_update(abs_ctx* ctx, int par) {
     q.st = ctx->at<DevState>(L.st); q.ri = ri; q.job = ctx->ctl.job; q.next_dur = ctx->ctl.next_dur; q.dur_job = ctx->ctl.dur_job;
     q.master = ctx->at<float>(L.master); q.ring = ctx->at<void>(L.ring); q.G = ctx->at<float>(L.G);
     q.d_pad = L.d_pad; q.d = ctx->m.dims[0]; q.P = ctx->lsq_grid; q.lr = ctx->m.lr;
+    q.loss_part = ctx->lsq_pipe ? ctx->at<float>(L.row_loss) : nullptr;
+    q.loss = ctx->ctl.loss; q.groups = (ctx->m.batch + lsqp::GROUP - 1) / lsqp::GROUP;
     const int blocks = std::max((q.d + 31) / 32, (ctx->W + 31) / 32);
     launch_ex(ctx, ABS_KC_UPDATE, lsq_update_kernel<T>, dim3(blocks), dim3(256), 0, q);
     return;
@@ -833,6 +846,19 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   if (model->kind == ABS_LSQ && model->dims[0] % 8 == 0 && model->dims[0] <= LSQ_MAX_D) {
     ctx->lsq_v2 = true;
     ctx->lsq_grid = std::min(W, 2 * ctx->sm_count);
+    // bf16 rows of up to 8 KB: stream them through shared memory with bulk copies, one CTA per SM
+    if (model->dtype == ABS_BF16_FP32MASTER && model->dims[0] <= 4096 && !(model->flags & ABS_FLAG_NO_BULK_PIPELINE)) {
+      int stages = lsqp::MAX_STAGES;
+      while (stages >= 2 && lsqp::smem_bytes(model->dims[0], stages) > 227 * 1024) --stages;
+      if (stages >= 2) {
+        const int sm = (int)lsqp::smem_bytes(model->dims[0], stages);
+        cudaError_t ep = cudaFuncSetAttribute(lsqp::lsq_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+        if (ep != cudaSuccess) return bail(cuda_fail(nullptr, ep, "cudaFuncSetAttribute(lsq_pipe_kernel)"));
+        ctx->lsq_pipe = true;
+        ctx->lsq_stages = stages;
+        ctx->lsq_grid = std::min(W, ctx->sm_count);
+      }
+    }
   }
   if (model->kind == ABS_LSQ && !(model->flags & ABS_FLAG_NO_PERSISTENT) && model->dims[0] % 8 == 0 &&
       model->dims[0] <= LSQ_ROUNDS_MAX_D && W <= LSQ_ROUNDS_NTG && (size_t)W * model->batch <= LSQ_ROUNDS_MAX_ROWS &&

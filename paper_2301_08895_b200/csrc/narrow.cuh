@@ -1015,10 +1015,13 @@ __global__ void __launch_bounds__(256, 2) lsq_grad_v2_kernel(LsqArgs a) {
 
 struct LsqUpdateArgs {
   const DevState* st;
-  const RoundInfo* ri;
+  RoundInfo* ri;
   const int* job; u64* next_dur; int* dur_job;
   float* master; void* ring; const float* G;
   size_t d_pad; int d; int P; float lr;
+  // when the gradient kernel leaves per-item loss sums (worker i, row group g): this kernel
+  // finishes the uploaded losses loss[i] = (sum_g loss_part[i * groups + g]) / B
+  const float* loss_part; float* loss; int groups;
 };
 
 // Eq. 3 for least squares: the P per-CTA partial sums are added in a fixed order (32 parameters x
@@ -1029,10 +1032,26 @@ __global__ void __launch_bounds__(256) lsq_update_kernel(LsqUpdateArgs a) {
   grid_dependency_sync();
   __shared__ float red[8][33];
   const DevState* st = a.st;
-  const RoundInfo* ri = a.ri;
+  RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   if (ri->diverged) return;
   const int K = ri->K;
+  if (a.loss_part != nullptr) {
+    // every block adds the loss sums up the same way, so all of them agree on whether a
+    // non-finite loss was uploaded (then Eq. 3 is not applied); block 0 publishes the losses
+    bool bad = false;
+    for (int i = threadIdx.x; i < K; i += 256) {
+      float s = 0.f;
+      for (int g = 0; g < a.groups; ++g) s += a.loss_part[(size_t)i * a.groups + g];
+      const float loss = __fdiv_rn(s, (float)st->B);
+      if (blockIdx.x == 0) a.loss[i] = loss;
+      bad |= !isfinite(loss);
+    }
+    if (__syncthreads_or(bad ? 1 : 0)) {
+      if (blockIdx.x == 0 && threadIdx.x == 0) ri->diverged = 1;
+      return;
+    }
+  }
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int j = blockIdx.x * 32 + lane;
   float acc = 0.f;

@@ -252,6 +252,22 @@ def test_cta_pair_gemms_match_single_cta_gemms():
     compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_TWO_CTA)
 
 
+@pytest.mark.parametrize("d,W,B,K0,S", [(4096, 200, 32, 25, 32), (1000, 160, 19, 7, 6), (2056, 300, 8, 300, 0)])
+def test_lsq_bulk_copy_pipeline_and_plain_load_kernels(d, W, B, K0, S):
+    """bf16 least squares streams the minibatch rows through shared memory with bulk copies (one
+    persistent CTA per SM, items of 8 rows); the flag keeps the kernel that reads rows with plain
+    16-byte loads.  Summation orders differ, so the two agree to rounding, and each agrees with
+    the oracle (integer trace exactly, with the oracle's K rule fed the uploaded losses)."""
+    cfg = _small_cfg(inputs.LSQ, (d, 1), inputs.BF16, W, B, K0, S, EXP, n=20000, lr=0.002)
+    X, y, w0 = _problem(cfg)
+    rows_a, _, err_a, _ = compare_with_oracle(cfg, X, y, w0, 30, TOL_BF16, forced=True)
+    rows_b, _, err_b, _ = compare_with_oracle(cfg, X, y, w0, 30, TOL_BF16, forced=True, flags=gpu.FLAG_NO_BULK_PIPELINE)
+    la = np.concatenate([r["sel_loss"] for r in rows_a])
+    lb = np.concatenate([r["sel_loss"] for r in rows_b])
+    if [r["sel"] for r in rows_a] == [r["sel"] for r in rows_b]:
+        assert np.allclose(la, lb, rtol=1e-4, atol=1e-6)
+
+
 # Small least-squares problems run all enqueued rounds inside one persistent kernel; the flag
 # keeps the one-launch-per-step path in use, and both must agree with the oracle.
 @pytest.mark.parametrize("flags", [0, gpu.FLAG_NO_PERSISTENT])
