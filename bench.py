@@ -27,9 +27,11 @@ sys.path.insert(0, ROOT)
 from paper_2301_08895_b200 import inputs  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes (read + write) per launch of the tensor-core GEMM kernel at K = N on configuration 4, from the ncu
-# capture summarised in profiles/tc_gemm_kernel_cfg4.md; valid only for the kernel source it was taken from.
-GEMM_TRAFFIC = {"config": 4, "bytes_per_launch": 38.6e6, "tc_cuh_sha256_16": "ab2a2a44b30ac923"}
+# DRAM bytes (read + write) per launch at K = N on configuration 4, from the ncu captures summarised in
+# profiles/tc_gemm_kernel_cfg4.md and profiles/update_kernel_cfg4.md; each figure is valid only for the kernel
+# source it was taken from (first 16 hex digits of the file's sha256).
+TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 39.7e6, "file": "tc.cuh", "sha256_16": "b1e563028d097907"},
+           "update": {"config": 4, "bytes_per_launch": 75.7e6, "file": "simt.cuh", "sha256_16": "3da31ad4d03aac5c"}}
 METRIC = "worker_gradients_per_sec"
 UNIT = "worker-gradients/s"
 
@@ -46,20 +48,20 @@ def load_peaks():
     return p
 
 
-def gemm_traffic(config_index):
+def measured_traffic(which, config_index, full_size):
     import hashlib
-    path = os.path.join(ROOT, "paper_2301_08895_b200", "csrc", "tc.cuh")
+    t = TRAFFIC[which]
+    path = os.path.join(ROOT, "paper_2301_08895_b200", "csrc", t["file"])
     with open(path, "rb") as f:
         sha = hashlib.sha256(f.read()).hexdigest()[:16]
-    if config_index == GEMM_TRAFFIC["config"] and sha == GEMM_TRAFFIC["tc_cuh_sha256_16"]:
-        return GEMM_TRAFFIC["bytes_per_launch"]
+    if full_size and config_index == t["config"] and sha == t["sha256_16"]:
+        return t["bytes_per_launch"]
     return None            # kernel changed since the counters were taken (or another workload)
 
 
 def workload_name(cfg, rounds):
-    return "config%s %s: dims %s, W=%d, B=%d, K0=%d, S=%d, %d rounds" % (
-        cfg.name.split("_")[0], cfg.name, "-".join(str(d) for d in cfg.dims), cfg.W, cfg.batch,
-        cfg.K0, cfg.S, rounds)
+    return "%s: dims %s, W=%d, B=%d, K0=%d, S=%d, %d samples, %d rounds" % (
+        cfg.name, "-".join(str(d) for d in cfg.dims), cfg.W, cfg.batch, cfg.K0, cfg.S, cfg.n_samples, rounds)
 
 
 # ------------------------------------------------------------------ flop / byte models
@@ -175,6 +177,8 @@ def main():
     ap.add_argument("--workers", type=int, default=None, help="W of configuration 5")
     ap.add_argument("--rounds", type=int, default=None, help="rounds per step (default: the configuration's)")
     ap.add_argument("--flags", type=int, default=0, help="ABS_FLAG_* bits passed to abs_init")
+    ap.add_argument("--samples", type=int, default=None,
+                    help="dataset rows (default: the configuration's; smaller for profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work")
     args = ap.parse_args()
 
@@ -183,6 +187,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
     cfg = inputs.config(args.config, args.workers)
+    if args.samples:
+        cfg = cfg.scaled(n_samples=args.samples)
     if world > 1:
         from paper_2301_08895_b200 import multi
         cfg.run_seed = multi.replica_seed(cfg.run_seed, rank)   # independent replicas, one per GPU
@@ -353,7 +359,8 @@ def main():
         ach = wg_p * bytes_wg / (t_l * 1e-3) / 1e9
         out["roofline"] = {"bound": "hbm",
                            "kernel": "abs_lsq_rounds_kernel (whole rounds, latency-bound)" if persistent
-                           else "lsq_grad_kernel", "achieved": ach,
+                           else ("lsq_pipe_kernel" if bf16 and cfg.dims[0] <= 4096 and not (args.flags & 32)
+                                 else "lsq_grad_v2_kernel"), "achieved": ach,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                            "traffic": None, "peak_source": peaks["source"],
                            "share_of_profiled_time": t_l / tot_prof}
@@ -364,7 +371,7 @@ def main():
         peak = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
         out["roofline"] = {"bound": "tensor", "kernel": "tc_gemm_kernel (fwd+dgrad+wgrad launches)",
                            "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                           "traffic": gemm_traffic(args.config), "peak_source": peaks["source"] + " (sustained bf16)",
+                           "traffic": measured_traffic("gemm", args.config, not args.samples), "peak_source": peaks["source"] + " (sustained bf16)",
                            "frac_of_burst_peak": ach / peaks["bf16_tflops"],
                            "share_of_profiled_time": t_g / tot_prof,
                            "per_class_tflops": {c: wg_p * flops[c] / (prof[c][1] * 1e-3) / 1e12
@@ -384,7 +391,8 @@ def main():
                                   "avg_us": 1e3 * t_u / n_u, "partials": P,
                                   "bytes_per_launch": bytes_launch, "achieved": ach,
                                   "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                  "frac": ach / peaks["hbm_gbs"], "traffic": None}
+                                  "frac": ach / peaks["hbm_gbs"],
+                                  "traffic": measured_traffic("update", args.config, not args.samples)}
     out["plan"] = plan
     out["_profiled_worker_gradients"] = wg_p
     out["cpu_baseline"] = time_oracle(cfg, X, y, w0, rounds, args.cpu_budget)
