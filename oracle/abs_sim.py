@@ -36,7 +36,7 @@ import numpy as np
 from . import models, philox, timing
 
 K_ADAPTIVE, K_FIXED = 0, 1
-BOUND_ADAPTIVE, BOUND_FIXED = 0, 1
+BOUND_ADAPTIVE, BOUND_FIXED, BOUND_OFFSET = 0, 1, 2
 
 
 class Diverged(Exception):
@@ -115,6 +115,14 @@ def theta_rule(W, k0, S, k):
     return min(S, max(1, math.floor(real_threshold)))
 
 
+def theta_offset_rule(W, S, k, a):
+    """Eq. 4 as printed, with the constant a given: max{1, N/K + a}, floored
+    (an integer age exceeds a real threshold iff it exceeds its floor; a is an
+    integer here, as in the paper's experiments, Sec. V-B) and capped by the
+    staleness bound S the model store is sized for."""
+    return min(S, max(1, math.floor(Fraction(W, k) + a)))
+
+
 class ABSOracle:
     """State of one simulated run.
 
@@ -127,7 +135,8 @@ class ABSOracle:
     dist, seed     time distribution and the Philox seed
     quant          round to bfloat16 at the storage points (bf16 configurations)
     k_mode         K_ADAPTIVE (Eq. 5) or K_FIXED
-    bound_mode     BOUND_ADAPTIVE (Eq. 4) or BOUND_FIXED (theta = S always)
+    bound_mode     BOUND_ADAPTIVE (Eq. 4 with a = S - N/K^0), BOUND_FIXED (theta = S
+                   always) or BOUND_OFFSET (Eq. 4 with the integer `bound_offset` as a)
     literal_eq6    test the pre-increment age against the threshold exactly as
                    Eq. 6 is printed (one round later than Algorithm 1's order)
     integer_only   play only the server's integer machinery (arrivals, Eq. 4-6,
@@ -137,7 +146,7 @@ class ABSOracle:
 
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, dist, seed,
                  quant=False, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE,
-                 literal_eq6=False, x_is_bf16_bits=False, integer_only=False):
+                 literal_eq6=False, x_is_bf16_bits=False, integer_only=False, bound_offset=0):
         if not (1 <= K0 <= W):
             raise ValueError("need 1 <= K0 <= W")
         if S < 0:
@@ -151,6 +160,9 @@ class ABSOracle:
         self.dist, self.seed = dist, int(seed)
         self.quant = bool(quant)
         self.k_mode, self.bound_mode = k_mode, bound_mode
+        self.bound_offset = int(bound_offset)
+        if bound_mode == BOUND_OFFSET and theta_offset_rule(self.W, 10 ** 9, self.K0, self.bound_offset) > self.S:
+            raise ValueError("staleness bound below the initial threshold N/K0 + a")
         self.literal_eq6 = literal_eq6
         self.integer_only = integer_only
         self.w = np.array(w0, dtype=np.float64)
@@ -238,6 +250,8 @@ class ABSOracle:
             K_next = K
         if self.bound_mode == BOUND_ADAPTIVE:
             theta = theta_rule(self.W, self.K0, self.S, K_next)         # Eq. 4
+        elif self.bound_mode == BOUND_OFFSET:
+            theta = theta_offset_rule(self.W, self.S, K_next, self.bound_offset)
         else:
             theta = self.S
 

@@ -78,6 +78,16 @@ def duration_word(seed, n, j):
     return philox4x32_10((n, j, TAG_DURATION, 0), seed_key(seed))[0]
 
 
+def duration_words(seed, n, j, count):
+    """`count` words of the job-duration stream of job j of worker n: word i is
+    word (i mod 4) of block (n, j, TAG_DURATION, i // 4); word 0 is
+    `duration_word`."""
+    out = []
+    for blk in range((count + 3) // 4):
+        out.extend(int(x) for x in philox4x32_10((n, j, TAG_DURATION, blk), seed_key(seed)))
+    return out[:count]
+
+
 def minibatch_words(seed, n, j, batch):
     """`batch` 32-bit words for the minibatch of job j of worker n:
     sample b uses word (b mod 4) of block (n, j, TAG_MINIBATCH, b // 4)."""

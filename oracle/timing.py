@@ -13,6 +13,11 @@ bit for bit:
            -ln_spec(u) / rate                             EXP
            shift + (-ln_spec(u) / rate)                   SHIFTED_EXP
            scale / sqrt(u)                                PARETO2 (shape 2)
+           shift + (e_0 + e_1 + ... + e_{k-1}) / rate     GAMMA, integer shape k >= 1:
+               e_i = -ln_spec(u_i), u_i from word i mod 4 of Philox block
+               (n, j, 0, i div 4); the sum runs left to right.  A sum of k
+               independent Exp(rate) times is Gamma(k, rate), the law the paper
+               draws its execution times from (Sec. V-A); k = 1 is SHIFTED_EXP
     dur *= slow_factor   if slow_mod > 0 and n mod slow_mod == slow_rem
     ticks = floor(dur * 2**20), at least 1, and below 2**53
 
@@ -27,7 +32,8 @@ import struct
 
 from . import philox
 
-CONST, EXP, SHIFTED_EXP, PARETO2 = 0, 1, 2, 3
+CONST, EXP, SHIFTED_EXP, PARETO2, GAMMA = 0, 1, 2, 3, 4
+MAX_SHAPE = 64
 TICKS_PER_UNIT = 2.0 ** 20
 MAX_TICKS = 1 << 53
 
@@ -39,7 +45,7 @@ class TimeDist:
     """Plain record of the distribution parameters."""
 
     def __init__(self, kind, shift=0.0, rate=1.0, scale=1.0,
-                 slow_mod=0, slow_rem=0, slow_factor=1.0):
+                 slow_mod=0, slow_rem=0, slow_factor=1.0, shape=1):
         self.kind = int(kind)
         self.shift = float(shift)
         self.rate = float(rate)
@@ -47,6 +53,7 @@ class TimeDist:
         self.slow_mod = int(slow_mod)
         self.slow_rem = int(slow_rem)
         self.slow_factor = float(slow_factor)
+        self.shape = int(shape)
 
 
 def ln_spec(u):
@@ -79,10 +86,18 @@ def uniform_from_word(r):
     return (float(r) + 0.5) * (2.0 ** -32)
 
 
-def duration_from_word(dist, n, r):
-    """Ticks of a job of worker n whose Philox word is r."""
+def duration_from_word(dist, n, r, more_words=None):
+    """Ticks of a job of worker n whose Philox word is r (GAMMA: `more_words`
+    are the words 1 .. shape-1 of the job)."""
     u = uniform_from_word(r)
-    if dist.kind == CONST:
+    if dist.kind == GAMMA:
+        if not (1 <= dist.shape <= MAX_SHAPE):
+            raise ValueError("gamma shape out of range")
+        total = -ln_spec(u)
+        for i in range(1, dist.shape):
+            total = total + (-ln_spec(uniform_from_word(more_words[i - 1])))
+        dur = dist.shift + total / dist.rate
+    elif dist.kind == CONST:
         dur = dist.shift
     elif dist.kind == EXP:
         dur = (-ln_spec(u)) / dist.rate
@@ -103,4 +118,7 @@ def duration_from_word(dist, n, r):
 
 def duration_ticks(dist, seed, n, j):
     """Ticks of job j of worker n under `seed`."""
+    if dist.kind == GAMMA and dist.shape > 1:
+        words = philox.duration_words(seed, n, j, dist.shape)
+        return duration_from_word(dist, n, words[0], words[1:])
     return duration_from_word(dist, n, philox.duration_word(seed, n, j))

@@ -147,3 +147,41 @@ def test_minibatch_indices_stay_in_shard():
     # draws spread over the whole shard
     idx = np.concatenate([abs_sim.minibatch_indices(1, 0, j, 64, 2, 1000) for j in range(200)])
     assert idx.min() < 10 and idx.max() >= 490 and abs(idx.mean() - 249.5) < 5
+
+
+def test_gamma_shape_one_is_shifted_exponential():
+    """Gamma(1, rate) = Exp(rate): the same Philox word, the same operations, the same ticks."""
+    g1 = timing.TimeDist(timing.GAMMA, shift=0.5, rate=2.0, shape=1)
+    se = timing.TimeDist(timing.SHIFTED_EXP, shift=0.5, rate=2.0)
+    for n in range(12):
+        for j in range(12):
+            assert timing.duration_ticks(g1, 9, n, j) == timing.duration_ticks(se, 9, n, j)
+
+
+def test_gamma_is_a_sum_of_exponentials_of_distinct_words():
+    """Shape k adds k exponential draws taken from k different Philox words of the job (words
+    0..3 of block 0, then block 1, ...); a repeated or skipped word would break the sum below."""
+    seed, n, j, k, rate = 77, 3, 11, 6, 1.25
+    words = philox.duration_words(seed, n, j, k)
+    assert len(set(words)) == k and words[0] == philox.duration_word(seed, n, j)
+    blk1 = philox.philox4x32_10((n, j, philox.TAG_DURATION, 1), philox.seed_key(seed))
+    assert words[4] == blk1[0] and words[5] == blk1[1]
+    exp1 = timing.TimeDist(timing.EXP, rate=rate)
+    parts = [timing.duration_from_word(exp1, n, w) for w in words]           # ticks of each draw
+    g = timing.TimeDist(timing.GAMMA, shift=0.0, rate=rate, shape=k)
+    total = timing.duration_ticks(g, seed, n, j)
+    assert abs(total - sum(parts)) <= k            # each part was floored on its own
+
+
+def test_gamma_moments_and_cdf():
+    """Mean k/rate, variance k/rate^2, and the distribution function against scipy's."""
+    from scipy import stats
+    k, rate = 3, 1.5
+    g = timing.TimeDist(timing.GAMMA, shift=0.0, rate=rate, shape=k)
+    v = np.array([timing.duration_ticks(g, 5, n, j) for n in range(150) for j in range(100)]) / 2.0 ** 20
+    assert abs(v.mean() - k / rate) < 0.03
+    assert abs(v.var() - k / rate ** 2) < 0.06
+    for x in (0.5, 1.0, 2.0, 4.0):
+        assert abs((v < x).mean() - stats.gamma.cdf(x, a=k, scale=1.0 / rate)) < 0.015
+    with pytest.raises(ValueError):
+        timing.duration_ticks(timing.TimeDist(timing.GAMMA, shape=0), 1, 0, 0)

@@ -197,6 +197,41 @@ def test_theta_table():
     assert abs_sim.theta_rule(8, 8, 0, 8) == 0           # bound 0 overrides the floor of 1
 
 
+def test_theta_offset_table():
+    """Eq. 4 with the constant a given (values of the paper's sweep, Sec. V-B)."""
+    with open(os.path.join(GOLDEN, "theta_offset_table.txt")) as f:
+        rows = [tuple(int(v) for v in line.split()) for line in f
+                if line.strip() and not line.startswith("#")]
+    assert len(rows) >= 20
+    for W, S, K, a, theta in rows:
+        assert abs_sim.theta_offset_rule(W, S, K, a) == theta
+
+
+def test_offset_mode_equals_derived_offset_when_k0_divides_n():
+    """BOUND_ADAPTIVE derives a = S - N/K0 from the staleness bound; when K0 divides N that a is
+    an integer and BOUND_OFFSET with it must play the very same rounds."""
+    X, y, _ = _lsq_problem(400, 6, seed=3)
+    dist = timing.TimeDist(timing.GAMMA, shift=0.25, rate=1.0, shape=2)
+    W, K0, S = 12, 3, 6                      # N/K0 = 4, a = 2
+    a = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, W, K0, S, dist, 5)
+    b = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, W, K0, S, dist, 5,
+                  bound_mode=abs_sim.BOUND_OFFSET, bound_offset=S - W // K0)
+    ra, rb = a.run(60), b.run(60)
+    assert ra == rb
+    assert any(r["restart"] for r in ra)
+    # a smaller offset discards more: restarts cannot decrease (qualitative claim of Sec. V-B)
+    c = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, W, K0, S, dist, 5,
+                  k_mode=abs_sim.K_FIXED, bound_mode=abs_sim.BOUND_OFFSET, bound_offset=2)
+    d = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, W, K0, S, dist, 5,
+                  k_mode=abs_sim.K_FIXED, bound_mode=abs_sim.BOUND_OFFSET, bound_offset=-1)
+    n_c = sum(len(r["restart"]) for r in c.run(60))
+    n_d = sum(len(r["restart"]) for r in d.run(60))
+    assert n_d >= n_c and n_d > 0
+    with pytest.raises(ValueError):
+        ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, W, K0, 3, dist, 5,
+                  bound_mode=abs_sim.BOUND_OFFSET, bound_offset=2)
+
+
 def test_loss_estimate_order_and_rounding():
     f = np.float32
     assert abs_sim.tree_sum([1.0, 2.0, 3.0]) == 6.0
