@@ -135,7 +135,7 @@ def oracle_for(cfg, X, y, w0):
     bf16 = cfg.dtype == inputs.BF16
     return abs_sim.ABSOracle(cfg.kind, cfg.dims, X, y, w0, cfg.batch, cfg.lr, cfg.W, cfg.K0, cfg.S,
                              timing.TimeDist(ts.kind, ts.shift, ts.rate, ts.scale, ts.slow_mod,
-                                             ts.slow_rem, ts.slow_factor),
+                                             ts.slow_rem, ts.slow_factor, ts.shape),
                              cfg.run_seed, quant=bf16, x_is_bf16_bits=bf16)
 
 

@@ -58,12 +58,16 @@ extern "C" {
 #define ABS_K_FIXED         1   /* K^t = K0 for all t (K-sync / K-async / ASGD baselines, Sec. II-B) */
 #define ABS_BOUND_ADAPTIVE  0   /* threshold from Eq. 4, capped by the staleness bound */
 #define ABS_BOUND_FIXED     1   /* threshold = staleness bound in every round (Fig. 1 setting) */
+#define ABS_BOUND_OFFSET    2   /* Eq. 4 with the constant a given: max(1, floor(N/K) + bound_offset), capped by
+                                   the staleness bound (the sweep over a of Sec. V-B) */
 
 /* execution-time laws (random execution times with stragglers, Sec. V-A) */
 #define ABS_T_CONST        0    /* shift */
 #define ABS_T_EXP          1    /* Exp(rate) */
 #define ABS_T_SHIFTED_EXP  2    /* shift + Exp(rate) */
 #define ABS_T_PARETO2      3    /* Pareto, shape 2, minimum `scale` */
+#define ABS_T_GAMMA        4    /* shift + Gamma(shape, rate), integer shape in [1, 64]: the sum of `shape`
+                                   exponential draws (the law the paper draws execution times from) */
 
 #define ABS_FLAG_NO_TENSOR_CORES 1  /* run the hidden-layer contractions on the FP32-FMA kernels */
 #define ABS_FLAG_TWO_CTA         4  /* hidden-layer GEMMs with >= 256 output columns run on CTA pairs
@@ -110,6 +114,8 @@ typedef struct {
   int local_steps;          /* U of Eq. 2; must be 1 */
   int k_mode;               /* ABS_K_* */
   int bound_mode;           /* ABS_BOUND_* */
+  int bound_offset;         /* the constant a of Eq. 4 when bound_mode = ABS_BOUND_OFFSET (else ignored);
+                               floor(N/K0) + a must not exceed the staleness bound */
   int max_rounds;           /* trace capacity: total rounds this context may run */
   int flags;                /* ABS_FLAG_* bits */
   int data_on_host;         /* 0: X, y are device pointers owned by the caller and must outlive
@@ -129,6 +135,7 @@ typedef struct {
   double shift, rate, scale;
   int slow_mod, slow_rem;   /* workers with n % slow_mod == slow_rem are slow (slow_mod 0: none) */
   double slow_factor;       /* their durations are multiplied by this */
+  int shape;                /* ABS_T_GAMMA: number of exponential draws summed (else ignored) */
 } abs_time_dist;
 
 /* Caller-owned host arrays receiving rounds [first_round, first_round + n_rounds).

@@ -18,8 +18,8 @@ OK, EINVAL, ENOSPACE, EUNSUPPORTED, ESTATE, ECUDA, ETIMEOUT, EDIVERGED, ERANGE =
 LSQ, SOFTMAX, MLP = 0, 1, 2
 FP32, BF16_FP32MASTER = 0, 1
 K_ADAPTIVE, K_FIXED = 0, 1
-BOUND_ADAPTIVE, BOUND_FIXED = 0, 1
-T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2 = 0, 1, 2, 3
+BOUND_ADAPTIVE, BOUND_FIXED, BOUND_OFFSET = 0, 1, 2
+T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2, T_GAMMA = 0, 1, 2, 3, 4
 MAX_LAYERS = 7
 FLAG_NO_TENSOR_CORES = 1
 FLAG_NO_OVERLAP = 2
@@ -34,7 +34,7 @@ class ModelDesc(C.Structure):
     _fields_ = [("kind", C.c_int), ("n_layers", C.c_int), ("dims", C.c_int * (MAX_LAYERS + 1)),
                 ("batch", C.c_int), ("lr", C.c_float), ("dtype", C.c_int),
                 ("local_steps", C.c_int), ("k_mode", C.c_int), ("bound_mode", C.c_int),
-                ("max_rounds", C.c_int), ("flags", C.c_int), ("data_on_host", C.c_int),
+                ("bound_offset", C.c_int), ("max_rounds", C.c_int), ("flags", C.c_int), ("data_on_host", C.c_int),
                 ("X", C.c_void_p), ("y", C.c_void_p), ("n_samples", C.c_longlong),
                 ("w0", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("stream", C.c_void_p)]
@@ -43,7 +43,7 @@ class ModelDesc(C.Structure):
 class TimeDist(C.Structure):
     _fields_ = [("kind", C.c_int), ("shift", C.c_double), ("rate", C.c_double),
                 ("scale", C.c_double), ("slow_mod", C.c_int), ("slow_rem", C.c_int),
-                ("slow_factor", C.c_double)]
+                ("slow_factor", C.c_double), ("shape", C.c_int)]
 
 
 class Trace(C.Structure):
@@ -113,7 +113,7 @@ def n_params(kind, dims):
 
 
 def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-          local_steps=1, data_on_host=0, flags=0):
+          local_steps=1, data_on_host=0, flags=0, bound_offset=0):
     m = ModelDesc()
     m.kind, m.n_layers = kind, len(dims) - 1
     for i, v in enumerate(dims):
@@ -122,6 +122,7 @@ def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mod
     m.local_steps, m.k_mode, m.bound_mode = local_steps, k_mode, bound_mode
     m.max_rounds, m.data_on_host, m.n_samples = int(max_rounds), data_on_host, int(n_samples)
     m.flags = int(flags)
+    m.bound_offset = int(bound_offset)
     return m
 
 
@@ -143,14 +144,14 @@ class Context:
 
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, time, seed, max_rounds,
                  dtype=FP32, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE, local_steps=1,
-                 data_on_host=False, stream=None, device="cuda:0", flags=0):
+                 data_on_host=False, stream=None, device="cuda:0", flags=0, bound_offset=0):
         import torch
         self._torch = torch
         self.kind, self.dims, self.W, self.S = kind, list(dims), W, S
         self.max_rounds = max_rounds
         n_samples = X.shape[0]
         m = _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-                  local_steps, 1 if data_on_host else 0, flags)
+                  local_steps, 1 if data_on_host else 0, flags, bound_offset)
         need = C.c_size_t(0)
         _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(need)))
         self.device = torch.device(device)
@@ -172,7 +173,7 @@ class Context:
         m.workspace, m.workspace_bytes = self.workspace.data_ptr(), need.value
         m.stream = self.stream.cuda_stream
         td = TimeDist(time.kind, time.shift, time.rate, time.scale, time.slow_mod, time.slow_rem,
-                      time.slow_factor)
+                      time.slow_factor, getattr(time, "shape", 1))
         self._ctx = C.c_void_p(None)
         self._desc = m
         _check(lib().abs_init(C.byref(self._ctx), C.byref(m), W, K0, S, C.byref(td),

@@ -735,13 +735,22 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     return fail(ABS_EUNSUPPORTED, "local_steps = %d: only U = 1 is implemented", model->local_steps);
   if (K0 < 1 || K0 > W) return fail(ABS_EINVAL, "K0 %d outside [1, W]", K0);
   if (model->k_mode != ABS_K_ADAPTIVE && model->k_mode != ABS_K_FIXED) return fail(ABS_EINVAL, "k_mode");
-  if (model->bound_mode != ABS_BOUND_ADAPTIVE && model->bound_mode != ABS_BOUND_FIXED)
+  if (model->bound_mode != ABS_BOUND_ADAPTIVE && model->bound_mode != ABS_BOUND_FIXED &&
+      model->bound_mode != ABS_BOUND_OFFSET)
     return fail(ABS_EINVAL, "bound_mode");
+  if (model->bound_mode == ABS_BOUND_OFFSET) {
+    if (model->bound_offset < -ABS_MAX_WORKERS || model->bound_offset > ABS_MAX_BOUND)
+      return fail(ABS_EINVAL, "bound_offset %d out of range", model->bound_offset);
+    if (std::max(1, W / K0 + model->bound_offset) > staleness_bound)
+      return fail(ABS_EINVAL, "staleness_bound %d is below the initial threshold floor(N/K0) + a = %d",
+                  staleness_bound, W / K0 + model->bound_offset);
+  }
   if (!(model->lr >= 0.f) || !std::isfinite(model->lr)) return fail(ABS_EINVAL, "lr");
   if (!td) return fail(ABS_EINVAL, "time_dist is null");
-  if (td->kind < ABS_T_CONST || td->kind > ABS_T_PARETO2) return fail(ABS_EUNSUPPORTED, "time_dist kind %d", td->kind);
-  if ((td->kind == ABS_T_EXP || td->kind == ABS_T_SHIFTED_EXP) && !(td->rate > 0.0)) return fail(ABS_EINVAL, "rate must be > 0");
-  if ((td->kind == ABS_T_CONST || td->kind == ABS_T_SHIFTED_EXP) && !(td->shift >= 0.0)) return fail(ABS_EINVAL, "shift must be >= 0");
+  if (td->kind < ABS_T_CONST || td->kind > ABS_T_GAMMA) return fail(ABS_EUNSUPPORTED, "time_dist kind %d", td->kind);
+  if ((td->kind == ABS_T_EXP || td->kind == ABS_T_SHIFTED_EXP || td->kind == ABS_T_GAMMA) && !(td->rate > 0.0)) return fail(ABS_EINVAL, "rate must be > 0");
+  if ((td->kind == ABS_T_CONST || td->kind == ABS_T_SHIFTED_EXP || td->kind == ABS_T_GAMMA) && !(td->shift >= 0.0)) return fail(ABS_EINVAL, "shift must be >= 0");
+  if (td->kind == ABS_T_GAMMA && (td->shape < 1 || td->shape > 64)) return fail(ABS_EINVAL, "gamma shape %d outside [1, 64]", td->shape);
   if (td->kind == ABS_T_PARETO2 && !(td->scale > 0.0)) return fail(ABS_EINVAL, "scale must be > 0");
   if (td->slow_mod < 0 || (td->slow_mod > 0 && (td->slow_rem < 0 || td->slow_rem >= td->slow_mod)))
     return fail(ABS_EINVAL, "slow class");
@@ -793,6 +802,8 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   h.key0 = (uint32_t)(seed & 0xffffffffull); h.key1 = (uint32_t)(seed >> 32);
   h.dist.kind = td->kind; h.dist.shift = td->shift; h.dist.rate = td->rate; h.dist.scale = td->scale;
   h.dist.slow_mod = td->slow_mod; h.dist.slow_rem = td->slow_rem; h.dist.slow_factor = td->slow_factor;
+  h.dist.shape = td->kind == ABS_T_GAMMA ? td->shape : 1;
+  h.bound_offset = model->bound_offset;
   h.K = K0; h.theta = staleness_bound; h.comm = (u64)W;
   e = cudaMemcpyAsync(ctx->at<DevState>(L.st), &h, sizeof h, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return bail(cuda_fail(nullptr, e, "state copy"));

@@ -29,6 +29,7 @@ struct TimeDist {
   double shift, rate, scale;
   int slow_mod, slow_rem;
   double slow_factor;
+  int shape;
 };
 
 // Scalars of Algorithm 1 that live on the device between rounds.
@@ -36,6 +37,7 @@ struct DevState {
   // constants of the run
   int W, K0, S, B, RB;            // RB: every version group's rows are padded to a multiple of RB
   int k_mode, bound_mode, max_rounds;
+  int bound_offset;               // the constant a of Eq. 4 (ABS_BOUND_OFFSET)
   i64 n_samples;
   uint32_t key0, key1;            // Philox key = (seed low, seed high)
   TimeDist dist;

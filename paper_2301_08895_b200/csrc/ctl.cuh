@@ -49,7 +49,17 @@ __device__ __forceinline__ u64 job_ticks(const TimeDist& d, uint32_t k0, uint32_
   philox4x32_10((uint32_t)n, (uint32_t)j, 0u, 0u, k0, k1, w);
   const double u = __dmul_rn(__dadd_rn((double)w[0], 0.5), 2.3283064365386963e-10);  // 2^-32
   double dur;
-  if (d.kind == ABS_T_CONST) dur = d.shift;
+  if (d.kind == ABS_T_GAMMA) {
+    // sum of `shape` exponential draws, left to right; draw i uses word i % 4 of block i / 4
+    double total = -ln_series(u);
+    for (int i = 1; i < d.shape; ++i) {
+      if ((i & 3) == 0) philox4x32_10((uint32_t)n, (uint32_t)j, 0u, (uint32_t)(i >> 2), k0, k1, w);
+      const uint32_t wi = (i & 3) == 0 ? w[0] : (i & 3) == 1 ? w[1] : (i & 3) == 2 ? w[2] : w[3];
+      const double ui = __dmul_rn(__dadd_rn((double)wi, 0.5), 2.3283064365386963e-10);
+      total = __dadd_rn(total, -ln_series(ui));
+    }
+    dur = __dadd_rn(d.shift, __ddiv_rn(total, d.rate));
+  } else if (d.kind == ABS_T_CONST) dur = d.shift;
   else if (d.kind == ABS_T_EXP) dur = __ddiv_rn(-ln_series(u), d.rate);
   else if (d.kind == ABS_T_SHIFTED_EXP) dur = __dadd_rn(d.shift, __ddiv_rn(-ln_series(u), d.rate));
   else dur = __ddiv_rn(d.scale, __dsqrt_rn(u));
@@ -152,6 +162,7 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
   const int po = (t_sel - 1) & 1, pn = t_sel & 1;     // layout copy of the open / of the new round
   const int status0 = st->status, open0 = st->open, diverged0 = a.ri[po].diverged;
   const int k_mode = st->k_mode, bound_mode = st->bound_mode, max_rounds = st->max_rounds;
+  const int bound_offset = st->bound_offset;
   const uint32_t key0 = st->key0, key1 = st->key1;
   const i64 n_samples = st->n_samples;
   const u64 T_end0 = st->T_end;
@@ -255,6 +266,11 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
       if (th < 1) th = 1;
       if (th > S) th = S;
       theta = (int)th;
+    } else if (bound_mode == ABS_BOUND_OFFSET) {     // Eq. 4 with a given: floor(N/K + a) = floor(N/K) + a
+      int th = W / K_next + bound_offset;
+      if (th < 1) th = 1;
+      if (th > S) th = S;
+      theta = th;
     }
     // Eq. 6 in Algorithm 1's order: arrivals and over-stale workers get w^{t+1}
     int restart = 0, renew = 0;

@@ -17,7 +17,7 @@ import numpy as np
 
 LSQ, SOFTMAX, MLP = 0, 1, 2
 FP32, BF16 = 0, 1
-T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2 = 0, 1, 2, 3
+T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2, T_GAMMA = 0, 1, 2, 3, 4
 
 
 @dataclass
@@ -29,6 +29,7 @@ class TimeSpec:
     slow_mod: int = 0
     slow_rem: int = 0
     slow_factor: float = 1.0
+    shape: int = 1            # T_GAMMA: integer shape
 
 
 @dataclass

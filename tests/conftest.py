@@ -16,7 +16,7 @@ def oracle_dist(ts):
     """inputs.TimeSpec -> oracle TimeDist (plain field copy)."""
     from oracle import timing
     return timing.TimeDist(ts.kind, ts.shift, ts.rate, ts.scale, ts.slow_mod, ts.slow_rem,
-                           ts.slow_factor)
+                           ts.slow_factor, ts.shape)
 
 
 def make_oracle(cfg, X, y, w0, **kw):

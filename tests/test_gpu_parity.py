@@ -7,7 +7,7 @@ threshold, communication counter): bit-exact.  Parameters: relative L2 within
 import numpy as np
 import pytest
 
-from helpers import compare_with_oracle, gpu_run, rel_l2
+from helpers import compare_with_oracle, gpu_run, rel_l2, to_device
 from conftest import make_oracle
 from paper_2301_08895_b200 import abs as gpu
 from paper_2301_08895_b200 import inputs
@@ -109,6 +109,47 @@ def test_modes_fixed_k_traces_are_pure_integer(k_mode, bound_mode, K0, S):
         assert all(len(r["restart"]) == 11 - K0 and set(r["tau"]) == {0} for r in rows)
     if K0 == 1:
         assert max(max(r["tau"]) for r in rows) > 11
+
+
+GAMMA3 = inputs.TimeSpec(inputs.T_GAMMA, shift=0.25, rate=1.5, shape=3)
+GAMMA6 = inputs.TimeSpec(inputs.T_GAMMA, shift=0.0, rate=4.0, shape=6)
+
+
+@pytest.mark.parametrize("kind,dims,dtype,W,B,time", [
+    (inputs.LSQ, (24, 1), inputs.FP32, 12, 6, GAMMA3),          # persistent least-squares kernel
+    (inputs.SOFTMAX, (40, 6), inputs.FP32, 20, 16, GAMMA6),     # shape 6: second Philox block
+    (inputs.MLP, (64, 128, 10), inputs.BF16, 40, 16, GAMMA3),
+])
+def test_gamma_execution_times(kind, dims, dtype, W, B, time):
+    """Gamma-distributed job times (Sec. V-A): the arrival order, ticks and everything downstream
+    must match the oracle exactly."""
+    cfg = _small_cfg(kind, dims, dtype, W, B, 3, 5, time)
+    X, y, w0 = _problem(cfg)
+    bf16 = dtype == inputs.BF16
+    rows, _, _, _ = compare_with_oracle(cfg, X, y, w0, 50, TOL_BF16 if bf16 else TOL_FP32, forced=bf16,
+                                        loss_tol=5e-2 if bf16 else None)
+    assert len({r["T_end"] for r in rows}) > 40
+
+
+@pytest.mark.parametrize("a", [0, -2, -3])
+def test_threshold_offset_sweep(a):
+    """Eq. 4 with the constant a given, in the setting of the paper's sweep (Sec. V-B: N = 20,
+    K0 = 5, a in {0, -2, -3}): traces identical to the oracle's; a smaller a restarts more."""
+    cfg = _small_cfg(inputs.SOFTMAX, (40, 6), inputs.FP32, 20, 16, 5, 6, GAMMA3)
+    X, y, w0 = _problem(cfg)
+    rows, _, _, _ = compare_with_oracle(cfg, X, y, w0, 60, TOL_FP32, bound_mode=gpu.BOUND_OFFSET, bound_offset=a)
+    assert rows[0]["theta"] == max(1, 20 // 5 + a)
+    assert all(r["theta"] == max(1, 20 // r2["K"] + a) for r, r2 in zip(rows, rows[1:]))
+    assert all(max(r["tau"]) <= r0["theta"] for r0, r in zip(rows, rows[1:]))
+
+
+def test_threshold_offset_needs_a_large_enough_bound():
+    cfg = _small_cfg(inputs.SOFTMAX, (40, 6), inputs.FP32, 20, 16, 5, 3, EXP)
+    X, y, w0 = _problem(cfg)
+    Xd, yd = to_device(cfg, X, y)
+    with pytest.raises(gpu.AbsError) as e:
+        gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=5, bound_mode=gpu.BOUND_OFFSET, bound_offset=0)
+    assert e.value.code == gpu.EINVAL
 
 
 def test_lock_step_constant_times():
