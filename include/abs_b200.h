@@ -80,6 +80,8 @@ extern "C" {
                                        tile is shared by several column tiles (each re-gathers it) */
 #define ABS_FLAG_NO_BULK_PIPELINE 32 /* bf16 least squares: per-warp 16-byte loads (rows read from HBM, then again
                                        from L2) instead of the bulk-copy pipeline through shared memory */
+#define ABS_FLAG_NO_FUSED_BACKWARD 64 /* tensor-core networks: a layer's delta back-propagation and its weight
+                                       gradient always get a launch each */
 #define ABS_FLAG_NO_PERSISTENT   8  /* small least-squares problems: one kernel launch per step of a round
                                        instead of one persistent kernel that runs all enqueued rounds */
 

@@ -27,6 +27,7 @@ FLAG_TWO_CTA = 4
 FLAG_NO_PERSISTENT = 8
 FLAG_TMA_GATHER = 16
 FLAG_NO_BULK_PIPELINE = 32
+FLAG_NO_FUSED_BACKWARD = 64
 KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update", "rounds")
 
 

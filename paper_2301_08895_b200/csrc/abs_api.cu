@@ -61,6 +61,7 @@ struct Layout {
   bool gather_tma = false;              // first-layer GEMMs fetch the minibatch rows from the dataset themselves
   bool two_cta = false;                 // GEMMs with N >= 256 run on CTA pairs (tiles of 256 x 256)
   int cg_fwd[ABS_MAX_LAYERS] = {}, cg_dg[ABS_MAX_LAYERS] = {}, cg_wg[ABS_MAX_LAYERS] = {};
+  bool pair_bwd[ABS_MAX_LAYERS] = {};   // delta back-propagation and weight gradient of the layer share a launch
   int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
   bool out_mma = false;                 // output layer through the mma.sync kernel (bf16, 64 rows per CTA)
   size_t esz = 4;                       // bytes per stored element (4 or 2)
@@ -163,6 +164,16 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
         // unit of the version groups is not involved)
         L->cg_wg[l] = 2; L->bn_wg[l] = 256;
       }
+    }
+    // A short weight gradient (fewer tiles than SMs at the back-propagation's tile width) shares
+    // its launch with the layer's delta back-propagation: both have one or two tiles per CTA, so
+    // separate launches would pay the fixed costs of a launch twice.
+    for (int l = 1; l < m->n_layers; ++l) {
+      if (L->path[l] != PATH_TC || L->cg_dg[l] != 1 || L->cg_wg[l] != 1 || (m->flags & ABS_FLAG_NO_FUSED_BACKWARD)) continue;
+      const int in = m->dims[l], out = m->dims[l + 1], bn = L->bn_dg[l];
+      if (out < bn) continue;
+      const long wg_tiles_min = (long)((in + 127) / 128 + 1) * ((out + bn - 1) / bn);   // at P = 1
+      if (wg_tiles_min * 4 < 148) { L->pair_bwd[l] = true; L->bn_wg[l] = bn; }
     }
     // split count P of the row reduction: the one that minimises the modelled time of all weight
     // gradients (whole waves of 148 CTAs, one tile = 128 x BN x rows/P) plus the extra partial
@@ -415,23 +426,29 @@ bool make_g_map(CUtensorMap* map, const void* base, int in, int out, int P, size
   return make_map(map, base, 3, dims, strides, box, CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
 }
 
+// One problem (second = null), or two independent problems in one launch.
+struct TcProblem { const CUtensorMap* a; const CUtensorMap* b; const CUtensorMap* o; const tc::Params* p; int max_tiles; };
+
 template <int BN, int CG>
-void launch_tc(abs_ctx* ctx, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
-               const tc::Params& p, int max_tiles) {
+void launch_tc(abs_ctx* ctx, int cls, const TcProblem& x, const TcProblem* y) {
   const int units = ctx->sm_count / CG;           // CTAs, or CTA pairs
-  const int grid = CG * std::max(1, std::min(units, max_tiles));
+  const int grid = CG * std::max(1, std::min(units, x.max_tiles + (y ? y->max_tiles : 0)));
+  tc::Params none;
+  memset(&none, 0, sizeof none);
+  none.mode = -1;
   ctx->next_cluster = CG;
-  launch_ex(ctx, cls, tc::tc_gemm_kernel<BN, CG>, dim3(grid), dim3(tc::THREADS), tc::Cfg<BN, CG>::SMEM_BYTES, a, b,
-            ctx->ones_map, o, p);
+  launch_ex(ctx, cls, tc::tc_gemm_kernel<BN, CG>, dim3(grid), dim3(tc::THREADS), tc::Cfg<BN, CG>::SMEM_BYTES, *x.a, *x.b,
+            ctx->ones_map, *x.o, *x.p, *(y ? y->a : x.a), *(y ? y->b : x.b), *(y ? y->o : x.o), y ? *y->p : none);
 }
 
 // max_tiles counts tiles of (128 * cg) x bn
 void launch_tc_bn(abs_ctx* ctx, int bn, int cg, int cls, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& o,
-                  const tc::Params& p, int max_tiles) {
-  if (cg == 2) launch_tc<256, 2>(ctx, cls, a, b, o, p, max_tiles);
-  else if (bn == 256) launch_tc<256, 1>(ctx, cls, a, b, o, p, max_tiles);
-  else if (bn == 128) launch_tc<128, 1>(ctx, cls, a, b, o, p, max_tiles);
-  else launch_tc<64, 1>(ctx, cls, a, b, o, p, max_tiles);
+                  const tc::Params& p, int max_tiles, const TcProblem* second = nullptr) {
+  const TcProblem x = {&a, &b, &o, &p, max_tiles};
+  if (cg == 2) launch_tc<256, 2>(ctx, cls, x, second);
+  else if (bn == 256) launch_tc<256, 1>(ctx, cls, x, second);
+  else if (bn == 128) launch_tc<128, 1>(ctx, cls, x, second);
+  else launch_tc<64, 1>(ctx, cls, x, second);
 }
 
 int setup_tc(abs_ctx* ctx) {
@@ -617,19 +634,26 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
   // ---- backward: deltas, then the weight gradients summed over all selected workers (Eq. 3)
   for (int l = nl - 1; l >= 0 && phase == PH_BACKWARD; --l) {
     if (L.path[l] == PATH_TC) {
-      if (l > 0) {
-        tc::Params p = tc_params(l, tc::DGRAD);
-        p.N_total = la[l].in; p.K_total = la[l].out;
-        p.mask_src = (const __nv_bfloat16*)la[l].act_in;
-        p.mask_bits = L.bits[l] ? ctx->at<uint32_t>(L.bits[l]) : nullptr;
-        p.mask_words = (la[l].in + 31) / 32;
-        p.out_bf16 = (__nv_bfloat16*)la[l].delta_in;
-        const int bn = L.bn_dg[l];
-        launch_tc_bn(ctx, bn, L.cg_dg[l], ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, ctx->tcl[l].dg_out, p, (row_tiles128 / L.cg_dg[l]) * ((la[l].in + bn - 1) / bn));
-      }
+      tc::Params pd = tc_params(l, tc::DGRAD);
+      pd.N_total = la[l].in; pd.K_total = la[l].out;
+      pd.mask_src = (const __nv_bfloat16*)la[l].act_in;
+      pd.mask_bits = L.bits[l] ? ctx->at<uint32_t>(L.bits[l]) : nullptr;
+      pd.mask_words = (la[l].in + 31) / 32;
+      pd.out_bf16 = (__nv_bfloat16*)la[l].delta_in;
+      const int bnd = L.bn_dg[l];
+      const int dg_tiles = (row_tiles128 / std::max(1, L.cg_dg[l])) * ((la[l].in + std::max(1, bnd) - 1) / std::max(1, bnd));
       tc::Params p = tc_params(l, tc::WGRAD);
       p.M_total = la[l].in + 1; p.N_total = la[l].out;     // row `in` of the result is the bias gradient
       p.out_f32 = ctx->at<float>(L.G) + L.w_off[l];
+      if (l > 0 && L.pair_bwd[l]) {
+        // the layer's delta back-propagation shares the weight gradient's launch (same tile width)
+        const TcProblem second = {&ctx->tcl[l].dg_a, &ctx->tcl[l].dg_b, &ctx->tcl[l].dg_out, &pd, dg_tiles};
+        launch_tc_bn(ctx, bnd, 1, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
+                     ((la[l].in + 127) / 128 + 1) * ((la[l].out + bnd - 1) / bnd) * L.P, &second);
+        continue;
+      }
+      if (l > 0)
+        launch_tc_bn(ctx, bnd, L.cg_dg[l], ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, ctx->tcl[l].dg_out, pd, dg_tiles);
       const int bn = L.bn_wg[l];
       const int tmw = 128 * L.cg_wg[l];
       launch_tc_bn(ctx, bn, L.cg_wg[l], ABS_KC_WGRAD, (l == 0 && L.gather_tma) ? ctx->tcl[l].x_rows : (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,

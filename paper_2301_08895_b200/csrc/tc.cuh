@@ -210,16 +210,24 @@ template <int BN, int CG = 1> struct Cfg {
       (size_t)STAGES * STAGE_BYTES + OUT_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 2 * BN * 2 /*bias*/;
 };
 
-struct TileCoord { int a_row, b_col, slot, k_begin, n_kb, split, bias_tile; };
+struct TileCoord { int which, a_row, b_col, slot, k_begin, n_kb, split, bias_tile; };
+// Tiling of one problem of a launch.
+struct Prob { int mode, n_ct, n_mt_w, n_mt, n_tiles, chunk; };
 
+// A launch serves one problem (p0), or two independent ones (p1.mode >= 0): a layer's weight
+// gradient (p0) next to its delta back-propagation (p1).  Both are short (one or two tiles per CTA),
+// so sharing one launch halves their fixed costs; the weight gradient's few long tiles go to the
+// first CTAs, the remaining CTAs split the many short tiles of the back-propagation.
 // CG = 1: one CTA per tile of 128 x BN.  CG = 2: a cluster of two CTAs per tile of 256 x BN; the
 // leader (cluster rank 0) issues the MMAs for both, every CTA loads its own A rows and its half of
 // B and drains its own half of the accumulator.
 template <int BN, int CG>
 __global__ void __launch_bounds__(THREADS, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_ones, const __grid_constant__ CUtensorMap map_out,
-               const Params p) {
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_b0,
+               const __grid_constant__ CUtensorMap map_ones, const __grid_constant__ CUtensorMap map_out0,
+               const Params p0,
+               const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_b1,
+               const __grid_constant__ CUtensorMap map_out1, const Params p1) {
   grid_dependency_sync();
   using C = Cfg<BN, CG>;
   constexpr int TM_ROWS = BM * CG;              // rows of one tile
@@ -227,20 +235,42 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int rank = (CG == 2) ? (int)cluster_rank() : 0;
   const int unit = (int)blockIdx.x / CG;        // tile-processing unit (CTA or CTA pair)
   const int n_units = (int)gridDim.x / CG;
-  DevState* st = p.st;
-  RoundInfo* ri = p.ri;
+  DevState* st = p0.st;
+  RoundInfo* ri = p0.ri;
   if (st->status != ST_OK) return;
   const int n_rows = ri->n_rows;
   const int n_row_tiles = n_rows / TM_ROWS;
-  const int mode = p.mode;
-  const int n_ct = (p.N_total + BN - 1) / BN;
-  // WGRAD: one extra row tile multiplies a column of ones with the deltas, which yields the bias
-  // gradient (row `in` of the [in + 1][out] gradient block) on the tensor cores for free
-  const int n_mt_w = (p.M_total - 1 + TM_ROWS - 1) / TM_ROWS;
-  const int n_mt = (mode == WGRAD) ? n_mt_w + 1 : n_row_tiles;
-  const int n_tiles = (mode == WGRAD) ? n_mt * n_ct * p.P : n_row_tiles * n_ct;
-  if (unit >= n_tiles) return;                  // same decision in both CTAs of a pair
-  const int chunk = (mode == WGRAD) ? round_up((n_rows + p.P - 1) / p.P, BK) : 0;
+  auto make_prob = [&](const Params& q) -> Prob {
+    Prob r;
+    r.mode = q.mode;
+    r.n_ct = (q.N_total + BN - 1) / BN;
+    // WGRAD: one extra row tile multiplies a column of ones with the deltas, which yields the bias
+    // gradient (row `in` of the [in + 1][out] gradient block) on the tensor cores for free
+    r.n_mt_w = (q.M_total - 1 + TM_ROWS - 1) / TM_ROWS;
+    r.n_mt = (q.mode == WGRAD) ? r.n_mt_w + 1 : n_row_tiles;
+    r.n_tiles = (q.mode == WGRAD) ? r.n_mt * r.n_ct * q.P : n_row_tiles * r.n_ct;
+    r.chunk = (q.mode == WGRAD) ? round_up((n_rows + q.P - 1) / q.P, BK) : 0;
+    return r;
+  };
+  const Prob P0 = make_prob(p0);
+  Prob P1 = P0;
+  P1.n_tiles = 0;
+  if (p1.mode >= 0) P1 = make_prob(p1);
+  const int T0 = P0.n_tiles, T1 = P1.n_tiles;
+  // i-th tile of this unit, or -1.  Two problems with fewer long tiles than units: units [0, T0)
+  // take one tile of problem 0 each, the others stride over problem 1; otherwise all units stride
+  // over the concatenated tiles.
+  const bool split_units = T1 > 0 && T0 < n_units;
+  auto tile_at = [&](int i) -> int {
+    if (split_units) {
+      if (unit < T0) return i == 0 ? unit : -1;
+      const int t = T0 + (unit - T0) + i * (n_units - T0);
+      return t < T0 + T1 ? t : -1;
+    }
+    const int t = unit + i * n_units;
+    return t < T0 + T1 ? t : -1;
+  };
+  if (tile_at(0) < 0) return;                   // same decision in both CTAs of a pair
   const int RB = st->RB;
 
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -280,29 +310,33 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t acc_empty0_addr = (CG == 2) ? map_to_cta(smem_u32(&acc_empty[0]), 0) : smem_u32(&acc_empty[0]);
   const uint32_t tmem_base = *tmem_slot;
 
-  auto tile_coord = [&](int tile) -> TileCoord {
+  auto tile_coord = [&](int gtile) -> TileCoord {
     TileCoord c;
-    if (mode == WGRAD) {
-      const int per_split = n_mt * n_ct;
+    c.which = gtile >= T0 ? 1 : 0;
+    const int tile = c.which ? gtile - T0 : gtile;
+    const Prob& P = c.which ? P1 : P0;
+    const Params& q = c.which ? p1 : p0;
+    if (P.mode == WGRAD) {
+      const int per_split = P.n_mt * P.n_ct;
       c.split = tile / per_split;
       const int rem = tile - c.split * per_split;
-      const int mt = rem / n_ct;
-      c.bias_tile = (mt == n_mt_w);
+      const int mt = rem / P.n_ct;
+      c.bias_tile = (mt == P.n_mt_w);
       c.a_row = mt * TM_ROWS + rank * BM;    // m0 of this CTA
-      c.b_col = (rem % n_ct) * BN;           // n0
+      c.b_col = (rem % P.n_ct) * BN;         // n0
       c.slot = 0;
-      c.k_begin = min(n_rows, c.split * chunk);
-      const int k_end = min(n_rows, (c.split + 1) * chunk);
+      c.k_begin = min(n_rows, c.split * P.chunk);
+      const int k_end = min(n_rows, (c.split + 1) * P.chunk);
       c.n_kb = (k_end - c.k_begin) / BK;
     } else {
-      const int rt = tile / n_ct;
+      const int rt = tile / P.n_ct;
       c.split = 0;
       c.bias_tile = 0;
       c.a_row = rt * TM_ROWS + rank * BM;
-      c.b_col = (tile - rt * n_ct) * BN;
-      c.slot = p.tile_slot[(rt * TM_ROWS) / RB];
+      c.b_col = (tile - rt * P.n_ct) * BN;
+      c.slot = q.tile_slot[(rt * TM_ROWS) / RB];
       c.k_begin = 0;
-      c.n_kb = (p.K_total + BK - 1) / BK;
+      c.n_kb = (q.K_total + BK - 1) / BK;
     }
     return c;
   };
@@ -324,12 +358,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       else tma_load_3d(dst, map, &full[st_], x, y, z);
     };
     constexpr int BH = BN / CG;                  // B columns (rows of the B tile) this CTA loads
-    if (p.gather_a == 0) {
+    if (p0.gather_a == 0) {
       // one elected lane: the stage ring is shallow, so nothing may sit between a stage being
       // released and its next loads being issued
       if (lane == 0) {
-        for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
+        for (int it = 0; ok; ++it) {
+          const int tile = tile_at(it);
+          if (tile < 0) break;
           const TileCoord c = tile_coord(tile);
+          const int mode = c.which ? p1.mode : p0.mode;
+          const CUtensorMap& map_a = c.which ? map_a1 : map_a0;
+          const CUtensorMap& map_b = c.which ? map_b1 : map_b0;
           const int b0 = c.b_col + rank * BH;
           for (int kb = 0; kb < c.n_kb; ++kb) {
             if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) { ok = false; break; }
@@ -364,11 +403,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // then every lane issues one four-row gather (32 x 4 = the 128 rows of a K-major tile, or
       // the 64 rows x two 64-feature boxes of an MN-major one).  Rows of padding (index -1) lie
       // outside the tensor and arrive as zeros.
+      const Params& p = p0;                      // a launch with row gathers serves one problem
+      const int mode = p0.mode;
+      const CUtensorMap& map_a = map_a0;
+      const CUtensorMap& map_b = map_b0;
       auto ldg4 = [&](void* dst, int st_, int x, const int4& r) {
         if (CG == 2) tma2_gather4(dst, &map_a, full0_addr + 8u * (uint32_t)st_, x, r);
         else tma_gather4(dst, &map_a, &full[st_], x, r);
       };
-      for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
+      for (int it = 0; ok; ++it) {
+        const int tile = tile_at(it);
+        if (tile < 0) break;
         const TileCoord c = tile_coord(tile);
         const int b0 = c.b_col + rank * BH;
         const bool g_tile = !(mode == WGRAD && c.bias_tile);
@@ -430,19 +475,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {            // with a CTA pair only the leader issues MMAs
-      const bool a_mn = (mode == WGRAD), b_mn = (mode != DGRAD);
-      const uint32_t idesc = instr_desc(a_mn ? 1 : 0, b_mn ? 1 : 0, BN, TM_ROWS);
-      // K-major tile: rows of 128 B, 8-row groups 1024 B apart; a k step of 16 elements is 32 B.
-      // MN-major tile: 64-wide boxes 8192 B apart (leading offset), 8-k groups 1024 B apart;
-      // a k step of 16 rows is 2048 B.
-      const uint32_t a_lbo = a_mn ? 8192u : 16u, b_lbo = b_mn ? 8192u : 16u;
-      const uint32_t a_kstep = a_mn ? 2048u : 32u, b_kstep = b_mn ? 2048u : 32u;
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = unit; tile < n_tiles && ok; tile += n_units) {
+      for (int it = 0; ok; ++it) {
+        const int tile = tile_at(it);
+        if (tile < 0) break;
         const TileCoord c = tile_coord(tile);
         if (c.n_kb == 0) continue;
+        const int mode = c.which ? p1.mode : p0.mode;
+        const bool a_mn = (mode == WGRAD), b_mn = (mode != DGRAD);
+        const uint32_t idesc = instr_desc(a_mn ? 1 : 0, b_mn ? 1 : 0, BN, TM_ROWS);
+        // K-major tile: rows of 128 B, 8-row groups 1024 B apart; a k step of 16 elements is 32 B.
+        // MN-major tile: 64-wide boxes 8192 B apart (leading offset), 8-k groups 1024 B apart;
+        // a k step of 16 rows is 2048 B.
+        const uint32_t a_lbo = a_mn ? 8192u : 16u, b_lbo = b_mn ? 8192u : 16u;
+        const uint32_t a_kstep = a_mn ? 2048u : 32u, b_kstep = b_mn ? 2048u : 32u;
         if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
@@ -483,11 +531,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int sw = lane & 7;
     uint8_t* my_box = stage_out + ((warp - 2) << 12);
     uint8_t* my_row = my_box + lane * 128;
-    const int box_cols = (mode == WGRAD) ? 32 : 64;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int tile = unit; tile < n_tiles; tile += n_units) {
+    for (int it = 0; ; ++it) {
+      const int tile = tile_at(it);
+      if (tile < 0) break;
       const TileCoord c = tile_coord(tile);
+      const Params& p = c.which ? p1 : p0;
+      const int mode = p.mode;
+      const CUtensorMap& map_out = c.which ? map_out1 : map_out0;
+      const int box_cols = (mode == WGRAD) ? 32 : 64;
       const bool have = c.n_kb > 0;
       // output row (FWD/DGRAD) or gradient row m (WGRAD; the bias tile's row 0 is row `in`)
       const int r = (mode == WGRAD && c.bias_tile) ? (p.M_total - 1) + rank * BM + row_in_tile : c.a_row + row_in_tile;
@@ -641,7 +694,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
   }
   if (threadIdx.x == 0 && *abort) {
-    st->timeout_where = 100 + mode;
+    st->timeout_where = 100 + p0.mode;
     st->status = ST_TIMEOUT;
   }
 }

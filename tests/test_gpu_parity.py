@@ -282,6 +282,21 @@ def test_tma_row_gather_matches_the_copy_kernel(dims, B):
     compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_TMA_GATHER)
 
 
+@pytest.mark.parametrize("dims,W,B", [((3072, 1024, 512, 10), 32, 64), ((320, 520, 264, 10), 13, 40),
+                                      ((256, 512, 512, 256, 10), 24, 32)])
+def test_merged_backward_launch_matches_separate_launches(dims, W, B):
+    """A hidden layer's delta back-propagation and weight gradient share one GEMM launch (two
+    problems, tiles dealt to disjoint CTAs); the flag gives each its own launch.  Every output
+    element is accumulated over the same rows in the same order either way: identical bits."""
+    cfg = _small_cfg(inputs.MLP, dims, inputs.BF16, W, B, 3, 5, PARETO)
+    X, y, w0 = _problem(cfg)
+    rows_a, params_a = gpu_run(cfg, X, y, w0, 25)
+    rows_b, params_b = gpu_run(cfg, X, y, w0, 25, flags=gpu.FLAG_NO_FUSED_BACKWARD)
+    assert rows_a == rows_b
+    assert np.array_equal(params_a, params_b)
+    compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2)
+
+
 def test_cta_pair_gemms_match_single_cta_gemms():
     """Opt-in tcgen05 cta_group::2 tiles (256 x 256 over a CTA pair) against the default tiles."""
     cfg = _small_cfg(inputs.MLP, (320, 520, 264, 10), inputs.BF16, 13, 40, 3, 5, PARETO)
