@@ -30,7 +30,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) per launch at K = N on configuration 4, from the ncu captures summarised in
 # profiles/tc_gemm_kernel_cfg4.md and profiles/update_kernel_cfg4.md; each figure is valid only for the kernel
 # source it was taken from (first 16 hex digits of the file's sha256).
-TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 39.7e6, "file": "tc.cuh", "sha256_16": "b1e563028d097907"},
+TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.4e6, "file": "tc.cuh", "sha256_16": "7bdde9a563de088e"},
            "update": {"config": 4, "bytes_per_launch": 75.7e6, "file": "simt.cuh", "sha256_16": "3da31ad4d03aac5c"}}
 METRIC = "worker_gradients_per_sec"
 UNIT = "worker-gradients/s"
@@ -196,7 +196,8 @@ def main():
     config_obj = {"workload": workload_name(cfg, rounds), "lr": cfg.lr,
                   "parallelism": "replicas x%d (the round loop does not shard)" % world,
                   "l2": "flushed between steps (512 MiB write); per-round working set exceeds L2",
-                  "reinit": "abs_init between steps, outside the device-timed region"}
+                  "reinit": "abs_init between steps, outside the device-timed region",
+                  "per_kernel": "event pair around every launch in one extra step with all kernels on one stream"}
 
     if args.impl == "reference":
         if rank != 0:
@@ -246,15 +247,18 @@ def main():
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream(dev)
 
-    def new_ctx(host=False):
+    def new_ctx(host=False, flags=None):
+        flags = args.flags if flags is None else flags
         if host:
             return gpu.context_from_config(cfg, Xh, yh, w0, max_rounds=rounds, data_on_host=True,
-                                           device=str(dev), flags=args.flags)
-        return gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=rounds, device=str(dev), flags=args.flags)
+                                           device=str(dev), flags=flags)
+        return gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=rounds, device=str(dev), flags=flags)
 
     def device_step(profile=False):
         """One run; returns (ms on the stream, worker-gradients, launches, profile dict)."""
-        ctx = new_ctx()
+        # the per-kernel step runs every kernel on one stream, so that an event pair brackets the
+        # kernel alone and not its wait for an SM held by the other stream (same kernels, same bits)
+        ctx = new_ctx(flags=(args.flags | gpu.FLAG_NO_OVERLAP) if profile else None)
         flush.zero_()
         l0 = ctx.launch_count()
         if profile:
@@ -374,7 +378,11 @@ def main():
                            "traffic": measured_traffic("gemm", args.config, not args.samples), "peak_source": peaks["source"] + " (sustained bf16)",
                            "frac_of_burst_peak": ach / peaks["bf16_tflops"],
                            "share_of_profiled_time": t_g / tot_prof,
-                           "per_class_tflops": {c: wg_p * flops[c] / (prof[c][1] * 1e-3) / 1e12
+                           # a layer's delta back-propagation may share the weight gradient's launch:
+                           # its flops then count in the "wgrad" class
+                           "per_class_tflops": {c: wg_p * (flops[c] + (flops["dgrad"] if c == "wgrad" and
+                                                                       prof["dgrad"][1] == 0 else 0.0))
+                                                / (prof[c][1] * 1e-3) / 1e12
                                                 for c in ("fwd", "dgrad", "wgrad") if prof[c][1] > 0}}
     else:
         out["roofline"] = {"bound": "latency", "achieved": None, "peak": None, "unit": None,
