@@ -3,6 +3,12 @@
 Test infrastructure (see the package header).  One call of `run` plays rounds
 t = 0, 1, ... of Algorithm 1 with U = 1 local step:
 
+  (With `local_steps` = U > 1 a job is U local minibatch steps, Eq. 2: the worker
+  starts from the model it holds, moves its own copy by -eta * (mean minibatch
+  gradient) U times, each step on a fresh minibatch, and uploads the sum of its
+  U mean gradients, i.e. (w^{.,0} - w^{.,U}) / eta, and the average of its U mean
+  minibatch losses (Algorithm 1, last worker line); Eq. 3 is unchanged.)
+
   1. the server waits for the K^t fastest uploads (Sec. II-A; Algorithm 1,
      "waits for the uploads"): the K^t smallest pending completion events,
      ordered by (completion tick, worker id), ties to the lower id;
@@ -49,11 +55,12 @@ def shard_bounds(n, W, M):
     return (n * M) // W, ((n + 1) * M) // W
 
 
-def minibatch_indices(seed, n, j, batch, W, M):
-    """Sample indices of job j of worker n: independent uniform draws (with
-    replacement) inside the worker's shard, index = lo + floor(r * len / 2**32)."""
+def minibatch_indices(seed, n, j, batch, W, M, step=0):
+    """Sample indices of local step `step` of job j of worker n: independent
+    uniform draws (with replacement) inside the worker's shard,
+    index = lo + floor(r * len / 2**32)."""
     lo, hi = shard_bounds(n, W, M)
-    words = philox.minibatch_words(seed, n, j, batch).astype(np.uint64)
+    words = philox.minibatch_words(seed, n, j, batch, step).astype(np.uint64)
     return lo + ((words * np.uint64(hi - lo)) >> np.uint64(32)).astype(np.int64)
 
 
@@ -137,6 +144,7 @@ class ABSOracle:
     k_mode         K_ADAPTIVE (Eq. 5) or K_FIXED
     bound_mode     BOUND_ADAPTIVE (Eq. 4 with a = S - N/K^0), BOUND_FIXED (theta = S
                    always) or BOUND_OFFSET (Eq. 4 with the integer `bound_offset` as a)
+    local_steps    U of Eq. 2 (local minibatch steps per job)
     literal_eq6    test the pre-increment age against the threshold exactly as
                    Eq. 6 is printed (one round later than Algorithm 1's order)
     integer_only   play only the server's integer machinery (arrivals, Eq. 4-6,
@@ -146,7 +154,8 @@ class ABSOracle:
 
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, dist, seed,
                  quant=False, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE,
-                 literal_eq6=False, x_is_bf16_bits=False, integer_only=False, bound_offset=0):
+                 literal_eq6=False, x_is_bf16_bits=False, integer_only=False, bound_offset=0,
+                 local_steps=1):
         if not (1 <= K0 <= W):
             raise ValueError("need 1 <= K0 <= W")
         if S < 0:
@@ -161,6 +170,9 @@ class ABSOracle:
         self.quant = bool(quant)
         self.k_mode, self.bound_mode = k_mode, bound_mode
         self.bound_offset = int(bound_offset)
+        self.local_steps = int(local_steps)
+        if self.local_steps < 1:
+            raise ValueError("need U >= 1")
         if bound_mode == BOUND_OFFSET and theta_offset_rule(self.W, 10 ** 9, self.K0, self.bound_offset) > self.S:
             raise ValueError("staleness bound below the initial threshold N/K0 + a")
         self.literal_eq6 = literal_eq6
@@ -192,15 +204,23 @@ class ABSOracle:
         return rows.astype(np.float64)
 
     def upload(self, n):
-        """(mean loss, mean gradient) of worker n's current job (Eq. 2, U = 1),
-        evaluated at the model version the worker holds."""
-        idx = minibatch_indices(self.seed, n, self.job[n], self.batch, self.W, self.M)
-        Xb = self._rows(idx)
-        yb = self.y[idx]
-        if self.kind == models.LSQ:
-            yb = yb.astype(np.float64)
-        w_held = self.versions[self.version[n]]
-        return models.loss_grad(self.kind, self.dims, w_held, Xb, yb, quant=self.quant)
+        """Upload of worker n's current job (Eq. 2): the average of the U mean
+        minibatch losses and the sum of the U mean minibatch gradients along the
+        worker's local trajectory, which starts at the model version it holds."""
+        w_local = np.array(self.versions[self.version[n]], dtype=np.float64)
+        loss_sum, grad_sum = 0.0, np.zeros_like(w_local)
+        for u in range(self.local_steps):
+            idx = minibatch_indices(self.seed, n, self.job[n], self.batch, self.W, self.M, step=u)
+            Xb = self._rows(idx)
+            yb = self.y[idx]
+            if self.kind == models.LSQ:
+                yb = yb.astype(np.float64)
+            loss, grad = models.loss_grad(self.kind, self.dims, w_local, Xb, yb, quant=self.quant)
+            loss_sum += loss
+            grad_sum += grad
+            if u + 1 < self.local_steps:
+                w_local = w_local - self.lr * grad                       # Eq. 2
+        return loss_sum / self.local_steps, grad_sum
 
     def _start_job(self, n, now):
         """Worker n receives w^{t+1} at tick `now` and starts its next job."""

@@ -88,11 +88,12 @@ def duration_words(seed, n, j, count):
     return out[:count]
 
 
-def minibatch_words(seed, n, j, batch):
-    """`batch` 32-bit words for the minibatch of job j of worker n:
-    sample b uses word (b mod 4) of block (n, j, TAG_MINIBATCH, b // 4)."""
+def minibatch_words(seed, n, j, batch, step=0):
+    """`batch` 32-bit words for the minibatch of local step `step` of job j of
+    worker n: sample b uses word (b mod 4) of block
+    (n, j, TAG_MINIBATCH, step * ceil(batch / 4) + b // 4)."""
     nblk = (batch + 3) // 4
-    blk = np.arange(nblk, dtype=np.uint64)
+    blk = np.arange(nblk, dtype=np.uint64) + np.uint64(step * nblk)
     out = philox4x32_10_blocks(np.full(nblk, n), np.full(nblk, j),
                                np.full(nblk, TAG_MINIBATCH), blk, seed_key(seed))
     return out.reshape(-1)[:batch]

@@ -323,3 +323,106 @@ def test_integer_only_mode_replays_the_same_trace():
         for f in ("K", "sel", "tau", "restart", "T_end", "theta", "comm"):
             assert ra[f] == rb[f]
     assert np.array_equal(b.w, np.zeros(6))
+
+
+# ---------------------------------------------------------------- local SGD steps (U > 1)
+def test_local_steps_follow_the_affine_recursion_of_least_squares():
+    """For f = 1/2 (x.w - y)^2 one local step is w <- (I - eta A_u) w + eta b_u with
+    A_u = X_u^T X_u / B, b_u = X_u^T y_u / B; the upload is (w^0 - w^U) / eta (Eq. 2, Algorithm 1)."""
+    X, y, _ = _lsq_problem(M=300, d=5, seed=7)
+    W, B, lr, U, seed = 3, 6, 0.07, 4, 21
+    dist = timing.TimeDist(timing.CONST, shift=1.0)
+    w0 = np.linspace(-1.0, 1.0, 5)
+    o = ABSOracle(models.LSQ, [5, 1], X, y, w0, B, lr, W, W, 0, dist, seed, local_steps=U)
+    for n in range(W):
+        w = w0.copy()
+        losses = []
+        for u in range(U):
+            idx = abs_sim.minibatch_indices(seed, n, 0, B, W, X.shape[0], step=u)
+            Xu, yu = X[idx], y[idx]
+            losses.append(0.5 * np.mean((Xu @ w - yu) ** 2))
+            A, b = Xu.T @ Xu / B, Xu.T @ yu / B
+            w = (np.eye(5) - lr * A) @ w + lr * b
+        loss, grad_sum = o.upload(n)
+        assert np.allclose(w0 - lr * grad_sum, w, rtol=0, atol=1e-12)
+        assert abs(loss - np.mean(losses)) < 1e-12
+
+
+def test_local_step_minibatches_use_consecutive_philox_blocks():
+    from oracle import philox
+    seed, n, j, B = 9, 2, 5, 10                       # ceil(10 / 4) = 3 blocks per step
+    for u in (0, 1, 3):
+        words = philox.minibatch_words(seed, n, j, B, step=u)
+        for b in range(B):
+            blk = philox.philox4x32_10((n, j, philox.TAG_MINIBATCH, 3 * u + b // 4), philox.seed_key(seed))
+            assert int(words[b]) == blk[b % 4]
+    a = abs_sim.minibatch_indices(seed, n, j, B, 4, 1000, step=0)
+    b = abs_sim.minibatch_indices(seed, n, j, B, 4, 1000, step=1)
+    assert not np.array_equal(a, b)
+    assert np.array_equal(a, abs_sim.minibatch_indices(seed, n, j, B, 4, 1000))
+
+
+def test_synchronous_local_sgd_reduction():
+    """K = N and bound 0 with U local steps is synchronous local SGD (Sec. II-B): every round each
+    worker moves U steps from the global model and the server averages the N displacements."""
+    X, y, _ = _lsq_problem(M=400, d=6, seed=1)
+    W, B, lr, U, seed = 4, 8, 0.05, 3, 42
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), B, lr, W, W, 0, dist, seed, local_steps=U)
+    rows = o.run(12)
+    w = np.zeros(6)
+    for t in range(12):
+        moved = np.zeros(6)
+        for n in range(W):
+            wl = w.copy()
+            for u in range(U):
+                idx = abs_sim.minibatch_indices(seed, n, t, B, W, X.shape[0], step=u)
+                wl = wl - lr * X[idx].T @ (X[idx] @ wl - y[idx]) / B
+            moved += w - wl
+        w = w - moved / W
+    assert np.allclose(o.w, w, rtol=0, atol=1e-12)
+    assert all(r["K"] == W and not r["restart"] and set(r["tau"]) == {0} for r in rows)
+
+
+def test_zero_step_size_makes_every_local_step_see_the_same_model():
+    """With eta = 0 the U local steps are U minibatch evaluations at one model: the uploaded loss is
+    the mean sample loss over all U B draws and the uploaded sum is U times their mean gradient."""
+    X, y, _ = _lsq_problem(M=200, d=4, seed=2)
+    W, B, U, seed = 2, 5, 3, 8
+    w0 = np.array([0.3, -0.2, 0.1, 0.5])
+    o = ABSOracle(models.LSQ, [4, 1], X, y, w0, B, 0.0, W, 1, 2, timing.TimeDist(timing.EXP), seed,
+                  local_steps=U)
+    loss, grad_sum = o.upload(1)
+    idx = np.concatenate([abs_sim.minibatch_indices(seed, 1, 0, B, W, 200, step=u) for u in range(U)])
+    per_sample = [models.sample_loss(models.LSQ, [4, 1], w0, X[i], y[i]) for i in idx]
+    assert abs(loss - np.mean(per_sample)) < 1e-12
+    assert np.allclose(grad_sum, U * (X[idx].T @ (X[idx] @ w0 - y[idx])) / len(idx), atol=1e-12)
+
+
+def test_local_steps_soft_max_against_finite_differences_of_the_chain():
+    """The uploaded sum of a soft-max job equals (w^0 - w^U) / eta of a chain built from numerical
+    gradients of the mean sample loss (independent of the analytic gradient code)."""
+    rng = np.random.default_rng(4)
+    M, d_in, C, W, B, U, lr, seed = 120, 5, 3, 2, 4, 2, 0.1, 3
+    X = rng.standard_normal((M, d_in))
+    y = rng.integers(0, C, size=M).astype(np.int32)
+    w0 = 0.1 * rng.standard_normal(d_in * C + C)
+    o = ABSOracle(models.SOFTMAX, [d_in, C], X, y, w0, B, lr, W, 1, 2, timing.TimeDist(timing.EXP), seed,
+                  local_steps=U)
+    _, grad_sum = o.upload(0)
+
+    def mean_loss(w, idx):
+        return np.mean([models.sample_loss(models.SOFTMAX, [d_in, C], w, X[i], y[i]) for i in idx])
+
+    w = w0.copy()
+    total = np.zeros_like(w0)
+    for u in range(U):
+        idx = abs_sim.minibatch_indices(seed, 0, 0, B, W, M, step=u)
+        g = np.zeros_like(w)
+        for k in range(w.shape[0]):
+            e = np.zeros_like(w)
+            e[k] = 1e-6
+            g[k] = (mean_loss(w + e, idx) - mean_loss(w - e, idx)) / 2e-6
+        total += g
+        w = w - lr * g
+    assert np.allclose(grad_sum, total, atol=1e-7)
