@@ -129,14 +129,14 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ oracle (CPU) arm
-def oracle_for(cfg, X, y, w0):
+def oracle_for(cfg, X, y, w0, local_steps=1):
     from oracle import abs_sim, timing
     ts = cfg.time
     bf16 = cfg.dtype == inputs.BF16
     return abs_sim.ABSOracle(cfg.kind, cfg.dims, X, y, w0, cfg.batch, cfg.lr, cfg.W, cfg.K0, cfg.S,
                              timing.TimeDist(ts.kind, ts.shift, ts.rate, ts.scale, ts.slow_mod,
                                              ts.slow_rem, ts.slow_factor, ts.shape),
-                             cfg.run_seed, quant=bf16, x_is_bf16_bits=bf16)
+                             cfg.run_seed, quant=bf16, x_is_bf16_bits=bf16, local_steps=local_steps)
 
 
 def blas_threads():
@@ -148,10 +148,10 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def time_oracle(cfg, X, y, w0, rounds, budget_s):
+def time_oracle(cfg, X, y, w0, rounds, budget_s, local_steps=1):
     """Runs the oracle on the first rounds of the workload until `budget_s` of CPU work is spent
     (at least 2 rounds, at most `rounds`)."""
-    o = oracle_for(cfg, X, y, w0)
+    o = oracle_for(cfg, X, y, w0, local_steps)
     t0 = time.perf_counter()
     done = 0
     while done < rounds:
@@ -177,6 +177,8 @@ def main():
     ap.add_argument("--workers", type=int, default=None, help="W of configuration 5")
     ap.add_argument("--rounds", type=int, default=None, help="rounds per step (default: the configuration's)")
     ap.add_argument("--flags", type=int, default=0, help="ABS_FLAG_* bits passed to abs_init")
+    ap.add_argument("--local-steps", type=int, default=1,
+                    help="U of Eq. 2: local minibatch steps per job (configurations 1, 2 and 5)")
     ap.add_argument("--samples", type=int, default=None,
                     help="dataset rows (default: the configuration's; smaller for profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work")
@@ -193,7 +195,8 @@ def main():
         from paper_2301_08895_b200 import multi
         cfg.run_seed = multi.replica_seed(cfg.run_seed, rank)   # independent replicas, one per GPU
     rounds = args.rounds or cfg.rounds
-    config_obj = {"workload": workload_name(cfg, rounds), "lr": cfg.lr,
+    U = args.local_steps
+    config_obj = {"workload": workload_name(cfg, rounds) + (", U=%d local steps" % U if U > 1 else ""), "lr": cfg.lr,
                   "parallelism": "replicas x%d (the round loop does not shard)" % world,
                   "l2": "flushed between steps (512 MiB write); per-round working set exceeds L2",
                   "reinit": "abs_init between steps, outside the device-timed region",
@@ -207,8 +210,8 @@ def main():
         per_step = max(2.0, min(args.cpu_budget, 150.0 / max(1, args.steps + args.warmup)))
         res = None
         for _ in range(args.warmup):
-            time_oracle(cfg, X, y, w0, rounds, min(per_step, 3.0))
-        vals = [time_oracle(cfg, X, y, w0, rounds, per_step) for _ in range(args.steps)]
+            time_oracle(cfg, X, y, w0, rounds, min(per_step, 3.0), U)
+        vals = [time_oracle(cfg, X, y, w0, rounds, per_step, U) for _ in range(args.steps)]
         res = vals[-1]
         value = float(np.mean([v["value"] for v in vals]))
         res["value"] = value
@@ -251,8 +254,9 @@ def main():
         flags = args.flags if flags is None else flags
         if host:
             return gpu.context_from_config(cfg, Xh, yh, w0, max_rounds=rounds, data_on_host=True,
-                                           device=str(dev), flags=flags)
-        return gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=rounds, device=str(dev), flags=flags)
+                                           device=str(dev), flags=flags, local_steps=U)
+        return gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=rounds, device=str(dev), flags=flags,
+                                       local_steps=U)
 
     def device_step(profile=False):
         """One run; returns (ms on the stream, worker-gradients, launches, profile dict)."""
@@ -341,6 +345,7 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if bf16 else "f32", "data": "synthetic", "config": config_obj,
         "rounds_per_sec": world * rounds * args.steps / t_dev,
+        "minibatch_gradients_per_sec": U * wg_all / t_dev,
         "worker_gradients_per_step": wg_total / args.steps,
         "wall_s_timed_region": wall,
         "clocks": clocks,
@@ -354,7 +359,14 @@ def main():
     kernels = {k: {"launches": n, "ms": round(t, 4)} for k, (n, t) in prof.items() if n}
     out["kernel_ms_profiled_step"] = kernels
     tot_prof = sum(t for _, t in prof.values())
-    if cfg.kind == inputs.LSQ:
+    if U > 1:
+        # local steps: every worker's chain of U steps is sequential, one CTA per worker
+        n_l, t_l = prof["lsq"]
+        out["roofline"] = {"bound": "latency", "kernel": "local_sgd_kernel", "achieved": None, "peak": None,
+                           "unit": None, "frac": None, "traffic": None,
+                           "avg_us": 1e3 * t_l / max(1, n_l), "share_of_profiled_time": t_l / tot_prof,
+                           "note": "U sequential minibatch steps per job; see minibatch_gradients_per_sec"}
+    elif cfg.kind == inputs.LSQ:
         # least squares reads each minibatch row once: B*d*esz + B*4 bytes per worker-gradient
         esz = 2 if bf16 else 4
         bytes_wg = cfg.batch * cfg.dims[0] * esz + cfg.batch * 4
@@ -403,7 +415,7 @@ def main():
                                   "traffic": measured_traffic("update", args.config, not args.samples)}
     out["plan"] = plan
     out["_profiled_worker_gradients"] = wg_p
-    out["cpu_baseline"] = time_oracle(cfg, X, y, w0, rounds, args.cpu_budget)
+    out["cpu_baseline"] = time_oracle(cfg, X, y, w0, rounds, args.cpu_budget, U)
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

@@ -37,7 +37,7 @@ extern "C" {
 #define ABS_OK            0
 #define ABS_EINVAL       -1  /* bad argument (text names it) */
 #define ABS_ENOSPACE     -2  /* workspace, trace capacity or round capacity too small */
-#define ABS_EUNSUPPORTED -3  /* local_steps != 1, unknown kind */
+#define ABS_EUNSUPPORTED -3  /* unknown kind, or local_steps > 1 for a model the local-step kernel does not cover */
 #define ABS_ESTATE       -4  /* call order */
 #define ABS_ECUDA        -5  /* a CUDA call failed; sticky for the context */
 #define ABS_ETIMEOUT     -6  /* a bounded device-side wait expired */
@@ -93,7 +93,7 @@ extern "C" {
 #define ABS_KC_WGRAD   4  /* weight gradient summed over the selected workers (Eq. 3) */
 #define ABS_KC_OUTPUT  5  /* output layer: forward + loss, its back-propagation and gradient */
 #define ABS_KC_BIAS    6  /* bias gradients */
-#define ABS_KC_LSQ     7  /* least-squares residual + gradient */
+#define ABS_KC_LSQ     7  /* least-squares residual + gradient; with local_steps > 1: the workers' local steps */
 #define ABS_KC_UPDATE  8  /* Eq. 3 step + ring write */
 #define ABS_KC_ROUNDS  9  /* whole rounds (control step + Eq. 2 + Eq. 3) of a small least-squares problem
                              in one persistent kernel; one launch per abs_enqueue_rounds call */
@@ -113,7 +113,10 @@ typedef struct {
   int batch;                /* B of Eq. 2, 1..1024 */
   float lr;                 /* eta, constant */
   int dtype;                /* ABS_FP32 | ABS_BF16_FP32MASTER */
-  int local_steps;          /* U of Eq. 2; must be 1 */
+  int local_steps;          /* U of Eq. 2, 1..1024.  U > 1 (local SGD inside a job: the upload is the sum of
+                               the U minibatch-gradient sums along the worker's own trajectory, the loss the
+                               average of its U minibatch losses) is implemented for ABS_LSQ and ABS_SOFTMAX
+                               with <= 16 classes, <= 12288 parameters and batch x classes <= 8192 */
   int k_mode;               /* ABS_K_* */
   int bound_mode;           /* ABS_BOUND_* */
   int bound_offset;         /* the constant a of Eq. 4 when bound_mode = ABS_BOUND_OFFSET (else ignored);
@@ -162,7 +165,7 @@ typedef struct {
 
 /* Bytes of device workspace a context needs (Sec. II-A sizes: N workers, ring of S + 1 model
  * versions, activations for N*B rows, trace for max_rounds).  Only kind, dims, batch, dtype,
- * max_rounds, data_on_host and n_samples of `model` are read. */
+ * local_steps, flags, max_rounds, data_on_host and n_samples of `model` are read. */
 int abs_workspace_bytes(const abs_model_desc* model, int W, int staleness_bound, size_t* out);
 
 /* Algorithm 1, initialisation: K^0, threshold N/K^0 + a := staleness_bound, w^0 broadcast to all

@@ -15,6 +15,7 @@
 #include "tc.cuh"
 #include "outlayer.cuh"
 #include "lsqpipe.cuh"
+#include "local.cuh"
 #include "persist.cuh"
 
 using namespace absb;
@@ -222,7 +223,8 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   L->row_loss = cv.take(4 * (size_t)L->rows_cap);
   L->master = cv.take(4 * L->d_pad);
   L->ring = cv.take(L->esz * L->d_pad * (S + 1));
-  L->G = cv.take(4 * L->d_pad * (lsq ? W : L->P));
+  if (m->local_steps > 1) L->P = 0;      // Eq. 3 adds one upload per selected worker
+  L->G = cv.take(4 * L->d_pad * ((lsq || m->local_steps > 1) ? W : L->P));
   if (!lsq) {
     const int C = m->dims[m->n_layers];
     L->logits = cv.take(4 * (size_t)L->rows_cap * C);
@@ -308,6 +310,7 @@ struct abs_ctx {
   long long launches = 0;
   cudaError_t launch_error = cudaSuccess;
   int next_cluster = 1;              // cluster width of the next launch (consumed by launch_on)
+  bool local_sgd = false;            // U > 1: one CTA per selected worker runs the worker's local steps
   bool lsq_pipe = false;             // bf16 least squares through the bulk-copy pipeline kernel
   int lsq_stages = 0;
   bool lsq_v2 = false;               // least squares through the persistent 16-byte-load kernel
@@ -755,8 +758,18 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   *out = nullptr;
   int rc = check_model(model, W, staleness_bound);
   if (rc != ABS_OK) return rc;
-  if (model->local_steps != 1)
-    return fail(ABS_EUNSUPPORTED, "local_steps = %d: only U = 1 is implemented", model->local_steps);
+  if (model->local_steps < 1 || model->local_steps > 1024)
+    return fail(ABS_EINVAL, "local_steps %d outside [1, 1024]", model->local_steps);
+  if (model->local_steps > 1) {
+    // U > 1: the worker's local model lives in shared memory; single-layer models only
+    if (model->kind == ABS_MLP)
+      return fail(ABS_EUNSUPPORTED, "local_steps = %d: U > 1 is implemented for least squares and soft-max regression only", model->local_steps);
+    const int C = model->kind == ABS_LSQ ? 1 : model->dims[1];
+    const size_t n_par = model->kind == ABS_LSQ ? (size_t)model->dims[0] : (size_t)model->dims[0] * C + C;
+    if (C > local::MAX_C || n_par > (size_t)local::MAX_PARAMS || (size_t)model->batch * C > (size_t)local::MAX_BC)
+      return fail(ABS_EUNSUPPORTED, "local_steps > 1 needs at most %d classes, %d parameters and batch x classes <= %d",
+                  local::MAX_C, local::MAX_PARAMS, local::MAX_BC);
+  }
   if (K0 < 1 || K0 > W) return fail(ABS_EINVAL, "K0 %d outside [1, W]", K0);
   if (model->k_mode != ABS_K_ADAPTIVE && model->k_mode != ABS_K_FIXED) return fail(ABS_EINVAL, "k_mode");
   if (model->bound_mode != ABS_BOUND_ADAPTIVE && model->bound_mode != ABS_BOUND_FIXED &&
@@ -842,7 +855,8 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     c.row_idx[q] = ctx->at<int>(L.row_idx[q]); c.tile_slot[q] = ctx->at<int>(L.tile_slot[q]);
   }
   c.loss = ctx->at<float>(L.loss);
-  c.row_loss = model->kind == ABS_LSQ ? nullptr : ctx->at<float>(L.row_loss);
+  // with local steps a worker's loss is uploaded whole (no per-row losses, no row layout)
+  c.row_loss = (model->kind == ABS_LSQ || model->local_steps > 1) ? nullptr : ctx->at<float>(L.row_loss);
   c.tr_K = ctx->at<int>(L.tr_K); c.tr_R = ctx->at<int>(L.tr_R); c.tr_theta = ctx->at<int>(L.tr_theta);
   c.tr_T = ctx->at<u64>(L.tr_T); c.tr_loss = ctx->at<float>(L.tr_loss); c.tr_comm = ctx->at<u64>(L.tr_comm);
   c.tr_sel_off = ctx->at<i64>(L.tr_sel_off); c.tr_rst_off = ctx->at<i64>(L.tr_rst_off);
@@ -878,7 +892,16 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
       ef = cudaFuncSetAttribute(narrow_fused_cc_kernel<__nv_bfloat16, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (ef != cudaSuccess) return bail(cuda_fail(nullptr, ef, "cudaFuncSetAttribute(narrow_fused_kernel)"));
   }
-  if (model->kind == ABS_LSQ && model->dims[0] % 8 == 0 && model->dims[0] <= LSQ_MAX_D) {
+  if (model->local_steps > 1) {
+    const int C = model->kind == ABS_LSQ ? 1 : model->dims[1];
+    const int n_par = model->kind == ABS_LSQ ? model->dims[0] : model->dims[0] * C + C;
+    const int sm = (int)local::smem_bytes(n_par, model->batch, C);
+    cudaError_t el = cudaFuncSetAttribute(local::local_sgd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+    if (el == cudaSuccess) el = cudaFuncSetAttribute(local::local_sgd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+    if (el != cudaSuccess) return bail(cuda_fail(nullptr, el, "cudaFuncSetAttribute(local_sgd_kernel)"));
+    ctx->local_sgd = true;
+  }
+  if (!ctx->local_sgd && model->kind == ABS_LSQ && model->dims[0] % 8 == 0 && model->dims[0] <= LSQ_MAX_D) {
     ctx->lsq_v2 = true;
     ctx->lsq_grid = std::min(W, 2 * ctx->sm_count);
     // bf16 rows of up to 8 KB: stream them through shared memory with bulk copies, one CTA per SM
@@ -895,7 +918,7 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
       }
     }
   }
-  if (model->kind == ABS_LSQ && !(model->flags & ABS_FLAG_NO_PERSISTENT) && model->dims[0] % 8 == 0 &&
+  if (!ctx->local_sgd && model->kind == ABS_LSQ && !(model->flags & ABS_FLAG_NO_PERSISTENT) && model->dims[0] % 8 == 0 &&
       model->dims[0] <= LSQ_ROUNDS_MAX_D && W <= LSQ_ROUNDS_NTG && (size_t)W * model->batch <= LSQ_ROUNDS_MAX_ROWS &&
       (size_t)(staleness_bound + 1) * model->dims[0] * 4 <= 64 * 1024) {
     const size_t sm = lsq_rounds_smem(staleness_bound, model->dims[0]);
@@ -950,7 +973,28 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     if (f32) enqueue_update<float>(ctx, par);
     else enqueue_update<__nv_bfloat16>(ctx, par);
   };
-  if (n > 0 && ctx->lsq_rounds) {
+  if (n > 0 && ctx->local_sgd) {
+    local::Args q;
+    q.st = ctx->at<DevState>(ctx->L.st);
+    q.sel = nullptr; q.sel_tau = nullptr; q.ri = nullptr;
+    q.job = ctx->ctl.job; q.X = ctx->X; q.y = ctx->y;
+    q.ring = ctx->at<void>(ctx->L.ring); q.slot_stride = ctx->L.d_pad;
+    q.loss = ctx->ctl.loss; q.G = ctx->at<float>(ctx->L.G);
+    q.lsq = ctx->m.kind == ABS_LSQ ? 1 : 0;
+    q.in = ctx->m.dims[0]; q.C = q.lsq ? 1 : ctx->m.dims[1]; q.U = ctx->m.local_steps; q.lr = ctx->m.lr;
+    const size_t sm = local::smem_bytes(q.lsq ? q.in : q.in * q.C + q.C, ctx->m.batch, q.C);
+    for (int r = 0; r < n; ++r) {
+      const int t = ctx->rounds_enqueued + r, par = t & 1;
+      launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
+      launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
+      q.ri = ctx->at<RoundInfo>(ctx->L.ri) + par;
+      q.sel = ctx->ctl.sel[par]; q.sel_tau = ctx->ctl.sel_tau[par];
+      if (f32) launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<float>, dim3(ctx->W), dim3(256), sm, q);
+      else launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<__nv_bfloat16>, dim3(ctx->W), dim3(256), sm, q);
+      update(par);
+    }
+    launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+  } else if (n > 0 && ctx->lsq_rounds) {
     LsqRoundsArgs q;
     q.X = ctx->X; q.y = (const float*)ctx->y;
     q.master = ctx->at<float>(ctx->L.master); q.ring = ctx->at<void>(ctx->L.ring);

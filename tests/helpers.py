@@ -48,7 +48,7 @@ def compare_with_oracle(cfg, X, y, w0, rounds, tol, forced=False, loss_tol=None,
     traces must be identical.  forced=True: the oracle's K rule is fed the
     GPU's uploaded losses (its own losses and parameters are still its own),
     which separates the integer machinery from last-bit loss differences."""
-    gkw = {k: v for k, v in kw.items() if k in ("k_mode", "bound_mode", "bound_offset")}
+    gkw = {k: v for k, v in kw.items() if k in ("k_mode", "bound_mode", "bound_offset", "local_steps")}
     rows, params = gpu_run(cfg, X, y, w0, rounds, flags=kw.get("flags", 0), **gkw)
     assert len(rows) == rounds
     o = make_oracle(cfg, X, y, w0, **gkw)

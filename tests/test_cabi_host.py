@@ -95,7 +95,9 @@ def _init_args():
 
 
 @pytest.mark.parametrize("mutate,code", [
-    (lambda m, td: setattr(m, "local_steps", 10), gpu.EUNSUPPORTED),
+    (lambda m, td: setattr(m, "local_steps", 0), gpu.EINVAL),
+    (lambda m, td: setattr(m, "local_steps", 2000), gpu.EINVAL),
+    (lambda m, td: (setattr(m, "local_steps", 4), setattr(m, "batch", 1024), m.dims.__setitem__(0, 20000)), gpu.EUNSUPPORTED),
     (lambda m, td: setattr(m, "workspace", 0), gpu.EINVAL),
     (lambda m, td: setattr(m, "workspace", 0x10010), gpu.EINVAL),
     (lambda m, td: setattr(m, "workspace_bytes", 1024), gpu.ENOSPACE),

@@ -152,6 +152,34 @@ def test_threshold_offset_needs_a_large_enough_bound():
     assert e.value.code == gpu.EINVAL
 
 
+@pytest.mark.parametrize("kind,dims,dtype,W,B,U,forced", [
+    (inputs.LSQ, (24, 1), inputs.FP32, 8, 6, 10, False),        # the paper's U = 10, N = 8
+    (inputs.LSQ, (77, 1), inputs.FP32, 13, 19, 3, True),
+    (inputs.LSQ, (64, 1), inputs.BF16, 20, 8, 4, True),
+    (inputs.SOFTMAX, (40, 6), inputs.FP32, 11, 16, 5, False),
+    (inputs.SOFTMAX, (131, 7), inputs.FP32, 13, 24, 2, True),
+    (inputs.SOFTMAX, (48, 10), inputs.BF16, 16, 12, 3, True),
+])
+def test_local_sgd_steps(kind, dims, dtype, W, B, U, forced):
+    """Eq. 2 with U > 1: every job is U local minibatch steps on the worker's own copy of the model;
+    trace and parameters must match the oracle's local-SGD runs."""
+    cfg = _small_cfg(kind, dims, dtype, W, B, 3, 5, GAMMA3, lr=0.02)
+    X, y, w0 = _problem(cfg)
+    bf16 = dtype == inputs.BF16
+    rows, orows, err, o = compare_with_oracle(cfg, X, y, w0, 40, TOL_BF16 if bf16 else TOL_FP32, forced=forced,
+                                              loss_tol=5e-2 if bf16 else None, local_steps=U)
+    assert rows[-1]["loss_mean"] < rows[0]["loss_mean"]
+
+
+def test_local_sgd_steps_rejected_for_multi_layer_networks():
+    cfg = _small_cfg(inputs.MLP, (64, 128, 10), inputs.BF16, 8, 16, 3, 5, EXP)
+    X, y, w0 = _problem(cfg)
+    Xd, yd = to_device(cfg, X, y)
+    with pytest.raises(gpu.AbsError) as e:
+        gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=5, local_steps=4)
+    assert e.value.code == gpu.EUNSUPPORTED
+
+
 def test_lock_step_constant_times():
     cfg = _small_cfg(inputs.LSQ, (16, 1), inputs.FP32, 8, 4, 2, 3,
                      inputs.TimeSpec(inputs.T_CONST, shift=3.0))
