@@ -983,14 +983,15 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     q.lsq = ctx->m.kind == ABS_LSQ ? 1 : 0;
     q.in = ctx->m.dims[0]; q.C = q.lsq ? 1 : ctx->m.dims[1]; q.U = ctx->m.local_steps; q.lr = ctx->m.lr;
     const size_t sm = local::smem_bytes(q.lsq ? q.in : q.in * q.C + q.C, ctx->m.batch, q.C);
+    const int nt = local::threads_for(q.lsq ? q.in : q.in * q.C + q.C);
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
       launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
       launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
       q.ri = ctx->at<RoundInfo>(ctx->L.ri) + par;
       q.sel = ctx->ctl.sel[par]; q.sel_tau = ctx->ctl.sel_tau[par];
-      if (f32) launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<float>, dim3(ctx->W), dim3(256), sm, q);
-      else launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<__nv_bfloat16>, dim3(ctx->W), dim3(256), sm, q);
+      if (f32) launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<float>, dim3(ctx->W), dim3(nt), sm, q);
+      else launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<__nv_bfloat16>, dim3(ctx->W), dim3(nt), sm, q);
       update(par);
     }
     launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);

@@ -19,6 +19,8 @@ namespace local {
 constexpr int MAX_PARAMS = 12288;     // fp32 parameters of the local model (twice in shared memory)
 constexpr int MAX_C = 16;
 constexpr int MAX_BC = 8192;          // B * C deltas of one step
+constexpr int NT_MAX = 1024;          // threads per CTA: only K CTAs run, so a large model gets wide CTAs
+inline int threads_for(int n_par) { return n_par >= 2048 ? NT_MAX : 256; }
 
 struct Args {
   DevState* st;
@@ -38,7 +40,7 @@ inline size_t smem_bytes(int n_par, int B, int C) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256) local_sgd_kernel(Args a) {
+__global__ void __launch_bounds__(NT_MAX) local_sgd_kernel(Args a) {
   grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char loc_raw[];
   DevState* st = a.st;
@@ -55,6 +57,7 @@ __global__ void __launch_bounds__(256) local_sgd_kernel(Args a) {
   float* red = rl + B;                                   // [64]
   int* sidx = reinterpret_cast<int*>(red + 64);          // [B] sample indices of the step
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int NT = (int)blockDim.x;
   const int wn = a.sel[i], jb = a.job[wn];
   const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
   const T* w0 = (const T*)a.ring + (size_t)slot * a.slot_stride;
@@ -65,10 +68,10 @@ __global__ void __launch_bounds__(256) local_sgd_kernel(Args a) {
   const uint32_t key0 = st->key0, key1 = st->key1;
   const int nblk = (B + 3) >> 2;
   const float step = __fdiv_rn(a.lr, (float)B);
-  for (int p = tid; p < n_par; p += 256) { wl[p] = ldf(w0, p); gs[p] = 0.f; }
+  for (int p = tid; p < n_par; p += NT) { wl[p] = ldf(w0, p); gs[p] = 0.f; }
   float loss_sum = 0.f;
   for (int u = 0; u < U; ++u) {
-    for (int blk = tid; blk < nblk; blk += 256) {
+    for (int blk = tid; blk < nblk; blk += NT) {
       uint32_t w4[4];
       philox4x32_10((uint32_t)wn, (uint32_t)jb, 1u, (uint32_t)(u * nblk + blk), key0, key1, w4);
 #pragma unroll
@@ -77,7 +80,7 @@ __global__ void __launch_bounds__(256) local_sgd_kernel(Args a) {
     }
     __syncthreads();
     // ---- forward at the local model: one warp per row
-    for (int b = warp; b < B; b += 8) {
+    for (int b = warp; b < B; b += NT / 32) {
       const T* x = X + (size_t)sidx[b] * in;
       float acc[MAX_C];
 #pragma unroll
@@ -122,13 +125,13 @@ __global__ void __launch_bounds__(256) local_sgd_kernel(Args a) {
     // ---- mean loss of the step (fixed order: strided partial sums, then a shuffle tree, then the warps in order)
     {
       float part = 0.f;
-      for (int b = tid; b < B; b += 256) part += rl[b];
+      for (int b = tid; b < B; b += NT) part += rl[b];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
       if (lane == 0) red[warp] = part;
     }
     // ---- gradient sum of the step, one feature per thread (all classes), and the local step
-    for (int m = tid; m < in; m += 256) {
+    for (int m = tid; m < in; m += NT) {
       float acc[MAX_C];
 #pragma unroll
       for (int c = 0; c < MAX_C; ++c) acc[c] = 0.f;
@@ -155,12 +158,12 @@ __global__ void __launch_bounds__(256) local_sgd_kernel(Args a) {
     __syncthreads();
     if (tid == 0) {
       float tot = 0.f;
-      for (int q = 0; q < 8; ++q) tot += red[q];
+      for (int q = 0; q < NT / 32; ++q) tot += red[q];
       loss_sum += __fdiv_rn(tot, (float)B);
     }
   }
   float* g = a.G + (size_t)i * a.slot_stride;
-  for (int p = tid; p < n_par; p += 256) g[p] = gs[p];
+  for (int p = tid; p < n_par; p += NT) g[p] = gs[p];
   if (tid == 0) {
     const float loss = __fdiv_rn(loss_sum, (float)U);
     a.loss[i] = loss;
