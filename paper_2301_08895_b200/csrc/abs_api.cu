@@ -698,7 +698,7 @@ void enqueue_update(abs_ctx* ctx, int par) {
   RoundInfo* ri = ctx->at<RoundInfo>(L.ri) + par;
   if (ctx->lsq_v2) {
     LsqUpdateArgs q;
-    q.st = ctx->at<DevState>(L.st); q.ri = ri; q.job = ctx->ctl.job; q.next_dur = ctx->ctl.next_dur; q.dur_job = ctx->ctl.dur_job;
+    q.st = ctx->at<DevState>(L.st); q.ri = ri; q.job = ctx->ctl.job; q.next_dur = ctx->overlap ? nullptr : ctx->ctl.next_dur; q.dur_job = ctx->ctl.dur_job;
     q.master = ctx->at<float>(L.master); q.ring = ctx->at<void>(L.ring); q.G = ctx->at<float>(L.G);
     q.d_pad = L.d_pad; q.d = ctx->m.dims[0]; q.P = ctx->lsq_grid; q.lr = ctx->m.lr;
     q.loss_part = ctx->lsq_pipe ? ctx->at<float>(L.row_loss) : nullptr;
@@ -710,7 +710,9 @@ void enqueue_update(abs_ctx* ctx, int par) {
   UpdateArgs u;
   u.st = ctx->at<DevState>(L.st); u.ri = ri; u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
   u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
-  u.job = ctx->ctl.job; u.next_dur = ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
+  // on one stream the Eq. 3 kernel also prepares the next job durations (its first warps); with the
+  // side stream a small kernel of its own does
+  u.job = ctx->ctl.job; u.next_dur = ctx->overlap ? nullptr : ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
   const size_t n4 = L.d_pad / 4;
   const int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * 8), (size_t)(ctx->W + 31) / 32);
   launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T>, dim3(blocks), dim3(256), 0, u);
@@ -987,7 +989,6 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
       launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
-      launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
       q.ri = ctx->at<RoundInfo>(ctx->L.ri) + par;
       q.sel = ctx->ctl.sel[par]; q.sel_tau = ctx->ctl.sel_tau[par];
       if (f32) launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<float>, dim3(ctx->W), dim3(nt), sm, q);
@@ -1008,7 +1009,6 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
       // the control kernel completes the previous round (if any) and selects this round's arrivals
       launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
-      launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
       gradient(par, PH_GATHER);
       gradient(par, PH_FORWARD);
       gradient(par, PH_BACKWARD);

@@ -337,6 +337,9 @@ __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
   const DevState* st = a.st;
   const RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
+  // duration look-ahead for the workers whose job index moved (first warp of the first ceil(N/32) blocks)
+  if (a.next_dur != nullptr && threadIdx.x < 32 && (int)blockIdx.x * 32 < st->W)
+    refresh_next_durations(st, a.job, a.next_dur, a.dur_job, (int)blockIdx.x * 32 + (int)threadIdx.x);
   if (ri->diverged) return;
   const int K = ri->K;
   const int P = a.P > 0 ? a.P : K;
