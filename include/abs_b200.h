@@ -61,6 +61,13 @@ extern "C" {
 #define ABS_BOUND_OFFSET    2   /* Eq. 4 with the constant a given: max(1, floor(N/K) + bound_offset), capped by
                                    the staleness bound (the sweep over a of Sec. V-B) */
 
+#define ABS_RESTART_ALGORITHM1 0 /* Eq. 6 in the order Algorithm 1 performs it: ages are incremented first, then a
+                                   non-selected worker restarts iff its new age exceeds the threshold; consumed
+                                   staleness never exceeds the staleness bound */
+#define ABS_RESTART_EQ6        1 /* Eq. 6 as printed: the age before the increment is tested, so a worker restarts
+                                   one round later and a consumed gradient may be staleness bound + 1 rounds old
+                                   (the library then keeps one more model version) */
+
 /* execution-time laws (random execution times with stragglers, Sec. V-A) */
 #define ABS_T_CONST        0    /* shift */
 #define ABS_T_EXP          1    /* Exp(rate) */
@@ -121,6 +128,7 @@ typedef struct {
   int bound_mode;           /* ABS_BOUND_* */
   int bound_offset;         /* the constant a of Eq. 4 when bound_mode = ABS_BOUND_OFFSET (else ignored);
                                floor(N/K0) + a must not exceed the staleness bound */
+  int restart_rule;         /* ABS_RESTART_* */
   int max_rounds;           /* trace capacity: total rounds this context may run */
   int flags;                /* ABS_FLAG_* bits */
   int data_on_host;         /* 0: X, y are device pointers owned by the caller and must outlive

@@ -19,6 +19,7 @@ LSQ, SOFTMAX, MLP = 0, 1, 2
 FP32, BF16_FP32MASTER = 0, 1
 K_ADAPTIVE, K_FIXED = 0, 1
 BOUND_ADAPTIVE, BOUND_FIXED, BOUND_OFFSET = 0, 1, 2
+RESTART_ALGORITHM1, RESTART_EQ6 = 0, 1
 T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2, T_GAMMA = 0, 1, 2, 3, 4
 MAX_LAYERS = 7
 FLAG_NO_TENSOR_CORES = 1
@@ -35,7 +36,7 @@ class ModelDesc(C.Structure):
     _fields_ = [("kind", C.c_int), ("n_layers", C.c_int), ("dims", C.c_int * (MAX_LAYERS + 1)),
                 ("batch", C.c_int), ("lr", C.c_float), ("dtype", C.c_int),
                 ("local_steps", C.c_int), ("k_mode", C.c_int), ("bound_mode", C.c_int),
-                ("bound_offset", C.c_int), ("max_rounds", C.c_int), ("flags", C.c_int), ("data_on_host", C.c_int),
+                ("bound_offset", C.c_int), ("restart_rule", C.c_int), ("max_rounds", C.c_int), ("flags", C.c_int), ("data_on_host", C.c_int),
                 ("X", C.c_void_p), ("y", C.c_void_p), ("n_samples", C.c_longlong),
                 ("w0", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("stream", C.c_void_p)]
@@ -114,7 +115,7 @@ def n_params(kind, dims):
 
 
 def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-          local_steps=1, data_on_host=0, flags=0, bound_offset=0):
+          local_steps=1, data_on_host=0, flags=0, bound_offset=0, restart_rule=0):
     m = ModelDesc()
     m.kind, m.n_layers = kind, len(dims) - 1
     for i, v in enumerate(dims):
@@ -124,6 +125,7 @@ def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mod
     m.max_rounds, m.data_on_host, m.n_samples = int(max_rounds), data_on_host, int(n_samples)
     m.flags = int(flags)
     m.bound_offset = int(bound_offset)
+    m.restart_rule = int(restart_rule)
     return m
 
 
@@ -145,14 +147,15 @@ class Context:
 
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, time, seed, max_rounds,
                  dtype=FP32, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE, local_steps=1,
-                 data_on_host=False, stream=None, device="cuda:0", flags=0, bound_offset=0):
+                 data_on_host=False, stream=None, device="cuda:0", flags=0, bound_offset=0,
+                 restart_rule=0):
         import torch
         self._torch = torch
         self.kind, self.dims, self.W, self.S = kind, list(dims), W, S
         self.max_rounds = max_rounds
         n_samples = X.shape[0]
         m = _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-                  local_steps, 1 if data_on_host else 0, flags, bound_offset)
+                  local_steps, 1 if data_on_host else 0, flags, bound_offset, restart_rule)
         need = C.c_size_t(0)
         _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(need)))
         self.device = torch.device(device)

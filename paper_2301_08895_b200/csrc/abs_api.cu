@@ -102,6 +102,9 @@ int check_model(const abs_model_desc* m, int W, int S) {
   if (W < 1 || W > ABS_MAX_WORKERS) return fail(ABS_EINVAL, "W %d outside [1, %d]", W, ABS_MAX_WORKERS);
   if (m->n_samples < W) return fail(ABS_EINVAL, "fewer samples than workers");
   if (S < 0 || S > ABS_MAX_BOUND) return fail(ABS_EINVAL, "staleness_bound %d outside [0, %d]", S, ABS_MAX_BOUND);
+  if (m->restart_rule != ABS_RESTART_ALGORITHM1 && m->restart_rule != ABS_RESTART_EQ6) return fail(ABS_EINVAL, "restart_rule");
+  if (m->restart_rule == ABS_RESTART_EQ6 && S + 1 > ABS_MAX_BOUND)
+    return fail(ABS_EINVAL, "staleness_bound %d: Eq. 6 as printed keeps one more version, at most %d", S, ABS_MAX_BOUND - 1);
   return ABS_OK;
 }
 
@@ -748,7 +751,7 @@ int abs_workspace_bytes(const abs_model_desc* model, int W, int staleness_bound,
   const int rc = check_model(model, W, staleness_bound);
   if (rc != ABS_OK) return rc;
   Layout L;
-  make_layout(model, W, staleness_bound, &L);
+  make_layout(model, W, staleness_bound + (model->restart_rule == ABS_RESTART_EQ6 ? 1 : 0), &L);
   *out = L.total;
   return ABS_OK;
 }
@@ -799,14 +802,17 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   if (((uintptr_t)model->workspace & 255) != 0) return fail(ABS_EINVAL, "workspace must be 256-byte aligned");
   if (!model->data_on_host && (((uintptr_t)model->X & 15) != 0 || ((uintptr_t)model->y & 3) != 0))
     return fail(ABS_EINVAL, "X must be 16-byte aligned, y 4-byte aligned");
+  // Eq. 6 as printed lets a consumed gradient be one round older: one more ring slot, same threshold
+  const int literal = model->restart_rule == ABS_RESTART_EQ6 ? 1 : 0;
+  const int S_ring = staleness_bound + literal;
   Layout L;
-  make_layout(model, W, staleness_bound, &L);
+  make_layout(model, W, S_ring, &L);
   if (model->workspace_bytes < L.total)
     return fail(ABS_ENOSPACE, "workspace has %zu bytes, %zu needed", model->workspace_bytes, L.total);
 
   ctx = new (std::nothrow) abs_ctx();
   if (!ctx) return fail(ABS_EINVAL, "out of host memory");
-  ctx->m = *model; ctx->L = L; ctx->W = W; ctx->K0 = K0; ctx->S = staleness_bound;
+  ctx->m = *model; ctx->L = L; ctx->W = W; ctx->K0 = K0; ctx->S = S_ring;
   ctx->stream = (cudaStream_t)model->stream;
   ctx->ws = (char*)model->workspace;
   cudaStream_t s = ctx->stream;
@@ -835,7 +841,8 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   }
   DevState h;
   memset(&h, 0, sizeof h);
-  h.W = W; h.K0 = K0; h.S = staleness_bound; h.B = model->batch; h.RB = L.RB;
+  h.W = W; h.K0 = K0; h.S = S_ring; h.B = model->batch; h.RB = L.RB;
+  h.theta_cap = staleness_bound; h.literal_eq6 = literal;
   h.k_mode = model->k_mode; h.bound_mode = model->bound_mode; h.max_rounds = model->max_rounds;
   h.n_samples = model->n_samples;
   h.key0 = (uint32_t)(seed & 0xffffffffull); h.key1 = (uint32_t)(seed >> 32);
@@ -922,8 +929,8 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   }
   if (!ctx->local_sgd && model->kind == ABS_LSQ && !(model->flags & ABS_FLAG_NO_PERSISTENT) && model->dims[0] % 8 == 0 &&
       model->dims[0] <= LSQ_ROUNDS_MAX_D && W <= LSQ_ROUNDS_NTG && (size_t)W * model->batch <= LSQ_ROUNDS_MAX_ROWS &&
-      (size_t)(staleness_bound + 1) * model->dims[0] * 4 <= 64 * 1024) {
-    const size_t sm = lsq_rounds_smem(staleness_bound, model->dims[0]);
+      (size_t)(S_ring + 1) * model->dims[0] * 4 <= 64 * 1024) {
+    const size_t sm = lsq_rounds_smem(S_ring, model->dims[0]);
     cudaError_t er = cudaFuncSetAttribute(abs_lsq_rounds_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (er == cudaSuccess)
       er = cudaFuncSetAttribute(abs_lsq_rounds_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);

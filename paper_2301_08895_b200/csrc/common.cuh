@@ -35,9 +35,13 @@ struct TimeDist {
 // Scalars of Algorithm 1 that live on the device between rounds.
 struct DevState {
   // constants of the run
-  int W, K0, S, B, RB;            // RB: every version group's rows are padded to a multiple of RB
+  int W, K0, S, B, RB;            // S: the ring keeps S + 1 model versions; RB: every version group's rows are
+                                  // padded to a multiple of RB
   int k_mode, bound_mode, max_rounds;
   int bound_offset;               // the constant a of Eq. 4 (ABS_BOUND_OFFSET)
+  int theta_cap;                  // largest threshold = the caller's staleness bound
+  int literal_eq6;                // 1: the restart test reads the age before its increment (Eq. 6 as printed);
+                                  // S is then the caller's bound + 1 (oldest model version still in use)
   i64 n_samples;
   uint32_t key0, key1;            // Philox key = (seed low, seed high)
   TimeDist dist;

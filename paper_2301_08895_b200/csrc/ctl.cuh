@@ -162,7 +162,7 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
   const int po = (t_sel - 1) & 1, pn = t_sel & 1;     // layout copy of the open / of the new round
   const int status0 = st->status, open0 = st->open, diverged0 = a.ri[po].diverged;
   const int k_mode = st->k_mode, bound_mode = st->bound_mode, max_rounds = st->max_rounds;
-  const int bound_offset = st->bound_offset;
+  const int bound_offset = st->bound_offset, Scap = st->theta_cap, literal = st->literal_eq6;
   const uint32_t key0 = st->key0, key1 = st->key1;
   const i64 n_samples = st->n_samples;
   const u64 T_end0 = st->T_end;
@@ -259,24 +259,24 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
     int K_next = K;
     if (k_mode == ABS_K_ADAPTIVE) K_next = min(W, max(K, sh.scalar[2]));
     // Eq. 4 with a = S - N/K0, in integers
-    int theta = S;
+    int theta = Scap;
     if (bound_mode == ABS_BOUND_ADAPTIVE) {
       const i64 fl = floor_div((i64)W * (i64)(K0 - K_next), (i64)K_next * (i64)K0);
-      i64 th = (i64)S + fl;
+      i64 th = (i64)Scap + fl;
       if (th < 1) th = 1;
-      if (th > S) th = S;
+      if (th > Scap) th = Scap;
       theta = (int)th;
     } else if (bound_mode == ABS_BOUND_OFFSET) {     // Eq. 4 with a given: floor(N/K + a) = floor(N/K) + a
       int th = W / K_next + bound_offset;
       if (th < 1) th = 1;
-      if (th > S) th = S;
+      if (th > Scap) th = Scap;
       theta = th;
     }
     // Eq. 6 in Algorithm 1's order: arrivals and over-stale workers get w^{t+1}
     int restart = 0, renew = 0;
     if (tid < W) {
       const int sel_me = sh.flag[tid];
-      restart = (!sel_me) && ((t + 1 - my_version) > theta);
+      restart = (!sel_me) && ((t + 1 - literal - my_version) > theta);
       renew = sel_me || restart;
     }
     int range_err = 0;

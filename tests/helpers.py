@@ -49,9 +49,11 @@ def compare_with_oracle(cfg, X, y, w0, rounds, tol, forced=False, loss_tol=None,
     GPU's uploaded losses (its own losses and parameters are still its own),
     which separates the integer machinery from last-bit loss differences."""
     gkw = {k: v for k, v in kw.items() if k in ("k_mode", "bound_mode", "bound_offset", "local_steps")}
-    rows, params = gpu_run(cfg, X, y, w0, rounds, flags=kw.get("flags", 0), **gkw)
+    literal = kw.get("restart_rule", 0) == gpu.RESTART_EQ6
+    rows, params = gpu_run(cfg, X, y, w0, rounds, flags=kw.get("flags", 0),
+                           restart_rule=kw.get("restart_rule", 0), **gkw)
     assert len(rows) == rounds
-    o = make_oracle(cfg, X, y, w0, **gkw)
+    o = make_oracle(cfg, X, y, w0, literal_eq6=literal, **gkw)
     orows = o.run(rounds, forced_losses=[r["sel_loss"] for r in rows] if forced else None)
     mm = first_integer_mismatch(rows, orows)
     assert mm is None, "integer trace differs at round %s field %s: gpu %s oracle %s (oracle " \

@@ -143,6 +143,28 @@ def test_threshold_offset_sweep(a):
     assert all(max(r["tau"]) <= r0["theta"] for r0, r in zip(rows, rows[1:]))
 
 
+@pytest.mark.parametrize("kind,dims,dtype,W,B,K0,S,mode", [
+    (inputs.SOFTMAX, (40, 6), inputs.FP32, 20, 16, 5, 3, gpu.BOUND_ADAPTIVE),
+    (inputs.LSQ, (24, 1), inputs.FP32, 12, 6, 2, 2, gpu.BOUND_FIXED),          # persistent least-squares kernel
+    (inputs.MLP, (64, 128, 10), inputs.BF16, 40, 16, 4, 4, gpu.BOUND_ADAPTIVE),
+    (inputs.LSQ, (64, 1), inputs.BF16, 300, 8, 30, 1, gpu.BOUND_FIXED),         # bulk-copy pipeline
+])
+def test_restart_rule_of_eq6_as_printed(kind, dims, dtype, W, B, K0, S, mode):
+    """Eq. 6 tests the age before its increment; Algorithm 1 (the default) after it.  With the
+    printed rule a worker restarts one round later, so gradients of staleness S + 1 are consumed
+    and the model ring holds one more version; the trace must match the oracle's `literal_eq6` run."""
+    cfg = _small_cfg(kind, dims, dtype, W, B, K0, S, GAMMA3)
+    X, y, w0 = _problem(cfg)
+    bf16 = dtype == inputs.BF16
+    rows, _, _, _ = compare_with_oracle(cfg, X, y, w0, 50, TOL_BF16 if bf16 else TOL_FP32, forced=bf16,
+                                        loss_tol=5e-2 if bf16 else None, bound_mode=mode,
+                                        k_mode=gpu.K_FIXED, restart_rule=gpu.RESTART_EQ6)
+    assert max(max(r["tau"]) for r in rows) == S + 1          # one round older than Algorithm 1 allows
+    assert sum(len(r["restart"]) for r in rows) > 0
+    rows_b, _ = gpu_run(cfg, X, y, w0, 50, bound_mode=mode, k_mode=gpu.K_FIXED)
+    assert max(max(r["tau"]) for r in rows_b) <= S
+
+
 def test_threshold_offset_needs_a_large_enough_bound():
     cfg = _small_cfg(inputs.SOFTMAX, (40, 6), inputs.FP32, 20, 16, 5, 3, EXP)
     X, y, w0 = _problem(cfg)

@@ -138,6 +138,23 @@ def test_straggler_is_restarted_every_theta_plus_one_rounds():
         assert (4 in row["restart"]) == (t % (S + 2) == S + 1)
 
 
+def test_printed_eq6_equals_algorithm_order_with_threshold_plus_one():
+    """Testing the age before the increment against theta is the same as testing the incremented
+    age against theta + 1: with a fixed threshold the two readings play identical rounds."""
+    X, y, _ = _lsq_problem()
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    a = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.01, 9, 2, 2, dist, 3,
+                  k_mode=K_FIXED, bound_mode=BOUND_FIXED, literal_eq6=True)
+    b = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.01, 9, 2, 3, dist, 3,
+                  k_mode=K_FIXED, bound_mode=BOUND_FIXED)
+    ra, rb = a.run(80), b.run(80)
+    assert sum(len(r["restart"]) for r in ra) > 0
+    for x, z in zip(ra, rb):
+        assert x["theta"] + 1 == z["theta"]
+        assert {k: v for k, v in x.items() if k != "theta"} == {k: v for k, v in z.items() if k != "theta"}
+    assert max(max(r["tau"]) for r in ra) == 3          # one more than the bound of 2
+
+
 # ------------------------------------------------------------------- rules
 def test_selection_is_the_k_smallest_with_ties_to_lower_id():
     X, y, _ = _lsq_problem(d=2)
