@@ -87,6 +87,9 @@ extern "C" {
                                        tile is shared by several column tiles (each re-gathers it) */
 #define ABS_FLAG_NO_BULK_PIPELINE 32 /* bf16 least squares: per-warp 16-byte loads (rows read from HBM, then again
                                        from L2) instead of the bulk-copy pipeline through shared memory */
+#define ABS_FLAG_FUSED_FORWARD  128 /* tensor-core networks: two consecutive hidden layers with the same tile width
+                                       run their forward GEMMs in one launch, tiles of the second waiting on
+                                       completion counters of the first (same results; measured no faster end to end) */
 #define ABS_FLAG_NO_FUSED_BACKWARD 64 /* tensor-core networks: a layer's delta back-propagation and its weight
                                        gradient always get a launch each */
 #define ABS_FLAG_NO_PERSISTENT   8  /* small least-squares problems: one kernel launch per step of a round
@@ -251,6 +254,10 @@ int abs_get_plan(abs_ctx* ctx, int* partials, int* row_block, int* rows_cap, int
  * kernel class (ABS_KC_*; both arrays need ABS_KC_COUNT entries), and ends profiling. */
 int abs_profile_start(abs_ctx* ctx, int max_launches);
 int abs_profile_read(abs_ctx* ctx, long long* launches, double* total_ms);
+/* Before abs_profile_read: the recorded launches one by one, in launch order (both streams): kernel
+ * class and the times of the two bracketing events in ms since the first recorded launch.  The
+ * arrays need `cap` entries; *n_out receives the number filled.  Synchronises. */
+int abs_profile_timeline(abs_ctx* ctx, int cap, int* cls, float* start_ms, float* end_ms, int* n_out);
 
 int abs_destroy(abs_ctx* ctx);
 

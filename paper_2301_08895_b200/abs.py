@@ -29,6 +29,7 @@ FLAG_NO_PERSISTENT = 8
 FLAG_TMA_GATHER = 16
 FLAG_NO_BULK_PIPELINE = 32
 FLAG_NO_FUSED_BACKWARD = 64
+FLAG_FUSED_FORWARD = 128
 KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update", "rounds")
 
 
@@ -94,6 +95,8 @@ def lib():
                                    C.POINTER(C.c_int), C.POINTER(C.c_int)]
         l.abs_profile_start.argtypes = [C.c_void_p, C.c_int]
         l.abs_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
+        l.abs_profile_timeline.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.POINTER(C.c_int)]
         l.abs_destroy.argtypes = [C.c_void_p]
         _lib = l
     return _lib
@@ -246,6 +249,17 @@ class Context:
         ms = (C.c_double * len(KC_NAMES))()
         _check(lib().abs_profile_read(self._ctx, n, ms))
         return {KC_NAMES[i]: (int(n[i]), float(ms[i])) for i in range(len(KC_NAMES))}
+
+    def profile_timeline(self, cap=4096):
+        """[(class name, start ms, end ms)] of the launches recorded since profile_start (call
+        before profile_read)."""
+        cls = np.zeros(cap, np.int32)
+        t0 = np.zeros(cap, np.float32)
+        t1 = np.zeros(cap, np.float32)
+        n = C.c_int(0)
+        _check(lib().abs_profile_timeline(self._ctx, cap, cls.ctypes.data, t0.ctypes.data,
+                                          t1.ctypes.data, C.byref(n)))
+        return [(KC_NAMES[cls[i]], float(t0[i]), float(t1[i])) for i in range(n.value)]
 
     def close(self):
         if self._ctx:

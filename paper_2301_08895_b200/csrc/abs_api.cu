@@ -62,6 +62,8 @@ struct Layout {
   bool gather_tma = false;              // first-layer GEMMs fetch the minibatch rows from the dataset themselves
   bool two_cta = false;                 // GEMMs with N >= 256 run on CTA pairs (tiles of 256 x 256)
   int cg_fwd[ABS_MAX_LAYERS] = {}, cg_dg[ABS_MAX_LAYERS] = {}, cg_wg[ABS_MAX_LAYERS] = {};
+  bool pair_fwd[ABS_MAX_LAYERS] = {};   // forward GEMMs of layers l and l + 1 share a launch
+  size_t done;                          // completion counters per row tile (paired forward launches)
   bool pair_bwd[ABS_MAX_LAYERS] = {};   // delta back-propagation and weight gradient of the layer share a launch
   int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
   bool out_mma = false;                 // output layer through the mma.sync kernel (bf16, 64 rows per CTA)
@@ -169,6 +171,16 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
         L->cg_wg[l] = 2; L->bn_wg[l] = 256;
       }
     }
+    // Opt-in: two consecutive tensor-core layers with the same tile width run their forward GEMMs in
+    // one launch (the second behind per-row-tile completion counters): one set of fixed launch
+    // costs, and the second layer's tiles fill the first layer's last, partly empty wave.
+    for (int l = 0; l + 1 < m->n_layers; ++l) {
+      if (L->path[l] != PATH_TC || L->path[l + 1] != PATH_TC || !(m->flags & ABS_FLAG_FUSED_FORWARD)) continue;
+      if (L->cg_fwd[l] != 1 || L->cg_fwd[l + 1] != 1 || L->bn_fwd[l] != L->bn_fwd[l + 1]) continue;
+      if (l == 0 && L->gather_tma) continue;
+      if (l > 0 && L->pair_fwd[l - 1]) continue;
+      L->pair_fwd[l] = true;
+    }
     // A short weight gradient (fewer tiles than SMs at the back-propagation's tile width) shares
     // its launch with the layer's delta back-propagation: both have one or two tiles per CTA, so
     // separate launches would pay the fixed costs of a launch twice.
@@ -224,6 +236,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   }
   L->loss = cv.take(4 * W);
   L->row_loss = cv.take(4 * (size_t)L->rows_cap);
+  L->done = cv.take(4 * (size_t)L->n_tiles_cap);
   L->master = cv.take(4 * L->d_pad);
   L->ring = cv.take(L->esz * L->d_pad * (S + 1));
   if (m->local_steps > 1) L->P = 0;      // Eq. 3 adds one upload per selected worker
@@ -590,7 +603,25 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       p.relu_bits = L.bits[l + 1] ? ctx->at<uint32_t>(L.bits[l + 1]) : nullptr;
       p.mask_words = (la[l].out + 31) / 32;
       const int bn = L.bn_fwd[l];
-      launch_tc_bn(ctx, bn, L.cg_fwd[l], ABS_KC_FWD, (l == 0 && L.gather_tma) ? ctx->tcl[l].x_rows : (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, (row_tiles128 / L.cg_fwd[l]) * ((la[l].out + bn - 1) / bn));
+      const CUtensorMap& amap = (l == 0 && L.gather_tma) ? ctx->tcl[l].x_rows : (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a;
+      const int tiles = (row_tiles128 / L.cg_fwd[l]) * ((la[l].out + bn - 1) / bn);
+      if (L.pair_fwd[l]) {
+        // the next layer's forward GEMM rides in the same launch, behind completion counters
+        const int n = l + 1;
+        tc::Params p2 = tc_params(n, tc::FWD);
+        p2.N_total = la[n].out; p2.K_total = la[n].in;
+        p2.out_bf16 = (__nv_bfloat16*)la[n].act_out;
+        p2.relu_bits = L.bits[n + 1] ? ctx->at<uint32_t>(L.bits[n + 1]) : nullptr;
+        p2.mask_words = (la[n].out + 31) / 32;
+        p.done_signal = ctx->at<int>(L.done);
+        p2.done_wait = ctx->at<int>(L.done);
+        p2.done_target = ((la[l].out + bn - 1) / bn) * tc::EPI_WARPS;
+        const TcProblem second = {&ctx->tcl[n].fwd_a, &ctx->tcl[n].fwd_b, &ctx->tcl[n].fwd_out, &p2, row_tiles128 * ((la[n].out + bn - 1) / bn)};
+        launch_tc_bn(ctx, bn, 1, ABS_KC_FWD, amap, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, tiles, &second);
+        ++l;
+        continue;
+      }
+      launch_tc_bn(ctx, bn, L.cg_fwd[l], ABS_KC_FWD, amap, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, tiles);
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
       if (L.fused_R) {
@@ -716,6 +747,9 @@ void enqueue_update(abs_ctx* ctx, int par) {
   // on one stream the Eq. 3 kernel also prepares the next job durations (its first warps); with the
   // side stream a small kernel of its own does
   u.job = ctx->ctl.job; u.next_dur = ctx->overlap ? nullptr : ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
+  u.zero_words = nullptr; u.n_zero = 0;
+  for (int l = 0; l < ctx->m.n_layers; ++l)
+    if (L.pair_fwd[l]) { u.zero_words = ctx->at<int>(L.done); u.n_zero = L.n_tiles_cap; }
   const size_t n4 = L.d_pad / 4;
   const int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * 8), (size_t)(ctx->W + 31) / 32);
   launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T>, dim3(blocks), dim3(256), 0, u);
@@ -1163,6 +1197,20 @@ int abs_profile_read(abs_ctx* ctx, long long* launches, double* total_ms) {
   }
   ctx->ev_cap = 0;
   ctx->ev_class.clear();
+  return ABS_OK;
+}
+
+int abs_profile_timeline(abs_ctx* ctx, int cap, int* cls, float* start_ms, float* end_ms, int* n_out) {
+  if (!ctx || !cls || !start_ms || !end_ms || !n_out || cap < 0) return fail(ABS_EINVAL, "bad argument");
+  CU(cudaStreamSynchronize(ctx->stream));
+  if (ctx->side) CU(cudaStreamSynchronize(ctx->side));
+  const int n = std::min<int>(cap, (int)ctx->ev_class.size());
+  for (int i = 0; i < n; ++i) {
+    cls[i] = ctx->ev_class[i];
+    CU(cudaEventElapsedTime(&start_ms[i], ctx->ev[0], ctx->ev[2 * i]));
+    CU(cudaEventElapsedTime(&end_ms[i], ctx->ev[0], ctx->ev[2 * i + 1]));
+  }
+  *n_out = n;
   return ABS_OK;
 }
 

@@ -327,6 +327,7 @@ struct UpdateArgs {
   size_t d_pad;
   int P;                  // partial count, or 0: one partial per selected worker (K^t)
   float lr;
+  int* zero_words; int n_zero;   // counters of the round's kernels to clear for the next round (or null)
 };
 
 // Eq. 3 and the ring write: w^{t+1} = w^t - eta / (K^t B) * sum_p G_p, stored as the fp32
@@ -340,6 +341,8 @@ __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
   // duration look-ahead for the workers whose job index moved (first warp of the first ceil(N/32) blocks)
   if (a.next_dur != nullptr && threadIdx.x < 32 && (int)blockIdx.x * 32 < st->W)
     refresh_next_durations(st, a.job, a.next_dur, a.dur_job, (int)blockIdx.x * 32 + (int)threadIdx.x);
+  if (a.zero_words != nullptr && blockIdx.x == gridDim.x - 1)
+    for (int i = threadIdx.x; i < a.n_zero; i += blockDim.x) a.zero_words[i] = 0;
   if (ri->diverged) return;
   const int K = ri->K;
   const int P = a.P > 0 ? a.P : K;
