@@ -27,9 +27,9 @@ sys.path.insert(0, ROOT)
 from paper_2301_08895_b200 import inputs  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes (read + write) per launch at K = N on configuration 4, from the ncu captures summarised in
-# profiles/tc_gemm_kernel_cfg4.md and profiles/update_kernel_cfg4.md; each figure is valid only for the kernel
-# source it was taken from (first 16 hex digits of the file's sha256).
+# DRAM bytes (read + write) per launch at K = N on configuration 4, from ncu captures of the GEMM and the
+# Eq. 3 kernel (summaries under profiles/); each figure is valid only for the kernel source it was taken
+# from (first 16 hex digits of the file's sha256).
 TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.4e6, "file": "tc.cuh", "sha256_16": "7bdde9a563de088e"},
            "update": {"config": 4, "bytes_per_launch": 75.7e6, "file": "simt.cuh", "sha256_16": "3da31ad4d03aac5c"}}
 METRIC = "worker_gradients_per_sec"

@@ -916,6 +916,9 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     const cudaError_t ea = cudaFuncSetAttribute(abs_ctl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 (int)sizeof(CtlShared));
     if (ea != cudaSuccess) return bail(cuda_fail(nullptr, ea, "cudaFuncSetAttribute(abs_ctl_kernel)"));
+    const cudaError_t eb = cudaFuncSetAttribute(abs_ctl_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)sizeof(CtlShared));
+    if (eb != cudaSuccess) return bail(cuda_fail(nullptr, eb, "cudaFuncSetAttribute(abs_ctl_small_kernel)"));
   }
   if (L.out_mma) {
     const int osm = (int)outl::smem_bytes(model->dims[model->n_layers - 1], model->dims[model->n_layers]);
@@ -1006,6 +1009,8 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     return fail(ABS_ENOSPACE, "%d rounds requested, %d of capacity %d already used", n, ctx->rounds_enqueued, ctx->m.max_rounds);
   const bool f32 = ctx->m.dtype == ABS_FP32;
   const size_t csm = sizeof(CtlShared);
+  void (*ctl_kernel)(CtlArgs, int, int, int) = ctx->W <= 256 ? abs_ctl_small_kernel : abs_ctl_kernel;
+  const int ctl_threads = ctx->W <= 256 ? 256 : 1024;
   const int times_blocks = (ctx->W + 31) / 32;
   const DevState* stc = ctx->at<DevState>(ctx->L.st);
   auto gradient = [&](int par, int phase) {
@@ -1029,14 +1034,14 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     const int nt = local::threads_for(q.lsq ? q.in : q.in * q.C + q.C);
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
-      launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
+      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
       q.ri = ctx->at<RoundInfo>(ctx->L.ri) + par;
       q.sel = ctx->ctl.sel[par]; q.sel_tau = ctx->ctl.sel_tau[par];
       if (f32) launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<float>, dim3(ctx->W), dim3(nt), sm, q);
       else launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<__nv_bfloat16>, dim3(ctx->W), dim3(nt), sm, q);
       update(par);
     }
-    launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
   } else if (n > 0 && ctx->lsq_rounds) {
     LsqRoundsArgs q;
     q.X = ctx->X; q.y = (const float*)ctx->y;
@@ -1049,13 +1054,13 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
       // the control kernel completes the previous round (if any) and selects this round's arrivals
-      launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
+      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
       gradient(par, PH_GATHER);
       gradient(par, PH_FORWARD);
       gradient(par, PH_BACKWARD);
       update(par);
     }
-    launch_ex(ctx, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
   } else if (n > 0) {
     // Two streams.  Side stream per round t: control kernel (finish t-1, select t), row gather,
     // [event ctl], duration look-ahead.  Main stream: wait ctl, forward kernels, [event loss],
@@ -1066,7 +1071,7 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     CU(cudaStreamWaitEvent(B, ctx->ev_loss, 0));
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
-      launch_on(ctx, B, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 1, t);
+      launch_on(ctx, B, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
       gradient(par, PH_GATHER);
       CU(cudaEventRecord(ctx->ev_ctl, B));
       launch_on(ctx, B, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
@@ -1077,7 +1082,7 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
       gradient(par, PH_BACKWARD);
       update(par);
     }
-    launch_on(ctx, B, ABS_KC_CTL, abs_ctl_kernel, dim3(1), dim3(1024), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+    launch_on(ctx, B, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
     CU(cudaEventRecord(ctx->ev_ctl, B));
     CU(cudaStreamWaitEvent(A, ctx->ev_ctl, 0));       // the caller's stream covers all of it
   }

@@ -447,6 +447,15 @@ __global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_fini
   ctl_round<1024>(a, sh, do_finish, do_select, t_sel);
 }
 
+// The same step with 256 threads for runs of at most 256 workers (one thread per worker is all the
+// step needs; its block-wide barriers are cheaper with 8 warps than with 32).
+__global__ void __launch_bounds__(256, 1) abs_ctl_small_kernel(CtlArgs a, int do_finish, int do_select, int t_sel) {
+  grid_dependency_sync();
+  extern __shared__ __align__(16) unsigned char ctl_smem[];
+  CtlShared& sh = *reinterpret_cast<CtlShared*>(ctl_smem);
+  ctl_round<256>(a, sh, do_finish, do_select, t_sel);
+}
+
 // Duration look-ahead (see refresh_next_durations): one warp per 32 workers.
 __global__ void abs_times_kernel(const DevState* st, const int* job, u64* next_dur, int* dur_job) {
   grid_dependency_sync();
