@@ -744,15 +744,17 @@ void enqueue_update(abs_ctx* ctx, int par) {
   UpdateArgs u;
   u.st = ctx->at<DevState>(L.st); u.ri = ri; u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
   u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
-  // on one stream the Eq. 3 kernel also prepares the next job durations (its first warps); with the
-  // side stream a small kernel of its own does
-  u.job = ctx->ctl.job; u.next_dur = ctx->overlap ? nullptr : ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
+  // for the latency-bound models (always one stream) the Eq. 3 kernel also prepares the next job
+  // durations (its first warps); tensor-core networks keep a small kernel of their own for that
+  const bool look = !L.any_tc;
+  u.job = ctx->ctl.job; u.next_dur = ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
   u.zero_words = nullptr; u.n_zero = 0;
   for (int l = 0; l < ctx->m.n_layers; ++l)
     if (L.pair_fwd[l]) { u.zero_words = ctx->at<int>(L.done); u.n_zero = L.n_tiles_cap; }
   const size_t n4 = L.d_pad / 4;
   const int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * 8), (size_t)(ctx->W + 31) / 32);
-  launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T>, dim3(blocks), dim3(256), 0, u);
+  if (look) launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T, true>, dim3(blocks), dim3(256), 0, u);
+  else launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T, false>, dim3(blocks), dim3(256), 0, u);
 }
 
 int read_status(abs_ctx* ctx, DevState* host) {
@@ -1055,6 +1057,8 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
       // the control kernel completes the previous round (if any) and selects this round's arrivals
       launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
+      if (ctx->L.any_tc)    // the other models prepare the next durations inside their Eq. 3 kernel
+        launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
       gradient(par, PH_GATHER);
       gradient(par, PH_FORWARD);
       gradient(par, PH_BACKWARD);

@@ -332,14 +332,16 @@ struct UpdateArgs {
 
 // Eq. 3 and the ring write: w^{t+1} = w^t - eta / (K^t B) * sum_p G_p, stored as the fp32
 // master and, in storage type, as ring slot (t+1) mod (S+1).  One pass, 16-byte accesses.
-template <typename T>
+// LOOK: the first warps also prepare the next job durations (latency-bound models, one stream); the
+// bandwidth-bound networks keep that in a kernel of its own so that this one stays a pure stream.
+template <typename T, bool LOOK>
 __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
   grid_dependency_sync();
   const DevState* st = a.st;
   const RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
   // duration look-ahead for the workers whose job index moved (first warp of the first ceil(N/32) blocks)
-  if (a.next_dur != nullptr && threadIdx.x < 32 && (int)blockIdx.x * 32 < st->W)
+  if (LOOK && threadIdx.x < 32 && (int)blockIdx.x * 32 < st->W)
     refresh_next_durations(st, a.job, a.next_dur, a.dur_job, (int)blockIdx.x * 32 + (int)threadIdx.x);
   if (a.zero_words != nullptr && blockIdx.x == gridDim.x - 1)
     for (int i = threadIdx.x; i < a.n_zero; i += blockDim.x) a.zero_words[i] = 0;
