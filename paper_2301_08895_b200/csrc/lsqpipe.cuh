@@ -45,6 +45,14 @@ inline size_t smem_bytes(int d, int stages) {
          2 * MAX_STAGES * 8 + 64;
 }
 
+// (d0, d1) += (a0, a1) * (b0, b1): two binary32 FMAs in one instruction (each lane rounds like a
+// scalar fma); the consumers are bound by instruction issue, so this halves their FMA count.
+__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%0, %1};\n\t"
+      "fma.rn.f32x2 rc, ra, rb, rc;\n\tmov.b64 {%0, %1}, rc;\n\t}"
+      : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
 __device__ __forceinline__ void bulk_row(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(tc::smem_u32(dst)), "l"(src), "r"(bytes), "r"(tc::smem_u32(bar)) : "memory");
@@ -169,8 +177,7 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float2 f = __bfloat1622float2(xh[j]);
-            s0 = fmaf(f.x, wf[2 * j], s0);
-            s1 = fmaf(f.y, wf[2 * j + 1], s1);
+            ffma2(s0, s1, f.x, f.y, wf[2 * j], wf[2 * j + 1]);
           }
           pd[r] = s0 + s1;
         }
@@ -219,8 +226,7 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float2 f = __bfloat1622float2(xh[j]);
-            acc[2 * j] = fmaf(res[r], f.x, acc[2 * j]);
-            acc[2 * j + 1] = fmaf(res[r], f.y, acc[2 * j + 1]);
+            ffma2(acc[2 * j], acc[2 * j + 1], f.x, f.y, res[r], res[r]);
           }
         }
         buf ^= 1;
