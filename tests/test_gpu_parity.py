@@ -389,6 +389,26 @@ def test_lsq_bulk_copy_pipeline_and_plain_load_kernels(d, W, B, K0, S):
         assert np.allclose(la, lb, rtol=1e-4, atol=1e-6)
 
 
+@pytest.mark.parametrize("d,W,B,K0,S", [(8, 300, 1, 40, 3), (40, 280, 7, 280, 0), (4096, 260, 9, 20, 5),
+                                         (1032, 1024, 33, 128, 2), (4088, 257, 16, 257, 1)])
+def test_lsq_bulk_copy_pipeline_edge_shapes(d, W, B, K0, S):
+    """Ragged row groups (B not a multiple of 8, B = 1), one 16-byte vector per row, the widest row,
+    more workers than SMs, K = N from the first round."""
+    cfg = _small_cfg(inputs.LSQ, (d, 1), inputs.BF16, W, B, K0, S, EXP, n=12000, lr=0.001)
+    X, y, w0 = _problem(cfg)
+    compare_with_oracle(cfg, X, y, w0, 12, TOL_BF16, forced=True)
+
+
+@pytest.mark.parametrize("dims,B", [((64, 128, 2), 24), ((200, 256, 16), 40), ((96, 1024, 10), 16),
+                                    ((72, 128, 128, 3), 64)])
+def test_output_layer_tensor_core_kernel_shapes(dims, B):
+    """The mma.sync output-layer kernel at each supported width of the last hidden layer, with 2, 3,
+    10 and 16 classes (class rows are padded to 16 inside the kernel)."""
+    cfg = _small_cfg(inputs.MLP, dims, inputs.BF16, 13, B, 3, 5, PARETO)
+    X, y, w0 = _problem(cfg)
+    compare_with_oracle(cfg, X, y, w0, 30, TOL_BF16, forced=True, loss_tol=5e-2)
+
+
 # Small least-squares problems run all enqueued rounds inside one persistent kernel; the flag
 # keeps the one-launch-per-step path in use, and both must agree with the oracle.
 @pytest.mark.parametrize("flags", [0, gpu.FLAG_NO_PERSISTENT])
