@@ -39,6 +39,13 @@ inline size_t smem_bytes(int n_par, int B, int C) {
   return sizeof(float) * ((size_t)2 * n_par + (size_t)B * C + B + 64) + sizeof(int) * (size_t)B;
 }
 
+// (d0, d1) += x * (w0, w1) as one packed binary32 FMA (each lane rounds like a scalar fma).
+__device__ __forceinline__ void ffma2_bcast(float& d0, float& d1, float x, const float2 w) {
+  asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %2};\n\tmov.b64 rb, {%3, %4};\n\tmov.b64 rc, {%0, %1};\n\t"
+      "fma.rn.f32x2 rc, ra, rb, rc;\n\tmov.b64 {%0, %1}, rc;\n\t}"
+      : "+f"(d0), "+f"(d1) : "f"(x), "f"(w.x), "f"(w.y));
+}
+
 template <typename T>
 __global__ void __launch_bounds__(NT_MAX) local_sgd_kernel(Args a) {
   grid_dependency_sync();
@@ -58,6 +65,7 @@ __global__ void __launch_bounds__(NT_MAX) local_sgd_kernel(Args a) {
   int* sidx = reinterpret_cast<int*>(red + 64);          // [B] sample indices of the step
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int NT = (int)blockDim.x;
+  const bool even_c = (C & 1) == 0;
   const int wn = a.sel[i], jb = a.job[wn];
   const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
   const T* w0 = (const T*)a.ring + (size_t)slot * a.slot_stride;
@@ -88,9 +96,16 @@ __global__ void __launch_bounds__(NT_MAX) local_sgd_kernel(Args a) {
 #pragma unroll 8
       for (int m = lane; m < in; m += 32) {
         const float xv = ldf(x, m);
+        if (even_c) {                 // class pairs: one 8-byte shared-memory read and one packed FMA per pair
+          const float2* wp = reinterpret_cast<const float2*>(wl + m * C);
 #pragma unroll
-        for (int c = 0; c < MAX_C; ++c)
-          if (c < C) acc[c] = fmaf(xv, wl[m * C + c], acc[c]);
+          for (int c = 0; c < MAX_C; c += 2)
+            if (c < C) ffma2_bcast(acc[c], acc[c + 1], xv, wp[c >> 1]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < MAX_C; ++c)
+            if (c < C) acc[c] = fmaf(xv, wl[m * C + c], acc[c]);
+        }
       }
 #pragma unroll
       for (int c = 0; c < MAX_C; ++c)
@@ -138,9 +153,16 @@ __global__ void __launch_bounds__(NT_MAX) local_sgd_kernel(Args a) {
 #pragma unroll 8
       for (int b = 0; b < B; ++b) {
         const float xv = ldf(X, (size_t)sidx[b] * in + m);
+        if (even_c) {
+          const float2* dp = reinterpret_cast<const float2*>(dl + b * C);
 #pragma unroll
-        for (int c = 0; c < MAX_C; ++c)
-          if (c < C) acc[c] = fmaf(xv, dl[b * C + c], acc[c]);
+          for (int c = 0; c < MAX_C; c += 2)
+            if (c < C) ffma2_bcast(acc[c], acc[c + 1], xv, dp[c >> 1]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < MAX_C; ++c)
+            if (c < C) acc[c] = fmaf(xv, dl[b * C + c], acc[c]);
+        }
       }
 #pragma unroll
       for (int c = 0; c < MAX_C; ++c)
