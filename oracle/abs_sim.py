@@ -5,7 +5,8 @@ t = 0, 1, ... of Algorithm 1 with U = 1 local step:
 
   (With `local_steps` = U > 1 a job is U local minibatch steps, Eq. 2: the worker
   starts from the model it holds, moves its own copy by -eta * (mean minibatch
-  gradient) U times, each step on a fresh minibatch, and uploads the sum of its
+  gradient) U times, each step on a fresh minibatch (in the bf16 configurations
+  each step's gradient is evaluated at the bf16 rounding of that copy), and uploads the sum of its
   U mean gradients, i.e. (w^{.,0} - w^{.,U}) / eta, and the average of its U mean
   minibatch losses (Algorithm 1, last worker line); Eq. 3 is unchanged.)
 
@@ -215,7 +216,9 @@ class ABSOracle:
             yb = self.y[idx]
             if self.kind == models.LSQ:
                 yb = yb.astype(np.float64)
-            loss, grad = models.loss_grad(self.kind, self.dims, w_local, Xb, yb, quant=self.quant)
+            # bf16 configurations compute every step with the 16-bit rounding of the local copy
+            # (the copy itself keeps full precision); at step 0 that is the downloaded model
+            loss, grad = models.loss_grad(self.kind, self.dims, self._stored(w_local), Xb, yb, quant=self.quant)
             loss_sum += loss
             grad_sum += grad
             if u + 1 < self.local_steps:

@@ -1,6 +1,7 @@
 // Local SGD inside a job (Eq. 2 with U > 1): one CTA per selected worker runs the worker's U
 // minibatch steps one after the other on its own copy of the model, which starts at the version the
-// worker holds (its ring slot) and lives in shared memory as fp32.  Step u draws its minibatch from
+// worker holds (its ring slot) and lives in shared memory as fp32 (bf16 configurations compute each
+// step with the bf16 rounding of that copy, as their tensor-core paths must).  Step u draws its minibatch from
 // Philox blocks (n, j, 1, u * ceil(B/4) + b/4).  The upload is the sum over the steps of the
 // per-sample gradient sums, G = (B / eta) (w^{.,0} - w^{.,U}), and the average of the U mean
 // minibatch losses (Algorithm 1, last worker line); Eq. 3 then reads the K uploads like the
@@ -100,11 +101,16 @@ __global__ void __launch_bounds__(NT_MAX) local_sgd_kernel(Args a) {
           const float2* wp = reinterpret_cast<const float2*>(wl + m * C);
 #pragma unroll
           for (int c = 0; c < MAX_C; c += 2)
-            if (c < C) ffma2_bcast(acc[c], acc[c + 1], xv, wp[c >> 1]);
+            if (c < C) {
+              float2 w = wp[c >> 1];
+              w.x = round_store(w.x, (const T*)nullptr);
+              w.y = round_store(w.y, (const T*)nullptr);
+              ffma2_bcast(acc[c], acc[c + 1], xv, w);
+            }
         } else {
 #pragma unroll
           for (int c = 0; c < MAX_C; ++c)
-            if (c < C) acc[c] = fmaf(xv, wl[m * C + c], acc[c]);
+            if (c < C) acc[c] = fmaf(xv, round_store(wl[m * C + c], (const T*)nullptr), acc[c]);
         }
       }
 #pragma unroll
@@ -121,7 +127,7 @@ __global__ void __launch_bounds__(NT_MAX) local_sgd_kernel(Args a) {
         float zmax = -3.0e38f, zy = 0.f;
 #pragma unroll
         for (int c = 0; c < MAX_C; ++c)
-          if (c < C) { acc[c] += wl[n_w + c]; zmax = fmaxf(zmax, acc[c]); if (c == y) zy = acc[c]; }
+          if (c < C) { acc[c] += round_store(wl[n_w + c], (const T*)nullptr); zmax = fmaxf(zmax, acc[c]); if (c == y) zy = acc[c]; }
         float se = 0.f;
 #pragma unroll
         for (int c = 0; c < MAX_C; ++c)
