@@ -103,7 +103,8 @@ extern "C" {
 #define ABS_KC_WGRAD   4  /* weight gradient summed over the selected workers (Eq. 3) */
 #define ABS_KC_OUTPUT  5  /* output layer: forward + loss, its back-propagation and gradient */
 #define ABS_KC_BIAS    6  /* bias gradients */
-#define ABS_KC_LSQ     7  /* least-squares residual + gradient; with local_steps > 1: the workers' local steps */
+#define ABS_KC_LSQ     7  /* least-squares residual + gradient; with local_steps > 1: the workers' local steps
+                             (single-layer models), or their set-up, row layouts and local updates (networks) */
 #define ABS_KC_UPDATE  8  /* Eq. 3 step + ring write */
 #define ABS_KC_ROUNDS  9  /* whole rounds (control step + Eq. 2 + Eq. 3) of a small least-squares problem
                              in one persistent kernel; one launch per abs_enqueue_rounds call */
@@ -126,7 +127,12 @@ typedef struct {
   int local_steps;          /* U of Eq. 2, 1..1024.  U > 1 (local SGD inside a job: the upload is the sum of
                                the U minibatch-gradient sums along the worker's own trajectory, the loss the
                                average of its U minibatch losses) is implemented for ABS_LSQ and ABS_SOFTMAX
-                               with <= 16 classes, <= 12288 parameters and batch x classes <= 8192 */
+                               with <= 16 classes, <= 12288 parameters and batch x classes <= 8192 (the worker's
+                               copy lives in shared memory), and for multi-layer ABS_MLP in ABS_BF16_FP32MASTER
+                               whose hidden layers all take the tensor-core path (widths multiples of 8 and
+                               >= 64, last hidden width 128/256/512/1024, <= 16 classes; the selected workers'
+                               copies live in the workspace: 14 bytes per parameter and worker); in the bf16
+                               configurations each step is evaluated at the bf16 rounding of the fp32 copy */
   int k_mode;               /* ABS_K_* */
   int bound_mode;           /* ABS_BOUND_* */
   int bound_offset;         /* the constant a of Eq. 4 when bound_mode = ABS_BOUND_OFFSET (else ignored);

@@ -16,6 +16,7 @@
 #include "outlayer.cuh"
 #include "lsqpipe.cuh"
 #include "local.cuh"
+#include "localnet.cuh"
 #include "persist.cuh"
 
 using namespace absb;
@@ -80,6 +81,12 @@ struct Layout {
   size_t tr_K, tr_R, tr_theta, tr_T, tr_loss, tr_comm, tr_sel_off, tr_rst_off;
   size_t tr_sel_id, tr_sel_tau, tr_sel_loss, tr_rst_id;
   size_t data_X, data_y;
+  // U > 1 on a multi-layer network: the selected workers' own model copies and uploads
+  bool local_net = false;
+  int RBp = 0;                          // rows reserved per worker in a local step's row layout
+  size_t priv16 = 0, priv32 = 0, gsum = 0, loss_acc = 0;
+  size_t gring = 0;                     // the models the gradient kernels read: the ring, or the private copies
+  int gslots = 0;
   size_t total = 0;
 };
 
@@ -143,6 +150,11 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   L->RB = lsq ? m->batch : (L->any_tc ? (L->two_cta ? 256 : 128) : 64);
   const int groups = (W < S + 1) ? W : S + 1;
   L->rows_cap = round_up(W * m->batch, L->RB) + groups * L->RB;
+  L->local_net = !lsq && m->n_layers > 1 && m->local_steps > 1;
+  if (L->local_net) {
+    L->RBp = round_up(m->batch, L->RB);
+    L->rows_cap = std::max(L->rows_cap, W * L->RBp);
+  }
   L->n_tiles_cap = L->rows_cap / L->RB;
   if (lsq) {
     L->P = 0;
@@ -179,6 +191,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       if (L->cg_fwd[l] != 1 || L->cg_fwd[l + 1] != 1 || L->bn_fwd[l] != L->bn_fwd[l + 1]) continue;
       if (l == 0 && L->gather_tma) continue;
       if (l > 0 && L->pair_fwd[l - 1]) continue;
+      if (L->local_net) continue;
       L->pair_fwd[l] = true;
     }
     // A short weight gradient (fewer tiles than SMs at the back-propagation's tile width) shares
@@ -186,6 +199,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     // separate launches would pay the fixed costs of a launch twice.
     for (int l = 1; l < m->n_layers; ++l) {
       if (L->path[l] != PATH_TC || L->cg_dg[l] != 1 || L->cg_wg[l] != 1 || (m->flags & ABS_FLAG_NO_FUSED_BACKWARD)) continue;
+      if (L->local_net) continue;
       const int in = m->dims[l], out = m->dims[l + 1], bn = L->bn_dg[l];
       if (out < bn) continue;
       const long wg_tiles_min = (long)((in + 127) / 128 + 1) * ((out + bn - 1) / bn);   // at P = 1
@@ -241,6 +255,16 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   L->ring = cv.take(L->esz * L->d_pad * (S + 1));
   if (m->local_steps > 1) L->P = 0;      // Eq. 3 adds one upload per selected worker
   L->G = cv.take(4 * L->d_pad * ((lsq || m->local_steps > 1) ? W : L->P));
+  L->gring = L->ring;
+  L->gslots = S + 1;
+  if (L->local_net) {
+    L->priv16 = cv.take(2 * L->d_pad * W);
+    L->priv32 = cv.take(4 * L->d_pad * W);
+    L->gsum = cv.take(4 * L->d_pad * W);
+    L->loss_acc = cv.take(4 * W);
+    L->gring = L->priv16;
+    L->gslots = W;
+  }
   if (!lsq) {
     const int C = m->dims[m->n_layers];
     L->logits = cv.take(4 * (size_t)L->rows_cap * C);
@@ -480,7 +504,8 @@ int setup_tc(abs_ctx* ctx) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<64, 1>::SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::Cfg<256, 2>::SMEM_BYTES);
   if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaFuncSetAttribute(tc_gemm_kernel)");
-  const char* ring = ctx->at<char>(L.ring);
+  const char* ring = ctx->at<char>(L.gring);
+  const int n_splits = L.P > 0 ? L.P : ctx->W;     // P = 0: one weight-gradient split per selected worker
   if (!make_act_map(&ctx->ones_map, ctx->at<void>(L.ones), 64, L.rows_cap, 64))
     return fail(ABS_ECUDA, "cuTensorMapEncodeTiled failed for the ones matrix");
   ones_init_kernel<<<(L.rows_cap + 255) / 256, 256, 0, ctx->stream>>>(ctx->at<__nv_bfloat16>(L.ones), L.rows_cap);
@@ -494,11 +519,11 @@ int setup_tc(abs_ctx* ctx) {
     const void* delta_out = ctx->at<void>(L.delta[l + 1]);
     const void* wbase = ring + 2 * L.w_off[l];
     bool ok = (from_x || make_act_map(&t.fwd_a, act_in, in, L.rows_cap, 128)) &&
-              make_w_map(&t.fwd_b, wbase, in, out, ctx->S + 1, L.d_pad, 64) &&
+              make_w_map(&t.fwd_b, wbase, in, out, L.gslots, L.d_pad, 64) &&
               (from_x || make_act_map(&t.wg_a, act_in, in, L.rows_cap, 64)) &&
               make_act_map(&t.wg_b, delta_out, out, L.rows_cap, 64) &&
               make_act_map(&t.fwd_out, ctx->at<void>(L.act[l + 1]), out, L.rows_cap, 32) &&
-              make_g_map(&t.wg_out, ctx->at<float>(L.G) + L.w_off[l], in, out, L.P, L.d_pad);
+              make_g_map(&t.wg_out, ctx->at<float>(L.G) + L.w_off[l], in, out, n_splits, L.d_pad);
     if (ok && l == 0 && !L.gather_tma)
       ok = make_act_map(&t.fwd_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 128) &&
            make_act_map(&t.wg_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 64);
@@ -506,7 +531,7 @@ int setup_tc(abs_ctx* ctx) {
       ok = make_act_map(&t.x_rows, ctx->X, in, (int)m.n_samples, 1);
     if (ok && l > 0)
       ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
-           make_w_map(&t.dg_b, wbase, in, out, ctx->S + 1, L.d_pad, L.bn_dg[l] / L.cg_dg[l]) &&
+           make_w_map(&t.dg_b, wbase, in, out, L.gslots, L.d_pad, L.bn_dg[l] / L.cg_dg[l]) &&
            make_act_map(&t.dg_out, ctx->at<void>(L.delta[l]), in, L.rows_cap, 32);
     if (!ok) return fail(ABS_ECUDA, "cuTensorMapEncodeTiled failed for layer %d", l);
   }
@@ -554,11 +579,12 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
   const int row_tiles = L.rows_cap / TM;
   const int row_tiles128 = L.rows_cap / 128;
   const bool gathered = L.path[0] == PATH_TC;     // layer 0 reads the gathered copy act[0]
+  const int n_splits = L.P > 0 ? L.P : ctx->W;    // weight-gradient splits (P = 0: one per selected worker)
   LayerArgs la[ABS_MAX_LAYERS];
   for (int l = 0; l < nl; ++l) {
     LayerArgs& a = la[l];
     a.st = st; a.ri = ri; a.tile_slot = ctx->ctl.tile_slot[par]; a.row_idx = ctx->ctl.row_idx[par];
-    a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad; a.w_off = L.w_off[l];
+    a.ring = ctx->at<void>(L.gring); a.slot_stride = L.d_pad; a.w_off = L.w_off[l];
     a.in = m.dims[l]; a.out = m.dims[l + 1];
     a.gather = (l == 0 && !gathered);
     a.act_in = (l == 0 && !gathered) ? ctx->X : ctx->at<void>((l == 0 && par) ? L.act0b : L.act[l]);
@@ -571,7 +597,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     tc::Params p;
     memset(&p, 0, sizeof p);
     p.st = st; p.ri = ri; p.tile_slot = ctx->ctl.tile_slot[par]; p.mode = mode; p.P = L.P;
-    p.ring = ctx->at<__nv_bfloat16>(L.ring); p.slot_stride = L.d_pad;
+    p.ring = ctx->at<__nv_bfloat16>(L.gring); p.slot_stride = L.d_pad;
     p.b_off = L.w_off[l] + (size_t)m.dims[l] * m.dims[l + 1];
     if (l == 0 && L.gather_tma && mode != tc::DGRAD) { p.gather_a = 1; p.row_idx = ctx->ctl.row_idx[par]; }
     return p;
@@ -579,12 +605,12 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
   auto narrow_args = [&](int l) {
     NarrowArgs a;
     a.st = st; a.ri = ri; a.tile_slot = ctx->ctl.tile_slot[par]; a.row_idx = ctx->ctl.row_idx[par]; a.labels = (const int*)ctx->y;
-    a.ring = ctx->at<void>(L.ring); a.slot_stride = L.d_pad; a.w_off = L.w_off[l];
+    a.ring = ctx->at<void>(L.gring); a.slot_stride = L.d_pad; a.w_off = L.w_off[l];
     a.in = m.dims[l]; a.C = m.dims[l + 1];
     a.gather = la[l].gather; a.act_in = la[l].act_in;
     a.delta_out = ctx->at<void>(L.delta[l + 1]);
     a.delta_in = (l == 0) ? nullptr : ctx->at<void>(L.delta[l]);
-    a.row_loss = ctx->ctl.row_loss; a.G = ctx->at<float>(L.G); a.P = L.P;
+    a.row_loss = L.local_net ? ctx->at<float>(L.row_loss) : ctx->ctl.row_loss; a.G = ctx->at<float>(L.G); a.P = L.P;
     return a;
   };
   if (phase == PH_GATHER) {
@@ -646,7 +672,11 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
         } else {
           launch_ex(ctx, ABS_KC_OUTPUT, narrow_fused_kernel<T>, dim3(L.rows_cap / R), dim3(256), sm, a, part, R, has_dgrad);
         }
-        launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, R);
+        if (L.local_net)
+          launch_ex(ctx, ABS_KC_OUTPUT, lnet::chunk_reduce_worker_kernel, dim3((len + 31) / 32, ctx->W), dim3(256), 0, st, ri, part, len,
+                    dstw, L.d_pad, R, L.RBp);
+        else
+          launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, R);
       } else if (a.in % 8 == 0) {
         const size_t sm = sizeof(T) * (size_t)a.in * a.C + sizeof(float) * a.C;
         launch_ex(ctx, ABS_KC_OUTPUT, narrow_fwd_loss_v8_kernel<T>, dim3(L.rows_cap / NARROW_ROWS), dim3(256), sm, a);
@@ -686,7 +716,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
         // the layer's delta back-propagation shares the weight gradient's launch (same tile width)
         const TcProblem second = {&ctx->tcl[l].dg_a, &ctx->tcl[l].dg_b, &ctx->tcl[l].dg_out, &pd, dg_tiles};
         launch_tc_bn(ctx, bnd, 1, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
-                     ((la[l].in + 127) / 128 + 1) * ((la[l].out + bnd - 1) / bnd) * L.P, &second);
+                     ((la[l].in + 127) / 128 + 1) * ((la[l].out + bnd - 1) / bnd) * n_splits, &second);
         continue;
       }
       if (l > 0)
@@ -694,7 +724,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       const int bn = L.bn_wg[l];
       const int tmw = 128 * L.cg_wg[l];
       launch_tc_bn(ctx, bn, L.cg_wg[l], ABS_KC_WGRAD, (l == 0 && L.gather_tma) ? ctx->tcl[l].x_rows : (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
-                   ((la[l].in + tmw - 1) / tmw + 1) * ((la[l].out + bn - 1) / bn) * L.P);
+                   ((la[l].in + tmw - 1) / tmw + 1) * ((la[l].out + bn - 1) / bn) * n_splits);
     } else if (L.path[l] == PATH_NARROW && L.fused_R) {
       // forward, loss, delta of the layer below and the gradient were all done by the fused kernel
     } else if (L.path[l] == PATH_NARROW) {
@@ -743,7 +773,7 @@ void enqueue_update(abs_ctx* ctx, int par) {
   }
   UpdateArgs u;
   u.st = ctx->at<DevState>(L.st); u.ri = ri; u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
-  u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
+  u.G = ctx->at<float>(L.local_net ? L.gsum : L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
   // for the latency-bound models (always one stream) the Eq. 3 kernel also prepares the next job
   // durations (its first warps); tensor-core networks keep a small kernel of their own for that
   const bool look = !L.any_tc;
@@ -803,11 +833,20 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     return fail(ABS_EINVAL, "local_steps %d outside [1, 1024]", model->local_steps);
   if (model->local_steps > 1) {
     // U > 1: the worker's local model lives in shared memory; single-layer models only
-    if (model->kind == ABS_MLP)
-      return fail(ABS_EUNSUPPORTED, "local_steps = %d: U > 1 is implemented for least squares and soft-max regression only", model->local_steps);
+    if (model->kind == ABS_MLP && model->n_layers > 1) {
+      // multi-layer networks: private model copies in HBM, every step through the tensor-core kernels
+      Layout Lc;
+      make_layout(model, W, staleness_bound, &Lc);
+      bool ok = Lc.out_mma && !Lc.gather_tma && !Lc.two_cta;
+      for (int l = 0; l + 1 < model->n_layers; ++l) ok = ok && Lc.path[l] == PATH_TC;
+      if (!ok)
+        return fail(ABS_EUNSUPPORTED, "local_steps = %d on a multi-layer network needs the bf16 tensor-core path: hidden widths that are "
+                    "multiples of 8 and at least 64, a last hidden width of 128, 256, 512 or 1024 and at most 16 classes", model->local_steps);
+    }
+    const bool single = model->kind != ABS_MLP || model->n_layers == 1;
     const int C = model->kind == ABS_LSQ ? 1 : model->dims[1];
     const size_t n_par = model->kind == ABS_LSQ ? (size_t)model->dims[0] : (size_t)model->dims[0] * C + C;
-    if (C > local::MAX_C || n_par > (size_t)local::MAX_PARAMS || (size_t)model->batch * C > (size_t)local::MAX_BC)
+    if (single && (C > local::MAX_C || n_par > (size_t)local::MAX_PARAMS || (size_t)model->batch * C > (size_t)local::MAX_BC))
       return fail(ABS_EUNSUPPORTED, "local_steps > 1 needs at most %d classes, %d parameters and batch x classes <= %d",
                   local::MAX_C, local::MAX_PARAMS, local::MAX_BC);
   }
@@ -940,7 +979,7 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
       ef = cudaFuncSetAttribute(narrow_fused_cc_kernel<__nv_bfloat16, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (ef != cudaSuccess) return bail(cuda_fail(nullptr, ef, "cudaFuncSetAttribute(narrow_fused_kernel)"));
   }
-  if (model->local_steps > 1) {
+  if (model->local_steps > 1 && !L.local_net) {
     const int C = model->kind == ABS_LSQ ? 1 : model->dims[1];
     const int n_par = model->kind == ABS_LSQ ? model->dims[0] : model->dims[0] * C + C;
     const int sm = (int)local::smem_bytes(n_par, model->batch, C);
@@ -980,7 +1019,7 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   if (rc != ABS_OK) return bail(rc);
   // worth it only when a round has a long backward pass to hide behind (tensor-core networks);
   // for the latency-bound models the cross-stream events cost more than they hide
-  if (!(model->flags & ABS_FLAG_NO_OVERLAP) && L.any_tc) {
+  if (!(model->flags & ABS_FLAG_NO_OVERLAP) && L.any_tc && !L.local_net) {
     cudaError_t es = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
     if (es == cudaSuccess) es = cudaEventCreateWithFlags(&ctx->ev_loss, cudaEventDisableTiming);
     if (es == cudaSuccess) es = cudaEventCreateWithFlags(&ctx->ev_ctl, cudaEventDisableTiming);
@@ -1041,6 +1080,37 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
       q.sel = ctx->ctl.sel[par]; q.sel_tau = ctx->ctl.sel_tau[par];
       if (f32) launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<float>, dim3(ctx->W), dim3(nt), sm, q);
       else launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<__nv_bfloat16>, dim3(ctx->W), dim3(nt), sm, q);
+      update(par);
+    }
+    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+  } else if (n > 0 && ctx->L.local_net) {
+    // U > 1 on a multi-layer network: per round, the workers' copies are set up, then every local
+    // step is one pass of the gradient kernels over the private copies followed by the local updates
+    const Layout& L = ctx->L;
+    lnet::Args q;
+    q.st = ctx->at<DevState>(L.st);
+    q.job = ctx->ctl.job;
+    q.ring = ctx->at<__nv_bfloat16>(L.ring);
+    q.priv16 = ctx->at<__nv_bfloat16>(L.priv16); q.priv32 = ctx->at<float>(L.priv32); q.gsum = ctx->at<float>(L.gsum);
+    q.G = ctx->at<float>(L.G); q.row_loss = ctx->at<float>(L.row_loss);
+    q.loss_acc = ctx->at<float>(L.loss_acc); q.loss = ctx->ctl.loss;
+    q.d_pad = L.d_pad; q.RBp = L.RBp; q.U = ctx->m.local_steps; q.lr = ctx->m.lr;
+    const int bx = (int)std::max<size_t>(1, std::min<size_t>((L.d_pad / 4 + 1023) / 1024, 64));
+    for (int r = 0; r < n; ++r) {
+      const int t = ctx->rounds_enqueued + r, par = t & 1;
+      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
+      launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
+      q.ri = ctx->at<RoundInfo>(L.ri) + par;
+      q.sel = ctx->ctl.sel[par]; q.sel_tau = ctx->ctl.sel_tau[par];
+      q.row_idx = ctx->ctl.row_idx[par]; q.tile_slot = ctx->ctl.tile_slot[par];
+      launch_ex(ctx, ABS_KC_LSQ, lnet::local_begin_kernel, dim3(bx, ctx->W), dim3(256), 0, q);
+      for (int u = 0; u < q.U; ++u) {
+        launch_ex(ctx, ABS_KC_LSQ, lnet::local_layout_kernel, dim3(ctx->W), dim3(128), 0, q, u);
+        gradient(par, PH_GATHER);
+        gradient(par, PH_FORWARD);
+        gradient(par, PH_BACKWARD);
+        launch_ex(ctx, ABS_KC_LSQ, lnet::local_step_kernel, dim3(bx, ctx->W), dim3(256), 0, q, u == q.U - 1 ? 1 : 0);
+      }
       update(par);
     }
     launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);

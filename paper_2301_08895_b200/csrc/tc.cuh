@@ -257,8 +257,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     // gradient (row `in` of the [in + 1][out] gradient block) on the tensor cores for free
     r.n_mt_w = (q.M_total - 1 + TM_ROWS - 1) / TM_ROWS;
     r.n_mt = (q.mode == WGRAD) ? r.n_mt_w + 1 : n_row_tiles;
-    r.n_tiles = (q.mode == WGRAD) ? r.n_mt * r.n_ct * q.P : n_row_tiles * r.n_ct;
-    r.chunk = (q.mode == WGRAD) ? round_up((n_rows + q.P - 1) / q.P, BK) : 0;
+    const int n_splits = q.P > 0 ? q.P : ri->K;      // P = 0: one split per selected worker (its own rows)
+    r.n_tiles = (q.mode == WGRAD) ? r.n_mt * r.n_ct * n_splits : n_row_tiles * r.n_ct;
+    r.chunk = (q.mode == WGRAD) ? round_up((n_rows + n_splits - 1) / n_splits, BK) : 0;
     return r;
   };
   const Prob P0 = make_prob(p0);

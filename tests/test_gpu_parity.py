@@ -193,8 +193,22 @@ def test_local_sgd_steps(kind, dims, dtype, W, B, U, forced):
     assert rows[-1]["loss_mean"] < rows[0]["loss_mean"]
 
 
-def test_local_sgd_steps_rejected_for_multi_layer_networks():
-    cfg = _small_cfg(inputs.MLP, (64, 128, 10), inputs.BF16, 8, 16, 3, 5, EXP)
+@pytest.mark.parametrize("dims,W,B,U,K0,S", [
+    ((64, 128, 10), 8, 16, 4, 3, 5),             # one tensor-core layer; a worker's rows are 16 of a 128-row tile
+    ((72, 136, 256, 10), 12, 48, 3, 4, 6),       # two tensor-core layers, ragged widths
+    ((64, 64, 128, 7), 5, 130, 2, 2, 3),         # two row tiles per worker (B > 128), odd class count
+])
+def test_local_sgd_steps_multi_layer_network(dims, W, B, U, K0, S):
+    """Eq. 2 with U > 1 on a multi-layer bf16 network: every selected worker owns a copy of the
+    model in HBM; a local step of all of them is one pass of the grouped tensor-core kernels."""
+    cfg = _small_cfg(inputs.MLP, dims, inputs.BF16, W, B, K0, S, GAMMA3, lr=0.05)
+    X, y, w0 = _problem(cfg)
+    rows, orows, err, o = compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2, local_steps=U)
+    assert rows[-1]["loss_mean"] < rows[0]["loss_mean"]
+
+
+def test_local_sgd_steps_rejected_for_fp32_multi_layer_networks():
+    cfg = _small_cfg(inputs.MLP, (64, 128, 10), inputs.FP32, 8, 16, 3, 5, EXP)
     X, y, w0 = _problem(cfg)
     Xd, yd = to_device(cfg, X, y)
     with pytest.raises(gpu.AbsError) as e:
