@@ -30,7 +30,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) per launch at K = N on configuration 4, from ncu captures of the GEMM and the
 # Eq. 3 kernel (summaries under profiles/); each figure is valid only for the kernel source it was taken
 # from (first 16 hex digits of the file's sha256).
-TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.0e6, "file": "tc.cuh", "sha256_16": "a057a9df0c4454e7"},
+TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.3e6, "file": "tc.cuh", "sha256_16": "cd82f760f9fc1bad"},
            "update": {"config": 4, "bytes_per_launch": 76.6e6, "file": "simt.cuh", "sha256_16": "11a0b5ded60e0244"}}
 METRIC = "worker_gradients_per_sec"
 UNIT = "worker-gradients/s"
