@@ -128,11 +128,10 @@ typedef struct {
                                the U minibatch-gradient sums along the worker's own trajectory, the loss the
                                average of its U minibatch losses) is implemented for ABS_LSQ and ABS_SOFTMAX
                                with <= 16 classes, <= 12288 parameters and batch x classes <= 8192 (the worker's
-                               copy lives in shared memory), and for multi-layer ABS_MLP in ABS_BF16_FP32MASTER
-                               whose hidden layers all take the tensor-core path (widths multiples of 8 and
-                               >= 64, last hidden width 128/256/512/1024, <= 16 classes; the selected workers'
-                               copies live in the workspace: 14 bytes per parameter and worker); in the bf16
-                               configurations each step is evaluated at the bf16 rounding of the fp32 copy */
+                               copy lives in shared memory), and for multi-layer ABS_MLP (the selected workers'
+                               copies live in the workspace: 12 bytes per parameter and worker, 14 in bf16;
+                               not with ABS_FLAG_TMA_GATHER / ABS_FLAG_TWO_CTA); in the bf16 configurations
+                               each step is evaluated at the bf16 rounding of the fp32 copy */
   int k_mode;               /* ABS_K_* */
   int bound_mode;           /* ABS_BOUND_* */
   int bound_offset;         /* the constant a of Eq. 4 when bound_mode = ABS_BOUND_OFFSET (else ignored);

@@ -258,8 +258,8 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   L->gring = L->ring;
   L->gslots = S + 1;
   if (L->local_net) {
-    L->priv16 = cv.take(2 * L->d_pad * W);
     L->priv32 = cv.take(4 * L->d_pad * W);
+    L->priv16 = L->esz == 2 ? cv.take(2 * L->d_pad * W) : L->priv32;     // fp32: the local models are the operands
     L->gsum = cv.take(4 * L->d_pad * W);
     L->loss_acc = cv.take(4 * W);
     L->gring = L->priv16;
@@ -693,7 +693,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
         LossArgs lo;
         lo.st = st; lo.ri = ri; lo.row_idx = ctx->ctl.row_idx[par]; lo.labels = (const int*)ctx->y;
         lo.logits = ctx->at<float>(L.logits); lo.delta = ctx->at<void>(L.delta[nl]);
-        lo.row_loss = ctx->ctl.row_loss; lo.C = m.dims[nl];
+        lo.row_loss = L.local_net ? ctx->at<float>(L.row_loss) : ctx->ctl.row_loss; lo.C = m.dims[nl];
         launch_ex(ctx, ABS_KC_OUTPUT, net_loss_kernel<T>, dim3((L.rows_cap + 255) / 256), dim3(256), 0, lo);
       }
     }
@@ -743,14 +743,18 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       float* dstw = ctx->at<float>(L.G) + L.w_off[l];
       const int len = (a.in + 1) * a.C;
       launch_ex(ctx, ABS_KC_OUTPUT, narrow_wgrad_chunk_kernel<T>, dim3(L.rows_cap / 64), dim3(256), 0, a, part);
-      launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, 64);
+      if (L.local_net)
+        launch_ex(ctx, ABS_KC_OUTPUT, lnet::chunk_reduce_worker_kernel, dim3((len + 31) / 32, ctx->W), dim3(256), 0, st, ri, part, len,
+                  dstw, L.d_pad, 64, L.RBp);
+      else
+        launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, 64);
     } else {
       const bool last = l == nl - 1;
       if (l > 0) {
         dim3 grid((la[l].in + TN - 1) / TN, row_tiles);
         launch_ex(ctx, last ? ABS_KC_OUTPUT : ABS_KC_DGRAD, simt_dgrad_kernel<T>, dim3(grid), dim3(256), 0, la[l]);
       }
-      dim3 gridw((la[l].out + TN - 1) / TN, (la[l].in + 1 + TM - 1) / TM, L.P);
+      dim3 gridw((la[l].out + TN - 1) / TN, (la[l].in + 1 + TM - 1) / TM, n_splits);
       launch_ex(ctx, last ? ABS_KC_OUTPUT : ABS_KC_WGRAD, simt_wgrad_kernel<T>, dim3(gridw), dim3(256), 0, la[l]);
     }
   }
@@ -837,11 +841,8 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
       // multi-layer networks: private model copies in HBM, every step through the tensor-core kernels
       Layout Lc;
       make_layout(model, W, staleness_bound, &Lc);
-      bool ok = Lc.out_mma && !Lc.gather_tma && !Lc.two_cta;
-      for (int l = 0; l + 1 < model->n_layers; ++l) ok = ok && Lc.path[l] == PATH_TC;
-      if (!ok)
-        return fail(ABS_EUNSUPPORTED, "local_steps = %d on a multi-layer network needs the bf16 tensor-core path: hidden widths that are "
-                    "multiples of 8 and at least 64, a last hidden width of 128, 256, 512 or 1024 and at most 16 classes", model->local_steps);
+      if (Lc.gather_tma || Lc.two_cta)
+        return fail(ABS_EUNSUPPORTED, "local_steps = %d on a multi-layer network: not with ABS_FLAG_TMA_GATHER or ABS_FLAG_TWO_CTA", model->local_steps);
     }
     const bool single = model->kind != ABS_MLP || model->n_layers == 1;
     const int C = model->kind == ABS_LSQ ? 1 : model->dims[1];
@@ -1090,7 +1091,7 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     lnet::Args q;
     q.st = ctx->at<DevState>(L.st);
     q.job = ctx->ctl.job;
-    q.ring = ctx->at<__nv_bfloat16>(L.ring);
+    q.ring = ctx->at<void>(L.ring);
     q.priv16 = ctx->at<__nv_bfloat16>(L.priv16); q.priv32 = ctx->at<float>(L.priv32); q.gsum = ctx->at<float>(L.gsum);
     q.G = ctx->at<float>(L.G); q.row_loss = ctx->at<float>(L.row_loss);
     q.loss_acc = ctx->at<float>(L.loss_acc); q.loss = ctx->ctl.loss;
@@ -1099,17 +1100,20 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
       launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
-      launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
+      if (L.any_tc)
+        launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
       q.ri = ctx->at<RoundInfo>(L.ri) + par;
       q.sel = ctx->ctl.sel[par]; q.sel_tau = ctx->ctl.sel_tau[par];
       q.row_idx = ctx->ctl.row_idx[par]; q.tile_slot = ctx->ctl.tile_slot[par];
-      launch_ex(ctx, ABS_KC_LSQ, lnet::local_begin_kernel, dim3(bx, ctx->W), dim3(256), 0, q);
+      if (f32) launch_ex(ctx, ABS_KC_LSQ, lnet::local_begin_kernel<float>, dim3(bx, ctx->W), dim3(256), 0, q);
+      else launch_ex(ctx, ABS_KC_LSQ, lnet::local_begin_kernel<__nv_bfloat16>, dim3(bx, ctx->W), dim3(256), 0, q);
       for (int u = 0; u < q.U; ++u) {
         launch_ex(ctx, ABS_KC_LSQ, lnet::local_layout_kernel, dim3(ctx->W), dim3(128), 0, q, u);
         gradient(par, PH_GATHER);
         gradient(par, PH_FORWARD);
         gradient(par, PH_BACKWARD);
-        launch_ex(ctx, ABS_KC_LSQ, lnet::local_step_kernel, dim3(bx, ctx->W), dim3(256), 0, q, u == q.U - 1 ? 1 : 0);
+        if (f32) launch_ex(ctx, ABS_KC_LSQ, lnet::local_step_kernel<float>, dim3(bx, ctx->W), dim3(256), 0, q, u == q.U - 1 ? 1 : 0);
+        else launch_ex(ctx, ABS_KC_LSQ, lnet::local_step_kernel<__nv_bfloat16>, dim3(bx, ctx->W), dim3(256), 0, q, u == q.U - 1 ? 1 : 0);
       }
       update(par);
     }

@@ -1,9 +1,10 @@
-// Local SGD inside a job (Eq. 2 with U > 1) for multi-layer networks on the tensor cores.
+// Local SGD inside a job (Eq. 2 with U > 1) for multi-layer networks.
 // After its first local step every selected worker computes with weights of its own, so the
-// workers' copies live in HBM: a bf16 copy (the GEMM operand), an fp32 copy (the local model) and
-// the fp32 sum of the steps' gradient sums (the upload), each [W][d_pad] and indexed by the
-// worker's position in the round's selection.  One local step of all selected workers is one pass of
-// the grouped forward / backward kernels in which
+// workers' copies live in HBM: an fp32 copy (the local model), for the bf16 configurations a bf16
+// copy of it (the operand the gradient kernels read), and the fp32 sum of the steps' gradient sums
+// (the upload), each [W][d_pad] and indexed by the worker's position in the round's selection.
+// One local step of all selected workers is one pass of the grouped forward / backward kernels
+// (tensor-core or FP32-FMA, as for U = 1) in which
 //   - the rows of worker i are rows [i * RBp, i * RBp + B) (RBp = B rounded up to the row-tile
 //     height; the rest is padding with sample index -1),
 //   - the "model version" of a row tile is the worker's own copy (slot i of the private store), and
@@ -22,8 +23,8 @@ struct Args {
   RoundInfo* ri;
   const int* sel; const int* job; const int* sel_tau;
   int* row_idx; int* tile_slot;        // the round's row layout, rewritten for every local step
-  const __nv_bfloat16* ring;           // [S+1][d_pad] model versions
-  __nv_bfloat16* priv16;               // [W][d_pad] operand copies of the local models
+  const void* ring;                    // [S+1][d_pad] model versions, storage type
+  __nv_bfloat16* priv16;               // [W][d_pad] bf16 operand copies of the local models (bf16 configurations)
   float* priv32;                       // [W][d_pad] local models
   float* gsum;                         // [W][d_pad] uploads: sum over the steps of the gradient sums
   const float* G;                      // [W][d_pad] gradient sums of the current step, per worker
@@ -37,6 +38,7 @@ struct Args {
 };
 
 // Start of a job's local steps: the worker's copies are the model version it holds.
+template <typename T>
 __global__ void __launch_bounds__(256) local_begin_kernel(Args a) {
   grid_dependency_sync();
   const DevState* st = a.st;
@@ -45,18 +47,22 @@ __global__ void __launch_bounds__(256) local_begin_kernel(Args a) {
   const int i = blockIdx.y;
   if (i >= ri->K) return;
   const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
-  const uint2* src = reinterpret_cast<const uint2*>(a.ring + (size_t)slot * a.d_pad);
+  const T* ring_slot = (const T*)a.ring + (size_t)slot * a.d_pad;
   uint2* d16 = reinterpret_cast<uint2*>(a.priv16 + (size_t)i * a.d_pad);
   float4* d32 = reinterpret_cast<float4*>(a.priv32 + (size_t)i * a.d_pad);
   float4* gs = reinterpret_cast<float4*>(a.gsum + (size_t)i * a.d_pad);
   const size_t n4 = a.d_pad / 4;
   for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < n4; v += (size_t)gridDim.x * blockDim.x) {
-    const uint2 pk = src[v];
-    d16[v] = pk;
-    const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&pk.x);
-    const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&pk.y);
-    const float2 f0 = __bfloat1622float2(lo), f1 = __bfloat1622float2(hi);
-    d32[v] = make_float4(f0.x, f0.y, f1.x, f1.y);
+    if (sizeof(T) == 4) {
+      d32[v] = reinterpret_cast<const float4*>(ring_slot)[v];
+    } else {
+      const uint2 pk = reinterpret_cast<const uint2*>(ring_slot)[v];
+      d16[v] = pk;
+      const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&pk.x);
+      const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&pk.y);
+      const float2 f0 = __bfloat1622float2(lo), f1 = __bfloat1622float2(hi);
+      d32[v] = make_float4(f0.x, f0.y, f1.x, f1.y);
+    }
     gs[v] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) a.loss_acc[i] = 0.f;
@@ -120,8 +126,10 @@ __global__ void __launch_bounds__(256) chunk_reduce_worker_kernel(const DevState
 }
 
 // The workers' local updates after step u (Eq. 2): w_i -= eta / B * G_i, upload += G_i, new
-// operand copy; block (0, i) also adds the step's mean loss and, after the last step, writes the
-// uploaded loss (the average of the U mean minibatch losses; Algorithm 1, last worker line).
+// operand copy (bf16 configurations); block (0, i) also adds the step's mean loss and, after the
+// last step, writes the uploaded loss (the average of the U mean minibatch losses; Algorithm 1,
+// last worker line).
+template <typename T>
 __global__ void __launch_bounds__(256) local_step_kernel(Args a, int last) {
   grid_dependency_sync();
   __shared__ float red[8];
@@ -146,11 +154,13 @@ __global__ void __launch_bounds__(256) local_step_kernel(Args a, int last) {
     m.x = fmaf(-step, gv.x, m.x); m.y = fmaf(-step, gv.y, m.y);
     m.z = fmaf(-step, gv.z, m.z); m.w = fmaf(-step, gv.w, m.w);
     w32[v] = m;
-    const __nv_bfloat162 lo = __floats2bfloat162_rn(m.x, m.y), hi = __floats2bfloat162_rn(m.z, m.w);
-    uint2 pk;
-    pk.x = *reinterpret_cast<const unsigned*>(&lo);
-    pk.y = *reinterpret_cast<const unsigned*>(&hi);
-    w16[v] = pk;
+    if (sizeof(T) == 2) {
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(m.x, m.y), hi = __floats2bfloat162_rn(m.z, m.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<const unsigned*>(&lo);
+      pk.y = *reinterpret_cast<const unsigned*>(&hi);
+      w16[v] = pk;
+    }
   }
   if (blockIdx.x == 0) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;

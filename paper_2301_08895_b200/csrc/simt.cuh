@@ -164,7 +164,9 @@ __global__ void __launch_bounds__(256) simt_wgrad_kernel(LayerArgs a) {
   if (st->status != ST_OK) return;
   const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN, p = blockIdx.z;
   const int n_rows = ri->n_rows;
-  const int chunk = round_up((n_rows + a.P - 1) / a.P, TK);
+  const int P = a.P > 0 ? a.P : ri->K;        // P = 0: one split per selected worker (its own rows)
+  if (p >= P) return;
+  const int chunk = round_up((n_rows + P - 1) / P, TK);
   const int k_begin = min(n_rows, p * chunk), k_end = min(n_rows, (p + 1) * chunk);
   const T* src = (const T*)a.act_in;
   const T* dl = (const T*)a.delta_out;

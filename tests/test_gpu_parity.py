@@ -207,12 +207,28 @@ def test_local_sgd_steps_multi_layer_network(dims, W, B, U, K0, S):
     assert rows[-1]["loss_mean"] < rows[0]["loss_mean"]
 
 
-def test_local_sgd_steps_rejected_for_fp32_multi_layer_networks():
-    cfg = _small_cfg(inputs.MLP, (64, 128, 10), inputs.FP32, 8, 16, 3, 5, EXP)
+@pytest.mark.parametrize("dims,dtype,W,B,U,K0,S,forced", [
+    ((20, 32, 10), inputs.FP32, 8, 16, 4, 3, 5, False),          # FP32-FMA hidden layer, fused output layer; free running
+    ((33, 50, 17, 5), inputs.FP32, 9, 70, 3, 2, 4, True),        # odd widths (plain output-layer kernels), two row tiles per worker
+    ((24, 40, 24), inputs.FP32, 6, 12, 2, 2, 3, True),           # 24 classes: output layer through the generic tiles
+    ((30, 44, 10), inputs.BF16, 7, 20, 3, 3, 5, True),           # bf16 without tensor-core layers (widths not multiples of 8)
+])
+def test_local_sgd_steps_multi_layer_network_fma_paths(dims, dtype, W, B, U, K0, S, forced):
+    """The per-worker local steps through the FP32-FMA layer kernels: fp32 at the fp32 tolerance."""
+    cfg = _small_cfg(inputs.MLP, dims, dtype, W, B, K0, S, GAMMA3, lr=0.05)
+    X, y, w0 = _problem(cfg)
+    bf16 = dtype == inputs.BF16
+    rows, orows, err, o = compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16 if bf16 else TOL_FP32, forced=forced,
+                                              loss_tol=5e-2 if bf16 else None, local_steps=U)
+    assert rows[-1]["loss_mean"] < rows[0]["loss_mean"]
+
+
+def test_local_sgd_steps_rejected_with_row_gather_by_tma():
+    cfg = _small_cfg(inputs.MLP, (64, 128, 10), inputs.BF16, 8, 16, 3, 5, EXP)
     X, y, w0 = _problem(cfg)
     Xd, yd = to_device(cfg, X, y)
     with pytest.raises(gpu.AbsError) as e:
-        gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=5, local_steps=4)
+        gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=5, local_steps=4, flags=gpu.FLAG_TMA_GATHER)
     assert e.value.code == gpu.EUNSUPPORTED
 
 
