@@ -31,7 +31,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # Eq. 3 kernel (summaries under profiles/); each figure is valid only for the kernel source it was taken
 # from (first 16 hex digits of the file's sha256).
 TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.3e6, "file": "tc.cuh", "sha256_16": "cd82f760f9fc1bad"},
-           "update": {"config": 4, "bytes_per_launch": 76.6e6, "file": "simt.cuh", "sha256_16": "11a0b5ded60e0244"}}
+           "update": {"config": 4, "bytes_per_launch": 75.9e6, "file": "simt.cuh", "sha256_16": "c91b022072db4098"}}
 METRIC = "worker_gradients_per_sec"
 UNIT = "worker-gradients/s"
 
@@ -266,7 +266,7 @@ def main():
         flush.zero_()
         l0 = ctx.launch_count()
         if profile:
-            ctx.profile_start(rounds * 24 + 8)
+            ctx.profile_start(rounds * (24 if U == 1 else 4 + 12 * U) + 8)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record(stream)
@@ -367,8 +367,9 @@ def main():
             # selected worker and step, the step's gradient (4 B/parameter), the upload sum (read + write,
             # 8 B), the fp32 copy (8 B) and the new bf16 operand copy (2 B)
             d_pad = plan.get("d_pad") or sum(cfg.dims[l] * cfg.dims[l + 1] + cfg.dims[l + 1] for l in range(len(cfg.dims) - 1))
-            n_upd = U * rounds
-            bytes_l = 22.0 * d_pad * wg_p / max(1, rounds)        # per local-update launch: 22 B x d x K^t
+            n_rounds_prof = max(1, prof["update"][0])             # rounds the recorded launches cover
+            n_upd = U * n_rounds_prof
+            bytes_l = 22.0 * d_pad * float(np.mean(ks[:n_rounds_prof]))   # per local-update launch: 22 B x d x K^t
             # the class also holds the begin and layout kernels (1 + U launches per round, small)
             out["roofline"] = {"bound": "hbm", "kernel": "local_step_kernel (+ local_begin / local_layout launches)",
                                "launches": n_l, "avg_us": 1e3 * t_l / max(1, n_l),
@@ -419,7 +420,7 @@ def main():
     if n_u:
         # Eq. 3 step: read fp32 master + P fp32 partial sums, write master + storage-type ring slot
         esz = 2 if bf16 else 4
-        P = plan["partials"] if plan["partials"] > 0 else float(np.mean(ks))
+        P = plan["partials"] if plan["partials"] > 0 else float(np.mean(ks[:n_u]))
         bytes_launch = (8 + esz + 4 * P) * d
         ach = bytes_launch / (t_u / n_u * 1e-3) / 1e9
         out["roofline_update"] = {"bound": "hbm", "kernel": "update_kernel", "launches": n_u,
