@@ -213,6 +213,20 @@ int abs_get_params(abs_ctx* ctx, float* dst_host, size_t cap, size_t* d_out);
  * K^t, the arrival-ordered selected workers, each gradient's staleness, the restarted workers. */
 int abs_get_trace(abs_ctx* ctx, int first_round, int n_rounds, abs_trace* out_host);
 
+/* Checkpoint of the simulation between rounds (Algorithm 1's whole state: the global model and the
+ * ring of model versions, every worker's held version, job index and completion tick, K^t, the
+ * threshold, f(w^0), the clock, and the trace so far; the Philox streams are counter-based, so
+ * nothing of the generators needs saving).  abs_state_bytes: size of the image.  abs_save_state:
+ * synchronises the stream and writes the image to dst_host (cap bytes; ABS_ENOSPACE if too small);
+ * *written receives its size.  abs_restore_state: loads an image into a context that abs_init
+ * created with the same model sizes, dtype, W, K0, staleness bound, modes, time distribution,
+ * seed and max_rounds (ABS_EINVAL otherwise, context unchanged); the context then continues with
+ * round `rounds completed in the image`, bit-identically to the context that saved it.  The
+ * dataset, w0 and profiling state are not part of the image.  Host memory is the caller's. */
+int abs_state_bytes(abs_ctx* ctx, size_t* out);
+int abs_save_state(abs_ctx* ctx, void* dst_host, size_t cap, size_t* written);
+int abs_restore_state(abs_ctx* ctx, const void* src_host, size_t bytes);
+
 /* Kernels of ours launched on behalf of this context so far (set-up included). */
 int abs_launch_count(abs_ctx* ctx, long long* launches);
 

@@ -84,6 +84,9 @@ def lib():
         l.abs_rounds_done.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
         l.abs_get_params.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
         l.abs_get_trace.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(Trace)]
+        l.abs_state_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
+        l.abs_save_state.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
+        l.abs_restore_state.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
         l.abs_launch_count.argtypes = [C.c_void_p, C.POINTER(C.c_longlong)]
         l.abs_lsq_gradient.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
                                        C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t,
@@ -205,6 +208,21 @@ class Context:
         _check(lib().abs_get_params(self._ctx, out.ctypes.data, d, C.byref(got)))
         assert got.value == d
         return out
+
+    def save_state(self):
+        """Checkpoint of the run between rounds as a uint8 array (abs_save_state)."""
+        n = C.c_size_t(0)
+        _check(lib().abs_state_bytes(self._ctx, C.byref(n)))
+        out = np.empty(n.value, dtype=np.uint8)
+        got = C.c_size_t(0)
+        _check(lib().abs_save_state(self._ctx, out.ctypes.data, n.value, C.byref(got)))
+        assert got.value == n.value
+        return out
+
+    def restore_state(self, image):
+        """Continue from a checkpoint taken by a context with the same arguments (abs_restore_state)."""
+        image = np.ascontiguousarray(image, dtype=np.uint8)
+        _check(lib().abs_restore_state(self._ctx, image.ctypes.data, image.size))
 
     def get_trace(self, first=0, n=None):
         if n is None:

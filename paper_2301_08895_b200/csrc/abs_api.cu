@@ -1202,6 +1202,96 @@ int abs_get_params(abs_ctx* ctx, float* dst, size_t cap, size_t* d_out) {
   return ABS_OK;
 }
 
+namespace {
+
+// Image of a context between rounds: header, then the two persistent regions of the workspace
+// (control state .. ring, and the trace arrays).
+struct StateHeader {
+  unsigned long long magic;
+  int version, rounds_enqueued;
+  unsigned long long d_pad, esz, block1, block2, max_rounds;
+  DevState st;                       // the saving context's state block (its constants are checked on restore)
+};
+constexpr unsigned long long STATE_MAGIC = 0x3130455441545341ull;   // "ASTATE01"
+
+void state_blocks(const Layout& L, size_t* b1_off, size_t* b1, size_t* b2_off, size_t* b2) {
+  *b1_off = L.st;  *b1 = L.G - L.st;                           // control state, per-worker arrays, layouts, master, ring
+  *b2_off = L.tr_K; *b2 = L.tr_rst_id - L.tr_K;                // trace arrays except the last ...
+}
+
+bool same_constants(const DevState& a, const DevState& b) {
+  return a.W == b.W && a.K0 == b.K0 && a.S == b.S && a.B == b.B && a.RB == b.RB && a.k_mode == b.k_mode &&
+         a.bound_mode == b.bound_mode && a.max_rounds == b.max_rounds && a.bound_offset == b.bound_offset &&
+         a.theta_cap == b.theta_cap && a.literal_eq6 == b.literal_eq6 && a.n_samples == b.n_samples &&
+         a.key0 == b.key0 && a.key1 == b.key1 && a.dist.kind == b.dist.kind && a.dist.shift == b.dist.shift &&
+         a.dist.rate == b.dist.rate && a.dist.scale == b.dist.scale && a.dist.slow_mod == b.dist.slow_mod &&
+         a.dist.slow_rem == b.dist.slow_rem && a.dist.slow_factor == b.dist.slow_factor && a.dist.shape == b.dist.shape;
+}
+
+}  // namespace
+
+int abs_state_bytes(abs_ctx* ctx, size_t* out) {
+  if (!ctx || !out) return fail(ABS_EINVAL, "null argument");
+  size_t o1, b1, o2, b2;
+  state_blocks(ctx->L, &o1, &b1, &o2, &b2);
+  b2 += 4 * (size_t)ctx->m.max_rounds * ctx->W;                // ... plus the last trace array (restarted ids)
+  *out = sizeof(StateHeader) + b1 + b2;
+  return ABS_OK;
+}
+
+int abs_save_state(abs_ctx* ctx, void* dst, size_t cap, size_t* written) {
+  if (!ctx || !dst) return fail(ABS_EINVAL, "null argument");
+  if (ctx->sticky != ABS_OK) return fail(ctx->sticky, "context is in a failed state (%d)", ctx->sticky);
+  size_t total = 0;
+  abs_state_bytes(ctx, &total);
+  if (written) *written = total;
+  if (cap < total) return fail(ABS_ENOSPACE, "destination holds %zu bytes, %zu needed", cap, total);
+  size_t o1, b1, o2, b2;
+  state_blocks(ctx->L, &o1, &b1, &o2, &b2);
+  b2 += 4 * (size_t)ctx->m.max_rounds * ctx->W;
+  StateHeader h;
+  memset(&h, 0, sizeof h);
+  int rc = read_status(ctx, &h.st);                            // synchronises the stream
+  if (rc != ABS_OK) return rc;
+  if (h.st.status != ST_OK) return fail(ABS_ESTATE, "the run has ended (status %d): nothing to continue from", h.st.status);
+  if (h.st.open) return fail(ABS_ESTATE, "a round is open");
+  h.magic = STATE_MAGIC; h.version = 1; h.rounds_enqueued = ctx->rounds_enqueued;
+  h.d_pad = ctx->L.d_pad; h.esz = ctx->L.esz; h.block1 = b1; h.block2 = b2; h.max_rounds = (unsigned long long)ctx->m.max_rounds;
+  char* p = (char*)dst;
+  memcpy(p, &h, sizeof h);
+  CU(cudaMemcpyAsync(p + sizeof h, ctx->ws + o1, b1, cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaMemcpyAsync(p + sizeof h + b1, ctx->ws + o2, b2, cudaMemcpyDeviceToHost, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  return ABS_OK;
+}
+
+int abs_restore_state(abs_ctx* ctx, const void* src, size_t bytes) {
+  if (!ctx || !src) return fail(ABS_EINVAL, "null argument");
+  if (ctx->sticky != ABS_OK) return fail(ctx->sticky, "context is in a failed state (%d)", ctx->sticky);
+  if (bytes < sizeof(StateHeader)) return fail(ABS_EINVAL, "image shorter than its header");
+  StateHeader h;
+  memcpy(&h, src, sizeof h);
+  if (h.magic != STATE_MAGIC || h.version != 1) return fail(ABS_EINVAL, "not a state image of this library version");
+  size_t o1, b1, o2, b2;
+  state_blocks(ctx->L, &o1, &b1, &o2, &b2);
+  b2 += 4 * (size_t)ctx->m.max_rounds * ctx->W;
+  DevState cur;
+  int rc = read_status(ctx, &cur);
+  if (rc != ABS_OK) return rc;
+  if (h.d_pad != ctx->L.d_pad || h.esz != ctx->L.esz || h.block1 != b1 || h.block2 != b2 ||
+      h.max_rounds != (unsigned long long)ctx->m.max_rounds || !same_constants(h.st, cur))
+    return fail(ABS_EINVAL, "the image was saved by a context with other sizes, modes, time distribution or seed");
+  if (bytes != sizeof h + b1 + b2) return fail(ABS_EINVAL, "image has %zu bytes, %zu expected", bytes, sizeof h + b1 + b2);
+  if (h.rounds_enqueued < 0 || h.rounds_enqueued > ctx->m.max_rounds || h.st.t != h.rounds_enqueued)
+    return fail(ABS_EINVAL, "image is inconsistent (rounds %d, completed %d)", h.rounds_enqueued, h.st.t);
+  const char* p = (const char*)src;
+  CU(cudaMemcpyAsync(ctx->ws + o1, p + sizeof h, b1, cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaMemcpyAsync(ctx->ws + o2, p + sizeof h + b1, b2, cudaMemcpyHostToDevice, ctx->stream));
+  CU(cudaStreamSynchronize(ctx->stream));
+  ctx->rounds_enqueued = h.rounds_enqueued;
+  return ABS_OK;
+}
+
 int abs_get_trace(abs_ctx* ctx, int first, int n, abs_trace* o) {
   if (!ctx || !o) return fail(ABS_EINVAL, "null argument");
   if (ctx->sticky == ABS_ECUDA) return fail(ABS_ECUDA, "context is in a failed state");

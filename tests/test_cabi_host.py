@@ -129,4 +129,7 @@ def test_null_context_calls():
     l = gpu.lib()
     assert l.abs_run_rounds(None, 1) == gpu.EINVAL
     assert l.abs_get_params(None, None, 0, None) == gpu.EINVAL
+    assert l.abs_state_bytes(None, None) == gpu.EINVAL
+    assert l.abs_save_state(None, None, 0, None) == gpu.EINVAL
+    assert l.abs_restore_state(None, None, 0) == gpu.EINVAL
     assert l.abs_destroy(None) == gpu.OK
