@@ -363,20 +363,22 @@ def main():
         # local steps: every worker's chain of U steps is sequential, one CTA per worker
         n_l, t_l = prof["lsq"]
         if cfg.kind == inputs.MLP and len(cfg.dims) > 2:
-            # multi-layer network: the workers' copies live in HBM; the local-update kernel streams, per
-            # selected worker and step, the step's gradient (4 B/parameter), the upload sum (read + write,
-            # 8 B), the fp32 copy (8 B) and the new bf16 operand copy (2 B)
+            # multi-layer network: the workers' copies live in HBM; after each step but the last the refresh
+            # kernel streams, per selected worker, the upload sum (4 B/parameter), the model version the
+            # worker started from and the new copy (storage type each)
             d_pad = plan.get("d_pad") or sum(cfg.dims[l] * cfg.dims[l + 1] + cfg.dims[l + 1] for l in range(len(cfg.dims) - 1))
             n_rounds_prof = max(1, prof["update"][0])             # rounds the recorded launches cover
-            n_upd = U * n_rounds_prof
-            bytes_l = 22.0 * d_pad * float(np.mean(ks[:n_rounds_prof]))   # per local-update launch: 22 B x d x K^t
+            n_upd = (U - 1) * n_rounds_prof
+            per_par = 4.0 + 2.0 * (2 if bf16 else 4)
+            bytes_l = per_par * d_pad * float(np.mean(ks[:n_rounds_prof]))   # per refresh launch: bytes x d x K^t
             # the class also holds the begin and layout kernels (1 + U launches per round, small)
             out["roofline"] = {"bound": "hbm", "kernel": "local_step_kernel (+ local_begin / local_layout launches)",
                                "launches": n_l, "avg_us": 1e3 * t_l / max(1, n_l),
                                "achieved": bytes_l * n_upd / (t_l * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": bytes_l * n_upd / (t_l * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
                                "peak_source": peaks["source"], "share_of_profiled_time": t_l / tot_prof,
-                               "note": "algorithmic bytes of the local updates only, over the time of the whole class"}
+                               "note": "algorithmic bytes of the U - 1 copy refreshes per round only, over the time of the "
+                                       "whole class (begin, layout and last-step launches included)"}
         else:
             out["roofline"] = {"bound": "latency", "kernel": "local_sgd_kernel", "achieved": None, "peak": None,
                                "unit": None, "frac": None, "traffic": None,

@@ -129,7 +129,7 @@ typedef struct {
                                average of its U minibatch losses) is implemented for ABS_LSQ and ABS_SOFTMAX
                                with <= 16 classes, <= 12288 parameters and batch x classes <= 8192 (the worker's
                                copy lives in shared memory), and for multi-layer ABS_MLP (the selected workers'
-                               copies live in the workspace: 12 bytes per parameter and worker, 14 in bf16;
+                               copies live in the workspace: 8 bytes per parameter and worker, 6 in bf16;
                                not with ABS_FLAG_TMA_GATHER / ABS_FLAG_TWO_CTA); in the bf16 configurations
                                each step is evaluated at the bf16 rounding of the fp32 copy */
   int k_mode;               /* ABS_K_* */

@@ -84,7 +84,7 @@ struct Layout {
   // U > 1 on a multi-layer network: the selected workers' own model copies and uploads
   bool local_net = false;
   int RBp = 0;                          // rows reserved per worker in a local step's row layout
-  size_t priv16 = 0, priv32 = 0, gsum = 0, loss_acc = 0;
+  size_t priv = 0, loss_acc = 0;          // the workers' copies (storage type); their uploads live in G
   size_t gring = 0;                     // the models the gradient kernels read: the ring, or the private copies
   int gslots = 0;
   size_t total = 0;
@@ -258,11 +258,9 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   L->gring = L->ring;
   L->gslots = S + 1;
   if (L->local_net) {
-    L->priv32 = cv.take(4 * L->d_pad * W);
-    L->priv16 = L->esz == 2 ? cv.take(2 * L->d_pad * W) : L->priv32;     // fp32: the local models are the operands
-    L->gsum = cv.take(4 * L->d_pad * W);
+    L->priv = cv.take(L->esz * L->d_pad * W);
     L->loss_acc = cv.take(4 * W);
-    L->gring = L->priv16;
+    L->gring = L->priv;
     L->gslots = W;
   }
   if (!lsq) {
@@ -777,7 +775,7 @@ void enqueue_update(abs_ctx* ctx, int par) {
   }
   UpdateArgs u;
   u.st = ctx->at<DevState>(L.st); u.ri = ri; u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
-  u.G = ctx->at<float>(L.local_net ? L.gsum : L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
+  u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
   // for the latency-bound models (always one stream) the Eq. 3 kernel also prepares the next job
   // durations (its first warps); tensor-core networks keep a small kernel of their own for that
   const bool look = !L.any_tc;
@@ -1092,8 +1090,8 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     q.st = ctx->at<DevState>(L.st);
     q.job = ctx->ctl.job;
     q.ring = ctx->at<void>(L.ring);
-    q.priv16 = ctx->at<__nv_bfloat16>(L.priv16); q.priv32 = ctx->at<float>(L.priv32); q.gsum = ctx->at<float>(L.gsum);
-    q.G = ctx->at<float>(L.G); q.row_loss = ctx->at<float>(L.row_loss);
+    q.priv = ctx->at<void>(L.priv); q.gsum = ctx->at<float>(L.G);
+    q.row_loss = ctx->at<float>(L.row_loss);
     q.loss_acc = ctx->at<float>(L.loss_acc); q.loss = ctx->ctl.loss;
     q.d_pad = L.d_pad; q.RBp = L.RBp; q.U = ctx->m.local_steps; q.lr = ctx->m.lr;
     const int bx = (int)std::max<size_t>(1, std::min<size_t>((L.d_pad / 4 + 1023) / 1024, 64));

@@ -1,16 +1,18 @@
 // Local SGD inside a job (Eq. 2 with U > 1) for multi-layer networks.
 // After its first local step every selected worker computes with weights of its own, so the
-// workers' copies live in HBM: an fp32 copy (the local model), for the bf16 configurations a bf16
-// copy of it (the operand the gradient kernels read), and the fp32 sum of the steps' gradient sums
-// (the upload), each [W][d_pad] and indexed by the worker's position in the round's selection.
+// workers' copies live in HBM, each [W][d_pad] and indexed by the worker's position in the round's
+// selection: the copy the gradient kernels read (storage type) and the fp32 upload, i.e. the sum of
+// the steps' gradient sums so far.  The local model after u steps is the model version the worker
+// started from minus eta / B times that sum (Eq. 2 unrolled), so no third copy is kept.
 // One local step of all selected workers is one pass of the grouped forward / backward kernels
 // (tensor-core or FP32-FMA, as for U = 1) in which
 //   - the rows of worker i are rows [i * RBp, i * RBp + B) (RBp = B rounded up to the row-tile
 //     height; the rest is padding with sample index -1),
 //   - the "model version" of a row tile is the worker's own copy (slot i of the private store), and
-//   - the weight gradient is split per worker (split i = the rows of worker i) instead of summed,
-// followed by the workers' local updates.  Eq. 3 then adds the K uploads like the partial sums of
-// the U = 1 path.  Minibatch of step u: Philox blocks (n, j, 1, u * ceil(B/4) + b/4).
+//   - the weight gradient is split per worker (split i = the rows of worker i) and added to the
+//     worker's upload instead of summed over the workers,
+// followed by the refresh of the workers' copies.  Eq. 3 then adds the K uploads like the partial
+// sums of the U = 1 path.  Minibatch of step u: Philox blocks (n, j, 1, u * ceil(B/4) + b/4).
 #pragma once
 #include "common.cuh"
 #include "ctl.cuh"
@@ -24,10 +26,8 @@ struct Args {
   const int* sel; const int* job; const int* sel_tau;
   int* row_idx; int* tile_slot;        // the round's row layout, rewritten for every local step
   const void* ring;                    // [S+1][d_pad] model versions, storage type
-  __nv_bfloat16* priv16;               // [W][d_pad] bf16 operand copies of the local models (bf16 configurations)
-  float* priv32;                       // [W][d_pad] local models
+  void* priv;                          // [W][d_pad] the workers' copies, storage type
   float* gsum;                         // [W][d_pad] uploads: sum over the steps of the gradient sums
-  const float* G;                      // [W][d_pad] gradient sums of the current step, per worker
   const float* row_loss;               // sample losses of the current step, by row
   float* loss_acc;                     // [W] sum of the steps' mean losses
   float* loss;                         // [W] uploaded losses
@@ -37,7 +37,7 @@ struct Args {
   float lr;
 };
 
-// Start of a job's local steps: the worker's copies are the model version it holds.
+// Start of a job's local steps: the worker's copy is the model version it holds, its upload zero.
 template <typename T>
 __global__ void __launch_bounds__(256) local_begin_kernel(Args a) {
   grid_dependency_sync();
@@ -47,22 +47,12 @@ __global__ void __launch_bounds__(256) local_begin_kernel(Args a) {
   const int i = blockIdx.y;
   if (i >= ri->K) return;
   const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
-  const T* ring_slot = (const T*)a.ring + (size_t)slot * a.d_pad;
-  uint2* d16 = reinterpret_cast<uint2*>(a.priv16 + (size_t)i * a.d_pad);
-  float4* d32 = reinterpret_cast<float4*>(a.priv32 + (size_t)i * a.d_pad);
+  const uint4* src = reinterpret_cast<const uint4*>((const T*)a.ring + (size_t)slot * a.d_pad);
+  uint4* dst = reinterpret_cast<uint4*>((T*)a.priv + (size_t)i * a.d_pad);
   float4* gs = reinterpret_cast<float4*>(a.gsum + (size_t)i * a.d_pad);
-  const size_t n4 = a.d_pad / 4;
+  const size_t n16 = a.d_pad * sizeof(T) / 16, n4 = a.d_pad / 4;
   for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < n4; v += (size_t)gridDim.x * blockDim.x) {
-    if (sizeof(T) == 4) {
-      d32[v] = reinterpret_cast<const float4*>(ring_slot)[v];
-    } else {
-      const uint2 pk = reinterpret_cast<const uint2*>(ring_slot)[v];
-      d16[v] = pk;
-      const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&pk.x);
-      const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&pk.y);
-      const float2 f0 = __bfloat1622float2(lo), f1 = __bfloat1622float2(hi);
-      d32[v] = make_float4(f0.x, f0.y, f1.x, f1.y);
-    }
+    if (v < n16) dst[v] = src[v];
     gs[v] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) a.loss_acc[i] = 0.f;
@@ -100,7 +90,8 @@ __global__ void __launch_bounds__(128) local_layout_kernel(Args a, int u) {
   for (int q = threadIdx.x; q < tiles; q += blockDim.x) a.tile_slot[i * tiles + q] = i;
 }
 
-// Output-layer gradient of every worker: dst_i[j] = sum over the worker's row chunks of part[q][j].
+// Output-layer gradient of every worker, added to its upload: dst_i[j] += sum over the worker's row
+// chunks of part[q][j].
 // Block = 32 outputs x 8 chunk lanes (lane w adds chunks w, w+8, ... in order, then the lanes in order).
 __global__ void __launch_bounds__(256) chunk_reduce_worker_kernel(const DevState* st, const RoundInfo* ri, const float* part, int len,
                                                                   float* dst, size_t d_pad, int chunk_rows, int RBp) {
@@ -121,14 +112,14 @@ __global__ void __launch_bounds__(256) chunk_reduce_worker_kernel(const DevState
     float tot = 0.f;
 #pragma unroll
     for (int q = 0; q < 8; ++q) tot += red[q][lane];
-    dst[(size_t)i * d_pad + j] = tot;
+    dst[(size_t)i * d_pad + j] += tot;
   }
 }
 
-// The workers' local updates after step u (Eq. 2): w_i -= eta / B * G_i, upload += G_i, new
-// operand copy (bf16 configurations); block (0, i) also adds the step's mean loss and, after the
-// last step, writes the uploaded loss (the average of the U mean minibatch losses; Algorithm 1,
-// last worker line).
+// After step u (Eq. 2 unrolled): w_i^{u+1} = w_i^0 - eta / B * (sum of the gradient sums so far), written
+// as the copy the next step reads (skipped after the last step); block (0, i) also adds the
+// step's mean loss and, after the last step, writes the uploaded loss (the average of the U mean
+// minibatch losses; Algorithm 1, last worker line).
 template <typename T>
 __global__ void __launch_bounds__(256) local_step_kernel(Args a, int last) {
   grid_dependency_sync();
@@ -139,27 +130,35 @@ __global__ void __launch_bounds__(256) local_step_kernel(Args a, int last) {
   const int i = blockIdx.y;
   if (i >= ri->K) return;
   const int B = st->B;
-  const float step = __fdiv_rn(a.lr, (float)B);
-  const float4* g = reinterpret_cast<const float4*>(a.G + (size_t)i * a.d_pad);
-  float4* gs = reinterpret_cast<float4*>(a.gsum + (size_t)i * a.d_pad);
-  float4* w32 = reinterpret_cast<float4*>(a.priv32 + (size_t)i * a.d_pad);
-  uint2* w16 = reinterpret_cast<uint2*>(a.priv16 + (size_t)i * a.d_pad);
-  const size_t n4 = a.d_pad / 4;
-  for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < n4; v += (size_t)gridDim.x * blockDim.x) {
-    const float4 gv = g[v];
-    float4 s = gs[v];
-    s.x += gv.x; s.y += gv.y; s.z += gv.z; s.w += gv.w;
-    gs[v] = s;
-    float4 m = w32[v];
-    m.x = fmaf(-step, gv.x, m.x); m.y = fmaf(-step, gv.y, m.y);
-    m.z = fmaf(-step, gv.z, m.z); m.w = fmaf(-step, gv.w, m.w);
-    w32[v] = m;
-    if (sizeof(T) == 2) {
-      const __nv_bfloat162 lo = __floats2bfloat162_rn(m.x, m.y), hi = __floats2bfloat162_rn(m.z, m.w);
-      uint2 pk;
-      pk.x = *reinterpret_cast<const unsigned*>(&lo);
-      pk.y = *reinterpret_cast<const unsigned*>(&hi);
-      w16[v] = pk;
+  if (!last) {
+    const float step = __fdiv_rn(a.lr, (float)B);
+    const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
+    const T* w0 = (const T*)a.ring + (size_t)slot * a.d_pad;
+    T* w = (T*)a.priv + (size_t)i * a.d_pad;
+    const float4* gs = reinterpret_cast<const float4*>(a.gsum + (size_t)i * a.d_pad);
+    const size_t n4 = a.d_pad / 4;
+    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < n4; v += (size_t)gridDim.x * blockDim.x) {
+      const float4 g = gs[v];
+      float4 m;
+      if (sizeof(T) == 4) {
+        m = reinterpret_cast<const float4*>(w0)[v];
+      } else {
+        const uint2 pk = reinterpret_cast<const uint2*>(w0)[v];
+        const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.x));
+        const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.y));
+        m = make_float4(f0.x, f0.y, f1.x, f1.y);
+      }
+      m.x = fmaf(-step, g.x, m.x); m.y = fmaf(-step, g.y, m.y);
+      m.z = fmaf(-step, g.z, m.z); m.w = fmaf(-step, g.w, m.w);
+      if (sizeof(T) == 4) {
+        reinterpret_cast<float4*>(w)[v] = m;
+      } else {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(m.x, m.y), hi = __floats2bfloat162_rn(m.z, m.w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const unsigned*>(&lo);
+        pk.y = *reinterpret_cast<const unsigned*>(&hi);
+        reinterpret_cast<uint2*>(w)[v] = pk;
+      }
     }
   }
   if (blockIdx.x == 0) {

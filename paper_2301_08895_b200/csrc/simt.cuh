@@ -65,7 +65,7 @@ struct LayerArgs {
   const void* delta_out;    // bwd: [rows][out] deltas of this layer's output
   void* delta_in;           // dgrad result [rows][in]
   float* G;                 // wgrad partials [P][slot_stride]
-  int P;
+  int P;                    // 0: one split per selected worker (its rows), added to G[worker]
 };
 
 // Forward of one affine layer for all rows of the round: act_out = [relu](act_in W_s + b_s).
@@ -196,7 +196,10 @@ __global__ void __launch_bounds__(256) simt_wgrad_kernel(LayerArgs a) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tx * 4 + j;
-      if (m <= in && n < out) G[(size_t)m * out + n] = acc[i][j];
+      if (m <= in && n < out) {
+        if (a.P == 0) G[(size_t)m * out + n] += acc[i][j];      // per-worker split: adds to the worker's upload
+        else G[(size_t)m * out + n] = acc[i][j];
+      }
     }
   }
 }

@@ -36,7 +36,7 @@ struct Params {
   int M_total;             // WGRAD: in + 1 (weight rows and the bias row of G); FWD/DGRAD: unused
   int N_total;             // FWD: out, DGRAD: in, WGRAD: out
   int K_total;             // FWD: in,  DGRAD: out, WGRAD: unused (rows come from the device state)
-  int P;                   // WGRAD split count
+  int P;                   // WGRAD split count; 0: one split per selected worker, added to its upload
   const __nv_bfloat16* ring; size_t slot_stride; size_t b_off;   // FWD bias: ring + slot*stride + b_off
   const __nv_bfloat16* mask_src;   // DGRAD: H[r][N_total] (used when mask_bits is null)
   const uint32_t* mask_bits;       // DGRAD: word [r][n/32] holds (H[r][n] > 0) for its 32 columns, column j of
@@ -652,8 +652,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
               float* dst = p.out_f32 + (size_t)c.split * p.slot_stride + (size_t)r * p.N_total + n0;
 #pragma unroll
               for (int i = 0; i < 32; i += 4)
-                if (n0 + i < p.N_total)
-                  *reinterpret_cast<uint4*>(dst + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                if (n0 + i < p.N_total) {
+                  uint4 o = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                  if (p.P == 0) {              // per-worker splits add to the worker's upload
+                    const float4 old = *reinterpret_cast<const float4*>(dst + i);
+                    o.x = __float_as_uint(old.x + __uint_as_float(o.x));
+                    o.y = __float_as_uint(old.y + __uint_as_float(o.y));
+                    o.z = __float_as_uint(old.z + __uint_as_float(o.z));
+                    o.w = __float_as_uint(old.w + __uint_as_float(o.w));
+                  }
+                  *reinterpret_cast<uint4*>(dst + i) = o;
+                }
             }
           } else {
 #pragma unroll
@@ -713,7 +722,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (issuer && !(mode == WGRAD && c.bias_tile)) {
-          if (mode == WGRAD)
+          if (mode == WGRAD && p.P == 0)       // one split per worker: the tile adds to that worker's upload
+            asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                         ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(smem_u32(my_box)), "r"(n0), "r"(c.a_row + q * 32), "r"(c.split)
+                         : "memory");
+          else if (mode == WGRAD)
             asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
                          ::"l"(reinterpret_cast<uint64_t>(&map_out)), "r"(smem_u32(my_box)), "r"(n0), "r"(c.a_row + q * 32), "r"(c.split)
                          : "memory");
