@@ -33,20 +33,21 @@ def check_invariants(cfg, rows):
         assert np.all(np.isfinite(r["sel_loss"]))
 
 
-def full_run_checks(cfg, prefix_rounds, tol, loss_tol):
+def full_run_checks(cfg, prefix_rounds, tol, loss_tol, rounds=None, **kw):
     X, y, _ = inputs.make_data(cfg)
     w0 = inputs.make_w0(cfg)
-    rows, params = gpu_run(cfg, X, y, w0, cfg.rounds)
-    assert len(rows) == cfg.rounds and np.all(np.isfinite(params))
+    rounds = rounds or cfg.rounds
+    rows, params = gpu_run(cfg, X, y, w0, rounds, **kw)
+    assert len(rows) == rounds and np.all(np.isfinite(params))
     check_invariants(cfg, rows)
     # (1) integer trace of the whole run against the oracle's server logic
-    o = make_oracle(cfg, X, y, w0, integer_only=True)
-    orows = o.run(cfg.rounds, forced_losses=[r["sel_loss"] for r in rows])
+    o = make_oracle(cfg, X, y, w0, integer_only=True, **kw)
+    orows = o.run(rounds, forced_losses=[r["sel_loss"] for r in rows])
     mm = first_integer_mismatch(rows, orows)
     assert mm is None, "full-run integer trace differs: %s" % (mm,)
     assert rows[-1]["loss_mean"] < 0.2 * rows[0]["loss_mean"]
     # (2) first rounds in lock step, floats included
-    compare_with_oracle(cfg, X, y, w0, prefix_rounds, tol, forced=True, loss_tol=loss_tol)
+    compare_with_oracle(cfg, X, y, w0, prefix_rounds, tol, forced=True, loss_tol=loss_tol, **kw)
     return rows
 
 
@@ -60,6 +61,17 @@ def test_config3_full_size():
     rows = full_run_checks(inputs.config(3), 60, 2e-2, 5e-2)
     assert rows[0]["K"] == 8 and rows[-1]["K"] == 64
     assert any(r["restart"] for r in rows)
+
+
+def test_config3_full_size_ten_local_steps():
+    """The paper's U = 10 on the benchmark's network configuration, in the launch shape bench.py times."""
+    rows = full_run_checks(inputs.config(3), 6, 2e-2, 5e-2, local_steps=10)
+    assert rows[0]["K"] == 8 and rows[-1]["K"] == 64
+
+
+def test_config4_ten_local_steps():
+    rows = full_run_checks(inputs.config(4), 1, 2e-2, 5e-2, rounds=120, local_steps=10)
+    assert rows[0]["K"] == 16 and rows[-1]["K"] > 64
 
 
 def test_config2_full_size_is_covered_by_the_free_running_test():
