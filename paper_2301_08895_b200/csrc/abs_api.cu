@@ -671,7 +671,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
           launch_ex(ctx, ABS_KC_OUTPUT, narrow_fused_kernel<T>, dim3(L.rows_cap / R), dim3(256), sm, a, part, R, has_dgrad);
         }
         if (L.local_net)
-          launch_ex(ctx, ABS_KC_OUTPUT, lnet::chunk_reduce_worker_kernel, dim3((len + 31) / 32, ctx->W), dim3(256), 0, st, ri, part, len,
+          launch_ex(ctx, ABS_KC_OUTPUT, lnet::chunk_reduce_worker_kernel, dim3((len + 255) / 256, ctx->W), dim3(256), 0, st, ri, part, len,
                     dstw, L.d_pad, R, L.RBp);
         else
           launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, R);
@@ -742,7 +742,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       const int len = (a.in + 1) * a.C;
       launch_ex(ctx, ABS_KC_OUTPUT, narrow_wgrad_chunk_kernel<T>, dim3(L.rows_cap / 64), dim3(256), 0, a, part);
       if (L.local_net)
-        launch_ex(ctx, ABS_KC_OUTPUT, lnet::chunk_reduce_worker_kernel, dim3((len + 31) / 32, ctx->W), dim3(256), 0, st, ri, part, len,
+        launch_ex(ctx, ABS_KC_OUTPUT, lnet::chunk_reduce_worker_kernel, dim3((len + 255) / 256, ctx->W), dim3(256), 0, st, ri, part, len,
                   dstw, L.d_pad, 64, L.RBp);
       else
         launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, 64);

@@ -91,29 +91,19 @@ __global__ void __launch_bounds__(128) local_layout_kernel(Args a, int u) {
 }
 
 // Output-layer gradient of every worker, added to its upload: dst_i[j] += sum over the worker's row
-// chunks of part[q][j].
-// Block = 32 outputs x 8 chunk lanes (lane w adds chunks w, w+8, ... in order, then the lanes in order).
+// chunks, in order, of part[q][j].  One thread per output (a worker has only RBp / chunk_rows chunks).
 __global__ void __launch_bounds__(256) chunk_reduce_worker_kernel(const DevState* st, const RoundInfo* ri, const float* part, int len,
                                                                   float* dst, size_t d_pad, int chunk_rows, int RBp) {
   grid_dependency_sync();
-  __shared__ float red[8][33];
   if (st->status != ST_OK) return;
   const int i = blockIdx.y;
   if (i >= ri->K) return;
   const int per = RBp / chunk_rows, q0 = i * per;
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int j = blockIdx.x * 32 + lane;
-  float acc = 0.f;
-  if (j < len)
-    for (int q = w; q < per; q += 8) acc += part[(size_t)(q0 + q) * len + j];
-  red[w][lane] = acc;
-  __syncthreads();
-  if (w == 0 && j < len) {
-    float tot = 0.f;
-#pragma unroll
-    for (int q = 0; q < 8; ++q) tot += red[q][lane];
-    dst[(size_t)i * d_pad + j] += tot;
-  }
+  const int j = blockIdx.x * 256 + threadIdx.x;
+  if (j >= len) return;
+  float tot = 0.f;
+  for (int q = 0; q < per; ++q) tot += part[(size_t)(q0 + q) * len + j];
+  dst[(size_t)i * d_pad + j] += tot;
 }
 
 // After step u (Eq. 2 unrolled): w_i^{u+1} = w_i^0 - eta / B * (sum of the gradient sums so far), written
