@@ -348,6 +348,7 @@ struct abs_ctx {
   long long launches = 0;
   cudaError_t launch_error = cudaSuccess;
   int next_cluster = 1;              // cluster width of the next launch (consumed by launch_on)
+  int upd_blocks_per_sm = 8;         // resident blocks per SM of the Eq. 3 kernel
   bool local_sgd = false;            // U > 1: one CTA per selected worker runs the worker's local steps
   bool lsq_pipe = false;             // bf16 least squares through the bulk-copy pipeline kernel
   int lsq_stages = 0;
@@ -783,8 +784,9 @@ void enqueue_update(abs_ctx* ctx, int par) {
   u.zero_words = nullptr; u.n_zero = 0;
   for (int l = 0; l < ctx->m.n_layers; ++l)
     if (L.pair_fwd[l]) { u.zero_words = ctx->at<int>(L.done); u.n_zero = L.n_tiles_cap; }
+  // one wave of resident blocks striding over the vector (a partly filled second wave would only add a tail)
   const size_t n4 = L.d_pad / 4;
-  const int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * 8), (size_t)(ctx->W + 31) / 32);
+  const int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * ctx->upd_blocks_per_sm), (size_t)(ctx->W + 31) / 32);
   if (look) launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T, true>, dim3(blocks), dim3(256), 0, u);
   else launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T, false>, dim3(blocks), dim3(256), 0, u);
 }
@@ -1016,6 +1018,18 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);
+  {
+    int occ = 0;
+    cudaError_t eo;
+    if (model->dtype == ABS_FP32)
+      eo = L.any_tc ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, update_kernel<float, false>, 256, 0)
+                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, update_kernel<float, true>, 256, 0);
+    else
+      eo = L.any_tc ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, update_kernel<__nv_bfloat16, false>, 256, 0)
+                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, update_kernel<__nv_bfloat16, true>, 256, 0);
+    if (eo != cudaSuccess) return bail(cuda_fail(nullptr, eo, "cudaOccupancyMaxActiveBlocksPerMultiprocessor(update_kernel)"));
+    ctx->upd_blocks_per_sm = std::max(1, std::min(occ, 8));
+  }
   // worth it only when a round has a long backward pass to hide behind (tensor-core networks);
   // for the latency-bound models the cross-stream events cost more than they hide
   if (!(model->flags & ABS_FLAG_NO_OVERLAP) && L.any_tc && !L.local_net) {

@@ -357,14 +357,9 @@ __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
   const int slot = (ri->t + 1) % (st->S + 1);
   T* dst = (T*)a.ring + (size_t)slot * a.d_pad;
   const size_t n4 = a.d_pad / 4;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
-       i += (size_t)gridDim.x * blockDim.x) {
-    float4 g = reinterpret_cast<const float4*>(a.G)[i];
-    for (int p = 1; p < P; ++p) {
-      const float4 q = reinterpret_cast<const float4*>(a.G + (size_t)p * a.d_pad)[i];
-      g.x += q.x; g.y += q.y; g.z += q.z; g.w += q.w;
-    }
-    float4 m = reinterpret_cast<float4*>(a.master)[i];
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  auto finish = [&](size_t i, float4 g, float4 m) {
     m.x = fmaf(-step, g.x, m.x); m.y = fmaf(-step, g.y, m.y);
     m.z = fmaf(-step, g.z, m.z); m.w = fmaf(-step, g.w, m.w);
     reinterpret_cast<float4*>(a.master)[i] = m;
@@ -377,6 +372,38 @@ __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
       pk.y = *reinterpret_cast<unsigned*>(&hi);
       reinterpret_cast<uint2*>(dst)[i] = pk;
     }
+  };
+  // few partials (the split counts of the weight-gradient GEMMs): two vectors per thread and
+  // iteration, all loads of both issued before the first use (same sums, same order per element)
+  if (P <= 4) {
+    for (; i + stride < n4; i += 2 * stride) {
+      const size_t j = i + stride;
+      float4 ga[4], gb[4];
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+        if (p < P) {
+          ga[p] = reinterpret_cast<const float4*>(a.G + (size_t)p * a.d_pad)[i];
+          gb[p] = reinterpret_cast<const float4*>(a.G + (size_t)p * a.d_pad)[j];
+        }
+      const float4 ma = reinterpret_cast<float4*>(a.master)[i], mb = reinterpret_cast<float4*>(a.master)[j];
+      float4 g = ga[0], h = gb[0];
+#pragma unroll
+      for (int p = 1; p < 4; ++p)
+        if (p < P) {
+          g.x += ga[p].x; g.y += ga[p].y; g.z += ga[p].z; g.w += ga[p].w;
+          h.x += gb[p].x; h.y += gb[p].y; h.z += gb[p].z; h.w += gb[p].w;
+        }
+      finish(i, g, ma);
+      finish(j, h, mb);
+    }
+  }
+  for (; i < n4; i += stride) {
+    float4 g = reinterpret_cast<const float4*>(a.G)[i];
+    for (int p = 1; p < P; ++p) {
+      const float4 q = reinterpret_cast<const float4*>(a.G + (size_t)p * a.d_pad)[i];
+      g.x += q.x; g.y += q.y; g.z += q.z; g.w += q.w;
+    }
+    finish(i, g, reinterpret_cast<float4*>(a.master)[i]);
   }
 }
 

@@ -269,8 +269,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   const int T0 = P0.n_tiles, T1 = P1.n_tiles;
   // i-th tile of this unit, or -1.  Two problems with fewer long tiles than units: units [0, T0)
   // take one tile of problem 0 each, the others stride over problem 1; otherwise all units stride
-  // over the concatenated tiles.
+  // over the concatenated tiles.  Weight gradient + back-propagation: a long tile costs about as
+  // much as `lead` short ones (k-blocks at 0.34 us plus about 3.5 us of fixed cost per tile), so
+  // the other units take `lead` short tiles each and what is left is strided over ALL units.
   const bool split_units = T1 > 0 && T0 < n_units;
+  const int R_units = n_units - T0;
+  int lead = 1 << 20;
+  if (split_units && p0.mode == WGRAD && p1.mode == DGRAD) {
+    const float long_t = (float)(P0.chunk / BK) * 0.34f + 3.5f;
+    const float short_t = (float)((p1.K_total + BK - 1) / BK) * 0.34f + 3.5f;
+    lead = max(1, (int)(long_t / short_t + 0.5f));
+  }
+  const int n_lead = split_units ? min(T1, lead * R_units) : 0;      // short tiles handed out before the long-tile units join
   // Second problem reading the first's output (two forward layers) when the first has between one
   // and two waves of tiles: the units left idle by its second wave take the tiles of the second
   // problem whose inputs the FIRST wave produced (row tiles [0, n_units / n_ct0)), and whatever is
@@ -300,9 +310,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       return t < T0 + T1 ? t : -1;
     }
     if (split_units) {
-      if (unit < T0) return i == 0 ? unit : -1;
-      const int t = T0 + (unit - T0) + i * (n_units - T0);
-      return t < T0 + T1 ? t : -1;
+      if (unit < T0) {
+        if (i == 0) return unit;
+        const int t1 = n_lead + unit + (i - 1) * n_units;
+        return t1 < T1 ? T0 + t1 : -1;
+      }
+      if (i < lead) {
+        const int t1 = (unit - T0) + i * R_units;
+        return t1 < n_lead ? T0 + t1 : -1;
+      }
+      const int t1 = n_lead + unit + (i - lead) * n_units;
+      return t1 < T1 ? T0 + t1 : -1;
     }
     const int t = unit + i * n_units;
     return t < T0 + T1 ? t : -1;
