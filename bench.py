@@ -30,8 +30,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) per launch at K = N on configuration 4, from ncu captures of the GEMM and the
 # Eq. 3 kernel (summaries under profiles/); each figure is valid only for the kernel source it was taken
 # from (first 16 hex digits of the file's sha256).
-TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.4e6, "file": "tc.cuh", "sha256_16": "5bbc5c03a639a578"},
-           "update": {"config": 4, "bytes_per_launch": 76.0e6, "file": "simt.cuh", "sha256_16": "c83254d5da04ead1"}}
+TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.3e6, "file": "tc.cuh", "sha256_16": "b4893775bfc39d3d"},
+           "update": {"config": 4, "bytes_per_launch": 75.8e6, "file": "simt.cuh", "sha256_16": "1e0e90dac7748f95"}}
 METRIC = "worker_gradients_per_sec"
 UNIT = "worker-gradients/s"
 
