@@ -24,8 +24,17 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const DevState* st, co
     if (s < 0) {
       for (int v = lane; v < vec_per_row; v += 32) dst[v] = make_uint4(0u, 0u, 0u, 0u);
     } else {
+      // four 16-byte loads per lane in flight before the first store
       const uint4* src = reinterpret_cast<const uint4*>(X + (size_t)s * in);
-      for (int v = lane; v < vec_per_row; v += 32) dst[v] = __ldg(src + v);
+      for (int v = lane; v < vec_per_row; v += 128) {
+        uint4 q[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (v + 32 * k < vec_per_row) q[k] = __ldg(src + v + 32 * k);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (v + 32 * k < vec_per_row) dst[v + 32 * k] = q[k];
+      }
     }
   }
 }
