@@ -136,8 +136,8 @@ def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mod
 
 
 def workspace_bytes(kind, dims, batch, dtype, W, S, max_rounds, n_samples, data_on_host=0,
-                    flags=0):
-    m = _desc(kind, dims, batch, 0.0, dtype, max_rounds, n_samples, 0, 0, 1, data_on_host, flags)
+                    flags=0, local_steps=1):
+    m = _desc(kind, dims, batch, 0.0, dtype, max_rounds, n_samples, 0, 0, local_steps, data_on_host, flags)
     out = C.c_size_t(0)
     _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(out)))
     return out.value

@@ -66,6 +66,10 @@ def test_workspace_bytes_grows_with_problem():
     d = 3072 * 1024 + 1024 + 1024 * 512 + 512 + 512 * 10 + 10
     assert c >= 17 * d * 2 + d * 4          # ring of S + 1 bf16 versions + fp32 master
     assert c < 4 << 30
+    # local steps on a network: every worker's own copy (bf16) and its fp32 upload
+    u = gpu.workspace_bytes(gpu.MLP, [3072, 1024, 512, 10], 64, gpu.BF16_FP32MASTER, 128, 16, 2000,
+                            50000, local_steps=10)
+    assert u - c >= 128 * d * 2 + (128 - 4) * d * 4 and u < 8 << 30
 
 
 @pytest.mark.parametrize("kw,code", [
@@ -98,6 +102,9 @@ def _init_args():
     (lambda m, td: setattr(m, "local_steps", 0), gpu.EINVAL),
     (lambda m, td: setattr(m, "local_steps", 2000), gpu.EINVAL),
     (lambda m, td: (setattr(m, "local_steps", 4), setattr(m, "batch", 1024), m.dims.__setitem__(0, 20000)), gpu.EUNSUPPORTED),
+    (lambda m, td: (setattr(m, "kind", gpu.MLP), setattr(m, "n_layers", 2), setattr(m, "dtype", gpu.BF16_FP32MASTER),
+                    m.dims.__setitem__(0, 64), m.dims.__setitem__(1, 128), m.dims.__setitem__(2, 10),
+                    setattr(m, "local_steps", 4), setattr(m, "flags", gpu.FLAG_TMA_GATHER)), gpu.EUNSUPPORTED),
     (lambda m, td: setattr(m, "workspace", 0), gpu.EINVAL),
     (lambda m, td: setattr(m, "workspace", 0x10010), gpu.EINVAL),
     (lambda m, td: setattr(m, "workspace_bytes", 1024), gpu.ENOSPACE),
