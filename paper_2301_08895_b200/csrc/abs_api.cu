@@ -671,11 +671,10 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
         } else {
           launch_ex(ctx, ABS_KC_OUTPUT, narrow_fused_kernel<T>, dim3(L.rows_cap / R), dim3(256), sm, a, part, R, has_dgrad);
         }
+        // U = 1: the chunk partials are added up by extra blocks of the Eq. 3 kernel (one launch less)
         if (L.local_net)
           launch_ex(ctx, ABS_KC_OUTPUT, lnet::chunk_reduce_worker_kernel, dim3((len + 255) / 256, ctx->W), dim3(256), 0, st, ri, part, len,
                     dstw, L.d_pad, R, L.RBp);
-        else
-          launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, R);
       } else if (a.in % 8 == 0) {
         const size_t sm = sizeof(T) * (size_t)a.in * a.C + sizeof(float) * a.C;
         launch_ex(ctx, ABS_KC_OUTPUT, narrow_fwd_loss_v8_kernel<T>, dim3(L.rows_cap / NARROW_ROWS), dim3(256), sm, a);
@@ -786,7 +785,17 @@ void enqueue_update(abs_ctx* ctx, int par) {
     if (L.pair_fwd[l]) { u.zero_words = ctx->at<int>(L.done); u.n_zero = L.n_tiles_cap; }
   // one wave of resident blocks striding over the vector (a partly filled second wave would only add a tail)
   const size_t n4 = L.d_pad / 4;
-  const int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * ctx->upd_blocks_per_sm), (size_t)(ctx->W + 31) / 32);
+  int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * ctx->upd_blocks_per_sm), (size_t)(ctx->W + 31) / 32);
+  u.part = nullptr; u.part_len = 0; u.part_chunk_rows = 1; u.part_off = 0; u.n_main_blocks = blocks;
+  const int last = ctx->m.n_layers - 1;
+  if (ctx->m.kind != ABS_LSQ && L.fused_R && L.path[last] == PATH_NARROW && !L.local_net && !ctx->local_sgd) {
+    // the fused output-layer kernel left its gradient as per-chunk partial sums
+    u.part = ctx->at<float>(L.red);
+    u.part_len = (ctx->m.dims[last] + 1) * ctx->m.dims[last + 1];
+    u.part_chunk_rows = L.out_mma ? outl::ROWS : L.fused_R;
+    u.part_off = L.w_off[last];
+    blocks += (u.part_len + 31) / 32;
+  }
   if (look) launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T, true>, dim3(blocks), dim3(256), 0, u);
   else launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T, false>, dim3(blocks), dim3(256), 0, u);
 }

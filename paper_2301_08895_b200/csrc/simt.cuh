@@ -333,6 +333,14 @@ struct UpdateArgs {
   int P;                  // partial count, or 0: one partial per selected worker (K^t)
   float lr;
   int* zero_words; int n_zero;   // counters of the round's kernels to clear for the next round (or null)
+  // Output-layer gradient still in per-chunk partial sums (or null): blocks [n_main_blocks, gridDim.x)
+  // add the chunks of 32 outputs each in a fixed order and apply Eq. 3 to those parameters; the
+  // streaming blocks skip the range.
+  const float* part;      // [chunks][part_len]
+  int part_len;           // (in + 1) * C parameters of the output layer
+  int part_chunk_rows;    // gradient rows per chunk
+  size_t part_off;        // element offset of the output layer inside the parameter vector (multiple of 4)
+  int n_main_blocks;
 };
 
 // Eq. 3 and the ring write: w^{t+1} = w^t - eta / (K^t B) * sum_p G_p, stored as the fp32
@@ -356,10 +364,38 @@ __global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
   const float step = __fdiv_rn(a.lr, (float)(K * st->B));
   const int slot = (ri->t + 1) % (st->S + 1);
   T* dst = (T*)a.ring + (size_t)slot * a.d_pad;
+  if (a.part != nullptr && (int)blockIdx.x >= a.n_main_blocks) {
+    // lane w adds chunks w, w + 8, ... in order, then the 8 lanes are added in order
+    __shared__ float red[8][33];
+    const int n_chunks = ri->n_rows / a.part_chunk_rows;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int j = ((int)blockIdx.x - a.n_main_blocks) * 32 + lane;
+    float acc = 0.f;
+    if (j < a.part_len) {
+#pragma unroll 8
+      for (int q = w; q < n_chunks; q += 8) acc += a.part[(size_t)q * a.part_len + j];
+    }
+    red[w][lane] = acc;
+    __syncthreads();
+    if (w == 0 && j < a.part_len) {
+      float tot = 0.f;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) tot += red[q][lane];
+      const size_t e = a.part_off + (size_t)j;
+      const float m = fmaf(-step, tot, a.master[e]);
+      a.master[e] = m;
+      stf(dst, e, m);
+    }
+    return;
+  }
   const size_t n4 = a.d_pad / 4;
-  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  const size_t part_lo4 = a.part != nullptr ? a.part_off / 4 : n4;
+  const size_t part_hi4 = a.part != nullptr ? (a.part_off + (size_t)a.part_len + 3) / 4 : n4;
+  const int n_blocks = a.part != nullptr ? a.n_main_blocks : (int)gridDim.x;
+  const size_t stride = (size_t)n_blocks * blockDim.x;
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   auto finish = [&](size_t i, float4 g, float4 m) {
+    if (i >= part_lo4 && i < part_hi4) return;     // the output layer is done by the reduce blocks
     m.x = fmaf(-step, g.x, m.x); m.y = fmaf(-step, g.y, m.y);
     m.z = fmaf(-step, g.z, m.z); m.w = fmaf(-step, g.w, m.w);
     reinterpret_cast<float4*>(a.master)[i] = m;
