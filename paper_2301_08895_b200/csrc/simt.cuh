@@ -348,7 +348,7 @@ struct UpdateArgs {
 // LOOK: the first warps also prepare the next job durations (latency-bound models, one stream); the
 // bandwidth-bound networks keep that in a kernel of its own so that this one stays a pure stream.
 template <typename T, bool LOOK>
-__global__ void __launch_bounds__(256) update_kernel(UpdateArgs a) {
+__global__ void __launch_bounds__(256, 4) update_kernel(UpdateArgs a) {
   grid_dependency_sync();
   const DevState* st = a.st;
   const RoundInfo* ri = a.ri;
