@@ -104,7 +104,7 @@ extern "C" {
 #define ABS_KC_OUTPUT  5  /* output layer: forward + loss, its back-propagation and gradient */
 #define ABS_KC_BIAS    6  /* bias gradients */
 #define ABS_KC_LSQ     7  /* least-squares residual + gradient; with local_steps > 1: the workers' local steps
-                             (single-layer models), or their set-up, row layouts and local updates (networks) */
+                             (single-layer models), or their set-up, row layouts and copy refreshes (networks) */
 #define ABS_KC_UPDATE  8  /* Eq. 3 step + ring write */
 #define ABS_KC_ROUNDS  9  /* whole rounds (control step + Eq. 2 + Eq. 3) of a small least-squares problem
                              in one persistent kernel; one launch per abs_enqueue_rounds call */
