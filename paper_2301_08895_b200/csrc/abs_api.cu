@@ -1107,7 +1107,8 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
   } else if (n > 0 && ctx->L.local_net) {
     // U > 1 on a multi-layer network: per round, the workers' copies are set up, then every local
-    // step is one pass of the gradient kernels over the private copies (which add each worker's gradient to its upload) followed by the refresh of the copies
+    // step is one pass of the gradient kernels over the private copies (which add each worker's
+    // gradient to its upload) followed by the refresh of the copies
     const Layout& L = ctx->L;
     lnet::Args q;
     q.st = ctx->at<DevState>(L.st);
