@@ -1130,12 +1130,11 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
       if (f32) launch_ex(ctx, ABS_KC_LSQ, lnet::local_begin_kernel<float>, dim3(bx, ctx->W), dim3(256), 0, q);
       else launch_ex(ctx, ABS_KC_LSQ, lnet::local_begin_kernel<__nv_bfloat16>, dim3(bx, ctx->W), dim3(256), 0, q);
       for (int u = 0; u < q.U; ++u) {
-        launch_ex(ctx, ABS_KC_LSQ, lnet::local_layout_kernel, dim3(ctx->W), dim3(128), 0, q, u);
         gradient(par, PH_GATHER);
         gradient(par, PH_FORWARD);
         gradient(par, PH_BACKWARD);
-        if (f32) launch_ex(ctx, ABS_KC_LSQ, lnet::local_step_kernel<float>, dim3(bx, ctx->W), dim3(256), 0, q, u == q.U - 1 ? 1 : 0);
-        else launch_ex(ctx, ABS_KC_LSQ, lnet::local_step_kernel<__nv_bfloat16>, dim3(bx, ctx->W), dim3(256), 0, q, u == q.U - 1 ? 1 : 0);
+        if (f32) launch_ex(ctx, ABS_KC_LSQ, lnet::local_step_kernel<float>, dim3(bx, ctx->W), dim3(256), 0, q, u);
+        else launch_ex(ctx, ABS_KC_LSQ, lnet::local_step_kernel<__nv_bfloat16>, dim3(bx, ctx->W), dim3(256), 0, q, u);
       }
       update(par);
     }

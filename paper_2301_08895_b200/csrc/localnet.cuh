@@ -37,38 +37,9 @@ struct Args {
   float lr;
 };
 
-// Start of a job's local steps: the worker's copy is the model version it holds, its upload zero.
-template <typename T>
-__global__ void __launch_bounds__(256) local_begin_kernel(Args a) {
-  grid_dependency_sync();
-  const DevState* st = a.st;
-  const RoundInfo* ri = a.ri;
-  if (st->status != ST_OK) return;
-  const int i = blockIdx.y;
-  if (i >= ri->K) return;
-  const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
-  const uint4* src = reinterpret_cast<const uint4*>((const T*)a.ring + (size_t)slot * a.d_pad);
-  uint4* dst = reinterpret_cast<uint4*>((T*)a.priv + (size_t)i * a.d_pad);
-  float4* gs = reinterpret_cast<float4*>(a.gsum + (size_t)i * a.d_pad);
-  const size_t n16 = a.d_pad * sizeof(T) / 16, n4 = a.d_pad / 4;
-  for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < n4; v += (size_t)gridDim.x * blockDim.x) {
-    if (v < n16) dst[v] = src[v];
-    gs[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  if (blockIdx.x == 0 && threadIdx.x == 0) a.loss_acc[i] = 0.f;
-}
-
-// Row layout of local step u: sample indices of every selected worker's minibatch, the owner of
-// every row tile, and the row count of the pass.
-__global__ void __launch_bounds__(128) local_layout_kernel(Args a, int u) {
-  grid_dependency_sync();
-  const DevState* st = a.st;
-  RoundInfo* ri = a.ri;
-  if (st->status != ST_OK) return;
-  const int K = ri->K;
-  if (blockIdx.x == 0 && threadIdx.x == 0) ri->n_rows = K * a.RBp;
-  const int i = blockIdx.x;
-  if (i >= K) return;
+// Row layout of local step u for selected worker i (one block): the sample indices of its minibatch
+// and the owner of its row tiles.
+__device__ __forceinline__ void write_layout(const Args& a, const DevState* st, int i, int u) {
   const int B = st->B, W = st->W, RB = st->RB;
   const int wn = a.sel[i], jb = a.job[wn];
   const i64 M = st->n_samples;
@@ -90,6 +61,32 @@ __global__ void __launch_bounds__(128) local_layout_kernel(Args a, int u) {
   for (int q = threadIdx.x; q < tiles; q += blockDim.x) a.tile_slot[i * tiles + q] = i;
 }
 
+// Start of a job's local steps: the worker's copy is the model version it holds, its upload zero;
+// block (0, i) also writes the row layout of step 0 (and block (0, 0) the row count of the passes).
+template <typename T>
+__global__ void __launch_bounds__(256) local_begin_kernel(Args a) {
+  grid_dependency_sync();
+  const DevState* st = a.st;
+  RoundInfo* ri = a.ri;
+  if (st->status != ST_OK) return;
+  const int i = blockIdx.y;
+  if (i >= ri->K) return;
+  if (blockIdx.x == 0) {
+    if (i == 0 && threadIdx.x == 0) ri->n_rows = ri->K * a.RBp;
+    write_layout(a, st, i, 0);
+  }
+  const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
+  const uint4* src = reinterpret_cast<const uint4*>((const T*)a.ring + (size_t)slot * a.d_pad);
+  uint4* dst = reinterpret_cast<uint4*>((T*)a.priv + (size_t)i * a.d_pad);
+  float4* gs = reinterpret_cast<float4*>(a.gsum + (size_t)i * a.d_pad);
+  const size_t n16 = a.d_pad * sizeof(T) / 16, n4 = a.d_pad / 4;
+  for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < n4; v += (size_t)gridDim.x * blockDim.x) {
+    if (v < n16) dst[v] = src[v];
+    gs[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) a.loss_acc[i] = 0.f;
+}
+
 // Output-layer gradient of every worker, added to its upload: dst_i[j] += sum over the worker's row
 // chunks, in order, of part[q][j].  One thread per output (a worker has only RBp / chunk_rows chunks).
 __global__ void __launch_bounds__(256) chunk_reduce_worker_kernel(const DevState* st, const RoundInfo* ri, const float* part, int len,
@@ -109,9 +106,9 @@ __global__ void __launch_bounds__(256) chunk_reduce_worker_kernel(const DevState
 // After step u (Eq. 2 unrolled): w_i^{u+1} = w_i^0 - eta / B * (sum of the gradient sums so far), written
 // as the copy the next step reads (skipped after the last step); block (0, i) also adds the
 // step's mean loss and, after the last step, writes the uploaded loss (the average of the U mean
-// minibatch losses; Algorithm 1, last worker line).
+// minibatch losses; Algorithm 1, last worker line) or else the row layout of step u + 1.
 template <typename T>
-__global__ void __launch_bounds__(256) local_step_kernel(Args a, int last) {
+__global__ void __launch_bounds__(256) local_step_kernel(Args a, int u) {
   grid_dependency_sync();
   __shared__ float red[8];
   const DevState* st = a.st;
@@ -120,7 +117,9 @@ __global__ void __launch_bounds__(256) local_step_kernel(Args a, int last) {
   const int i = blockIdx.y;
   if (i >= ri->K) return;
   const int B = st->B;
+  const int last = u == a.U - 1;
   if (!last) {
+    if (blockIdx.x == 0) write_layout(a, st, i, u + 1);
     const float step = __fdiv_rn(a.lr, (float)B);
     const int slot = (ri->t - a.sel_tau[i]) % (st->S + 1);
     const T* w0 = (const T*)a.ring + (size_t)slot * a.d_pad;
