@@ -372,13 +372,13 @@ def main():
             per_par = 4.0 + 2.0 * (2 if bf16 else 4)
             bytes_l = per_par * d_pad * float(np.mean(ks[:n_rounds_prof]))   # per refresh launch: bytes x d x K^t
             # the class also holds the begin and layout kernels (1 + U launches per round, small)
-            out["roofline"] = {"bound": "hbm", "kernel": "local_step_kernel (+ local_begin / local_layout launches)",
+            out["roofline"] = {"bound": "hbm", "kernel": "local_step_kernel (+ local_begin launches)",
                                "launches": n_l, "avg_us": 1e3 * t_l / max(1, n_l),
                                "achieved": bytes_l * n_upd / (t_l * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": bytes_l * n_upd / (t_l * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
                                "peak_source": peaks["source"], "share_of_profiled_time": t_l / tot_prof,
                                "note": "algorithmic bytes of the U - 1 copy refreshes per round only, over the time of the "
-                                       "whole class (begin, layout and last-step launches included)"}
+                                       "whole class (begin and last-step launches included)"}
         else:
             out["roofline"] = {"bound": "latency", "kernel": "local_sgd_kernel", "achieved": None, "peak": None,
                                "unit": None, "frac": None, "traffic": None,
