@@ -208,7 +208,8 @@ class ABSOracle:
         """Upload of worker n's current job (Eq. 2): the average of the U mean
         minibatch losses and the sum of the U mean minibatch gradients along the
         worker's local trajectory, which starts at the model version it holds."""
-        w_local = np.array(self.versions[self.version[n]], dtype=np.float64)
+        held = self.versions[self.version[n]]        # the stored copy the worker downloaded
+        w_local = np.array(held, dtype=np.float64)
         loss_sum, grad_sum = 0.0, np.zeros_like(w_local)
         for u in range(self.local_steps):
             idx = minibatch_indices(self.seed, n, self.job[n], self.batch, self.W, self.M, step=u)
@@ -217,8 +218,10 @@ class ABSOracle:
             if self.kind == models.LSQ:
                 yb = yb.astype(np.float64)
             # bf16 configurations compute every step with the 16-bit rounding of the local copy
-            # (the copy itself keeps full precision); at step 0 that is the downloaded model
-            loss, grad = models.loss_grad(self.kind, self.dims, self._stored(w_local), Xb, yb, quant=self.quant)
+            # (the copy itself keeps full precision); at step 0 that is the downloaded model, which
+            # is stored rounded already (rounding it again would change nothing)
+            w_eval = held if u == 0 else self._stored(w_local)
+            loss, grad = models.loss_grad(self.kind, self.dims, w_eval, Xb, yb, quant=self.quant)
             loss_sum += loss
             grad_sum += grad
             if u + 1 < self.local_steps:

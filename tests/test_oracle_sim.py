@@ -443,3 +443,38 @@ def test_local_steps_soft_max_against_finite_differences_of_the_chain():
         total += g
         w = w - lr * g
     assert np.allclose(grad_sum, total, atol=1e-7)
+
+
+def test_bf16_local_steps_round_the_evaluation_point_not_the_copy():
+    """Eq. 2 with 16-bit stored models, three local steps worked by hand.
+
+    One worker, one sample x = 1, y = 0, so f(w) = w^2 / 2, the minibatch gradient is the
+    model value the step is evaluated at, and every minibatch is that sample.  eta = 3/1024,
+    w^{.,0} = 1.  bfloat16 has spacing 2^-8 just below 1.
+      step 0: evaluated at 1                      -> g0 = 1,          copy -> 1 - 3/1024
+      step 1: the copy 1 - 0.75 * 2^-8 is evaluated at its rounding 1 - 2^-8 = 0.99609375
+              -> g1 = 0.99609375, copy (kept unrounded) -> 1 - 3/1024 - (3/1024) * 0.99609375
+      step 2: that copy is 1 - 1.497 * 2^-8 and rounds to 1 - 2^-8 again -> g2 = 0.99609375
+    Without the rounding g1 would be 1 - 3/1024; with the copy itself rounded after step 1,
+    step 2 would start from 0.99609375 * (1 - 3/1024) = 1 - 1.747 * 2^-8, which rounds to
+    1 - 2^-7, so g2 would be 0.9921875.
+    """
+    lr = 3.0 / 1024.0
+    X, y = np.array([[1.0]]), np.array([0.0], dtype=np.float32)
+    o = abs_sim.ABSOracle(models.LSQ, (1, 1), X, y, np.array([1.0]), 1, lr, 1, 1, 0,
+                          timing.TimeDist(timing.CONST, shift=1.0), 3, quant=True, local_steps=3)
+    loss, g = o.upload(0)
+    g0, g1, g2 = 1.0, 0.99609375, 0.99609375
+    assert g[0] == g0 + g1 + g2 == 2.9921875
+    assert loss == (0.5 * g0 * g0 + 0.5 * g1 * g1 + 0.5 * g2 * g2) / 3.0
+    # the two other readings give other numbers (the pin has teeth)
+    assert g[0] != 1.0 + (1.0 - lr) + 0.99609375
+    assert g[0] != 1.0 + 0.99609375 + 0.9921875
+    # Eq. 3 with the upload: w^1 = w^0 - eta * (g0 + g1 + g2)
+    o.round()
+    assert o.w[0] == 1.0 - lr * 2.9921875
+    # full precision (fp32 configurations): plain chained steps
+    o2 = abs_sim.ABSOracle(models.LSQ, (1, 1), X, y, np.array([1.0]), 1, lr, 1, 1, 0,
+                           timing.TimeDist(timing.CONST, shift=1.0), 3, quant=False, local_steps=3)
+    _, gf = o2.upload(0)
+    assert gf[0] == 1.0 + (1.0 - lr) + (1.0 - lr) * (1.0 - lr)
