@@ -40,7 +40,7 @@ extern "C" {
 #define ABS_EUNSUPPORTED -3  /* unknown kind, or local_steps > 1 for a model the local-step kernel does not cover */
 #define ABS_ESTATE       -4  /* call order */
 #define ABS_ECUDA        -5  /* a CUDA call failed; sticky for the context */
-#define ABS_ETIMEOUT     -6  /* a bounded device-side wait expired */
+#define ABS_ETIMEOUT     -6  /* a bounded device-side wait (100 ms) expired */
 #define ABS_EDIVERGED    -7  /* a non-finite loss was uploaded; see abs_run_rounds */
 #define ABS_ERANGE       -8  /* simulated time left the 2^53 tick range */
 
@@ -277,6 +277,16 @@ int abs_profile_read(abs_ctx* ctx, long long* launches, double* total_ms);
  * class and the times of the two bracketing events in ms since the first recorded launch.  The
  * arrays need `cap` entries; *n_out receives the number filled.  Synchronises. */
 int abs_profile_timeline(abs_ctx* ctx, int cap, int* cls, float* start_ms, float* end_ms, int* n_out);
+
+/* Test aid for the failure path of the device-side waits (the paper has no counterpart).  Every wait
+ * inside the library's kernels (on an mbarrier or a completion counter) gives up after a time limit,
+ * raises the context's device status and lets the kernel return normally.  This call launches a
+ * one-warp kernel that waits, with the library's own wait routine and a limit of limit_us
+ * microseconds (1 .. 1000000), on a barrier that nothing ever signals, then synchronises.  It is
+ * expected to return ABS_ETIMEOUT (abs_last_error names site 900); the context is then in the same
+ * sticky state as after a real expiry: no further rounds, while abs_get_params, abs_get_trace and
+ * abs_destroy keep working.  Nothing faults, traps or hangs. */
+int abs_selftest_wait_timeout(abs_ctx* ctx, int limit_us);
 
 int abs_destroy(abs_ctx* ctx);
 

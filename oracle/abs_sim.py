@@ -28,6 +28,14 @@ t = 0, 1, ... of Algorithm 1 with U = 1 local step:
   7. the communication counter grows by one per worker that talks to the
      server (Sec. V-B).
 
+Comparison systems of the paper's evaluation (Sec. I, Sec. II-B, Sec. V) in the same loop:
+  * AdaSync: K adapts as above but no worker is ever forced to restart (`restarts=False`), so
+    the staleness of a consumed gradient is unbounded; the oracle keeps every model version
+    some worker still holds.
+  * Staleness-aware step size (SA): a stale gradient's step size is penalised linearly in its
+    delay (`sa_penalty=True`): upload k enters Eq. 3 as g_k / max(1, tau_k).  SA-AdaSync is
+    both switches together.
+
 Symbols: N workers (W in the code), K, S, theta, B, eta as in the paper.
 `version[n]` is the round index of the model worker n holds, so its age is
 t - version[n].  Times are integer ticks (module `timing`).
@@ -151,12 +159,15 @@ class ABSOracle:
     integer_only   play only the server's integer machinery (arrivals, Eq. 4-6,
                    ticks): no gradient is evaluated and the model stays at w^0;
                    every round must then be given its uploaded losses
+    restarts       False: Eq. 6 never forces a restart (AdaSync, K-async SGD): ages grow until
+                   the worker's own upload arrives; the threshold is still computed and recorded
+    sa_penalty     staleness-aware step size: upload k is divided by max(1, tau_k) in Eq. 3
     """
 
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, dist, seed,
                  quant=False, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE,
                  literal_eq6=False, x_is_bf16_bits=False, integer_only=False, bound_offset=0,
-                 local_steps=1):
+                 local_steps=1, restarts=True, sa_penalty=False):
         if not (1 <= K0 <= W):
             raise ValueError("need 1 <= K0 <= W")
         if S < 0:
@@ -178,6 +189,8 @@ class ABSOracle:
             raise ValueError("staleness bound below the initial threshold N/K0 + a")
         self.literal_eq6 = literal_eq6
         self.integer_only = integer_only
+        self.restarts = bool(restarts)
+        self.sa_penalty = bool(sa_penalty)
         self.w = np.array(w0, dtype=np.float64)
         assert self.w.shape[0] == models.n_params(kind, dims)
         # the oracle may keep every past model; the bound is what lets a real
@@ -253,9 +266,11 @@ class ABSOracle:
             assert forced_losses is not None and len(forced_losses) == K
             own_losses = [np.float32(x) for x in forced_losses]
         else:
-            for n in arrivals:
+            for n, tau in zip(arrivals, taus):
                 loss, grad = self.upload(n)
                 own_losses.append(np.float32(loss))
+                if self.sa_penalty:
+                    grad = grad / max(1, tau)          # step size penalised linearly in the delay
                 grad_sum += grad
         losses = own_losses if forced_losses is None else \
             [np.float32(x) for x in forced_losses]
@@ -288,7 +303,7 @@ class ABSOracle:
                 continue
             age_now = t - self.version[n]
             over = (age_now > theta) if self.literal_eq6 else (age_now + 1 > theta)
-            if over:
+            if over and self.restarts:
                 restarted.append(n)
         for n in arrivals + restarted:
             self._start_job(n, T_end)

@@ -100,6 +100,7 @@ def lib():
         l.abs_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
         l.abs_profile_timeline.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.POINTER(C.c_int)]
+        l.abs_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_int]
         l.abs_destroy.argtypes = [C.c_void_p]
         _lib = l
     return _lib
@@ -278,6 +279,10 @@ class Context:
         _check(lib().abs_profile_timeline(self._ctx, cap, cls.ctypes.data, t0.ctypes.data,
                                           t1.ctypes.data, C.byref(n)))
         return [(KC_NAMES[cls[i]], float(t0[i]), float(t1[i])) for i in range(n.value)]
+
+    def selftest_wait_timeout(self, limit_us=1000):
+        """abs_selftest_wait_timeout: lets a bounded device wait run out; raises AbsError(ETIMEOUT)."""
+        _check(lib().abs_selftest_wait_timeout(self._ctx, int(limit_us)))
 
     def close(self):
         if self._ctx:

@@ -1408,6 +1408,19 @@ int abs_profile_timeline(abs_ctx* ctx, int cap, int* cls, float* start_ms, float
   return ABS_OK;
 }
 
+int abs_selftest_wait_timeout(abs_ctx* ctx, int limit_us) {
+  if (!ctx) return fail(ABS_EINVAL, "ctx is null");
+  if (ctx->sticky != ABS_OK) return fail(ctx->sticky, "context is in a failed state (%d)", ctx->sticky);
+  if (limit_us < 1 || limit_us > 1000000) return fail(ABS_EINVAL, "limit_us %d outside [1, 1000000]", limit_us);
+  tc::wait_selftest_kernel<<<1, 32, 0, ctx->stream>>>(ctx->at<DevState>(ctx->L.st), 1000ull * (unsigned long long)limit_us);
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  DevState h;
+  const int rc = read_status(ctx, &h);
+  if (rc != ABS_OK) return rc;
+  return status_to_code(ctx, h);
+}
+
 int abs_destroy(abs_ctx* ctx) {
   if (!ctx) return ABS_OK;
   cudaStreamSynchronize(ctx->stream);

@@ -10,7 +10,7 @@
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the tensor-memory allocation),
 // warps 2..9 = epilogue (tensor memory -> registers -> global; two warps per tensor-memory lane
 // quarter, each draining one half of the tile's columns).  Two accumulators alternate so the
-// epilogue of one tile overlaps the main loop of the next.  Every mbarrier wait is bounded; on
+// epilogue of one tile overlaps the main loop of the next.  Every mbarrier wait is bounded (WAIT_LIMIT_NS); on
 // expiry the CTA raises ST_TIMEOUT, drains its own copies, frees tensor memory and returns.
 #pragma once
 #include <cuda.h>
@@ -82,16 +82,21 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait (about two seconds, and never more than 2^28 polls).  False = gave up, or another
-// role of this CTA already gave up; *abort is the CTA-wide flag.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+// Longest time a kernel of the round loop waits on a barrier or a counter: 100 ms, thousands of
+// times the longest tile, and short enough that a wait that can never end costs a shared GPU
+// next to nothing.
+constexpr unsigned long long WAIT_LIMIT_NS = 100000000ull;
+// Bounded wait (limit_ns, and never more than 2^28 polls).  False = gave up, or another role of
+// this CTA already gave up; *abort is the CTA-wide flag.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
   if (mbar_test(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t i = 1; i < (1u << 28); ++i) {
     if (mbar_test(bar, parity)) return true;
     if ((i & 63u) == 0u) {
       if (*abort) return false;
-      if (global_ns() - t0 > 2000000000ull) break;
+      if (global_ns() - t0 > limit_ns) break;
     }
   }
   *abort = 1;
@@ -438,7 +443,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
               for (uint32_t spin = 0;; ++spin) {
                 asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(dw + c.rt) : "memory");
                 if (seen >= target) break;
-                if ((spin & 63u) == 63u && (*abort || global_ns() - t0 > 2000000000ull)) { *abort = 1; ok = false; break; }
+                if ((spin & 63u) == 63u && (*abort || global_ns() - t0 > WAIT_LIMIT_NS)) { *abort = 1; ok = false; break; }
               }
               if (!ok) break;
               asm volatile("fence.proxy.async;" ::: "memory");
@@ -542,7 +547,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         for (int s = 0; s < C::STAGES; ++s)
           if (armed[s] >= 0) {
             const unsigned long long t0 = global_ns();
-            while (!mbar_test(&full[s], (uint32_t)armed[s]) && global_ns() - t0 < 100000000ull) {}
+            while (!mbar_test(&full[s], (uint32_t)armed[s]) && global_ns() - t0 < WAIT_LIMIT_NS) {}
           }
       }
     }
@@ -791,6 +796,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   }
   if (threadIdx.x == 0 && *abort) {
     st->timeout_where = 100 + p0.mode;
+    st->status = ST_TIMEOUT;
+  }
+}
+
+// Self-test of the bounded wait: one warp initialises a barrier that expects one arrival, nobody
+// ever arrives, and lane 0 waits on it with the given limit.  The wait must give up, and the
+// kernel then reports it the way the round-loop kernels do (status word + site), and returns.
+constexpr int TIMEOUT_SITE_SELFTEST = 900;
+__global__ void wait_selftest_kernel(DevState* st, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && !mbar_wait(&bar, 0u, &abort_flag, limit_ns)) {
+    st->timeout_where = TIMEOUT_SITE_SELFTEST;
     st->status = ST_TIMEOUT;
   }
 }

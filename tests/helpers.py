@@ -43,6 +43,35 @@ def rel_l2(a, b):
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
 
 
+def layer_blocks(kind, dims):
+    """(name, slice) of every W_l and b_l inside the flat parameter vector (layout of w0)."""
+    if kind == inputs.LSQ:
+        return [("w", slice(0, dims[0]))]
+    out, off = [], 0
+    for l in range(len(dims) - 1):
+        n_w, n_b = dims[l] * dims[l + 1], dims[l + 1]
+        out.append(("W%d" % (l + 1), slice(off, off + n_w)))
+        out.append(("b%d" % (l + 1), slice(off + n_w, off + n_w + n_b)))
+        off += n_w + n_b
+    return out
+
+
+def assert_params_close(cfg, params, ref, tol):
+    """Relative L2 of the whole vector and of every layer block (each W_l, each b_l) within tol:
+    a wrong bias vector moves the norm of millions of weights by less than any tolerance, so the
+    whole-vector figure alone would not see it."""
+    err = rel_l2(params, ref)
+    assert err <= tol, "parameters differ: rel L2 %.3g > %.3g" % (err, tol)
+    ref = np.asarray(ref, np.float64)
+    for name, sl in layer_blocks(cfg.kind, cfg.dims):
+        if np.linalg.norm(ref[sl]) == 0.0:
+            assert np.linalg.norm(np.asarray(params, np.float64)[sl]) == 0.0, "block %s should be zero" % name
+            continue
+        e = rel_l2(np.asarray(params)[sl], ref[sl])
+        assert e <= tol, "parameter block %s differs: rel L2 %.3g > %.3g" % (name, e, tol)
+    return err
+
+
 def compare_with_oracle(cfg, X, y, w0, rounds, tol, forced=False, loss_tol=None, **kw):
     """GPU run vs oracle run.  forced=False: both run freely and the integer
     traces must be identical.  forced=True: the oracle's K rule is fed the
@@ -58,8 +87,7 @@ def compare_with_oracle(cfg, X, y, w0, rounds, tol, forced=False, loss_tol=None,
     mm = first_integer_mismatch(rows, orows)
     assert mm is None, "integer trace differs at round %s field %s: gpu %s oracle %s (oracle " \
         "decision margin %.3g)" % (mm + (o.min_margin,))
-    err = rel_l2(params, o.w)
-    assert err <= tol, "parameters differ: rel L2 %.3g > %.3g" % (err, tol)
+    err = assert_params_close(cfg, params, o.w, tol)
     lt = loss_tol if loss_tol is not None else tol * 10
     for t, (a, b) in enumerate(zip(rows, orows)):
         la, lb = np.array(a["sel_loss"]), np.array(b["sel_loss"])

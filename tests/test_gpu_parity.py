@@ -392,6 +392,18 @@ def test_paired_forward_launch_matches_separate_launches(dims, W, B):
     compare_with_oracle(cfg, X, y, w0, 12, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_FUSED_FORWARD)
 
 
+def test_bf16_network_without_tensor_cores():
+    """ABS_FLAG_NO_TENSOR_CORES: the hidden layers of a bf16 network on the FP32-FMA tile kernels
+    (same storage points, other summation order)."""
+    cfg = _small_cfg(inputs.MLP, (320, 520, 264, 10), inputs.BF16, 13, 40, 3, 5, PARETO)
+    X, y, w0 = _problem(cfg)
+    Xd, yd = to_device(cfg, X, y)
+    ctx = gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=1, flags=gpu.FLAG_NO_TENSOR_CORES)
+    assert ctx.plan()["path"] == [0, 0, 2]        # no layer on the tensor-core path
+    ctx.close()
+    compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_NO_TENSOR_CORES)
+
+
 def test_cta_pair_gemms_match_single_cta_gemms():
     """Opt-in tcgen05 cta_group::2 tiles (256 x 256 over a CTA pair) against the default tiles."""
     cfg = _small_cfg(inputs.MLP, (320, 520, 264, 10), inputs.BF16, 13, 40, 3, 5, PARETO)

@@ -478,3 +478,95 @@ def test_bf16_local_steps_round_the_evaluation_point_not_the_copy():
                            timing.TimeDist(timing.CONST, shift=1.0), 3, quant=False, local_steps=3)
     _, gf = o2.upload(0)
     assert gf[0] == 1.0 + (1.0 - lr) + (1.0 - lr) * (1.0 - lr)
+
+
+# ---------------------------------------------------------------- comparison systems (Sec. II-B, Sec. V)
+def test_staleness_aware_step_size_by_hand():
+    """SA penalises a stale gradient's step size linearly in its delay (Sec. I).  Three workers in
+    lock step (constant times, K = 1): the arriving gradient has staleness min(t, 2).  One sample
+    x = 1, y = 0, so f = w^2 / 2 and a gradient is the model value it was computed at; eta = 1/4.
+      w^1 = 1 - 1/4 (tau 0) = 3/4;  w^2 = 3/4 - 1/4 * w^0 (tau 1) = 1/2;
+      w^3 = 1/2 - 1/4 * w^0 / 2 (tau 2) = 3/8;  w^4 = 3/8 - 1/4 * w^1 / 2 (tau 2) = 9/32.
+    Without the penalty the last two steps are whole: w^3 = 1/4, w^4 = 1/16."""
+    X, y = np.ones((3, 1)), np.zeros(3)
+    dist = timing.TimeDist(timing.CONST, shift=1.0)
+    kw = dict(k_mode=K_FIXED, bound_mode=BOUND_FIXED)
+    o = ABSOracle(models.LSQ, [1, 1], X, y, np.array([1.0]), 1, 0.25, 3, 1, 2, dist, 5, sa_penalty=True, **kw)
+    seen = []
+    for row in (o.round() for _ in range(4)):
+        seen.append(o.w[0])
+        assert row["restart"] == []
+    assert [r["tau"] for r in o.trace] == [[0], [1], [2], [2]]
+    assert seen == [0.75, 0.5, 0.375, 0.28125]
+    o = ABSOracle(models.LSQ, [1, 1], X, y, np.array([1.0]), 1, 0.25, 3, 1, 2, dist, 5, **kw)
+    o.run(4)
+    assert o.w[0] == 0.0625
+
+
+def test_staleness_aware_step_size_changes_nothing_without_staleness():
+    """With bound 0 every consumed gradient has age 0 and with bound 1 at most 1: the penalty
+    1 / max(1, tau) is then 1 and the run is ABS bit for bit."""
+    X, y, _ = _lsq_problem()
+    dist = timing.TimeDist(timing.SHIFTED_EXP, shift=1.0, rate=1.0)
+    for S in (0, 1):
+        a = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 6, 2, S, dist, 9)
+        b = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 6, 2, S, dist, 9, sa_penalty=True)
+        assert a.run(40) == b.run(40) and np.array_equal(a.w, b.w)
+    # and with real staleness it does change the model, never the integer decisions of a fixed-K run
+    a = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 6, 2, 4, dist, 9, k_mode=K_FIXED)
+    b = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 6, 2, 4, dist, 9, k_mode=K_FIXED, sa_penalty=True)
+    ra, rb = a.run(40), b.run(40)
+    assert max(max(r["tau"]) for r in ra) >= 2
+    assert [(r["sel"], r["tau"], r["restart"]) for r in ra] == [(r["sel"], r["tau"], r["restart"]) for r in rb]
+    assert not np.array_equal(a.w, b.w)
+
+
+def test_without_restarts_equals_abs_while_no_restart_would_fire():
+    """AdaSync is the loop without Eq. 6's forced restarts.  With a bound so large that Eq. 6 never
+    fires, both runs are the same; with a small bound they part at the first restart."""
+    X, y, _ = _lsq_problem()
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    a = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 8, 2, 200, dist, 4, bound_mode=BOUND_FIXED)
+    b = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 8, 2, 200, dist, 4, bound_mode=BOUND_FIXED, restarts=False)
+    ra, rb = a.run(60), b.run(60)
+    assert all(r["restart"] == [] for r in ra) and ra == rb and np.array_equal(a.w, b.w)
+    a = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 8, 2, 2, dist, 4, k_mode=K_FIXED)
+    b = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.05, 8, 2, 2, dist, 4, k_mode=K_FIXED, restarts=False)
+    ra, rb = a.run(60), b.run(60)
+    first = next(t for t, r in enumerate(ra) if r["restart"])
+    assert ra[:first] == rb[:first]
+    assert all(r["restart"] == [] for r in rb)
+    assert max(max(r["tau"]) for r in rb) > 2 >= max(max(r["tau"]) for r in ra)     # unbounded vs bounded
+    # communication counter: only the K uploads per round (Sec. V-B)
+    assert rb[-1]["comm"] == 8 + 2 * 60
+
+
+def test_without_restarts_a_straggler_arrives_with_its_full_age():
+    """One worker 50 times slower than the others, K = 2 of 5, constant times: with restarts it
+    would be sent the fresh model every theta + 1 rounds; without, it keeps computing on w^0 and
+    its upload is consumed with the age it has then (K-async SGD, Sec. I)."""
+    X, y, _ = _lsq_problem()
+    W, K = 5, 2
+    dist = timing.TimeDist(timing.CONST, shift=1.0, slow_mod=W, slow_rem=4, slow_factor=50.0)
+    o = ABSOracle(models.LSQ, [6, 1], X, y, np.zeros(6), 4, 0.01, W, K, 3, dist, 1,
+                  k_mode=K_FIXED, bound_mode=BOUND_FIXED, restarts=False)
+    rows = o.run(120)
+    hits = [(t, r["tau"][r["sel"].index(4)]) for t, r in enumerate(rows) if 4 in r["sel"]]
+    # the four fast workers finish one job per time unit: two rounds per unit, so the slow job
+    # (50 units) arrives in round 100 at the latest, with staleness equal to the round index
+    assert hits and hits[0][1] == hits[0][0] and 96 <= hits[0][0] <= 100
+    assert all(r["restart"] == [] for r in rows)
+
+
+def test_k_async_without_restarts_statistics():
+    """K = 1, no restarts, i.i.d. exponential times: the arriving worker is uniform (memoryless),
+    so the consumed staleness is geometric with mean N - 1 whatever the bound says."""
+    X, y, _ = _lsq_problem(d=3)
+    W, rounds = 5, 6000
+    dist = timing.TimeDist(timing.EXP, rate=1.0)
+    o = ABSOracle(models.LSQ, [3, 1], X, y, np.zeros(3), 2, 0.01, W, 1, 1, dist, 3,
+                  k_mode=K_FIXED, restarts=False, sa_penalty=True)
+    rows = o.run(rounds)
+    taus = np.array([row["tau"][0] for row in rows[200:]])
+    assert abs(taus.mean() - (W - 1)) < 5 * math.sqrt(W * (W - 1) / len(taus))
+    assert taus.max() > 10

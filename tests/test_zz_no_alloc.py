@@ -15,6 +15,7 @@ from a run that stops at the first failure.
 import numpy as np
 import pytest
 
+from oracle import models
 from paper_2301_08895_b200 import abs as gpu
 
 pytestmark = pytest.mark.gpu
@@ -32,6 +33,18 @@ def _inputs(n, B, d, bf16, seed):
     return X.to(dt).cuda(), y.cuda(), w.to(dt).cuda(), idx.cuda()
 
 
+def _oracle(X, y, w, idx):
+    """Eq. 2 (U = 1) per worker and the mean of the uploads (the sum of Eq. 3 over n), by the oracle."""
+    Xh, yh = X.float().cpu().numpy().astype(np.float64), y.cpu().numpy().astype(np.float64)
+    wh, ih = w.float().cpu().numpy().astype(np.float64), idx.cpu().numpy()
+    losses, g = [], np.zeros(Xh.shape[1])
+    for i in range(ih.shape[0]):
+        loss, grad = models.lsq_loss_grad(wh, Xh[ih[i]], yh[ih[i]])
+        losses.append(loss)
+        g += grad
+    return g / ih.shape[0], np.array(losses)
+
+
 def _both(n, B, d, bf16, seed):
     import torch
     X, y, w, idx = _inputs(n, B, d, bf16, seed)
@@ -40,16 +53,20 @@ def _both(n, B, d, bf16, seed):
     gpu.lsq_gradient(X, y, w, idx, g_ref, l_ref, torch.empty(n * d, device="cuda"))
     gpu.lsq_gradient_noalloc(X, y, w, idx, g_new, l_new)
     torch.cuda.synchronize()
-    return g_ref.cpu().numpy(), l_ref.cpu().numpy(), g_new.cpu().numpy(), l_new.cpu().numpy()
+    g_o, l_o = _oracle(X, y, w, idx)
+    return g_ref.cpu().numpy(), l_ref.cpu().numpy(), g_new.cpu().numpy(), l_new.cpu().numpy(), g_o, l_o
 
 
 def test_noalloc_matches_scratch_variant_on_two_calls_in_a_row():
     # second call is smaller and of another type: stale partial sums of the first call sit right
     # behind (and under) the region it uses
     for n, B, d, bf16, seed in ((200, 32, 4096, True, 1), (37, 19, 301, False, 2)):
-        g_ref, l_ref, g_new, l_new = _both(n, B, d, bf16, seed)
+        g_ref, l_ref, g_new, l_new, g_o, l_o = _both(n, B, d, bf16, seed)
         assert np.linalg.norm(g_new - g_ref) <= 1e-5 * np.linalg.norm(g_ref)
         assert np.allclose(l_new, l_ref, rtol=1e-5, atol=0.0)
+        # and against the oracle itself, not only through the other entry point
+        assert np.linalg.norm(g_new - g_o) <= 1e-5 * np.linalg.norm(g_o)
+        assert np.allclose(l_new, l_o, rtol=2e-5, atol=1e-6)
         assert np.all(np.isfinite(g_new)) and not np.any(l_new == 7.0)
 
 
