@@ -30,8 +30,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) per launch at K = N on configuration 4, from ncu captures of the GEMM and the
 # Eq. 3 kernel (summaries under profiles/); each figure is valid only for the kernel source it was taken
 # from (first 16 hex digits of the file's sha256).
-TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.3e6, "file": "tc.cuh", "sha256_16": "b4893775bfc39d3d"},
-           "update": {"config": 4, "bytes_per_launch": 79.8e6, "file": "simt.cuh", "sha256_16": "089a55733700ff7d"}}
+TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 47.3e6, "file": "tc.cuh", "sha256_16": "b4893775bfc39d3d",
+                    "source": "ncu capture of the four GEMM launches of one round, profiles/tc_gemm_kernel_cfg4.md"},
+           "update": {"config": 4, "bytes_per_launch": 79.8e6, "file": "simt.cuh", "sha256_16": "089a55733700ff7d",
+                      "source": "ncu capture of two launches, profiles/update_kernel_cfg4.md"}}
 METRIC = "worker_gradients_per_sec"
 UNIT = "worker-gradients/s"
 
@@ -82,6 +84,19 @@ def n_params(cfg):
     return inputs.n_params(cfg.kind, cfg.dims)
 
 
+def padded_rows(tr, B, RB):
+    """Gradient rows the kernels process per round: the arrivals are grouped by staleness (= model
+    version) and every group's rows are padded to a multiple of RB, so that a row tile never
+    straddles two versions.  Returns (rows with padding, real rows) summed over the rounds."""
+    padded = real = 0
+    off, tau = tr["sel_off"], tr["sel_tau"]
+    for t in range(len(tr["K"])):
+        _, counts = np.unique(tau[off[t]:off[t + 1]], return_counts=True)
+        padded += int(sum((c * B + RB - 1) // RB * RB for c in counts))
+        real += int(counts.sum()) * B
+    return padded, real
+
+
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -129,14 +144,15 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ oracle (CPU) arm
-def oracle_for(cfg, X, y, w0, local_steps=1):
+def oracle_for(cfg, X, y, w0, local_steps=1, k_fixed=False):
     from oracle import abs_sim, timing
     ts = cfg.time
     bf16 = cfg.dtype == inputs.BF16
     return abs_sim.ABSOracle(cfg.kind, cfg.dims, X, y, w0, cfg.batch, cfg.lr, cfg.W, cfg.K0, cfg.S,
                              timing.TimeDist(ts.kind, ts.shift, ts.rate, ts.scale, ts.slow_mod,
                                              ts.slow_rem, ts.slow_factor, ts.shape),
-                             cfg.run_seed, quant=bf16, x_is_bf16_bits=bf16, local_steps=local_steps)
+                             cfg.run_seed, quant=bf16, x_is_bf16_bits=bf16, local_steps=local_steps,
+                             k_mode=abs_sim.K_FIXED if k_fixed else abs_sim.K_ADAPTIVE)
 
 
 def blas_threads():
@@ -148,10 +164,10 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def time_oracle(cfg, X, y, w0, rounds, budget_s, local_steps=1):
+def time_oracle(cfg, X, y, w0, rounds, budget_s, local_steps=1, k_fixed=False):
     """Runs the oracle on the first rounds of the workload until `budget_s` of CPU work is spent
     (at least 2 rounds, at most `rounds`)."""
-    o = oracle_for(cfg, X, y, w0, local_steps)
+    o = oracle_for(cfg, X, y, w0, local_steps, k_fixed)
     t0 = time.perf_counter()
     done = 0
     while done < rounds:
@@ -179,6 +195,8 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="ABS_FLAG_* bits passed to abs_init")
     ap.add_argument("--local-steps", type=int, default=1,
                     help="U of Eq. 2: local minibatch steps per job (configurations 1, 2 and 5)")
+    ap.add_argument("--k-fixed", type=int, default=None,
+                    help="run with K^t fixed at this value (ABS_K_FIXED, K0 = K): the many-version-groups regime")
     ap.add_argument("--samples", type=int, default=None,
                     help="dataset rows (default: the configuration's; smaller for profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work")
@@ -191,12 +209,15 @@ def main():
     cfg = inputs.config(args.config, args.workers)
     if args.samples:
         cfg = cfg.scaled(n_samples=args.samples)
+    if args.k_fixed:
+        cfg = cfg.scaled(K0=args.k_fixed)
     if world > 1:
         from paper_2301_08895_b200 import multi
         cfg.run_seed = multi.replica_seed(cfg.run_seed, rank)   # independent replicas, one per GPU
     rounds = args.rounds or cfg.rounds
     U = args.local_steps
-    config_obj = {"workload": workload_name(cfg, rounds) + (", U=%d local steps" % U if U > 1 else ""), "lr": cfg.lr,
+    config_obj = {"workload": workload_name(cfg, rounds) + (", U=%d local steps" % U if U > 1 else "") +
+                  (", K fixed" if args.k_fixed else ""), "lr": cfg.lr,
                   "parallelism": "replicas x%d (the round loop does not shard)" % world,
                   "l2": "flushed between steps (512 MiB write); per-round working set exceeds L2",
                   "reinit": "abs_init between steps, outside the device-timed region",
@@ -210,8 +231,8 @@ def main():
         per_step = max(2.0, min(args.cpu_budget, 150.0 / max(1, args.steps + args.warmup)))
         res = None
         for _ in range(args.warmup):
-            time_oracle(cfg, X, y, w0, rounds, min(per_step, 3.0), U)
-        vals = [time_oracle(cfg, X, y, w0, rounds, per_step, U) for _ in range(args.steps)]
+            time_oracle(cfg, X, y, w0, rounds, min(per_step, 3.0), U, bool(args.k_fixed))
+        vals = [time_oracle(cfg, X, y, w0, rounds, per_step, U, bool(args.k_fixed)) for _ in range(args.steps)]
         res = vals[-1]
         value = float(np.mean([v["value"] for v in vals]))
         res["value"] = value
@@ -250,13 +271,15 @@ def main():
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream(dev)
 
+    k_mode = gpu.K_FIXED if args.k_fixed else gpu.K_ADAPTIVE
+
     def new_ctx(host=False, flags=None):
         flags = args.flags if flags is None else flags
         if host:
             return gpu.context_from_config(cfg, Xh, yh, w0, max_rounds=rounds, data_on_host=True,
-                                           device=str(dev), flags=flags, local_steps=U)
+                                           device=str(dev), flags=flags, local_steps=U, k_mode=k_mode)
         return gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=rounds, device=str(dev), flags=flags,
-                                       local_steps=U)
+                                       local_steps=U, k_mode=k_mode)
 
     def device_step(profile=False):
         """One run; returns (ms on the stream, worker-gradients, launches, profile dict)."""
@@ -281,6 +304,7 @@ def main():
         wg = int(tr["K"].sum())
         launches = ctx.launch_count() - l0
         ks = tr["K"].copy()
+        plan["padded_rows"] = padded_rows(tr, cfg.batch, plan["row_block"]) if cfg.kind != inputs.LSQ else None
         ctx.close()
         return e0.elapsed_time(e1), wg, launches, prof, ks, plan
 
@@ -405,7 +429,8 @@ def main():
         peak = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
         out["roofline"] = {"bound": "tensor", "kernel": "tc_gemm_kernel (fwd+dgrad+wgrad launches)",
                            "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                           "traffic": measured_traffic("gemm", args.config, not args.samples), "peak_source": peaks["source"] + " (sustained bf16)",
+                           "traffic": measured_traffic("gemm", args.config, not args.samples and not args.k_fixed),
+                           "traffic_source": TRAFFIC["gemm"]["source"], "peak_source": peaks["source"] + " (sustained bf16)",
                            "frac_of_burst_peak": ach / peaks["bf16_tflops"],
                            "share_of_profiled_time": t_g / tot_prof,
                            # a layer's delta back-propagation may share the weight gradient's launch:
@@ -425,15 +450,27 @@ def main():
         P = plan["partials"] if plan["partials"] > 0 else float(np.mean(ks[:n_u]))
         bytes_launch = (8 + esz + 4 * P) * d
         ach = bytes_launch / (t_u / n_u * 1e-3) / 1e9
+        traffic_u = measured_traffic("update", args.config, not args.samples)
+        sec_u = t_u / n_u * 1e-3
         out["roofline_update"] = {"bound": "hbm", "kernel": "update_kernel", "launches": n_u,
                                   "avg_us": 1e3 * t_u / n_u, "partials": P,
                                   "bytes_per_launch": bytes_launch, "achieved": ach,
                                   "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                   "frac": ach / peaks["hbm_gbs"],
-                                  "traffic": measured_traffic("update", args.config, not args.samples)}
+                                  # the same launch time against the bytes Eq. 3 needs at the least (one gradient
+                                  # vector: P = 1) and against the DRAM bytes an ncu capture counted (the partial
+                                  # sums the GEMMs just wrote are partly still in L2)
+                                  "min_bytes_per_launch": (8 + esz + 4) * d,
+                                  "frac_min_bytes": (8 + esz + 4) * d / sec_u / 1e9 / peaks["hbm_gbs"],
+                                  "frac_dram": (traffic_u / sec_u / 1e9 / peaks["hbm_gbs"]) if traffic_u else None,
+                                  "traffic": traffic_u,
+                                  "traffic_source": TRAFFIC["update"]["source"] if traffic_u else None}
+    if plan.get("padded_rows"):
+        padded, real = plan["padded_rows"]
+        out["padded_row_ratio"] = padded / max(1, real)      # rows the GEMMs process / rows of real samples
     out["plan"] = plan
     out["_profiled_worker_gradients"] = wg_p
-    out["cpu_baseline"] = time_oracle(cfg, X, y, w0, rounds, args.cpu_budget, U)
+    out["cpu_baseline"] = time_oracle(cfg, X, y, w0, rounds, args.cpu_budget, U, bool(args.k_fixed))
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

@@ -43,6 +43,8 @@ extern "C" {
 #define ABS_ETIMEOUT     -6  /* a bounded device-side wait (100 ms) expired */
 #define ABS_EDIVERGED    -7  /* a non-finite loss was uploaded; see abs_run_rounds */
 #define ABS_ERANGE       -8  /* simulated time left the 2^53 tick range */
+#define ABS_ESTALE       -9  /* ABS_RESTART_NONE: an upload older than the staleness bound arrived, i.e. older than
+                                the model versions the context keeps; the rounds before it stay valid */
 
 /* model kinds: the sample loss f of Eq. 1 */
 #define ABS_LSQ      0  /* f = 1/2 (x.w - y)^2, dims = {d, 1}, no bias */
@@ -67,6 +69,12 @@ extern "C" {
 #define ABS_RESTART_EQ6        1 /* Eq. 6 as printed: the age before the increment is tested, so a worker restarts
                                    one round later and a consumed gradient may be staleness bound + 1 rounds old
                                    (the library then keeps one more model version) */
+#define ABS_RESTART_NONE       2 /* no forced restarts at all: AdaSync (with ABS_K_ADAPTIVE) and K-async SGD (with
+                                   ABS_K_FIXED), the comparison systems of Sec. II-B and Sec. V.  Staleness is then
+                                   unbounded in principle; the library still keeps staleness bound + 1 model
+                                   versions, and a run in which an older upload arrives ends with ABS_ESTALE at
+                                   that round (choose the bound, at most 255, above the staleness the time law
+                                   can produce).  The threshold of Eq. 4 is still computed and reported */
 
 /* execution-time laws (random execution times with stragglers, Sec. V-A) */
 #define ABS_T_CONST        0    /* shift */
@@ -102,13 +110,12 @@ extern "C" {
 #define ABS_KC_DGRAD   3  /* hidden-layer delta back-propagation */
 #define ABS_KC_WGRAD   4  /* weight gradient summed over the selected workers (Eq. 3) */
 #define ABS_KC_OUTPUT  5  /* output layer: forward + loss, its back-propagation and gradient */
-#define ABS_KC_BIAS    6  /* bias gradients */
-#define ABS_KC_LSQ     7  /* least-squares residual + gradient; with local_steps > 1: the workers' local steps
+#define ABS_KC_LSQ     6  /* least-squares residual + gradient; with local_steps > 1: the workers' local steps
                              (single-layer models), or their set-up, row layouts and copy refreshes (networks) */
-#define ABS_KC_UPDATE  8  /* Eq. 3 step + ring write */
-#define ABS_KC_ROUNDS  9  /* whole rounds (control step + Eq. 2 + Eq. 3) of a small least-squares problem
+#define ABS_KC_UPDATE  7  /* Eq. 3 step + ring write */
+#define ABS_KC_ROUNDS  8  /* whole rounds (control step + Eq. 2 + Eq. 3) of a small least-squares problem
                              in one persistent kernel; one launch per abs_enqueue_rounds call */
-#define ABS_KC_COUNT   10
+#define ABS_KC_COUNT   9
 
 #define ABS_MAX_LAYERS   7
 #define ABS_MAX_WORKERS  1024
@@ -137,6 +144,9 @@ typedef struct {
   int bound_offset;         /* the constant a of Eq. 4 when bound_mode = ABS_BOUND_OFFSET (else ignored);
                                floor(N/K0) + a must not exceed the staleness bound */
   int restart_rule;         /* ABS_RESTART_* */
+  int sa_penalty;           /* 0 | 1.  1: staleness-aware step size (Sec. I, Sec. V: "SA"): the step size of a stale
+                               gradient is penalised linearly in its delay, i.e. upload k enters the sum of Eq. 3
+                               as g_k / max(1, tau_k).  With ABS_RESTART_NONE this is SA-AdaSync */
   int max_rounds;           /* trace capacity: total rounds this context may run */
   int flags;                /* ABS_FLAG_* bits */
   int data_on_host;         /* 0: X, y are device pointers owned by the caller and must outlive
@@ -219,8 +229,9 @@ int abs_get_trace(abs_ctx* ctx, int first_round, int n_rounds, abs_trace* out_ho
  * nothing of the generators needs saving).  abs_state_bytes: size of the image.  abs_save_state:
  * synchronises the stream and writes the image to dst_host (cap bytes; ABS_ENOSPACE if too small);
  * *written receives its size.  abs_restore_state: loads an image into a context that abs_init
- * created with the same model sizes, dtype, W, K0, staleness bound, modes, time distribution,
- * seed and max_rounds (ABS_EINVAL otherwise, context unchanged); the context then continues with
+ * created with the same model kind and sizes, batch, step size, dtype, local steps, flags, W, K0,
+ * staleness bound, modes, time distribution, seed and max_rounds (ABS_EINVAL otherwise, context
+ * unchanged); the context then continues with
  * round `rounds completed in the image`, bit-identically to the context that saved it.  The
  * dataset, w0 and profiling state are not part of the image.  Host memory is the caller's. */
 int abs_state_bytes(abs_ctx* ctx, size_t* out);

@@ -13,13 +13,13 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libabs_b200.so")
 
-OK, EINVAL, ENOSPACE, EUNSUPPORTED, ESTATE, ECUDA, ETIMEOUT, EDIVERGED, ERANGE = \
-    0, -1, -2, -3, -4, -5, -6, -7, -8
+OK, EINVAL, ENOSPACE, EUNSUPPORTED, ESTATE, ECUDA, ETIMEOUT, EDIVERGED, ERANGE, ESTALE = \
+    0, -1, -2, -3, -4, -5, -6, -7, -8, -9
 LSQ, SOFTMAX, MLP = 0, 1, 2
 FP32, BF16_FP32MASTER = 0, 1
 K_ADAPTIVE, K_FIXED = 0, 1
 BOUND_ADAPTIVE, BOUND_FIXED, BOUND_OFFSET = 0, 1, 2
-RESTART_ALGORITHM1, RESTART_EQ6 = 0, 1
+RESTART_ALGORITHM1, RESTART_EQ6, RESTART_NONE = 0, 1, 2
 T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2, T_GAMMA = 0, 1, 2, 3, 4
 MAX_LAYERS = 7
 FLAG_NO_TENSOR_CORES = 1
@@ -30,14 +30,14 @@ FLAG_TMA_GATHER = 16
 FLAG_NO_BULK_PIPELINE = 32
 FLAG_NO_FUSED_BACKWARD = 64
 FLAG_FUSED_FORWARD = 128
-KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "bias", "lsq", "update", "rounds")
+KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "lsq", "update", "rounds")
 
 
 class ModelDesc(C.Structure):
     _fields_ = [("kind", C.c_int), ("n_layers", C.c_int), ("dims", C.c_int * (MAX_LAYERS + 1)),
                 ("batch", C.c_int), ("lr", C.c_float), ("dtype", C.c_int),
                 ("local_steps", C.c_int), ("k_mode", C.c_int), ("bound_mode", C.c_int),
-                ("bound_offset", C.c_int), ("restart_rule", C.c_int), ("max_rounds", C.c_int), ("flags", C.c_int), ("data_on_host", C.c_int),
+                ("bound_offset", C.c_int), ("restart_rule", C.c_int), ("sa_penalty", C.c_int), ("max_rounds", C.c_int), ("flags", C.c_int), ("data_on_host", C.c_int),
                 ("X", C.c_void_p), ("y", C.c_void_p), ("n_samples", C.c_longlong),
                 ("w0", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("stream", C.c_void_p)]
@@ -122,7 +122,7 @@ def n_params(kind, dims):
 
 
 def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-          local_steps=1, data_on_host=0, flags=0, bound_offset=0, restart_rule=0):
+          local_steps=1, data_on_host=0, flags=0, bound_offset=0, restart_rule=0, sa_penalty=0):
     m = ModelDesc()
     m.kind, m.n_layers = kind, len(dims) - 1
     for i, v in enumerate(dims):
@@ -133,6 +133,7 @@ def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mod
     m.flags = int(flags)
     m.bound_offset = int(bound_offset)
     m.restart_rule = int(restart_rule)
+    m.sa_penalty = int(sa_penalty)
     return m
 
 
@@ -155,14 +156,14 @@ class Context:
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, time, seed, max_rounds,
                  dtype=FP32, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE, local_steps=1,
                  data_on_host=False, stream=None, device="cuda:0", flags=0, bound_offset=0,
-                 restart_rule=0):
+                 restart_rule=0, sa_penalty=0):
         import torch
         self._torch = torch
         self.kind, self.dims, self.W, self.S = kind, list(dims), W, S
         self.max_rounds = max_rounds
         n_samples = X.shape[0]
         m = _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-                  local_steps, 1 if data_on_host else 0, flags, bound_offset, restart_rule)
+                  local_steps, 1 if data_on_host else 0, flags, bound_offset, restart_rule, sa_penalty)
         need = C.c_size_t(0)
         _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(need)))
         self.device = torch.device(device)

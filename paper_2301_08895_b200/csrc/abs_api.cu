@@ -111,7 +111,9 @@ int check_model(const abs_model_desc* m, int W, int S) {
   if (W < 1 || W > ABS_MAX_WORKERS) return fail(ABS_EINVAL, "W %d outside [1, %d]", W, ABS_MAX_WORKERS);
   if (m->n_samples < W) return fail(ABS_EINVAL, "fewer samples than workers");
   if (S < 0 || S > ABS_MAX_BOUND) return fail(ABS_EINVAL, "staleness_bound %d outside [0, %d]", S, ABS_MAX_BOUND);
-  if (m->restart_rule != ABS_RESTART_ALGORITHM1 && m->restart_rule != ABS_RESTART_EQ6) return fail(ABS_EINVAL, "restart_rule");
+  if (m->restart_rule != ABS_RESTART_ALGORITHM1 && m->restart_rule != ABS_RESTART_EQ6 && m->restart_rule != ABS_RESTART_NONE)
+    return fail(ABS_EINVAL, "restart_rule");
+  if (m->sa_penalty != 0 && m->sa_penalty != 1) return fail(ABS_EINVAL, "sa_penalty must be 0 or 1");
   if (m->restart_rule == ABS_RESTART_EQ6 && S + 1 > ABS_MAX_BOUND)
     return fail(ABS_EINVAL, "staleness_bound %d: Eq. 6 as printed keeps one more version, at most %d", S, ABS_MAX_BOUND - 1);
   return ABS_OK;
@@ -689,7 +691,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       else launch_ex(ctx, cls, simt_fwd_kernel<T, false>, dim3(grid), dim3(256), 0, la[l]);
       if (last) {
         LossArgs lo;
-        lo.st = st; lo.ri = ri; lo.row_idx = ctx->ctl.row_idx[par]; lo.labels = (const int*)ctx->y;
+        lo.st = st; lo.ri = ri; lo.tile_slot = ctx->ctl.tile_slot[par]; lo.row_idx = ctx->ctl.row_idx[par]; lo.labels = (const int*)ctx->y;
         lo.logits = ctx->at<float>(L.logits); lo.delta = ctx->at<void>(L.delta[nl]);
         lo.row_loss = L.local_net ? ctx->at<float>(L.row_loss) : ctx->ctl.row_loss; lo.C = m.dims[nl];
         launch_ex(ctx, ABS_KC_OUTPUT, net_loss_kernel<T>, dim3((L.rows_cap + 255) / 256), dim3(256), 0, lo);
@@ -776,6 +778,7 @@ void enqueue_update(abs_ctx* ctx, int par) {
   UpdateArgs u;
   u.st = ctx->at<DevState>(L.st); u.ri = ri; u.master = ctx->at<float>(L.master); u.ring = ctx->at<void>(L.ring);
   u.G = ctx->at<float>(L.G); u.d_pad = L.d_pad; u.P = L.P; u.lr = ctx->m.lr;
+  u.sel_tau = ctx->ctl.sel_tau[par];
   // for the latency-bound models (always one stream) the Eq. 3 kernel also prepares the next job
   // durations (its first warps); tensor-core networks keep a small kernel of their own for that
   const bool look = !L.any_tc;
@@ -814,6 +817,10 @@ int status_to_code(abs_ctx* ctx, const DevState& h) {
       return fail(ABS_EDIVERGED, "non-finite loss uploaded in round %d; state is that of %d completed rounds", h.t, h.t);
     case ST_RANGE: ctx->sticky = ABS_ERANGE; return fail(ABS_ERANGE, "simulated time left the 2^53 tick range in round %d", h.t);
     case ST_NOSPACE: ctx->sticky = ABS_ENOSPACE; return fail(ABS_ENOSPACE, "round capacity %d exhausted", h.max_rounds);
+    case ST_STALE:
+      ctx->sticky = ABS_ESTALE;
+      return fail(ABS_ESTALE, "round %d: an upload older than the staleness bound arrived (no forced restarts); "
+                  "%d completed rounds stay valid", h.t, h.t);
     case ST_TIMEOUT: ctx->sticky = ABS_ETIMEOUT; return fail(ABS_ETIMEOUT, "bounded device wait expired (site %d)", h.timeout_where);
     default: ctx->sticky = ABS_ECUDA; return fail(ABS_ECUDA, "internal invariant failed (status %d, round %d)", h.status, h.t);
   }
@@ -928,6 +935,11 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   memset(&h, 0, sizeof h);
   h.W = W; h.K0 = K0; h.S = S_ring; h.B = model->batch; h.RB = L.RB;
   h.theta_cap = staleness_bound; h.literal_eq6 = literal;
+  h.no_restart = model->restart_rule == ABS_RESTART_NONE ? 1 : 0;
+  // staleness-aware step size: applied to the delta rows / residuals by the gradient kernels, except
+  // with local steps on a network, whose local copies need the plain gradient sums (there Eq. 3
+  // weights the uploads)
+  h.sa_penalty = model->sa_penalty ? (L.local_net ? 2 : 1) : 0;
   h.k_mode = model->k_mode; h.bound_mode = model->bound_mode; h.max_rounds = model->max_rounds;
   h.n_samples = model->n_samples;
   h.key0 = (uint32_t)(seed & 0xffffffffull); h.key1 = (uint32_t)(seed >> 32);
@@ -1231,9 +1243,27 @@ struct StateHeader {
   unsigned long long magic;
   int version, rounds_enqueued;
   unsigned long long d_pad, esz, block1, block2, max_rounds;
-  DevState st;                       // the saving context's state block (its constants are checked on restore)
+  // what the saving context was created with (checked on restore)
+  int kind, n_layers, dims[ABS_MAX_LAYERS + 1], batch, dtype, local_steps, flags, restart_rule, sa_penalty;
+  float lr;
+  DevState st;                       // its state block (constants checked on restore)
 };
-constexpr unsigned long long STATE_MAGIC = 0x3130455441545341ull;   // "ASTATE01"
+constexpr unsigned long long STATE_MAGIC = 0x3230455441545341ull;   // "ASTATE02"
+
+void describe_model(const abs_model_desc& m, StateHeader* h) {
+  h->kind = m.kind; h->n_layers = m.n_layers;
+  for (int l = 0; l <= ABS_MAX_LAYERS; ++l) h->dims[l] = l <= m.n_layers ? m.dims[l] : 0;
+  h->batch = m.batch; h->dtype = m.dtype; h->local_steps = m.local_steps; h->flags = m.flags;
+  h->restart_rule = m.restart_rule; h->sa_penalty = m.sa_penalty; h->lr = m.lr;
+}
+
+bool same_model(const StateHeader& a, const StateHeader& b) {
+  bool same = a.kind == b.kind && a.n_layers == b.n_layers && a.batch == b.batch && a.dtype == b.dtype &&
+              a.local_steps == b.local_steps && a.flags == b.flags && a.restart_rule == b.restart_rule &&
+              a.sa_penalty == b.sa_penalty && a.lr == b.lr;
+  for (int l = 0; l <= ABS_MAX_LAYERS; ++l) same = same && a.dims[l] == b.dims[l];
+  return same;
+}
 
 void state_blocks(const Layout& L, size_t* b1_off, size_t* b1, size_t* b2_off, size_t* b2) {
   *b1_off = L.st;  *b1 = L.G - L.st;                           // control state, per-worker arrays, layouts, master, ring
@@ -1243,7 +1273,8 @@ void state_blocks(const Layout& L, size_t* b1_off, size_t* b1, size_t* b2_off, s
 bool same_constants(const DevState& a, const DevState& b) {
   return a.W == b.W && a.K0 == b.K0 && a.S == b.S && a.B == b.B && a.RB == b.RB && a.k_mode == b.k_mode &&
          a.bound_mode == b.bound_mode && a.max_rounds == b.max_rounds && a.bound_offset == b.bound_offset &&
-         a.theta_cap == b.theta_cap && a.literal_eq6 == b.literal_eq6 && a.n_samples == b.n_samples &&
+         a.theta_cap == b.theta_cap && a.literal_eq6 == b.literal_eq6 && a.no_restart == b.no_restart &&
+         a.sa_penalty == b.sa_penalty && a.n_samples == b.n_samples &&
          a.key0 == b.key0 && a.key1 == b.key1 && a.dist.kind == b.dist.kind && a.dist.shift == b.dist.shift &&
          a.dist.rate == b.dist.rate && a.dist.scale == b.dist.scale && a.dist.slow_mod == b.dist.slow_mod &&
          a.dist.slow_rem == b.dist.slow_rem && a.dist.slow_factor == b.dist.slow_factor && a.dist.shape == b.dist.shape;
@@ -1276,7 +1307,8 @@ int abs_save_state(abs_ctx* ctx, void* dst, size_t cap, size_t* written) {
   if (rc != ABS_OK) return rc;
   if (h.st.status != ST_OK) return fail(ABS_ESTATE, "the run has ended (status %d): nothing to continue from", h.st.status);
   if (h.st.open) return fail(ABS_ESTATE, "a round is open");
-  h.magic = STATE_MAGIC; h.version = 1; h.rounds_enqueued = ctx->rounds_enqueued;
+  h.magic = STATE_MAGIC; h.version = 2; h.rounds_enqueued = ctx->rounds_enqueued;
+  describe_model(ctx->m, &h);
   h.d_pad = ctx->L.d_pad; h.esz = ctx->L.esz; h.block1 = b1; h.block2 = b2; h.max_rounds = (unsigned long long)ctx->m.max_rounds;
   char* p = (char*)dst;
   memcpy(p, &h, sizeof h);
@@ -1292,7 +1324,12 @@ int abs_restore_state(abs_ctx* ctx, const void* src, size_t bytes) {
   if (bytes < sizeof(StateHeader)) return fail(ABS_EINVAL, "image shorter than its header");
   StateHeader h;
   memcpy(&h, src, sizeof h);
-  if (h.magic != STATE_MAGIC || h.version != 1) return fail(ABS_EINVAL, "not a state image of this library version");
+  if (h.magic != STATE_MAGIC || h.version != 2) return fail(ABS_EINVAL, "not a state image of this library version");
+  StateHeader mine;
+  memset(&mine, 0, sizeof mine);
+  describe_model(ctx->m, &mine);
+  if (!same_model(h, mine))
+    return fail(ABS_EINVAL, "the image was saved by a context with another model, batch, step size, dtype, local steps, flags or modes");
   size_t o1, b1, o2, b2;
   state_blocks(ctx->L, &o1, &b1, &o2, &b2);
   b2 += 4 * (size_t)ctx->m.max_rounds * ctx->W;

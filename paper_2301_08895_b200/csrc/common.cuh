@@ -19,6 +19,7 @@ enum : int {
   ST_NOSPACE = 3,    // round index reached the trace capacity
   ST_INTERNAL = 4,   // an invariant failed (consumed staleness above the bound)
   ST_TIMEOUT = 5,    // a bounded wait inside a kernel expired
+  ST_STALE = 6,      // runs without forced restarts: an arrival is older than the model versions kept
 };
 
 constexpr int MAX_W = ABS_MAX_WORKERS;
@@ -42,6 +43,11 @@ struct DevState {
   int theta_cap;                  // largest threshold = the caller's staleness bound
   int literal_eq6;                // 1: the restart test reads the age before its increment (Eq. 6 as printed);
                                   // S is then the caller's bound + 1 (oldest model version still in use)
+  int no_restart;                 // 1: Eq. 6 never forces a restart (AdaSync / K-async SGD, Sec. II-B); an arrival
+                                  // older than S rounds ends the run with ST_STALE
+  int sa_penalty;                 // staleness-aware step size (Sec. I): 0 off; 1 the gradient kernels scale the
+                                  // rows of a tile by the weight of the tile's staleness; 2 the Eq. 3 kernel
+                                  // weights each selected worker's upload (runs with local steps on networks)
   i64 n_samples;
   uint32_t key0, key1;            // Philox key = (seed low, seed high)
   TimeDist dist;
@@ -106,6 +112,16 @@ __device__ __forceinline__ void stf(__nv_bfloat16* p, size_t i, float v) { p[i] 
 __device__ __forceinline__ void grid_dependency_sync() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Staleness-aware step size (Sec. I: the step size of a stale gradient is penalised linearly in its
+// delay): weight of a gradient of staleness tau in the sum of Eq. 3.
+__device__ __forceinline__ float sa_weight(int tau) { return tau > 1 ? __fdiv_rn(1.f, (float)tau) : 1.f; }
+// Weight of the gradient rows of a tile that reads ring slot `slot` in round t: a consumed gradient
+// is at most S rounds old, so its staleness is (t - slot) mod (S + 1) (slot = version mod (S + 1)
+// and version <= t, so t - slot is never negative).
+__device__ __forceinline__ float sa_slot_weight(const DevState* st, int t, int slot) {
+  return st->sa_penalty == 1 ? sa_weight((t - slot) % (st->S + 1)) : 1.f;
 }
 
 __host__ __device__ inline int round_up(int a, int b) { return (a + b - 1) / b * b; }

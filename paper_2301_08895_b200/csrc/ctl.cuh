@@ -163,6 +163,7 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
   const int status0 = st->status, open0 = st->open, diverged0 = a.ri[po].diverged;
   const int k_mode = st->k_mode, bound_mode = st->bound_mode, max_rounds = st->max_rounds;
   const int bound_offset = st->bound_offset, Scap = st->theta_cap, literal = st->literal_eq6;
+  const int no_restart = st->no_restart;
   const uint32_t key0 = st->key0, key1 = st->key1;
   const i64 n_samples = st->n_samples;
   const u64 T_end0 = st->T_end;
@@ -276,7 +277,7 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
     int restart = 0, renew = 0;
     if (tid < W) {
       const int sel_me = sh.flag[tid];
-      restart = (!sel_me) && ((t + 1 - literal - my_version) > theta);
+      restart = (!sel_me) && !no_restart && ((t + 1 - literal - my_version) > theta);
       renew = sel_me || restart;
     }
     int range_err = 0;
@@ -346,7 +347,10 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
     }
     const int tau_bad = __syncthreads_or(tid < K && (tau < 0 || tau > S));
     if (tau_bad) {
-      if (tid == 0) st->status = ST_INTERNAL;
+      // with forced restarts this cannot happen (consumed staleness <= threshold <= S); without
+      // them the arrival's model version may have left the ring: the run ends here, before any
+      // kernel reads the slot that was overwritten
+      if (tid == 0) st->status = no_restart ? ST_STALE : ST_INTERNAL;
       return 1;
     }
     // network models: group the arrivals by staleness (all members of a group read the same

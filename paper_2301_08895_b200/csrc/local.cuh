@@ -191,7 +191,8 @@ __global__ void __launch_bounds__(NT_MAX) local_sgd_kernel(Args a) {
     }
   }
   float* g = a.G + (size_t)i * a.slot_stride;
-  for (int p = tid; p < n_par; p += NT) g[p] = gs[p];
+  const float sa = st->sa_penalty ? sa_weight(a.sel_tau[i]) : 1.f;   // staleness-aware step size: weight of the upload in Eq. 3
+  for (int p = tid; p < n_par; p += NT) g[p] = gs[p] * sa;
   if (tid == 0) {
     const float loss = __fdiv_rn(loss_sum, (float)U);
     a.loss[i] = loss;

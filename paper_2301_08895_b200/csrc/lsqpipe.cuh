@@ -41,7 +41,7 @@ struct Args {
 
 inline size_t stage_bytes(int d) { return (size_t)(GROUP + 1) * d * 2; }
 inline size_t smem_bytes(int d, int stages) {
-  return (size_t)stages * stage_bytes(d) + (size_t)MAX_ITEMS * GROUP * 8 + MAX_ITEMS * 4 + 2 * NWARPS * GROUP * 4 +
+  return (size_t)stages * stage_bytes(d) + (size_t)MAX_ITEMS * GROUP * 8 + MAX_ITEMS * 8 + 2 * NWARPS * GROUP * 4 +
          2 * MAX_STAGES * 8 + 64;
 }
 
@@ -75,7 +75,8 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
   int* m_idx = reinterpret_cast<int*>(lsm + (size_t)STAGES * stg);         // [MAX_ITEMS][GROUP] sample index
   float* m_y = reinterpret_cast<float*>(m_idx + MAX_ITEMS * GROUP);        // [MAX_ITEMS][GROUP] target
   int* m_slot = reinterpret_cast<int*>(m_y + MAX_ITEMS * GROUP);           // [MAX_ITEMS] ring slot of the worker
-  float* red = reinterpret_cast<float*>(m_slot + MAX_ITEMS);               // [2][NWARPS][GROUP] partial dots
+  float* m_sa = reinterpret_cast<float*>(m_slot + MAX_ITEMS);              // [MAX_ITEMS] weight of the worker's gradient in Eq. 3
+  float* red = m_sa + MAX_ITEMS;                                           // [2][NWARPS][GROUP] partial dots
   uint64_t* full = reinterpret_cast<uint64_t*>(red + 2 * NWARPS * GROUP);  // [STAGES]
   uint64_t* empty = full + MAX_STAGES;                                     // [STAGES]
   volatile int* abort = reinterpret_cast<volatile int*>(empty + MAX_STAGES);
@@ -107,7 +108,10 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
       const int i = it / groups, g = it - i * groups;
       const int b = g * GROUP + r;
       const int wn = a.sel[i];
-      if (r == 0) m_slot[q] = (t - a.sel_tau[i]) % (S + 1);
+      if (r == 0) {
+        m_slot[q] = (t - a.sel_tau[i]) % (S + 1);
+        m_sa[q] = st->sa_penalty ? sa_weight(a.sel_tau[i]) : 1.f;     // staleness-aware step size
+      }
       int idx = -1;
       float yv = 0.f;
       if (b < B) {
@@ -220,8 +224,10 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
           lsum += 0.5f * res[r] * res[r];
         }
         if (tid == 0) a.loss_part[it] = lsum;
+        const float sa = m_sa[q];
 #pragma unroll
         for (int r = 0; r < GROUP; ++r) {
+          res[r] *= sa;
           const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xr[r]);
 #pragma unroll
           for (int j = 0; j < 4; ++j) {

@@ -39,32 +39,6 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const DevState* st, co
   }
 }
 
-// Bias gradient of a hidden layer: G_p[b_off + n] = sum over the rows of chunk p of delta[r][n].
-// Block = 32 column lanes x 32 row lanes; fixed-order reduction.
-template <typename T>
-__global__ void __launch_bounds__(1024) colsum_kernel(const DevState* st, const RoundInfo* ri, const T* delta, float* G, size_t slot_stride,
-                                                      size_t b_off, int out, int P) {
-  grid_dependency_sync();
-  __shared__ float red[32][33];
-  if (st->status != ST_OK) return;
-  const int n_rows = ri->n_rows;
-  const int chunk = round_up((n_rows + P - 1) / P, 64);
-  const int p = blockIdx.y;
-  const int k_begin = min(n_rows, p * chunk), k_end = min(n_rows, (p + 1) * chunk);
-  const int cl = threadIdx.x & 31, rl = threadIdx.x >> 5;
-  const int n = blockIdx.x * 32 + cl;
-  float acc = 0.f;
-  if (n < out)
-    for (int r = k_begin + rl; r < k_end; r += 32) acc += ldf(delta, (size_t)r * out + n);
-  red[rl][cl] = acc;
-  __syncthreads();
-  if (rl == 0 && n < out) {
-    float tot = 0.f;
-    for (int q = 0; q < 32; ++q) tot += red[q][cl];
-    G[(size_t)p * slot_stride + b_off + n] = tot;
-  }
-}
-
 struct NarrowArgs {
   DevState* st;
   RoundInfo* ri;
@@ -94,6 +68,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_kernel(NarrowArgs a) {
   if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   const int slot = a.tile_slot[r0 / st->RB];
+  const float sa = sa_slot_weight(st, ri->t, slot);     // staleness-aware step size: weight of these rows in Eq. 3
   const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
   for (int i = threadIdx.x; i < in * C + C; i += 256) wsm[i] = ldf(Wm, i);
   __syncthreads();
@@ -141,7 +116,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_kernel(NarrowArgs a) {
     float mine = 0.f;
 #pragma unroll
     for (int c = 0; c < NARROW_MAX_C; ++c)
-      if (c == lane) mine = acc[c] * inv - (c == y ? 1.f : 0.f);
+      if (c == lane) mine = (acc[c] * inv - (c == y ? 1.f : 0.f)) * sa;
     if (lane < C) stf(d, lane, mine);
     const float loss = logf(se) - (zy - zmax);
     if (lane == 0) a.row_loss[r] = loss;
@@ -182,57 +157,6 @@ __global__ void __launch_bounds__(256) narrow_dgrad_kernel(NarrowArgs a) {
         if (c < C) acc = fmaf(dsm[rr * C + c], w[c], acc);
       const size_t o = (size_t)(r0 + rr) * in + m;
       stf(out, o, ldf(h, o) > 0.f ? acc : 0.f);
-    }
-  }
-}
-
-// Weight and bias gradient of the output layer over the rows of chunk p:
-// G_p[m][c] = sum_r act_in[r][m] delta_out[r][c], row m = `in` is the bias gradient.
-// Block = 32 feature lanes x 32 row lanes, fixed-order reduction over the row lanes.
-template <typename T>
-__global__ void __launch_bounds__(1024) narrow_wgrad_kernel(NarrowArgs a) {
-  grid_dependency_sync();
-  __shared__ float red[32][33];
-  DevState* st = a.st;
-  RoundInfo* ri = a.ri;
-  if (st->status != ST_OK) return;
-  const int in = a.in, C = a.C;
-  const int n_rows = ri->n_rows;
-  const int chunk = round_up((n_rows + a.P - 1) / a.P, 64);
-  const int p = blockIdx.y;
-  const int k_begin = min(n_rows, p * chunk), k_end = min(n_rows, (p + 1) * chunk);
-  const int ml = threadIdx.x & 31, rl = threadIdx.x >> 5;
-  const int m = blockIdx.x * 32 + ml;
-  const T* src = (const T*)a.act_in;
-  const T* dl = (const T*)a.delta_out;
-  float acc[NARROW_MAX_C];
-#pragma unroll
-  for (int c = 0; c < NARROW_MAX_C; ++c) acc[c] = 0.f;
-  if (m <= in) {
-    for (int r = k_begin + rl; r < k_end; r += 32) {
-      float xv;
-      if (m == in) xv = 1.f;
-      else if (a.gather) {
-        const int s = a.row_idx[r];
-        xv = s < 0 ? 0.f : ldf(src, (size_t)s * in + m);
-      } else xv = ldf(src, (size_t)r * in + m);
-#pragma unroll
-      for (int c = 0; c < NARROW_MAX_C; ++c)
-        if (c < C) acc[c] = fmaf(xv, ldf(dl, (size_t)r * C + c), acc[c]);
-    }
-  }
-  float* G = a.G + (size_t)p * a.slot_stride + a.w_off;
-#pragma unroll
-  for (int c = 0; c < NARROW_MAX_C; ++c) {
-    if (c < C) {                                // C is uniform across the block
-      red[rl][ml] = acc[c];
-      __syncthreads();
-      if (rl == 0 && m <= in) {
-        float tot = 0.f;
-        for (int q = 0; q < 32; ++q) tot += red[q][ml];
-        G[(size_t)m * C + c] = tot;
-      }
-      __syncthreads();
     }
   }
 }
@@ -280,6 +204,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_v8_kernel(NarrowArgs a) {
   const int in = a.in, C = a.C;
   float* bias = reinterpret_cast<float*>(wT + (size_t)C * in);
   const int slot = a.tile_slot[r0 / st->RB];
+  const float sa = sa_slot_weight(st, ri->t, slot);     // staleness-aware step size: weight of these rows in Eq. 3
   const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
 #pragma unroll 8
   for (int i = threadIdx.x; i < in * C; i += 256) {
@@ -338,7 +263,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_v8_kernel(NarrowArgs a) {
     float mine = 0.f;
 #pragma unroll
     for (int c = 0; c < NARROW_MAX_C; ++c)
-      if (c == lane) mine = acc[c] * inv - (c == y ? 1.f : 0.f);
+      if (c == lane) mine = (acc[c] * inv - (c == y ? 1.f : 0.f)) * sa;
     if (lane < C) stf(d, lane, mine);
     const float loss = logf(se) - (zy - zmax);
     if (lane == 0) a.row_loss[r] = loss;
@@ -471,57 +396,6 @@ __global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, f
   }
 }
 
-// Stage 1 of a hidden layer's bias gradient: part[q][n] = sum over the 64 rows of chunk q of
-// delta[r][n]; `out` a multiple of 8.
-template <typename T>
-__global__ void __launch_bounds__(256) colsum_chunk_kernel(const DevState* st, const RoundInfo* ri, const T* delta, int out, float* part) {
-  grid_dependency_sync();
-  extern __shared__ __align__(16) unsigned char nsm_raw[];
-  float* red = reinterpret_cast<float*>(nsm_raw);        // [row lanes][out]
-  if (st->status != ST_OK) return;
-  const int r0 = blockIdx.x * 64;
-  if (r0 >= ri->n_rows) return;
-  const int nvec = out >> 3;
-  const int per = min(nvec, 256);                         // threads along a row
-  const int lanes = 256 / per;                            // rows worked on side by side
-  for (int v0 = 0; v0 < nvec; v0 += 256) {
-    const int v = v0 + (int)threadIdx.x % per;
-    const int rl = (int)threadIdx.x / per;
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-    const bool active = rl < lanes && v < nvec;
-    if (active)
-      for (int rr = rl; rr < 64; rr += lanes) {
-        float dv[8];
-        load8(delta + (size_t)(r0 + rr) * out + (size_t)v * 8, dv);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] += dv[j];
-      }
-    if (lanes == 1) {
-      if (active) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) part[(size_t)blockIdx.x * out + v * 8 + j] = acc[j];
-      }
-      continue;
-    }
-    if (active) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) red[(size_t)rl * out + v * 8 + j] = acc[j];
-    }
-    __syncthreads();
-    if (active && rl == 0) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        float tot = 0.f;
-        for (int q = 0; q < lanes; ++q) tot += red[(size_t)q * out + v * 8 + j];
-        part[(size_t)blockIdx.x * out + v * 8 + j] = tot;
-      }
-    }
-    __syncthreads();
-  }
-}
-
 // Stage 2: dst[i] = sum over the active chunks q of part[q][i], i < len.  Block = 32 outputs x 8
 // chunk lanes; lane w adds chunks w, w+8, ... in order, then the 8 lanes are added in order.
 __global__ void __launch_bounds__(256) chunk_reduce_kernel(const DevState* st, const RoundInfo* ri, const float* part, int len, float* dst,
@@ -602,6 +476,7 @@ __global__ void __launch_bounds__(256) narrow_fused_kernel(NarrowArgs a, float* 
     }
   }
   const int slot = a.tile_slot[r0 / st->RB];
+  const float sa = sa_slot_weight(st, ri->t, slot);     // staleness-aware step size: weight of these rows in Eq. 3
   const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
   {
     // weights + bias are contiguous and start on a 128-byte boundary; copy whole 16-byte pieces
@@ -664,7 +539,7 @@ __global__ void __launch_bounds__(256) narrow_fused_kernel(NarrowArgs a, float* 
     float mine = 0.f;
 #pragma unroll
     for (int c = 0; c < NARROW_MAX_C; ++c)
-      if (c == lane) mine = acc[c] * inv - (c == y ? 1.f : 0.f);
+      if (c == lane) mine = (acc[c] * inv - (c == y ? 1.f : 0.f)) * sa;
     // the delta is a stored quantity: round it to the storage type like every other delta
     if (lane < NARROW_MAX_C) d3[rr * NARROW_MAX_C + lane] = lane < C ? round_store(mine, (const T*)nullptr) : 0.f;
     const float loss = logf(se) - (zy - zmax);
@@ -761,6 +636,7 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
     }
   }
   const int slot = a.tile_slot[r0 / st->RB];
+  const float sa = sa_slot_weight(st, ri->t, slot);     // staleness-aware step size: weight of these rows in Eq. 3
   const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
   {
     const int n16 = (int)(((size_t)(in + 1) * CC * sizeof(T) + 15) / 16);
@@ -828,7 +704,7 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
       float mine = 0.f;
 #pragma unroll
       for (int c = 0; c < CC; ++c)
-        if (c == lane) mine = z[c] * inv - (c == y ? 1.f : 0.f);
+        if (c == lane) mine = (z[c] * inv - (c == y ? 1.f : 0.f)) * sa;
       // the delta is a stored quantity: round it to the storage type like every other delta
       if (lane < CC) d3[rr * CC + lane] = round_store(mine, (const T*)nullptr);
       const float loss = logf(se) - (zy - zmax);
@@ -989,7 +865,9 @@ __global__ void __launch_bounds__(256, 2) lsq_grad_v2_kernel(LsqArgs a) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
     if (lane == 0) red[warp] = part;
-    // pass 2: this worker's gradient into the running sums (rows come from L2 now)
+    // pass 2: this worker's gradient into the running sums (rows come from L2 now), with the
+    // weight of its staleness when the staleness-aware step size is on
+    const float sa = st->sa_penalty ? sa_weight(a.sel_tau[i]) : 1.f;
 #pragma unroll
     for (int q = 0; q < NV; ++q) {
       const int v = tid + q * 256;
@@ -998,7 +876,7 @@ __global__ void __launch_bounds__(256, 2) lsq_grad_v2_kernel(LsqArgs a) {
         for (int b = 0; b < B; ++b) {
           float xv[8];
           load8(X + (size_t)sidx[b] * d + (size_t)v * 8, xv);
-          const float rb = res[b];
+          const float rb = res[b] * sa;
 #pragma unroll
           for (int j = 0; j < 8; ++j) acc[q][j] = fmaf(rb, xv[j], acc[q][j]);
         }

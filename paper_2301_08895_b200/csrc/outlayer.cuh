@@ -77,6 +77,7 @@ __global__ void __launch_bounds__(THREADS) out_layer_mma_kernel(NarrowArgs a, fl
                  "l"(src + (size_t)rr * IN + v * 8) : "memory");
   }
   const int slot = a.tile_slot[r0 / st->RB];
+  const float sa = sa_slot_weight(st, ri->t, slot);     // staleness-aware step size: weight of these rows in Eq. 3
   const __nv_bfloat16* Wm = (const __nv_bfloat16*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
   {
     // weights + bias are contiguous and start on a 128-byte boundary: whole 16-byte pieces
@@ -164,7 +165,7 @@ __global__ void __launch_bounds__(THREADS) out_layer_mma_kernel(NarrowArgs a, fl
         float d[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          d[i] = (y >= 0 && cls[i] < C) ? e[i] * inv - (cls[i] == y ? 1.f : 0.f) : 0.f;   // padding rows add nothing to Eq. 3
+          d[i] = (y >= 0 && cls[i] < C) ? (e[i] * inv - (cls[i] == y ? 1.f : 0.f)) * sa : 0.f;   // padding rows add nothing to Eq. 3
         dpk[h][0] = pack_bf16(d[0], d[1]);
         dpk[h][1] = pack_bf16(d[2], d[3]);
         const int rr = 16 * mt + g + 8 * h;

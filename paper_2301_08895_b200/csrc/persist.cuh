@@ -159,8 +159,10 @@ abs_lsq_rounds_kernel(CtlArgs a, LsqRoundsArgs q, int t_first, int n_rounds) {
           }
           const float res = dot - __shfl_sync(0xffffffffu, yv[k], sub * lpr);
           if (valid && v == 0) rowloss_s[row] = 0.5f * res * res;
+          // staleness-aware step size: the row's weight follows from the ring slot it was computed on
+          const float rg = res * (valid ? sa_slot_weight(st, t, rslot_s[row]) : 1.f);
 #pragma unroll
-          for (int j = 0; j < 8; ++j) acc[j] = fmaf(res, xv[k][j], acc[j]);   // xv = 0 where there is no row
+          for (int j = 0; j < 8; ++j) acc[j] = fmaf(rg, xv[k][j], acc[j]);   // xv = 0 where there is no row
         }
       }
 #pragma unroll

@@ -207,6 +207,7 @@ __global__ void __launch_bounds__(256) simt_wgrad_kernel(LayerArgs a) {
 struct LossArgs {
   DevState* st;
   RoundInfo* ri;
+  const int* tile_slot;   // ring slot of every row tile (RB rows)
   const int* row_idx;
   const int* labels;      // [n_samples]
   const float* logits;    // [rows][C]
@@ -240,7 +241,8 @@ __global__ void __launch_bounds__(256) net_loss_kernel(LossArgs a) {
   float se = 0.f;
   for (int c = 0; c < C; ++c) se += expf(z[c] - zmax);
   const float inv = 1.f / se;
-  for (int c = 0; c < C; ++c) stf(d, c, expf(z[c] - zmax) * inv - (c == y ? 1.f : 0.f));
+  const float sa = sa_slot_weight(st, ri->t, a.tile_slot[r / st->RB]);   // staleness-aware step size
+  for (int c = 0; c < C; ++c) stf(d, c, (expf(z[c] - zmax) * inv - (c == y ? 1.f : 0.f)) * sa);
   const float loss = logf(se) - (z[y] - zmax);
   a.row_loss[r] = loss;
   if (!isfinite(loss)) ri->diverged = 1;
@@ -315,10 +317,11 @@ __global__ void __launch_bounds__(256) lsq_grad_kernel(LsqArgs a) {
     if (!isfinite(loss)) ri->diverged = 1;
   }
   float* g = a.G + (size_t)i * a.slot_stride;
+  const float sa = st->sa_penalty ? sa_weight(a.sel_tau[i]) : 1.f;   // staleness-aware step size
   for (int j = tid; j < d; j += 256) {
     float acc = 0.f;
     for (int b = 0; b < B; ++b) acc = fmaf(res[b], ldf(X, (size_t)sidx[b] * d + j), acc);
-    g[j] = acc;
+    g[j] = acc * sa;
   }
 }
 
@@ -331,6 +334,8 @@ struct UpdateArgs {
   const float* G;         // [P][d_pad]
   size_t d_pad;
   int P;                  // partial count, or 0: one partial per selected worker (K^t)
+  const int* sel_tau;     // [K^t] staleness of each selected worker's upload (read when the staleness-aware
+                          // step size is applied to whole uploads: DevState::sa_penalty == 2, P == 0)
   float lr;
   int* zero_words; int n_zero;   // counters of the round's kernels to clear for the next round (or null)
   // Output-layer gradient still in per-chunk partial sums (or null): blocks [n_main_blocks, gridDim.x)
@@ -411,7 +416,8 @@ __global__ void __launch_bounds__(256, 4) update_kernel(UpdateArgs a) {
   };
   // few partials (the split counts of the weight-gradient GEMMs): two vectors per thread and
   // iteration, all loads of both issued before the first use (same sums, same order per element)
-  if (P <= 4) {
+  const bool weigh = a.P == 0 && st->sa_penalty == 2;
+  if (P <= 4 && !weigh) {
     for (; i + stride < n4; i += 2 * stride) {
       const size_t j = i + stride;
       float4 ga[4], gb[4];
@@ -435,9 +441,20 @@ __global__ void __launch_bounds__(256, 4) update_kernel(UpdateArgs a) {
   }
   for (; i < n4; i += stride) {
     float4 g = reinterpret_cast<const float4*>(a.G)[i];
-    for (int p = 1; p < P; ++p) {
-      const float4 q = reinterpret_cast<const float4*>(a.G + (size_t)p * a.d_pad)[i];
-      g.x += q.x; g.y += q.y; g.z += q.z; g.w += q.w;
+    if (weigh) {
+      // staleness-aware step size on whole uploads: upload p counts with weight 1 / max(1, tau_p)
+      const float w0 = sa_weight(a.sel_tau[0]);
+      g.x *= w0; g.y *= w0; g.z *= w0; g.w *= w0;
+      for (int p = 1; p < P; ++p) {
+        const float4 q = reinterpret_cast<const float4*>(a.G + (size_t)p * a.d_pad)[i];
+        const float wp = sa_weight(a.sel_tau[p]);
+        g.x = fmaf(wp, q.x, g.x); g.y = fmaf(wp, q.y, g.y); g.z = fmaf(wp, q.z, g.z); g.w = fmaf(wp, q.w, g.w);
+      }
+    } else {
+      for (int p = 1; p < P; ++p) {
+        const float4 q = reinterpret_cast<const float4*>(a.G + (size_t)p * a.d_pad)[i];
+        g.x += q.x; g.y += q.y; g.z += q.z; g.w += q.w;
+      }
     }
     finish(i, g, reinterpret_cast<float4*>(a.master)[i]);
   }

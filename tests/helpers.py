@@ -56,19 +56,29 @@ def layer_blocks(kind, dims):
     return out
 
 
+# A bias block is a few dozen numbers, each the sum of many rounds of signed updates: the result is
+# smaller than the terms that were added, so its relative rounding error is a small multiple of the
+# whole vector's (seen: up to 1.7x with fp32 storage), while a block that is actually wrong (a
+# dropped or doubled contribution) is off by 1e-1 or more.  fp32 blocks get this factor on top of
+# the run's tolerance; bf16 runs keep the plain 2e-2.
+BLOCK_SLACK_FP32 = 4.0
+
+
 def assert_params_close(cfg, params, ref, tol):
-    """Relative L2 of the whole vector and of every layer block (each W_l, each b_l) within tol:
-    a wrong bias vector moves the norm of millions of weights by less than any tolerance, so the
-    whole-vector figure alone would not see it."""
+    """Relative L2 of the whole vector within tol, and of every layer block (each W_l, each b_l)
+    within tol (bf16 storage) or BLOCK_SLACK_FP32 * tol (fp32 storage): a wrong bias vector moves
+    the norm of millions of weights by less than any tolerance, so the whole-vector figure alone
+    would not see it."""
     err = rel_l2(params, ref)
     assert err <= tol, "parameters differ: rel L2 %.3g > %.3g" % (err, tol)
     ref = np.asarray(ref, np.float64)
+    btol = tol if cfg.dtype == inputs.BF16 else BLOCK_SLACK_FP32 * tol
     for name, sl in layer_blocks(cfg.kind, cfg.dims):
         if np.linalg.norm(ref[sl]) == 0.0:
             assert np.linalg.norm(np.asarray(params, np.float64)[sl]) == 0.0, "block %s should be zero" % name
             continue
         e = rel_l2(np.asarray(params)[sl], ref[sl])
-        assert e <= tol, "parameter block %s differs: rel L2 %.3g > %.3g" % (name, e, tol)
+        assert e <= btol, "parameter block %s differs: rel L2 %.3g > %.3g" % (name, e, btol)
     return err
 
 
@@ -79,10 +89,12 @@ def compare_with_oracle(cfg, X, y, w0, rounds, tol, forced=False, loss_tol=None,
     which separates the integer machinery from last-bit loss differences."""
     gkw = {k: v for k, v in kw.items() if k in ("k_mode", "bound_mode", "bound_offset", "local_steps")}
     literal = kw.get("restart_rule", 0) == gpu.RESTART_EQ6
+    sa = int(kw.get("sa_penalty", 0))
     rows, params = gpu_run(cfg, X, y, w0, rounds, flags=kw.get("flags", 0),
-                           restart_rule=kw.get("restart_rule", 0), **gkw)
+                           restart_rule=kw.get("restart_rule", 0), sa_penalty=sa, **gkw)
     assert len(rows) == rounds
-    o = make_oracle(cfg, X, y, w0, literal_eq6=literal, **gkw)
+    o = make_oracle(cfg, X, y, w0, literal_eq6=literal, sa_penalty=bool(sa),
+                    restarts=kw.get("restart_rule", 0) != gpu.RESTART_NONE, **gkw)
     orows = o.run(rounds, forced_losses=[r["sel_loss"] for r in rows] if forced else None)
     mm = first_integer_mismatch(rows, orows)
     assert mm is None, "integer trace differs at round %s field %s: gpu %s oracle %s (oracle " \

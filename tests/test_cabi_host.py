@@ -39,18 +39,18 @@ def test_struct_sizes_match_header_layout(tmp_path):
     src = tmp_path / "layout.c"
     src.write_text(
         '#include <stdio.h>\n#include <stddef.h>\n#include "abs_b200.h"\n'
-        'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(abs_time_dist), '
+        'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(abs_time_dist), '
         'sizeof(abs_trace), sizeof(abs_model_desc), offsetof(abs_model_desc, X), '
         'offsetof(abs_model_desc, bound_offset), offsetof(abs_model_desc, max_rounds), '
         'offsetof(abs_model_desc, stream), offsetof(abs_time_dist, shape), '
-        'offsetof(abs_time_dist, slow_factor)); return 0; }\n')
+        'offsetof(abs_time_dist, slow_factor), offsetof(abs_model_desc, sa_penalty)); return 0; }\n')
     exe = tmp_path / "layout"
     subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
     got = [int(v) for v in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
     assert got == [C.sizeof(gpu.TimeDist), C.sizeof(gpu.Trace), C.sizeof(gpu.ModelDesc),
                    gpu.ModelDesc.X.offset, gpu.ModelDesc.bound_offset.offset,
                    gpu.ModelDesc.max_rounds.offset, gpu.ModelDesc.stream.offset,
-                   gpu.TimeDist.shape.offset, gpu.TimeDist.slow_factor.offset]
+                   gpu.TimeDist.shape.offset, gpu.TimeDist.slow_factor.offset, gpu.ModelDesc.sa_penalty.offset]
     assert C.sizeof(gpu.Trace) == 14 * 8
 
 
