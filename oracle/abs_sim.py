@@ -142,7 +142,8 @@ def theta_offset_rule(W, S, k, a):
 class ABSOracle:
     """State of one simulated run.
 
-    kind, dims     model kind (models.LSQ/SOFTMAX/MLP) and layer sizes
+    kind, dims     model kind (models.LSQ/SOFTMAX/MLP/CNN) and layer sizes (CNN: of its fully
+                   connected part; `conv` = (H, W, C_in, k, C1, C2) describes the two convolution blocks)
     X, y           dataset; X either float array [M, in] or, with
                    `x_is_bf16_bits`, uint16 bfloat16 patterns
     w0             initial parameters (flat, layout of module `models`)
@@ -167,7 +168,7 @@ class ABSOracle:
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, dist, seed,
                  quant=False, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE,
                  literal_eq6=False, x_is_bf16_bits=False, integer_only=False, bound_offset=0,
-                 local_steps=1, restarts=True, sa_penalty=False):
+                 local_steps=1, restarts=True, sa_penalty=False, conv=None):
         if not (1 <= K0 <= W):
             raise ValueError("need 1 <= K0 <= W")
         if S < 0:
@@ -192,7 +193,11 @@ class ABSOracle:
         self.restarts = bool(restarts)
         self.sa_penalty = bool(sa_penalty)
         self.w = np.array(w0, dtype=np.float64)
-        assert self.w.shape[0] == models.n_params(kind, dims)
+        self.conv = None if conv is None else tuple(int(v) for v in conv)
+        if kind == models.CNN:
+            assert self.w.shape[0] == models.cnn_n_params(self.conv, dims)
+        else:
+            assert self.w.shape[0] == models.n_params(kind, dims)
         # the oracle may keep every past model; the bound is what lets a real
         # implementation keep only S + 1 of them
         self.versions = {0: self._stored(self.w)}
@@ -234,7 +239,7 @@ class ABSOracle:
             # (the copy itself keeps full precision); at step 0 that is the downloaded model, which
             # is stored rounded already (rounding it again would change nothing)
             w_eval = held if u == 0 else self._stored(w_local)
-            loss, grad = models.loss_grad(self.kind, self.dims, w_eval, Xb, yb, quant=self.quant)
+            loss, grad = models.loss_grad(self.kind, self.dims, w_eval, Xb, yb, quant=self.quant, conv=self.conv)
             loss_sum += loss
             grad_sum += grad
             if u + 1 < self.local_steps:
