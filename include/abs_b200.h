@@ -85,14 +85,8 @@ extern "C" {
                                    exponential draws (the law the paper draws execution times from) */
 
 #define ABS_FLAG_NO_TENSOR_CORES 1  /* run the hidden-layer contractions on the FP32-FMA kernels */
-#define ABS_FLAG_TWO_CTA         4  /* hidden-layer GEMMs with >= 256 output columns run on CTA pairs
-                                       (tcgen05 cta_group::2, tiles of 256 x 256) */
 #define ABS_FLAG_NO_OVERLAP      2  /* enqueue every kernel on the caller's stream (no side stream for the
                                        server-side kernels of the next round) */
-#define ABS_FLAG_TMA_GATHER     16  /* tensor-core networks: the first layer's GEMMs fetch the minibatch rows
-                                       from the dataset by row index (TMA four-row gathers) instead of reading
-                                       a dense copy made by a separate kernel; same results, slower when a row
-                                       tile is shared by several column tiles (each re-gathers it) */
 #define ABS_FLAG_NO_BULK_PIPELINE 32 /* bf16 least squares: per-warp 16-byte loads (rows read from HBM, then again
                                        from L2) instead of the bulk-copy pipeline through shared memory */
 #define ABS_FLAG_FUSED_FORWARD  128 /* tensor-core networks: two consecutive hidden layers with the same tile width
@@ -136,8 +130,8 @@ typedef struct {
                                average of its U minibatch losses) is implemented for ABS_LSQ and ABS_SOFTMAX
                                with <= 16 classes, <= 12288 parameters and batch x classes <= 8192 (the worker's
                                copy lives in shared memory), and for multi-layer ABS_MLP (the selected workers'
-                               copies live in the workspace: 8 bytes per parameter and worker, 6 in bf16;
-                               not with ABS_FLAG_TMA_GATHER / ABS_FLAG_TWO_CTA); in the bf16 configurations
+                               copies live in the workspace: 8 bytes per parameter and worker, 6 in bf16);
+                               in the bf16 configurations
                                each step is evaluated at the bf16 rounding of the fp32 copy */
   int k_mode;               /* ABS_K_* */
   int bound_mode;           /* ABS_BOUND_* */

@@ -24,9 +24,7 @@ T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2, T_GAMMA = 0, 1, 2, 3, 4
 MAX_LAYERS = 7
 FLAG_NO_TENSOR_CORES = 1
 FLAG_NO_OVERLAP = 2
-FLAG_TWO_CTA = 4
 FLAG_NO_PERSISTENT = 8
-FLAG_TMA_GATHER = 16
 FLAG_NO_BULK_PIPELINE = 32
 FLAG_NO_FUSED_BACKWARD = 64
 FLAG_FUSED_FORWARD = 128

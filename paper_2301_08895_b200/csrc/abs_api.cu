@@ -60,8 +60,6 @@ struct Layout {
   int path[ABS_MAX_LAYERS] = {};        // how each layer's contractions run
   int bn_fwd[ABS_MAX_LAYERS] = {}, bn_dg[ABS_MAX_LAYERS] = {}, bn_wg[ABS_MAX_LAYERS] = {};
   bool any_tc = false;
-  bool gather_tma = false;              // first-layer GEMMs fetch the minibatch rows from the dataset themselves
-  bool two_cta = false;                 // GEMMs with N >= 256 run on CTA pairs (tiles of 256 x 256)
   int cg_fwd[ABS_MAX_LAYERS] = {}, cg_dg[ABS_MAX_LAYERS] = {}, cg_wg[ABS_MAX_LAYERS] = {};
   bool pair_fwd[ABS_MAX_LAYERS] = {};   // forward GEMMs of layers l and l + 1 share a launch
   size_t done;                          // completion counters per row tile (paired forward launches)
@@ -147,9 +145,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       L->any_tc = true;
     } else L->path[l] = PATH_SIMT;
   }
-  L->two_cta = L->any_tc && (m->flags & ABS_FLAG_TWO_CTA);
-  L->gather_tma = !lsq && L->path[0] == PATH_TC && (m->flags & ABS_FLAG_TMA_GATHER);
-  L->RB = lsq ? m->batch : (L->any_tc ? (L->two_cta ? 256 : 128) : 64);
+  L->RB = lsq ? m->batch : (L->any_tc ? 128 : 64);
   const int groups = (W < S + 1) ? W : S + 1;
   L->rows_cap = round_up(W * m->batch, L->RB) + groups * L->RB;
   L->local_net = !lsq && m->n_layers > 1 && m->local_steps > 1;
@@ -175,10 +171,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       L->bn_dg[l] = pick(in, row_tiles);
       L->bn_wg[l] = pick(out, ((in + 127) / 128 + 1) * 3);
       L->cg_fwd[l] = L->cg_dg[l] = L->cg_wg[l] = 1;
-      if (L->two_cta) {
-        if (out >= 256) { L->cg_fwd[l] = 2; L->bn_fwd[l] = 256; L->cg_wg[l] = 2; L->bn_wg[l] = 256; }
-        if (in >= 256) { L->cg_dg[l] = 2; L->bn_dg[l] = 256; }
-      } else if ((size_t)in * out >= ((size_t)1 << 21) && in >= 256 && out >= 256 && W * m->batch >= 4096) {
+      if ((size_t)in * out >= ((size_t)1 << 21) && in >= 256 && out >= 256 && W * m->batch >= 4096) {
         // a large weight gradient is bound by operand traffic into shared memory: CTA pairs halve
         // the B operand each CTA has to stage (its tiles are features x outputs, so the row padding
         // unit of the version groups is not involved)
@@ -191,7 +184,6 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     for (int l = 0; l + 1 < m->n_layers; ++l) {
       if (L->path[l] != PATH_TC || L->path[l + 1] != PATH_TC || !(m->flags & ABS_FLAG_FUSED_FORWARD)) continue;
       if (L->cg_fwd[l] != 1 || L->cg_fwd[l + 1] != 1 || L->bn_fwd[l] != L->bn_fwd[l + 1]) continue;
-      if (l == 0 && L->gather_tma) continue;
       if (l > 0 && L->pair_fwd[l - 1]) continue;
       if (L->local_net) continue;
       L->pair_fwd[l] = true;
@@ -287,7 +279,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     for (int l = 0; l <= m->n_layers; ++l) L->bits[l] = 0;
     for (int l = 0; l + 1 < m->n_layers; ++l)
       if (L->path[l] == PATH_TC) L->bits[l + 1] = cv.take(4 * (size_t)L->rows_cap * ((m->dims[l + 1] + 31) / 32));
-    const bool copy0 = L->path[0] == PATH_TC && !L->gather_tma;     // gathered copies of the input rows
+    const bool copy0 = L->path[0] == PATH_TC;     // gathered copies of the input rows
     L->act[0] = copy0 ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     L->act0b = copy0 ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     for (int l = 1; l <= m->n_layers; ++l) {
@@ -321,7 +313,6 @@ struct TcLayer {
   CUtensorMap fwd_a, fwd_b, dg_a, dg_b, wg_a, wg_b;
   CUtensorMap fwd_out, dg_out, wg_out;     // result tensors written by bulk tensor stores
   CUtensorMap fwd_a_odd, wg_a_odd;         // layer 0 only: operand maps over the second gathered copy
-  CUtensorMap x_rows;                      // layer 0 only: the dataset with a one-row box (row gathers)
 };
 
 // ones[r][0] = 1 (bf16), the rest of the 64-wide rows stays zero: the extra operand row that turns
@@ -515,21 +506,18 @@ int setup_tc(abs_ctx* ctx) {
     if (L.path[l] != PATH_TC) continue;
     const int in = m.dims[l], out = m.dims[l + 1];
     TcLayer& t = ctx->tcl[l];
-    const bool from_x = l == 0 && L.gather_tma;      // no gathered copy: fwd_a / wg_a stay unused
-    const void* act_in = from_x ? ctx->X : ctx->at<void>(L.act[l]);
+    const void* act_in = ctx->at<void>(L.act[l]);
     const void* delta_out = ctx->at<void>(L.delta[l + 1]);
     const void* wbase = ring + 2 * L.w_off[l];
-    bool ok = (from_x || make_act_map(&t.fwd_a, act_in, in, L.rows_cap, 128)) &&
+    bool ok = make_act_map(&t.fwd_a, act_in, in, L.rows_cap, 128) &&
               make_w_map(&t.fwd_b, wbase, in, out, L.gslots, L.d_pad, 64) &&
-              (from_x || make_act_map(&t.wg_a, act_in, in, L.rows_cap, 64)) &&
+              make_act_map(&t.wg_a, act_in, in, L.rows_cap, 64) &&
               make_act_map(&t.wg_b, delta_out, out, L.rows_cap, 64) &&
               make_act_map(&t.fwd_out, ctx->at<void>(L.act[l + 1]), out, L.rows_cap, 32) &&
               make_g_map(&t.wg_out, ctx->at<float>(L.G) + L.w_off[l], in, out, n_splits, L.d_pad);
-    if (ok && l == 0 && !L.gather_tma)
+    if (ok && l == 0)
       ok = make_act_map(&t.fwd_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 128) &&
            make_act_map(&t.wg_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 64);
-    if (ok && l == 0 && L.gather_tma)
-      ok = make_act_map(&t.x_rows, ctx->X, in, (int)m.n_samples, 1);
     if (ok && l > 0)
       ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
            make_w_map(&t.dg_b, wbase, in, out, L.gslots, L.d_pad, L.bn_dg[l] / L.cg_dg[l]) &&
@@ -600,7 +588,6 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     p.st = st; p.ri = ri; p.tile_slot = ctx->ctl.tile_slot[par]; p.mode = mode; p.P = L.P;
     p.ring = ctx->at<__nv_bfloat16>(L.gring); p.slot_stride = L.d_pad;
     p.b_off = L.w_off[l] + (size_t)m.dims[l] * m.dims[l + 1];
-    if (l == 0 && L.gather_tma && mode != tc::DGRAD) { p.gather_a = 1; p.row_idx = ctx->ctl.row_idx[par]; }
     return p;
   };
   auto narrow_args = [&](int l) {
@@ -615,7 +602,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     return a;
   };
   if (phase == PH_GATHER) {
-    if (gathered && !L.gather_tma)
+    if (gathered)
       launch_on(ctx, ctx->overlap ? ctx->side : s, ABS_KC_GATHER, gather_rows_kernel, dim3(ctx->sm_count * 8), dim3(256), 0,
                 st, ri, ctx->ctl.row_idx[par], (const __nv_bfloat16*)ctx->X, ctx->at<__nv_bfloat16>(par ? L.act0b : L.act[0]), m.dims[0]);
     return;
@@ -630,7 +617,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       p.relu_bits = L.bits[l + 1] ? ctx->at<uint32_t>(L.bits[l + 1]) : nullptr;
       p.mask_words = (la[l].out + 31) / 32;
       const int bn = L.bn_fwd[l];
-      const CUtensorMap& amap = (l == 0 && L.gather_tma) ? ctx->tcl[l].x_rows : (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a;
+      const CUtensorMap& amap = (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a;
       const int tiles = (row_tiles128 / L.cg_fwd[l]) * ((la[l].out + bn - 1) / bn);
       if (L.pair_fwd[l]) {
         // the next layer's forward GEMM rides in the same launch, behind completion counters
@@ -723,7 +710,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
         launch_tc_bn(ctx, bnd, L.cg_dg[l], ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, ctx->tcl[l].dg_out, pd, dg_tiles);
       const int bn = L.bn_wg[l];
       const int tmw = 128 * L.cg_wg[l];
-      launch_tc_bn(ctx, bn, L.cg_wg[l], ABS_KC_WGRAD, (l == 0 && L.gather_tma) ? ctx->tcl[l].x_rows : (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
+      launch_tc_bn(ctx, bn, L.cg_wg[l], ABS_KC_WGRAD, (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
                    ((la[l].in + tmw - 1) / tmw + 1) * ((la[l].out + bn - 1) / bn) * n_splits);
     } else if (L.path[l] == PATH_NARROW && L.fused_R) {
       // forward, loss, delta of the layer below and the gradient were all done by the fused kernel
@@ -853,13 +840,6 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     return fail(ABS_EINVAL, "local_steps %d outside [1, 1024]", model->local_steps);
   if (model->local_steps > 1) {
     // U > 1: the worker's local model lives in shared memory; single-layer models only
-    if (model->kind == ABS_MLP && model->n_layers > 1) {
-      // multi-layer networks: private model copies in HBM, every step through the tensor-core kernels
-      Layout Lc;
-      make_layout(model, W, staleness_bound, &Lc);
-      if (Lc.gather_tma || Lc.two_cta)
-        return fail(ABS_EUNSUPPORTED, "local_steps = %d on a multi-layer network: not with ABS_FLAG_TMA_GATHER or ABS_FLAG_TWO_CTA", model->local_steps);
-    }
     const bool single = model->kind != ABS_MLP || model->n_layers == 1;
     const int C = model->kind == ABS_LSQ ? 1 : model->dims[1];
     const size_t n_par = model->kind == ABS_LSQ ? (size_t)model->dims[0] : (size_t)model->dims[0] * C + C;

@@ -43,9 +43,6 @@ struct Params {
                                    // the word at bit (j >> 1) + 16 * (j & 1) (even columns low half, odd high)
   uint32_t* relu_bits;             // FWD: the same bits for this layer's output (may be null)
   int mask_words;                  // words per row of mask_bits / relu_bits = ceil(N_total / 32)
-  const int* row_idx;              // gather_a: sample index of every gradient row (-1 = padding row)
-  int gather_a;                    // FWD/WGRAD: operand A is the dataset, its rows fetched by row_idx
-                                   // (map_a then describes X with a one-row box)
   // Two forward problems in one launch: the second reads what the first writes.  Every epilogue
   // warp of the first adds 1 to done[row tile] once its stores of a tile have completed; the
   // producer of the second waits until done[row tile] reaches done_target before it loads rows
@@ -103,6 +100,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+__device__ __forceinline__ void prefetch_map(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -164,20 +164,6 @@ __device__ __forceinline__ void tma2_load_3d(void* dst, const CUtensorMap* map, 
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y), "r"(z)
-      : "memory");
-}
-// Four rows of a 2-D tensor (rows given by index, columns [x, x + box width)) into four consecutive
-// 128-byte rows of a swizzled tile.
-__device__ __forceinline__ void tma_gather4(void* dst, const CUtensorMap* map, uint64_t* bar, int x, const int4& r) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w)
-      : "memory");
-}
-__device__ __forceinline__ void tma2_gather4(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, const int4& r) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w)
       : "memory");
 }
 __device__ __forceinline__ void umma2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -242,7 +228,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                const Params p0,
                const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_b1,
                const __grid_constant__ CUtensorMap map_out1, const Params p1) {
-  grid_dependency_sync();
+  // The kernel in front of this one may still be running (programmatic stream serialization): the
+  // kernel behind this one may be scheduled as early, and everything that does not read the
+  // predecessors' results -- barriers, the tensor-memory allocation, descriptor prefetch -- is done
+  // before the wait for them.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   using C = Cfg<BN, CG>;
   constexpr int TM_ROWS = BM * CG;              // rows of one tile
   extern __shared__ uint8_t smem_raw[];
@@ -251,8 +241,50 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   const int n_units = (int)gridDim.x / CG;
   DevState* st = p0.st;
   RoundInfo* ri = p0.ri;
-  if (st->status != ST_OK) return;
-  const int n_rows = ri->n_rows;
+
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
+  uint8_t* stage_out = smem + (size_t)C::STAGES * C::STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stage_out + C::OUT_BYTES);
+  uint64_t* full = bars;                     // [STAGES] TMA bytes landed
+  uint64_t* empty = bars + C::STAGES;        // [STAGES] MMAs that read the stage are done
+  uint64_t* acc_full = bars + 2 * C::STAGES; // [2] accumulator complete
+  uint64_t* acc_empty = acc_full + 2;        // [2] accumulator drained by the epilogue
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  __nv_bfloat16* bias_s = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [2][BN]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS * CG); }
+    *abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    prefetch_map(&map_a0); prefetch_map(&map_b0); prefetch_map(&map_out0);
+    if (p1.mode >= 0) { prefetch_map(&map_a1); prefetch_map(&map_b1); prefetch_map(&map_out1); }
+  }
+  if (warp == 1) {
+    if (CG == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (CG == 2) cluster_sync_all();              // the peer's barriers exist before anything signals them
+  tc_fence_after();
+  // barriers that live in the leader CTA, as addresses valid from either CTA of the pair
+  const uint32_t full0_addr = (CG == 2) ? map_to_cta(smem_u32(&full[0]), 0) : smem_u32(&full[0]);
+  const uint32_t acc_empty0_addr = (CG == 2) ? map_to_cta(smem_u32(&acc_empty[0]), 0) : smem_u32(&acc_empty[0]);
+  const uint32_t tmem_base = *tmem_slot;
+
+  // from here on the kernel reads what its predecessors wrote (device state, layouts, operands)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const bool running = st->status == ST_OK;
+  const int n_rows = running ? ri->n_rows : 0;
   const int n_row_tiles = n_rows / TM_ROWS;
   auto make_prob = [&](const Params& q) -> Prob {
     Prob r;
@@ -262,7 +294,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     // gradient (row `in` of the [in + 1][out] gradient block) on the tensor cores for free
     r.n_mt_w = (q.M_total - 1 + TM_ROWS - 1) / TM_ROWS;
     r.n_mt = (q.mode == WGRAD) ? r.n_mt_w + 1 : n_row_tiles;
-    const int n_splits = q.P > 0 ? q.P : ri->K;      // P = 0: one split per selected worker (its own rows)
+    const int n_splits = max(1, q.P > 0 ? q.P : ri->K);   // P = 0: one split per selected worker (its own rows)
     r.n_tiles = (q.mode == WGRAD) ? r.n_mt * r.n_ct * n_splits : n_row_tiles * r.n_ct;
     r.chunk = (q.mode == WGRAD) ? round_up((n_rows + n_splits - 1) / n_splits, BK) : 0;
     return r;
@@ -330,45 +362,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     const int t = unit + i * n_units;
     return t < T0 + T1 ? t : -1;
   };
-  if (tile_at(0) < 0) return;                   // same decision in both CTAs of a pair
+  // a CTA (pair) without work, or a run that has ended, goes straight to the teardown (same
+  // decision in both CTAs of a pair)
+  const bool has_work = running && tile_at(0) >= 0;
   const int RB = st->RB;
-
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* stage_out = smem + (size_t)C::STAGES * C::STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stage_out + C::OUT_BYTES);
-  uint64_t* full = bars;                     // [STAGES] TMA bytes landed
-  uint64_t* empty = bars + C::STAGES;        // [STAGES] MMAs that read the stage are done
-  uint64_t* acc_full = bars + 2 * C::STAGES; // [2] accumulator complete
-  uint64_t* acc_empty = acc_full + 2;        // [2] accumulator drained by the epilogue
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
-  volatile int* abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  __nv_bfloat16* bias_s = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<uint8_t*>(bars) + 256);   // [2][BN]
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS * CG); }
-    *abort = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 1) {
-    if (CG == 2) {
-      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    } else {
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::TMEM_COLS) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (CG == 2) cluster_sync_all();              // the peer's barriers exist before anything signals them
-  tc_fence_after();
-  // barriers that live in the leader CTA, as addresses valid from either CTA of the pair
-  const uint32_t full0_addr = (CG == 2) ? map_to_cta(smem_u32(&full[0]), 0) : smem_u32(&full[0]);
-  const uint32_t acc_empty0_addr = (CG == 2) ? map_to_cta(smem_u32(&acc_empty[0]), 0) : smem_u32(&acc_empty[0]);
-  const uint32_t tmem_base = *tmem_slot;
 
   auto tile_coord = [&](int gtile) -> TileCoord {
     TileCoord c;
@@ -403,7 +400,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     return c;
   };
 
-  if (warp == 0) {
+  if (!has_work) {
+    // nothing to do
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     int stage = 0;
     uint32_t phase = 0;
@@ -420,116 +419,56 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       else tma_load_3d(dst, map, &full[st_], x, y, z);
     };
     constexpr int BH = BN / CG;                  // B columns (rows of the B tile) this CTA loads
-    if (p0.gather_a == 0) {
-      // one elected lane: the stage ring is shallow, so nothing may sit between a stage being
-      // released and its next loads being issued
-      if (lane == 0) {
-        for (int it = 0; ok; ++it) {
-          const int tile = tile_at(it);
-          if (tile < 0) break;
-          const TileCoord c = tile_coord(tile);
-          const int mode = c.which ? p1.mode : p0.mode;
-          const CUtensorMap& map_a = c.which ? map_a1 : map_a0;
-          const CUtensorMap& map_b = c.which ? map_b1 : map_b0;
-          const int b0 = c.b_col + rank * BH;
-          {
-            // rows written by the other problem of this launch: wait (bounded) until all of their
-            // stores are complete, then order the tensor loads below after what was observed
-            const int* dw = c.which ? p1.done_wait : p0.done_wait;
-            if (dw != nullptr) {
-              const int target = c.which ? p1.done_target : p0.done_target;
-              const unsigned long long t0 = global_ns();
-              int seen;
-              for (uint32_t spin = 0;; ++spin) {
-                asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(dw + c.rt) : "memory");
-                if (seen >= target) break;
-                if ((spin & 63u) == 63u && (*abort || global_ns() - t0 > WAIT_LIMIT_NS)) { *abort = 1; ok = false; break; }
-              }
-              if (!ok) break;
-              asm volatile("fence.proxy.async;" ::: "memory");
-            }
-          }
-          for (int kb = 0; kb < c.n_kb; ++kb) {
-            if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) { ok = false; break; }
-            uint8_t* sa = smem + (size_t)stage * C::STAGE_BYTES;
-            uint8_t* sb = sa + C::A_BYTES;
-            if (rank == 0) {                     // the leader arms the barrier for the bytes of the whole pair
-              mbar_expect_tx(&full[stage], CG * C::STAGE_BYTES);
-              armed[stage] = (int)phase;
-            }
-            const int k0 = c.k_begin + kb * BK;
-            if (mode == FWD) {
-              ld2(sa, &map_a, stage, k0, c.a_row);
-              for (int j = 0; j < BH / 64; ++j) ld3(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0, c.slot);
-            } else if (mode == DGRAD) {
-              ld2(sa, &map_a, stage, k0, c.a_row);
-              ld3(sb, &map_b, stage, k0, b0, c.slot);
-            } else {
-              if (c.bias_tile) {   // only column 0 of the 64-wide ones matrix is non-zero; the rest is zero fill
-                for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_ones, stage, rank * BM + 64 * j, k0);
-              } else {
-                for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_a, stage, c.a_row + 64 * j, k0);
-              }
-              for (int j = 0; j < BH / 64; ++j) ld2(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0);
-            }
-            if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
-          }
-        }
-      }
-    } else {
-      // Operand A is the minibatch itself (first layer, FWD or WGRAD): its rows are fetched straight
-      // from the dataset by row index.  Lane 0 waits, arms the barrier and issues the tiled B loads;
-      // then every lane issues one four-row gather (32 x 4 = the 128 rows of a K-major tile, or
-      // the 64 rows x two 64-feature boxes of an MN-major one).  Rows of padding (index -1) lie
-      // outside the tensor and arrive as zeros.
-      const Params& p = p0;                      // a launch with row gathers serves one problem
-      const int mode = p0.mode;
-      const CUtensorMap& map_a = map_a0;
-      const CUtensorMap& map_b = map_b0;
-      auto ldg4 = [&](void* dst, int st_, int x, const int4& r) {
-        if (CG == 2) tma2_gather4(dst, &map_a, full0_addr + 8u * (uint32_t)st_, x, r);
-        else tma_gather4(dst, &map_a, &full[st_], x, r);
-      };
+    // one elected lane: the stage ring is shallow, so nothing may sit between a stage being
+    // released and its next loads being issued
+    if (lane == 0) {
       for (int it = 0; ok; ++it) {
         const int tile = tile_at(it);
         if (tile < 0) break;
         const TileCoord c = tile_coord(tile);
+        const int mode = c.which ? p1.mode : p0.mode;
+        const CUtensorMap& map_a = c.which ? map_a1 : map_a0;
+        const CUtensorMap& map_b = c.which ? map_b1 : map_b0;
         const int b0 = c.b_col + rank * BH;
-        const bool g_tile = !(mode == WGRAD && c.bias_tile);
-        // sample indices of the rows this lane gathers: fixed per tile (K-major A: the tile's
-        // rows), or per stage (MN-major A: the stage's 64 reduction rows, fetched one stage ahead)
-        int4 ridx = make_int4(-1, -1, -1, -1);
-        if (g_tile && c.n_kb > 0)
-          ridx = *reinterpret_cast<const int4*>(p.row_idx + (mode == WGRAD ? c.k_begin + 4 * (lane & 15) : c.a_row + 4 * lane));
+        {
+          // rows written by the other problem of this launch: wait (bounded) until all of their
+          // stores are complete, then order the tensor loads below after what was observed
+          const int* dw = c.which ? p1.done_wait : p0.done_wait;
+          if (dw != nullptr) {
+            const int target = c.which ? p1.done_target : p0.done_target;
+            const unsigned long long t0 = global_ns();
+            int seen;
+            for (uint32_t spin = 0;; ++spin) {
+              asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(dw + c.rt) : "memory");
+              if (seen >= target) break;
+              if ((spin & 63u) == 63u && (*abort || global_ns() - t0 > WAIT_LIMIT_NS)) { *abort = 1; ok = false; break; }
+            }
+            if (!ok) break;
+            asm volatile("fence.proxy.async;" ::: "memory");
+          }
+        }
         for (int kb = 0; kb < c.n_kb; ++kb) {
+          if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) { ok = false; break; }
           uint8_t* sa = smem + (size_t)stage * C::STAGE_BYTES;
           uint8_t* sb = sa + C::A_BYTES;
+          if (rank == 0) {                     // the leader arms the barrier for the bytes of the whole pair
+            mbar_expect_tx(&full[stage], CG * C::STAGE_BYTES);
+            armed[stage] = (int)phase;
+          }
           const int k0 = c.k_begin + kb * BK;
-          int4 rnext = ridx;
-          if (g_tile && mode == WGRAD && kb + 1 < c.n_kb)
-            rnext = *reinterpret_cast<const int4*>(p.row_idx + k0 + BK + 4 * (lane & 15));
-          if (lane == 0) {
-            ok = mbar_wait(&empty[stage], phase ^ 1u, abort);
-            if (ok && rank == 0) {
-              mbar_expect_tx(&full[stage], CG * C::STAGE_BYTES);
-              armed[stage] = (int)phase;
-            }
-          }
-          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-          if (!ok) break;
-          if (lane == 0) {
-            if (mode == FWD) {
-              for (int j = 0; j < BH / 64; ++j) ld3(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0, c.slot);
+          if (mode == FWD) {
+            ld2(sa, &map_a, stage, k0, c.a_row);
+            for (int j = 0; j < BH / 64; ++j) ld3(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0, c.slot);
+          } else if (mode == DGRAD) {
+            ld2(sa, &map_a, stage, k0, c.a_row);
+            ld3(sb, &map_b, stage, k0, b0, c.slot);
+          } else {
+            if (c.bias_tile) {   // only column 0 of the 64-wide ones matrix is non-zero; the rest is zero fill
+              for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_ones, stage, rank * BM + 64 * j, k0);
             } else {
-              if (c.bias_tile)
-                for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_ones, stage, rank * BM + 64 * j, k0);
-              for (int j = 0; j < BH / 64; ++j) ld2(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0);
+              for (int j = 0; j < BM / 64; ++j) ld2(sa + j * 8192, &map_a, stage, c.a_row + 64 * j, k0);
             }
-          }
-          if (g_tile) {
-            if (mode == WGRAD) ldg4(sa + (lane >> 4) * 8192 + (lane & 15) * 512, stage, c.a_row + 64 * (lane >> 4), ridx);
-            else ldg4(sa + lane * 512, stage, k0, ridx);
-            ridx = rnext;
+            for (int j = 0; j < BH / 64; ++j) ld2(sb + j * 8192, &map_b, stage, b0 + 64 * j, k0);
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }

@@ -102,9 +102,8 @@ def _init_args():
     (lambda m, td: setattr(m, "local_steps", 0), gpu.EINVAL),
     (lambda m, td: setattr(m, "local_steps", 2000), gpu.EINVAL),
     (lambda m, td: (setattr(m, "local_steps", 4), setattr(m, "batch", 1024), m.dims.__setitem__(0, 20000)), gpu.EUNSUPPORTED),
-    (lambda m, td: (setattr(m, "kind", gpu.MLP), setattr(m, "n_layers", 2), setattr(m, "dtype", gpu.BF16_FP32MASTER),
-                    m.dims.__setitem__(0, 64), m.dims.__setitem__(1, 128), m.dims.__setitem__(2, 10),
-                    setattr(m, "local_steps", 4), setattr(m, "flags", gpu.FLAG_TMA_GATHER)), gpu.EUNSUPPORTED),
+    (lambda m, td: setattr(m, "restart_rule", 3), gpu.EINVAL),
+    (lambda m, td: setattr(m, "sa_penalty", 2), gpu.EINVAL),
     (lambda m, td: setattr(m, "workspace", 0), gpu.EINVAL),
     (lambda m, td: setattr(m, "workspace", 0x10010), gpu.EINVAL),
     (lambda m, td: setattr(m, "workspace_bytes", 1024), gpu.ENOSPACE),

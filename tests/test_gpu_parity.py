@@ -223,15 +223,6 @@ def test_local_sgd_steps_multi_layer_network_fma_paths(dims, dtype, W, B, U, K0,
     assert rows[-1]["loss_mean"] < rows[0]["loss_mean"]
 
 
-def test_local_sgd_steps_rejected_with_row_gather_by_tma():
-    cfg = _small_cfg(inputs.MLP, (64, 128, 10), inputs.BF16, 8, 16, 3, 5, EXP)
-    X, y, w0 = _problem(cfg)
-    Xd, yd = to_device(cfg, X, y)
-    with pytest.raises(gpu.AbsError) as e:
-        gpu.context_from_config(cfg, Xd, yd, w0, max_rounds=5, local_steps=4, flags=gpu.FLAG_TMA_GATHER)
-    assert e.value.code == gpu.EUNSUPPORTED
-
-
 def test_lock_step_constant_times():
     cfg = _small_cfg(inputs.LSQ, (16, 1), inputs.FP32, 8, 4, 2, 3,
                      inputs.TimeSpec(inputs.T_CONST, shift=3.0))
@@ -347,21 +338,6 @@ def test_side_stream_overlap_changes_nothing(idx, rounds, n):
     assert np.array_equal(params_a, params_b)
 
 
-@pytest.mark.parametrize("dims,B", [((3072, 1024, 512, 10), 64), ((320, 520, 264, 10), 40), ((784, 256, 10), 128)])
-def test_tma_row_gather_matches_the_copy_kernel(dims, B):
-    """With the flag the first layer's GEMMs fetch the minibatch rows from the dataset by row index
-    (TMA four-row gathers) instead of reading the dense copy made by the gather kernel.  Both feed
-    the tensor cores the same operands, so traces and parameters must be identical bit for bit,
-    and both agree with the oracle."""
-    cfg = _small_cfg(inputs.MLP, dims, inputs.BF16, 13, B, 3, 5, PARETO)
-    X, y, w0 = _problem(cfg)
-    rows_a, params_a = gpu_run(cfg, X, y, w0, 25)
-    rows_b, params_b = gpu_run(cfg, X, y, w0, 25, flags=gpu.FLAG_TMA_GATHER)
-    assert rows_a == rows_b
-    assert np.array_equal(params_a, params_b)
-    compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_TMA_GATHER)
-
-
 @pytest.mark.parametrize("dims,W,B", [((3072, 1024, 512, 10), 32, 64), ((320, 520, 264, 10), 13, 40),
                                       ((256, 512, 512, 256, 10), 24, 32)])
 def test_merged_backward_launch_matches_separate_launches(dims, W, B):
@@ -402,17 +378,6 @@ def test_bf16_network_without_tensor_cores():
     assert ctx.plan()["path"] == [0, 0, 2]        # no layer on the tensor-core path
     ctx.close()
     compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_NO_TENSOR_CORES)
-
-
-def test_cta_pair_gemms_match_single_cta_gemms():
-    """Opt-in tcgen05 cta_group::2 tiles (256 x 256 over a CTA pair) against the default tiles."""
-    cfg = _small_cfg(inputs.MLP, (320, 520, 264, 10), inputs.BF16, 13, 40, 3, 5, PARETO)
-    X, y, w0 = _problem(cfg)
-    rows_a, params_a = gpu_run(cfg, X, y, w0, 25, k_mode=gpu.K_FIXED)
-    rows_b, params_b = gpu_run(cfg, X, y, w0, 25, k_mode=gpu.K_FIXED, flags=gpu.FLAG_TWO_CTA)
-    assert [r["sel"] for r in rows_a] == [r["sel"] for r in rows_b]
-    assert rel_l2(params_b, params_a) < 1e-4
-    compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_TWO_CTA)
 
 
 @pytest.mark.parametrize("d,W,B,K0,S", [(4096, 200, 32, 25, 32), (1000, 160, 19, 7, 6), (2056, 300, 8, 300, 0)])
