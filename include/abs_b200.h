@@ -50,6 +50,8 @@ extern "C" {
 #define ABS_LSQ      0  /* f = 1/2 (x.w - y)^2, dims = {d, 1}, no bias */
 #define ABS_SOFTMAX  1  /* one affine layer + soft-max cross-entropy */
 #define ABS_MLP      2  /* affine layers with ReLU between them + soft-max cross-entropy */
+#define ABS_CNN      3  /* the paper's model class (Sec. V-A): two blocks of k x k convolution (stride 1, no padding)
+                           + ReLU + 2 x 2 max-pool in front of an ABS_MLP of at least two layers; see `conv` */
 
 /* storage/arithmetic type */
 #define ABS_FP32             0  /* fp32 data, fp32 models, fp32 FMA */
@@ -122,6 +124,13 @@ typedef struct {
   int kind;                 /* ABS_LSQ | ABS_SOFTMAX | ABS_MLP */
   int n_layers;             /* affine layers; dims has n_layers + 1 entries */
   int dims[ABS_MAX_LAYERS + 1]; /* e.g. {3072,1024,512,10}; LSQ: {d,1}; last dim = classes (<= 64) */
+  int conv[6];              /* ABS_CNN only: {H, W, C_in, k, C1, C2}: image size and channels, kernel size, output
+                               channels of the two blocks.  Dataset rows are images stored [H][W][C_in]; both
+                               convolution outputs must be even-sized; dims[0] must equal the number of features
+                               the second block delivers, (rows x columns x C2) of its pooled maps, which are
+                               flattened in that order.  Parameter vector: W1[k][k][C_in][C1], b1[C1],
+                               W2[k][k][C1][C2], b2[C2], then the affine layers as for ABS_MLP.  A block has at
+                               most 4096 parameters; local_steps must be 1 */
   int batch;                /* B of Eq. 2, 1..1024 */
   float lr;                 /* eta, constant */
   int dtype;                /* ABS_FP32 | ABS_BF16_FP32MASTER */
@@ -146,7 +155,8 @@ typedef struct {
   int data_on_host;         /* 0: X, y are device pointers owned by the caller and must outlive
                                the context.  1: X, y are host pointers; abs_init copies them into
                                the workspace (abs_workspace_bytes accounts for the room) */
-  const void* X;            /* [n_samples][dims[0]] row-major; float (FP32) or bf16 bits (BF16) */
+  const void* X;            /* [n_samples][dims[0]] row-major (ABS_CNN: [n_samples][H*W*C_in]); float (FP32) or
+                               bf16 bits (BF16) */
   const void* y;            /* float targets (LSQ) or int32 labels in [0, classes) */
   long long n_samples;      /* M of Eq. 1; worker n owns samples [n*M/N, (n+1)*M/N) */
   const float* w0;          /* host, n_params floats, copied by abs_init */

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libabs_b200.so")
 
 OK, EINVAL, ENOSPACE, EUNSUPPORTED, ESTATE, ECUDA, ETIMEOUT, EDIVERGED, ERANGE, ESTALE = \
     0, -1, -2, -3, -4, -5, -6, -7, -8, -9
-LSQ, SOFTMAX, MLP = 0, 1, 2
+LSQ, SOFTMAX, MLP, CNN = 0, 1, 2, 3
 FP32, BF16_FP32MASTER = 0, 1
 K_ADAPTIVE, K_FIXED = 0, 1
 BOUND_ADAPTIVE, BOUND_FIXED, BOUND_OFFSET = 0, 1, 2
@@ -33,7 +33,7 @@ KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "lsq", "update",
 
 class ModelDesc(C.Structure):
     _fields_ = [("kind", C.c_int), ("n_layers", C.c_int), ("dims", C.c_int * (MAX_LAYERS + 1)),
-                ("batch", C.c_int), ("lr", C.c_float), ("dtype", C.c_int),
+                ("conv", C.c_int * 6), ("batch", C.c_int), ("lr", C.c_float), ("dtype", C.c_int),
                 ("local_steps", C.c_int), ("k_mode", C.c_int), ("bound_mode", C.c_int),
                 ("bound_offset", C.c_int), ("restart_rule", C.c_int), ("sa_penalty", C.c_int), ("max_rounds", C.c_int), ("flags", C.c_int), ("data_on_host", C.c_int),
                 ("X", C.c_void_p), ("y", C.c_void_p), ("n_samples", C.c_longlong),
@@ -113,14 +113,18 @@ def _check(rc):
         raise AbsError(rc, last_error())
 
 
-def n_params(kind, dims):
+def n_params(kind, dims, conv=None):
     if kind == LSQ:
         return dims[0]
-    return sum(dims[l] * dims[l + 1] + dims[l + 1] for l in range(len(dims) - 1))
+    n = sum(dims[l] * dims[l + 1] + dims[l + 1] for l in range(len(dims) - 1))
+    if kind == CNN:
+        _, _, c_in, k, c1, c2 = conv
+        n += k * k * c_in * c1 + c1 + k * k * c1 * c2 + c2
+    return n
 
 
 def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-          local_steps=1, data_on_host=0, flags=0, bound_offset=0, restart_rule=0, sa_penalty=0):
+          local_steps=1, data_on_host=0, flags=0, bound_offset=0, restart_rule=0, sa_penalty=0, conv=None):
     m = ModelDesc()
     m.kind, m.n_layers = kind, len(dims) - 1
     for i, v in enumerate(dims):
@@ -132,6 +136,8 @@ def _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mod
     m.bound_offset = int(bound_offset)
     m.restart_rule = int(restart_rule)
     m.sa_penalty = int(sa_penalty)
+    for i, v in enumerate(conv or ()):
+        m.conv[i] = int(v)
     return m
 
 
@@ -154,14 +160,15 @@ class Context:
     def __init__(self, kind, dims, X, y, w0, batch, lr, W, K0, S, time, seed, max_rounds,
                  dtype=FP32, k_mode=K_ADAPTIVE, bound_mode=BOUND_ADAPTIVE, local_steps=1,
                  data_on_host=False, stream=None, device="cuda:0", flags=0, bound_offset=0,
-                 restart_rule=0, sa_penalty=0):
+                 restart_rule=0, sa_penalty=0, conv=None):
         import torch
         self._torch = torch
         self.kind, self.dims, self.W, self.S = kind, list(dims), W, S
+        self.conv = None if conv is None else tuple(conv)
         self.max_rounds = max_rounds
         n_samples = X.shape[0]
         m = _desc(kind, dims, batch, lr, dtype, max_rounds, n_samples, k_mode, bound_mode,
-                  local_steps, 1 if data_on_host else 0, flags, bound_offset, restart_rule, sa_penalty)
+                  local_steps, 1 if data_on_host else 0, flags, bound_offset, restart_rule, sa_penalty, conv)
         need = C.c_size_t(0)
         _check(lib().abs_workspace_bytes(C.byref(m), W, S, C.byref(need)))
         self.device = torch.device(device)
@@ -178,7 +185,7 @@ class Context:
             assert X.is_cuda and y.is_cuda and X.is_contiguous() and y.is_contiguous()
             m.X, m.y = X.data_ptr(), y.data_ptr()
         w0 = np.ascontiguousarray(w0, dtype=np.float32)
-        assert w0.shape[0] == n_params(kind, dims)
+        assert w0.shape[0] == n_params(kind, dims, conv)
         m.w0 = w0.ctypes.data
         m.workspace, m.workspace_bytes = self.workspace.data_ptr(), need.value
         m.stream = self.stream.cuda_stream
@@ -202,7 +209,7 @@ class Context:
         return r.value, rc
 
     def get_params(self):
-        d = n_params(self.kind, self.dims)
+        d = n_params(self.kind, self.dims, self.conv)
         out = np.empty(d, dtype=np.float32)
         got = C.c_size_t(0)
         _check(lib().abs_get_params(self._ctx, out.ctypes.data, d, C.byref(got)))
@@ -341,4 +348,4 @@ def context_from_config(cfg, X, y, w0, max_rounds=None, **kw):
     """Context for an `inputs.Config`; X, y as produced by `inputs.make_data` moved to the
     device by the caller (or numpy with data_on_host=True)."""
     return Context(cfg.kind, cfg.dims, X, y, w0, cfg.batch, cfg.lr, cfg.W, cfg.K0, cfg.S, cfg.time,
-                   cfg.run_seed, max_rounds or cfg.rounds, dtype=cfg.dtype, **kw)
+                   cfg.run_seed, max_rounds or cfg.rounds, dtype=cfg.dtype, conv=getattr(cfg, "conv", None), **kw)

@@ -18,6 +18,7 @@
 #include "local.cuh"
 #include "localnet.cuh"
 #include "persist.cuh"
+#include "conv.cuh"
 
 using namespace absb;
 
@@ -74,6 +75,12 @@ struct Layout {
   size_t sel[2], sel_tau[2], sel_row0[2], row_idx[2], tile_slot[2];   // per-round layout, by round parity
   size_t act0b;                         // second copy of the gathered input rows (odd rounds)
   size_t master, ring, G, logits, red, ones;
+  // convolution blocks of ABS_CNN (two of them, in front of the affine layers)
+  bool cnn = false;
+  int cHi[2] = {}, cWi[2] = {}, cCi[2] = {}, cCo[2] = {}, ck = 0;   // input map, channels of each block
+  size_t c_off[2] = {}, c_src[2] = {}, c_len[2] = {};               // W[k][k][Ci][Co] + b[Co]: padded / caller offset, length
+  size_t x_len = 0;                       // elements of one dataset row
+  size_t pool1 = 0, dpool1 = 0, arg1 = 0, arg2 = 0, cpart[2] = {};  // pooled maps of block 1, their delta, pool positions, chunk sums
   size_t bits[ABS_MAX_LAYERS + 1];      // ReLU sign bits of act[l] (tensor-core layers)
   size_t act[ABS_MAX_LAYERS + 1], delta[ABS_MAX_LAYERS + 1];
   size_t tr_K, tr_R, tr_theta, tr_T, tr_loss, tr_comm, tr_sel_off, tr_rst_off;
@@ -90,7 +97,7 @@ struct Layout {
 
 int check_model(const abs_model_desc* m, int W, int S) {
   if (!m) return fail(ABS_EINVAL, "model is null");
-  if (m->kind != ABS_LSQ && m->kind != ABS_SOFTMAX && m->kind != ABS_MLP)
+  if (m->kind != ABS_LSQ && m->kind != ABS_SOFTMAX && m->kind != ABS_MLP && m->kind != ABS_CNN)
     return fail(ABS_EUNSUPPORTED, "unknown model kind %d", m->kind);
   if (m->dtype != ABS_FP32 && m->dtype != ABS_BF16_FP32MASTER)
     return fail(ABS_EUNSUPPORTED, "unknown dtype %d", m->dtype);
@@ -103,6 +110,23 @@ int check_model(const abs_model_desc* m, int W, int S) {
   if (m->kind == ABS_LSQ && m->dims[1] != 1) return fail(ABS_EINVAL, "least squares needs dims = {d, 1}");
   if (m->kind != ABS_LSQ && (m->dims[m->n_layers] < 2 || m->dims[m->n_layers] > 64))
     return fail(ABS_EINVAL, "class count %d outside [2, 64]", m->dims[m->n_layers]);
+  if (m->kind == ABS_CNN) {
+    const int H = m->conv[0], Wd = m->conv[1], Ci = m->conv[2], k = m->conv[3], C1 = m->conv[4], C2 = m->conv[5];
+    if (m->n_layers < 2) return fail(ABS_EINVAL, "ABS_CNN needs at least two affine layers behind the convolution blocks");
+    if (H < 1 || Wd < 1 || Ci < 1 || k < 1 || C1 < 1 || C2 < 1 || H > 1024 || Wd > 1024 || Ci > 1024 || C1 > 1024 || C2 > 1024)
+      return fail(ABS_EINVAL, "conv = {H, W, C_in, k, C1, C2} out of range");
+    const int H1 = H - k + 1, W1 = Wd - k + 1;
+    if (H1 < 2 || W1 < 2 || (H1 & 1) || (W1 & 1)) return fail(ABS_EINVAL, "first convolution output %d x %d must be even-sized and at least 2 x 2", H1, W1);
+    const int H2 = H1 / 2 - k + 1, W2 = W1 / 2 - k + 1;
+    if (H2 < 2 || W2 < 2 || (H2 & 1) || (W2 & 1)) return fail(ABS_EINVAL, "second convolution output %d x %d must be even-sized and at least 2 x 2", H2, W2);
+    if ((long long)(H2 / 2) * (W2 / 2) * C2 != m->dims[0])
+      return fail(ABS_EINVAL, "dims[0] = %d, but the second block delivers %d features", m->dims[0], (H2 / 2) * (W2 / 2) * C2);
+    if ((long long)k * k * Ci * C1 + C1 > 4096 || (long long)k * k * C1 * C2 + C2 > 4096)
+      return fail(ABS_EUNSUPPORTED, "a convolution block may have at most 4096 parameters");
+    if (conv::bwd_smem_bytes(H, Wd, Ci, k, C1) > 200 * 1024 || conv::bwd_smem_bytes(H1 / 2, W1 / 2, C1, k, C2) > 200 * 1024)
+      return fail(ABS_EUNSUPPORTED, "convolution maps too large for the shared-memory kernels");
+    if (m->local_steps > 1) return fail(ABS_EUNSUPPORTED, "local_steps > 1 is not implemented for ABS_CNN");
+  }
   if (m->batch < 1 || m->batch > 1024) return fail(ABS_EINVAL, "batch %d outside [1, 1024]", m->batch);
   if (m->max_rounds < 1) return fail(ABS_EINVAL, "max_rounds %d < 1", m->max_rounds);
   if (m->n_samples < 1 || m->n_samples > 0x7fffffffLL) return fail(ABS_EINVAL, "n_samples out of range");
@@ -123,6 +147,21 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   const bool lsq = m->kind == ABS_LSQ;
   // padded parameter vector: each layer's [W | b] block starts on a 64-element boundary
   size_t off = 0, src = 0;
+  L->cnn = m->kind == ABS_CNN;
+  L->x_len = (size_t)m->dims[0];
+  if (L->cnn) {
+    const int H = m->conv[0], Wd = m->conv[1], k = m->conv[3];
+    L->ck = k;
+    L->cHi[0] = H; L->cWi[0] = Wd; L->cCi[0] = m->conv[2]; L->cCo[0] = m->conv[4];
+    L->cHi[1] = (H - k + 1) / 2; L->cWi[1] = (Wd - k + 1) / 2; L->cCi[1] = m->conv[4]; L->cCo[1] = m->conv[5];
+    L->x_len = (size_t)H * Wd * m->conv[2];
+    for (int b = 0; b < 2; ++b) {
+      L->c_len[b] = (size_t)k * k * L->cCi[b] * L->cCo[b] + L->cCo[b];
+      L->c_off[b] = off; L->c_src[b] = src;
+      off = round_up_sz(off + L->c_len[b], 64);
+      src += L->c_len[b];
+    }
+  }
   for (int l = 0; l < m->n_layers; ++l) {
     L->w_off[l] = off;
     L->w_src[l] = src;
@@ -279,12 +318,21 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     for (int l = 0; l <= m->n_layers; ++l) L->bits[l] = 0;
     for (int l = 0; l + 1 < m->n_layers; ++l)
       if (L->path[l] == PATH_TC) L->bits[l + 1] = cv.take(4 * (size_t)L->rows_cap * ((m->dims[l + 1] + 31) / 32));
-    const bool copy0 = L->path[0] == PATH_TC;     // gathered copies of the input rows
+    const bool copy0 = L->path[0] == PATH_TC || L->cnn;     // gathered copies of the input rows (CNN: the features)
     L->act[0] = copy0 ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     L->act0b = copy0 ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]) : 0;
     for (int l = 1; l <= m->n_layers; ++l) {
       L->act[l] = (l < m->n_layers) ? cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]) : 0;
       L->delta[l] = cv.take(L->esz * (size_t)L->rows_cap * m->dims[l]);
+    }
+    if (L->cnn) {
+      const size_t n_p1 = (size_t)L->cHi[1] * L->cWi[1] * L->cCi[1];        // pooled maps of block 1 per row
+      L->delta[0] = cv.take(L->esz * (size_t)L->rows_cap * m->dims[0]);
+      L->pool1 = cv.take(L->esz * (size_t)L->rows_cap * n_p1);
+      L->dpool1 = cv.take(L->esz * (size_t)L->rows_cap * n_p1);
+      L->arg1 = cv.take((size_t)L->rows_cap * n_p1);
+      L->arg2 = cv.take((size_t)L->rows_cap * m->dims[0]);
+      for (int b = 0; b < 2; ++b) L->cpart[b] = cv.take(4 * L->c_len[b] * (size_t)(L->rows_cap / conv::CHUNK));
     }
   }
   const size_t R = (size_t)m->max_rounds;
@@ -301,7 +349,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   L->tr_sel_loss = cv.take(4 * R * W);
   L->tr_rst_id = cv.take(4 * R * W);
   if (m->data_on_host) {
-    L->data_X = cv.take(L->esz * (size_t)m->n_samples * m->dims[0]);
+    L->data_X = cv.take(L->esz * (size_t)m->n_samples * L->x_len);
     L->data_y = cv.take(4 * (size_t)m->n_samples);
   }
   L->total = cv.off;
@@ -518,7 +566,7 @@ int setup_tc(abs_ctx* ctx) {
     if (ok && l == 0)
       ok = make_act_map(&t.fwd_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 128) &&
            make_act_map(&t.wg_a_odd, ctx->at<void>(L.act0b), in, L.rows_cap, 64);
-    if (ok && l > 0)
+    if (ok && (l > 0 || L.cnn))
       ok = make_act_map(&t.dg_a, delta_out, out, L.rows_cap, 128) &&
            make_w_map(&t.dg_b, wbase, in, out, L.gslots, L.d_pad, L.bn_dg[l] / L.cg_dg[l]) &&
            make_act_map(&t.dg_out, ctx->at<void>(L.delta[l]), in, L.rows_cap, 32);
@@ -567,7 +615,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
   const int nl = m.n_layers;
   const int row_tiles = L.rows_cap / TM;
   const int row_tiles128 = L.rows_cap / 128;
-  const bool gathered = L.path[0] == PATH_TC;     // layer 0 reads the gathered copy act[0]
+  const bool gathered = L.path[0] == PATH_TC || L.cnn;     // layer 0 reads act[0]: the gathered rows, or the CNN's features
   const int n_splits = L.P > 0 ? L.P : ctx->W;    // weight-gradient splits (P = 0: one per selected worker)
   LayerArgs la[ABS_MAX_LAYERS];
   for (int l = 0; l < nl; ++l) {
@@ -579,9 +627,23 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     a.act_in = (l == 0 && !gathered) ? ctx->X : ctx->at<void>((l == 0 && par) ? L.act0b : L.act[l]);
     a.act_out = (l == nl - 1) ? ctx->at<void>(L.logits) : ctx->at<void>(L.act[l + 1]);
     a.delta_out = ctx->at<void>(L.delta[l + 1]);
-    a.delta_in = (l == 0) ? nullptr : ctx->at<void>(L.delta[l]);
+    a.delta_in = (l == 0 && !L.cnn) ? nullptr : ctx->at<void>(L.delta[l]);
     a.G = ctx->at<float>(L.G); a.P = L.P;
   }
+  // convolution block b of the CNN (0: images -> pooled maps, 1: pooled maps -> features)
+  auto conv_args = [&](int b) {
+    conv::Args c;
+    c.st = st; c.ri = ri; c.tile_slot = ctx->ctl.tile_slot[par]; c.row_idx = ctx->ctl.row_idx[par];
+    c.ring = ctx->at<void>(L.gring); c.slot_stride = L.d_pad; c.w_off = L.c_off[b];
+    c.Hi = L.cHi[b]; c.Wi = L.cWi[b]; c.Ci = L.cCi[b]; c.k = L.ck; c.Co = L.cCo[b];
+    c.in = b == 0 ? ctx->X : ctx->at<void>(L.pool1); c.from_dataset = b == 0 ? 1 : 0;
+    c.pooled = b == 0 ? ctx->at<void>(L.pool1) : ctx->at<void>(par ? L.act0b : L.act[0]);
+    c.arg = ctx->at<unsigned char>(b == 0 ? L.arg1 : L.arg2);
+    c.d_pooled = b == 0 ? ctx->at<void>(L.dpool1) : ctx->at<void>(L.delta[0]);
+    c.d_in = b == 0 ? nullptr : ctx->at<void>(L.dpool1);
+    c.part = ctx->at<float>(L.cpart[b]);
+    return c;
+  };
   auto tc_params = [&](int l, int mode) {
     tc::Params p;
     memset(&p, 0, sizeof p);
@@ -601,6 +663,15 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     a.row_loss = L.local_net ? ctx->at<float>(L.row_loss) : ctx->ctl.row_loss; a.G = ctx->at<float>(L.G); a.P = L.P;
     return a;
   };
+  if (phase == PH_GATHER && L.cnn) {
+    // Eq. 2 forward through the two convolution blocks: the features are the input rows of layer 0
+    for (int b = 0; b < 2; ++b) {
+      const conv::Args c = conv_args(b);
+      launch_ex(ctx, ABS_KC_FWD, conv::conv_block_fwd_kernel<T>, dim3(L.rows_cap), dim3(conv::THREADS),
+                conv::fwd_smem_bytes(c.Hi, c.Wi, c.Ci, c.k, c.Co), c);
+    }
+    return;
+  }
   if (phase == PH_GATHER) {
     if (gathered)
       launch_on(ctx, ctx->overlap ? ctx->side : s, ABS_KC_GATHER, gather_rows_kernel, dim3(ctx->sm_count * 8), dim3(256), 0,
@@ -706,7 +777,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
                      ((la[l].in + 127) / 128 + 1) * ((la[l].out + bnd - 1) / bnd) * n_splits, &second);
         continue;
       }
-      if (l > 0)
+      if (l > 0 || L.cnn)
         launch_tc_bn(ctx, bnd, L.cg_dg[l], ABS_KC_DGRAD, ctx->tcl[l].dg_a, ctx->tcl[l].dg_b, ctx->tcl[l].dg_out, pd, dg_tiles);
       const int bn = L.bn_wg[l];
       const int tmw = 128 * L.cg_wg[l];
@@ -737,13 +808,22 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
         launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, 64);
     } else {
       const bool last = l == nl - 1;
-      if (l > 0) {
+      if (l > 0 || L.cnn) {
         dim3 grid((la[l].in + TN - 1) / TN, row_tiles);
         launch_ex(ctx, last ? ABS_KC_OUTPUT : ABS_KC_DGRAD, simt_dgrad_kernel<T>, dim3(grid), dim3(256), 0, la[l]);
       }
       dim3 gridw((la[l].out + TN - 1) / TN, (la[l].in + 1 + TM - 1) / TM, n_splits);
       launch_ex(ctx, last ? ABS_KC_OUTPUT : ABS_KC_WGRAD, simt_wgrad_kernel<T>, dim3(gridw), dim3(256), 0, la[l]);
     }
+  }
+  // ---- CNN: back through the convolution blocks (second, then first); their weight gradients are
+  // per-chunk sums that a fixed-order reduction adds up into partial 0 of the gradient vector
+  for (int b = 1; b >= 0 && phase == PH_BACKWARD && L.cnn; --b) {
+    const conv::Args c = conv_args(b);
+    launch_ex(ctx, ABS_KC_WGRAD, conv::conv_block_bwd_kernel<T>, dim3(L.rows_cap / conv::CHUNK), dim3(conv::THREADS),
+              conv::bwd_smem_bytes(c.Hi, c.Wi, c.Ci, c.k, c.Co), c);
+    launch_ex(ctx, ABS_KC_WGRAD, chunk_reduce_kernel, dim3(((int)L.c_len[b] + 31) / 32), dim3(256), 0, st, ri, c.part, (int)L.c_len[b],
+              ctx->at<float>(L.G) + L.c_off[b], conv::CHUNK);
   }
 }
 
@@ -895,7 +975,7 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   cudaError_t e = cudaMemsetAsync(ctx->ws, 0, zero_bytes, s);
   if (e != cudaSuccess) return bail(cuda_fail(nullptr, e, "cudaMemsetAsync(workspace)"));
   if (model->data_on_host) {
-    e = cudaMemcpyAsync(ctx->ws + L.data_X, model->X, L.esz * (size_t)model->n_samples * model->dims[0], cudaMemcpyHostToDevice, s);
+    e = cudaMemcpyAsync(ctx->ws + L.data_X, model->X, L.esz * (size_t)model->n_samples * L.x_len, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->ws + L.data_y, model->y, 4 * (size_t)model->n_samples, cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return bail(cuda_fail(nullptr, e, "dataset copy"));
     ctx->X = ctx->ws + L.data_X;
@@ -909,6 +989,10 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     const size_t n = model->kind == ABS_LSQ ? (size_t)model->dims[0]
                                              : (size_t)model->dims[l] * model->dims[l + 1] + model->dims[l + 1];
     e = cudaMemcpyAsync(ctx->at<float>(L.master) + L.w_off[l], model->w0 + L.w_src[l], 4 * n, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return bail(cuda_fail(nullptr, e, "w0 copy"));
+  }
+  for (int b = 0; b < 2 && L.cnn; ++b) {
+    e = cudaMemcpyAsync(ctx->at<float>(L.master) + L.c_off[b], model->w0 + L.c_src[b], 4 * L.c_len[b], cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return bail(cuda_fail(nullptr, e, "w0 copy"));
   }
   DevState h;
@@ -1033,7 +1117,18 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
   }
   // worth it only when a round has a long backward pass to hide behind (tensor-core networks);
   // for the latency-bound models the cross-stream events cost more than they hide
-  if (!(model->flags & ABS_FLAG_NO_OVERLAP) && L.any_tc && !L.local_net) {
+  if (L.cnn) {
+    size_t need = 0;
+    for (int b = 0; b < 2; ++b)
+      need = std::max(need, std::max(conv::fwd_smem_bytes(L.cHi[b], L.cWi[b], L.cCi[b], L.ck, L.cCo[b]),
+                                     conv::bwd_smem_bytes(L.cHi[b], L.cWi[b], L.cCi[b], L.ck, L.cCo[b])));
+    cudaError_t ec = cudaFuncSetAttribute(conv::conv_block_fwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_fwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (ec != cudaSuccess) return bail(cuda_fail(nullptr, ec, "cudaFuncSetAttribute(conv_block kernels)"));
+  }
+  if (!(model->flags & ABS_FLAG_NO_OVERLAP) && L.any_tc && !L.local_net && !L.cnn) {
     cudaError_t es = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
     if (es == cudaSuccess) es = cudaEventCreateWithFlags(&ctx->ev_loss, cudaEventDisableTiming);
     if (es == cudaSuccess) es = cudaEventCreateWithFlags(&ctx->ev_ctl, cudaEventDisableTiming);
@@ -1211,6 +1306,8 @@ int abs_get_params(abs_ctx* ctx, float* dst, size_t cap, size_t* d_out) {
                                              : (size_t)ctx->m.dims[l] * ctx->m.dims[l + 1] + ctx->m.dims[l + 1];
     CU(cudaMemcpyAsync(dst + L.w_src[l], ctx->at<float>(L.master) + L.w_off[l], 4 * n, cudaMemcpyDeviceToHost, ctx->stream));
   }
+  for (int b = 0; b < 2 && L.cnn; ++b)
+    CU(cudaMemcpyAsync(dst + L.c_src[b], ctx->at<float>(L.master) + L.c_off[b], 4 * L.c_len[b], cudaMemcpyDeviceToHost, ctx->stream));
   CU(cudaStreamSynchronize(ctx->stream));
   return ABS_OK;
 }
@@ -1224,7 +1321,7 @@ struct StateHeader {
   int version, rounds_enqueued;
   unsigned long long d_pad, esz, block1, block2, max_rounds;
   // what the saving context was created with (checked on restore)
-  int kind, n_layers, dims[ABS_MAX_LAYERS + 1], batch, dtype, local_steps, flags, restart_rule, sa_penalty;
+  int kind, n_layers, dims[ABS_MAX_LAYERS + 1], conv[6], batch, dtype, local_steps, flags, restart_rule, sa_penalty;
   float lr;
   DevState st;                       // its state block (constants checked on restore)
 };
@@ -1233,6 +1330,7 @@ constexpr unsigned long long STATE_MAGIC = 0x3230455441545341ull;   // "ASTATE02
 void describe_model(const abs_model_desc& m, StateHeader* h) {
   h->kind = m.kind; h->n_layers = m.n_layers;
   for (int l = 0; l <= ABS_MAX_LAYERS; ++l) h->dims[l] = l <= m.n_layers ? m.dims[l] : 0;
+  for (int i = 0; i < 6; ++i) h->conv[i] = m.kind == ABS_CNN ? m.conv[i] : 0;
   h->batch = m.batch; h->dtype = m.dtype; h->local_steps = m.local_steps; h->flags = m.flags;
   h->restart_rule = m.restart_rule; h->sa_penalty = m.sa_penalty; h->lr = m.lr;
 }
@@ -1242,6 +1340,7 @@ bool same_model(const StateHeader& a, const StateHeader& b) {
               a.local_steps == b.local_steps && a.flags == b.flags && a.restart_rule == b.restart_rule &&
               a.sa_penalty == b.sa_penalty && a.lr == b.lr;
   for (int l = 0; l <= ABS_MAX_LAYERS; ++l) same = same && a.dims[l] == b.dims[l];
+  for (int i = 0; i < 6; ++i) same = same && a.conv[i] == b.conv[i];
   return same;
 }
 

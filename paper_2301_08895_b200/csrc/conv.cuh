@@ -1,0 +1,217 @@
+// The two convolution blocks in front of the fully connected layers of the paper's model class
+// (Sec. V-A: "two convolutional layers and three fully connected layers" on 32 x 32 x 3 images).
+// A block is a k x k convolution (stride 1, no padding), ReLU, and a 2 x 2 max-pool of stride 2.
+//
+//   forward   a[y][x][co] = relu( b[co] + sum_{dy,dx,ci} in[y+dy][x+dx][ci] W_s[dy][dx][ci][co] )   (stored rounded)
+//             p[py][px][co] = max of the 2 x 2 window of a, arg = position of its first maximum
+//   backward  the delta of p goes to the window position `arg` (it arrives already zeroed where
+//             p is not positive, i.e. where the ReLU was inactive);
+//             G[dy][dx][ci][co] = sum over rows and pooled pixels of in[2py+ay+dy][2px+ax+dx][ci] dp[py][px][co]
+//             d_in[y][x][ci]    = ( sum_{dy,dx,co} dz[y-dy][x-dx][co] W_s[dy][dx][ci][co] ) [in[y][x][ci] > 0]
+// (Eq. 2 with U = 1 at the model version s the row's worker holds; Eq. 3 needs only the sum of G
+// over all rows.)  Maps are stored [row][y][x][channel] in the storage type; the images of the
+// first block are dataset rows fetched by sample index.  The channel counts of this model class
+// are far below a tensor-core tile (3 -> 6 -> 16 in the benchmark network), so these are FP32-FMA
+// kernels: one CTA per gradient row forward, one CTA per 16 rows backward, everything the CTA
+// needs staged in shared memory, fixed summation orders.
+#pragma once
+#include "common.cuh"
+#include "simt.cuh"
+
+namespace absb {
+namespace conv {
+
+constexpr int THREADS = 256;
+constexpr int CHUNK = 16;        // gradient rows per CTA of the backward kernel (divides the row padding unit)
+
+struct Args {
+  DevState* st;
+  RoundInfo* ri;
+  const int* tile_slot;     // ring slot per RB-row tile
+  const int* row_idx;       // sample index per gradient row (-1: padding)
+  const void* ring; size_t slot_stride;
+  size_t w_off;             // element offset of W[k][k][Ci][Co]; the bias b[Co] follows it
+  int Hi, Wi, Ci, k, Co;    // input map, kernel size, output channels
+  const void* in;           // input maps [rows][Hi][Wi][Ci], or the dataset when from_dataset
+  int from_dataset;         // 1: row r reads X[row_idx[r]]
+  void* pooled;             // [rows][Ph][Pw][Co] pooled ReLU outputs (storage type)
+  unsigned char* arg;       // [rows][Ph][Pw][Co] window position (0..3 = (wy, wx) row-major) of the first maximum
+  const void* d_pooled;     // backward: [rows][Ph][Pw][Co] delta of the pooled maps
+  void* d_in;               // backward: [rows][Hi][Wi][Ci] delta of the input maps, or null (first block)
+  float* part;              // backward: [chunks][k k Ci Co + Co] per-chunk sums of the weight and bias gradient
+};
+
+inline size_t fwd_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
+  return sizeof(float) * ((size_t)Hi * Wi * Ci + (size_t)k * k * Ci * Co + Co);
+}
+inline size_t bwd_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
+  const int Ho = Hi - k + 1, Wo = Wi - k + 1;
+  return sizeof(float) * ((size_t)Hi * Wi * Ci + (size_t)k * k * Ci * Co + (size_t)Ho * Wo * Co +
+                          (size_t)(Ho / 2) * (Wo / 2) * Co) + (size_t)(Ho / 2) * (Wo / 2) * Co + 16;
+}
+
+template <typename T>
+__device__ __forceinline__ float as_stored_value(float v) { return v; }
+template <>
+__device__ __forceinline__ float as_stored_value<__nv_bfloat16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
+// One block forward for every gradient row of the round; CTA = row.
+template <typename T>
+__global__ void __launch_bounds__(THREADS) conv_block_fwd_kernel(Args a) {
+  grid_dependency_sync();
+  extern __shared__ __align__(16) float csm[];
+  DevState* st = a.st;
+  RoundInfo* ri = a.ri;
+  if (st->status != ST_OK) return;
+  const int r = blockIdx.x;
+  if (r >= ri->n_rows) return;
+  const int Hi = a.Hi, Wi = a.Wi, Ci = a.Ci, k = a.k, Co = a.Co;
+  const int Ho = Hi - k + 1, Wo = Wi - k + 1, Ph = Ho >> 1, Pw = Wo >> 1;
+  const int n_in = Hi * Wi * Ci, n_w = k * k * Ci * Co, n_out = Ph * Pw * Co;
+  T* out = (T*)a.pooled + (size_t)r * n_out;
+  unsigned char* arg = a.arg + (size_t)r * n_out;
+  const int s = a.row_idx[r];
+  if (s < 0) {                               // padding row: its deltas are zero, its maps only have to be finite
+    for (int i = threadIdx.x; i < n_out; i += THREADS) { stf(out, i, 0.f); arg[i] = 0; }
+    return;
+  }
+  float* img = csm;                          // [Hi][Wi][Ci]
+  float* wk = img + n_in;                    // [k][k][Ci][Co]
+  float* bias = wk + n_w;                    // [Co]
+  const int slot = a.tile_slot[r / st->RB];
+  const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
+  const T* src = (const T*)a.in + (size_t)(a.from_dataset ? s : r) * n_in;
+  for (int i = threadIdx.x; i < n_in; i += THREADS) img[i] = ldf(src, i);
+  for (int i = threadIdx.x; i < n_w + Co; i += THREADS) wk[i] = ldf(Wm, i);     // the bias follows the weights
+  __syncthreads();
+  for (int e = threadIdx.x; e < n_out; e += THREADS) {
+    const int co = e % Co, px = (e / Co) % Pw, py = e / (Co * Pw);
+    float best = 0.f;
+    int where = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int y = 2 * py + (q >> 1), x = 2 * px + (q & 1);
+      float acc = 0.f;
+      for (int dy = 0; dy < k; ++dy)
+        for (int dx = 0; dx < k; ++dx) {
+          const float* ip = img + ((y + dy) * Wi + (x + dx)) * Ci;
+          const float* wp = wk + ((dy * k + dx) * Ci) * Co + co;
+          for (int ci = 0; ci < Ci; ++ci) acc = fmaf(ip[ci], wp[ci * Co], acc);
+        }
+      const float v = as_stored_value<T>(fmaxf(acc + bias[co], 0.f));      // the stored ReLU output
+      if (q == 0 || v > best) { best = v; where = q; }                      // first maximum wins a tie
+    }
+    stf(out, e, best);
+    arg[e] = (unsigned char)where;
+  }
+}
+
+// One block backward for CHUNK consecutive gradient rows (they share a model version): this CTA's
+// share of the weight and bias gradient, and (second block) the delta of the block's input maps.
+template <typename T>
+__global__ void __launch_bounds__(THREADS) conv_block_bwd_kernel(Args a) {
+  grid_dependency_sync();
+  extern __shared__ __align__(16) float csm[];
+  DevState* st = a.st;
+  RoundInfo* ri = a.ri;
+  if (st->status != ST_OK) return;
+  const int r0 = blockIdx.x * CHUNK;
+  if (r0 >= ri->n_rows) return;
+  const int Hi = a.Hi, Wi = a.Wi, Ci = a.Ci, k = a.k, Co = a.Co;
+  const int Ho = Hi - k + 1, Wo = Wi - k + 1, Ph = Ho >> 1, Pw = Wo >> 1;
+  const int n_in = Hi * Wi * Ci, n_w = k * k * Ci * Co, n_out = Ph * Pw * Co, n_z = Ho * Wo * Co;
+  float* img = csm;                          // [Hi][Wi][Ci] input maps of the current row
+  float* wk = img + n_in;                    // [k][k][Ci][Co]
+  float* dz = wk + n_w;                      // [Ho][Wo][Co] delta before the pool, dense (second block only)
+  float* dp = dz + n_z;                      // [Ph][Pw][Co] delta of the pooled maps
+  unsigned char* ag = reinterpret_cast<unsigned char*>(dp + n_out);   // [Ph][Pw][Co]
+  const bool dgrad = a.d_in != nullptr;
+  const int slot = a.tile_slot[r0 / st->RB];
+  const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
+  if (dgrad) for (int i = threadIdx.x; i < n_w; i += THREADS) wk[i] = ldf(Wm, i);
+  // weight-gradient elements this thread owns: e = tid, tid + THREADS, ... (at most MAXE);
+  // elements n_w .. n_w + Co - 1 are the bias sums
+  constexpr int MAXE = 16;
+  float acc[MAXE];
+#pragma unroll
+  for (int j = 0; j < MAXE; ++j) acc[j] = 0.f;
+  const int n_rows = ri->n_rows;
+  for (int rr = 0; rr < CHUNK && r0 + rr < n_rows; ++rr) {
+    const int r = r0 + rr;
+    const int s = a.row_idx[r];
+    __syncthreads();                         // the previous row's maps are no longer read
+    if (s < 0) {                             // padding row: zero deltas, nothing to add
+      if (dgrad) {
+        T* din = (T*)a.d_in + (size_t)r * n_in;
+        for (int i = threadIdx.x; i < n_in; i += THREADS) stf(din, i, 0.f);
+      }
+      continue;
+    }
+    const T* src = (const T*)a.in + (size_t)(a.from_dataset ? s : r) * n_in;
+    const T* dps = (const T*)a.d_pooled + (size_t)r * n_out;
+    const unsigned char* args = a.arg + (size_t)r * n_out;
+    for (int i = threadIdx.x; i < n_in; i += THREADS) img[i] = ldf(src, i);
+    for (int i = threadIdx.x; i < n_out; i += THREADS) { dp[i] = ldf(dps, i); ag[i] = args[i]; }
+    if (dgrad) for (int i = threadIdx.x; i < n_z; i += THREADS) dz[i] = 0.f;
+    __syncthreads();
+    if (dgrad) {
+      for (int e = threadIdx.x; e < n_out; e += THREADS) {
+        const int co = e % Co, px = (e / Co) % Pw, py = e / (Co * Pw);
+        const int q = ag[e];
+        dz[((2 * py + (q >> 1)) * Wo + 2 * px + (q & 1)) * Co + co] = dp[e];
+      }
+      __syncthreads();
+    }
+    // weight gradient: only the window position that supplied the maximum carries a delta
+#pragma unroll
+    for (int j = 0; j < MAXE; ++j) {
+      const int e = threadIdx.x + j * THREADS;
+      if (e < n_w) {
+        const int co = e % Co, ci = (e / Co) % Ci, dx = (e / (Co * Ci)) % k, dy = e / (Co * Ci * k);
+        float sum = 0.f;
+        for (int py = 0; py < Ph; ++py)
+          for (int px = 0; px < Pw; ++px) {
+            const int o = (py * Pw + px) * Co + co;
+            const int q = ag[o];
+            sum = fmaf(img[((2 * py + (q >> 1) + dy) * Wi + 2 * px + (q & 1) + dx) * Ci + ci], dp[o], sum);
+          }
+        acc[j] += sum;
+      } else if (e < n_w + Co) {
+        const int co = e - n_w;
+        float sum = 0.f;
+        for (int o = co; o < n_out; o += Co) sum += dp[o];
+        acc[j] += sum;
+      }
+    }
+    if (dgrad) {
+      // delta of the input maps: every tap of every output pixel that covers (y, x), masked by the
+      // ReLU that produced the input (it is a pooled ReLU output: positive where active)
+      T* din = (T*)a.d_in + (size_t)r * n_in;
+      for (int e = threadIdx.x; e < n_in; e += THREADS) {
+        const int ci = e % Ci, x = (e / Ci) % Wi, y = e / (Ci * Wi);
+        float sum = 0.f;
+        for (int dy = 0; dy < k; ++dy) {
+          const int oy = y - dy;
+          if (oy < 0 || oy >= Ho) continue;
+          for (int dx = 0; dx < k; ++dx) {
+            const int ox = x - dx;
+            if (ox < 0 || ox >= Wo) continue;
+            const float* zp = dz + (oy * Wo + ox) * Co;
+            const float* wp = wk + ((dy * k + dx) * Ci + ci) * Co;
+            for (int co = 0; co < Co; ++co) sum = fmaf(zp[co], wp[co], sum);
+          }
+        }
+        stf(din, e, img[e] > 0.f ? sum : 0.f);
+      }
+    }
+  }
+  float* dst = a.part + (size_t)blockIdx.x * (size_t)(n_w + Co);
+#pragma unroll
+  for (int j = 0; j < MAXE; ++j) {
+    const int e = threadIdx.x + j * THREADS;
+    if (e < n_w + Co) dst[e] = acc[j];
+  }
+}
+
+}  // namespace conv
+}  // namespace absb

@@ -80,6 +80,7 @@ abs_lsq_rounds_kernel(CtlArgs a, LsqRoundsArgs q, int t_first, int n_rounds) {
   const int sub = lane / lpr, v = lane - sub * lpr;
   __syncthreads();
 
+  const bool sa_on = st->sa_penalty != 0;          // staleness-aware step size
   for (int r = 0; r < n_rounds; ++r) {
     const int t = t_first + r;
     if (ctl_round<NT>(a, sh, 1, 1, t)) return;
@@ -160,7 +161,7 @@ abs_lsq_rounds_kernel(CtlArgs a, LsqRoundsArgs q, int t_first, int n_rounds) {
           const float res = dot - __shfl_sync(0xffffffffu, yv[k], sub * lpr);
           if (valid && v == 0) rowloss_s[row] = 0.5f * res * res;
           // staleness-aware step size: the row's weight follows from the ring slot it was computed on
-          const float rg = res * (valid ? sa_slot_weight(st, t, rslot_s[row]) : 1.f);
+          const float rg = (sa_on && valid) ? res * sa_weight((t - rslot_s[row]) % (S + 1)) : res;
 #pragma unroll
           for (int j = 0; j < 8; ++j) acc[j] = fmaf(rg, xv[k][j], acc[j]);   // xv = 0 where there is no row
         }

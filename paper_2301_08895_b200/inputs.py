@@ -15,7 +15,7 @@ from dataclasses import dataclass, field, replace
 
 import numpy as np
 
-LSQ, SOFTMAX, MLP = 0, 1, 2
+LSQ, SOFTMAX, MLP, CNN = 0, 1, 2, 3
 FP32, BF16 = 0, 1
 T_CONST, T_EXP, T_SHIFTED_EXP, T_PARETO2, T_GAMMA = 0, 1, 2, 3, 4
 
@@ -54,13 +54,23 @@ class Config:
     data_seed: int = 0
     run_seed: int = 0
     w0_seed: int = 0
+    conv: tuple = None        # CNN: (H, W, C_in, k, C1, C2); dims then describes the fully connected part
+
+    @property
+    def x_len(self):
+        """Elements of one dataset row."""
+        return self.conv[0] * self.conv[1] * self.conv[2] if self.kind == CNN else self.dims[0]
 
     def scaled(self, **kw):
         return replace(self, **kw)
 
 
 def config(i, W=None):
-    """Configuration i = 1..5 of the benchmark (5 takes W in {256, 512, 1024})."""
+    """Configuration i = 1..5 of the benchmark (5 takes W in {256, 512, 1024}); 6 is the paper's own
+    model class on image-shaped synthetic data (Sec. V-A: 32 x 32 x 3 inputs, two convolution
+    blocks and three fully connected layers, B = 32, N = 20, K^0 = 5, gamma-distributed execution
+    times; the step size is 0.003 instead of the paper's 0.1 because the synthetic features are
+    not normalised)."""
     if i == 1:
         c = Config("lsq64_w8", LSQ, (64, 1), FP32, 8, 32, 2, 4, 200, 0.05, 8192,
                    TimeSpec(T_SHIFTED_EXP, shift=1.0, rate=1.0), "lsq")
@@ -80,16 +90,24 @@ def config(i, W=None):
         W = 256 if W is None else W
         c = Config("lsq4096_w%d" % W, LSQ, (4096, 1), BF16, W, 32, W // 8, 32, 500, 0.01,
                    1_000_000, TimeSpec(T_EXP, rate=1.0), "lsq")
+    elif i == 6:
+        c = Config("cnn32_w20", CNN, (400, 120, 84, 10), BF16, 20, 32, 5, 8, 500, 0.003, 50000,
+                   TimeSpec(T_GAMMA, shift=0.0, rate=3.0, shape=3), "mixture", sigma=1.0, w0="he",
+                   conv=(32, 32, 3, 5, 6, 16))
     else:
-        raise ValueError("config index 1..5")
+        raise ValueError("config index 1..6")
     c.data_seed, c.run_seed, c.w0_seed = 1000 + i, 2000 + i, 3000 + i
     return c
 
 
-def n_params(kind, dims):
+def n_params(kind, dims, conv=None):
     if kind == LSQ:
         return dims[0]
-    return sum(dims[l] * dims[l + 1] + dims[l + 1] for l in range(len(dims) - 1))
+    n = sum(dims[l] * dims[l + 1] + dims[l + 1] for l in range(len(dims) - 1))
+    if kind == CNN:
+        _, _, c_in, k, c1, c2 = conv
+        n += k * k * c_in * c1 + c1 + k * k * c1 * c2 + c2
+    return n
 
 
 def to_bf16_bits(a32):
@@ -129,7 +147,7 @@ def make_data(cfg):
     uint16 bfloat16 patterns for BF16 ones; y is float32 (least squares) or
     int32 labels; extra carries the generating parameters (w_star or means).
     """
-    n, d_in = cfg.n_samples, cfg.dims[0]
+    n, d_in = cfg.n_samples, cfg.x_len
     rng = np.random.Generator(np.random.PCG64(cfg.data_seed))
     bf16 = cfg.dtype == BF16
     X = np.empty((n, d_in), dtype=np.uint16 if bf16 else np.float32)
@@ -168,12 +186,19 @@ def make_data(cfg):
 
 def make_w0(cfg):
     """Initial parameters, float32, layout: per layer W[in][out] then b[out]
-    (least squares: w[d])."""
-    d = n_params(cfg.kind, cfg.dims)
+    (least squares: w[d]; CNN: the two convolution blocks first)."""
+    d = n_params(cfg.kind, cfg.dims, cfg.conv)
     w0 = np.zeros(d, dtype=np.float32)
     if cfg.w0 == "he":
         rng = np.random.Generator(np.random.PCG64(cfg.w0_seed))
         off = 0
+        if cfg.kind == CNN:            # convolution blocks: W[k][k][C_in][C_out] with fan-in k k C_in, then b = 0
+            _, _, c_in, k, c1, c2 = cfg.conv
+            for ci, co in ((c_in, c1), (c1, c2)):
+                n_w = k * k * ci * co
+                w0[off:off + n_w] = rng.standard_normal(n_w).astype(np.float32) * np.float32(
+                    np.sqrt(2.0 / (k * k * ci)))
+                off += n_w + co
         for l in range(len(cfg.dims) - 1):
             i, o = cfg.dims[l], cfg.dims[l + 1]
             w0[off:off + i * o] = rng.standard_normal(i * o).astype(np.float32) * np.float32(

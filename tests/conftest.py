@@ -25,4 +25,4 @@ def make_oracle(cfg, X, y, w0, **kw):
     bf16 = cfg.dtype == inputs.BF16
     return abs_sim.ABSOracle(cfg.kind, cfg.dims, X, y, w0, cfg.batch, cfg.lr, cfg.W, cfg.K0, cfg.S,
                              oracle_dist(cfg.time), cfg.run_seed, quant=bf16,
-                             x_is_bf16_bits=bf16, **kw)
+                             x_is_bf16_bits=bf16, conv=getattr(cfg, "conv", None), **kw)
