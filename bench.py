@@ -76,12 +76,22 @@ def per_wg_flops(cfg):
     nl = len(dims) - 1
     hidden = [2.0 * B * dims[l] * dims[l + 1] for l in range(nl - 1)]
     last = 2.0 * B * dims[nl - 1] * dims[nl]
-    return {"fwd": sum(hidden), "wgrad": sum(hidden), "dgrad": sum(hidden[1:]),
-            "output": last * (3 if nl > 1 else 2)}
+    out = {"fwd": sum(hidden), "wgrad": sum(hidden), "dgrad": sum(hidden[1:]),
+           "output": last * (3 if nl > 1 else 2)}
+    if cfg.kind == inputs.CNN:
+        # convolution blocks: 2 k k C_in C_out flops per output pixel forward; the weight gradient only
+        # sees the pooled positions (a quarter of the pixels); the second block also back-propagates
+        H, W, c_in, k, c1, c2 = cfg.conv
+        h1, w1 = H - k + 1, W - k + 1
+        h2, w2 = h1 // 2 - k + 1, w1 // 2 - k + 1
+        f1, f2 = 2.0 * k * k * c_in * c1 * h1 * w1, 2.0 * k * k * c1 * c2 * h2 * w2
+        out["conv"] = B * (f1 + f2 + 0.25 * (f1 + f2) + f2)
+        out["dgrad"] = sum(hidden)          # the first affine layer back-propagates into the features too
+    return out
 
 
 def n_params(cfg):
-    return inputs.n_params(cfg.kind, cfg.dims)
+    return inputs.n_params(cfg.kind, cfg.dims, cfg.conv)
 
 
 def padded_rows(tr, B, RB):
@@ -152,7 +162,7 @@ def oracle_for(cfg, X, y, w0, local_steps=1, k_fixed=False):
                              timing.TimeDist(ts.kind, ts.shift, ts.rate, ts.scale, ts.slow_mod,
                                              ts.slow_rem, ts.slow_factor, ts.shape),
                              cfg.run_seed, quant=bf16, x_is_bf16_bits=bf16, local_steps=local_steps,
-                             k_mode=abs_sim.K_FIXED if k_fixed else abs_sim.K_ADAPTIVE)
+                             k_mode=abs_sim.K_FIXED if k_fixed else abs_sim.K_ADAPTIVE, conv=cfg.conv)
 
 
 def blas_threads():
@@ -189,7 +199,7 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
-    ap.add_argument("--config", type=int, default=4)
+    ap.add_argument("--config", type=int, default=4, help="1..5: the benchmark configurations; 6: the paper's CNN")
     ap.add_argument("--workers", type=int, default=None, help="W of configuration 5")
     ap.add_argument("--rounds", type=int, default=None, help="rounds per step (default: the configuration's)")
     ap.add_argument("--flags", type=int, default=0, help="ABS_FLAG_* bits passed to abs_init")
@@ -422,6 +432,15 @@ def main():
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                            "traffic": None, "peak_source": peaks["source"],
                            "share_of_profiled_time": t_l / tot_prof}
+    elif cfg.kind == inputs.CNN:
+        # FP32-FMA kernels: 148 SMs x 128 lanes x 2 flop per clock at the maximum SM clock
+        n_c, t_c = prof["conv"]
+        peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        ach = wg_p * flops["conv"] / (t_c * 1e-3) / 1e12
+        out["roofline"] = {"bound": "alu", "kernel": "conv_block_fwd_kernel + conv_block_bwd_kernel (+ chunk sums)",
+                           "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
+                           "peak_source": "148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz",
+                           "share_of_profiled_time": t_c / tot_prof}
     elif prof["fwd"][0] and bf16:
         t_g = prof["fwd"][1] + prof["dgrad"][1] + prof["wgrad"][1]
         fl = wg_p * (flops["fwd"] + flops["dgrad"] + flops["wgrad"])

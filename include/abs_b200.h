@@ -91,9 +91,6 @@ extern "C" {
                                        server-side kernels of the next round) */
 #define ABS_FLAG_NO_BULK_PIPELINE 32 /* bf16 least squares: per-warp 16-byte loads (rows read from HBM, then again
                                        from L2) instead of the bulk-copy pipeline through shared memory */
-#define ABS_FLAG_FUSED_FORWARD  128 /* tensor-core networks: two consecutive hidden layers with the same tile width
-                                       run their forward GEMMs in one launch, tiles of the second waiting on
-                                       completion counters of the first (same results; measured no faster end to end) */
 #define ABS_FLAG_NO_FUSED_BACKWARD 64 /* tensor-core networks: a layer's delta back-propagation and its weight
                                        gradient always get a launch each */
 #define ABS_FLAG_NO_PERSISTENT   8  /* small least-squares problems: one kernel launch per step of a round
@@ -111,7 +108,8 @@ extern "C" {
 #define ABS_KC_UPDATE  7  /* Eq. 3 step + ring write */
 #define ABS_KC_ROUNDS  8  /* whole rounds (control step + Eq. 2 + Eq. 3) of a small least-squares problem
                              in one persistent kernel; one launch per abs_enqueue_rounds call */
-#define ABS_KC_COUNT   9
+#define ABS_KC_CONV    9  /* ABS_CNN: the convolution blocks, forward and backward */
+#define ABS_KC_COUNT   10
 
 #define ABS_MAX_LAYERS   7
 #define ABS_MAX_WORKERS  1024

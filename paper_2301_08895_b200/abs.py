@@ -27,8 +27,7 @@ FLAG_NO_OVERLAP = 2
 FLAG_NO_PERSISTENT = 8
 FLAG_NO_BULK_PIPELINE = 32
 FLAG_NO_FUSED_BACKWARD = 64
-FLAG_FUSED_FORWARD = 128
-KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "lsq", "update", "rounds")
+KC_NAMES = ("ctl", "gather", "fwd", "dgrad", "wgrad", "output", "lsq", "update", "rounds", "conv")
 
 
 class ModelDesc(C.Structure):

@@ -62,8 +62,6 @@ struct Layout {
   int bn_fwd[ABS_MAX_LAYERS] = {}, bn_dg[ABS_MAX_LAYERS] = {}, bn_wg[ABS_MAX_LAYERS] = {};
   bool any_tc = false;
   int cg_fwd[ABS_MAX_LAYERS] = {}, cg_dg[ABS_MAX_LAYERS] = {}, cg_wg[ABS_MAX_LAYERS] = {};
-  bool pair_fwd[ABS_MAX_LAYERS] = {};   // forward GEMMs of layers l and l + 1 share a launch
-  size_t done;                          // completion counters per row tile (paired forward launches)
   bool pair_bwd[ABS_MAX_LAYERS] = {};   // delta back-propagation and weight gradient of the layer share a launch
   int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
   bool out_mma = false;                 // output layer through the mma.sync kernel (bf16, 64 rows per CTA)
@@ -217,16 +215,6 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
         L->cg_wg[l] = 2; L->bn_wg[l] = 256;
       }
     }
-    // Opt-in: two consecutive tensor-core layers with the same tile width run their forward GEMMs in
-    // one launch (the second behind per-row-tile completion counters): one set of fixed launch
-    // costs, and the second layer's tiles fill the first layer's last, partly empty wave.
-    for (int l = 0; l + 1 < m->n_layers; ++l) {
-      if (L->path[l] != PATH_TC || L->path[l + 1] != PATH_TC || !(m->flags & ABS_FLAG_FUSED_FORWARD)) continue;
-      if (L->cg_fwd[l] != 1 || L->cg_fwd[l + 1] != 1 || L->bn_fwd[l] != L->bn_fwd[l + 1]) continue;
-      if (l > 0 && L->pair_fwd[l - 1]) continue;
-      if (L->local_net) continue;
-      L->pair_fwd[l] = true;
-    }
     // A short weight gradient (fewer tiles than SMs at the back-propagation's tile width) shares
     // its launch with the layer's delta back-propagation: both have one or two tiles per CTA, so
     // separate launches would pay the fixed costs of a launch twice.
@@ -283,7 +271,6 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
   }
   L->loss = cv.take(4 * W);
   L->row_loss = cv.take(4 * (size_t)L->rows_cap);
-  L->done = cv.take(4 * (size_t)L->n_tiles_cap);
   L->master = cv.take(4 * L->d_pad);
   L->ring = cv.take(L->esz * L->d_pad * (S + 1));
   if (m->local_steps > 1) L->P = 0;      // Eq. 3 adds one upload per selected worker
@@ -667,7 +654,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     // Eq. 2 forward through the two convolution blocks: the features are the input rows of layer 0
     for (int b = 0; b < 2; ++b) {
       const conv::Args c = conv_args(b);
-      launch_ex(ctx, ABS_KC_FWD, conv::conv_block_fwd_kernel<T>, dim3(L.rows_cap), dim3(conv::THREADS),
+      launch_ex(ctx, ABS_KC_CONV, conv::conv_block_fwd_kernel<T>, dim3(L.rows_cap), dim3(conv::THREADS),
                 conv::fwd_smem_bytes(c.Hi, c.Wi, c.Ci, c.k, c.Co), c);
     }
     return;
@@ -690,22 +677,6 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       const int bn = L.bn_fwd[l];
       const CUtensorMap& amap = (l == 0 && par) ? ctx->tcl[l].fwd_a_odd : ctx->tcl[l].fwd_a;
       const int tiles = (row_tiles128 / L.cg_fwd[l]) * ((la[l].out + bn - 1) / bn);
-      if (L.pair_fwd[l]) {
-        // the next layer's forward GEMM rides in the same launch, behind completion counters
-        const int n = l + 1;
-        tc::Params p2 = tc_params(n, tc::FWD);
-        p2.N_total = la[n].out; p2.K_total = la[n].in;
-        p2.out_bf16 = (__nv_bfloat16*)la[n].act_out;
-        p2.relu_bits = L.bits[n + 1] ? ctx->at<uint32_t>(L.bits[n + 1]) : nullptr;
-        p2.mask_words = (la[n].out + 31) / 32;
-        p.done_signal = ctx->at<int>(L.done);
-        p2.done_wait = ctx->at<int>(L.done);
-        p2.done_target = ((la[l].out + bn - 1) / bn) * tc::EPI_WARPS;
-        const TcProblem second = {&ctx->tcl[n].fwd_a, &ctx->tcl[n].fwd_b, &ctx->tcl[n].fwd_out, &p2, row_tiles128 * ((la[n].out + bn - 1) / bn)};
-        launch_tc_bn(ctx, bn, 1, ABS_KC_FWD, amap, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, tiles, &second);
-        ++l;
-        continue;
-      }
       launch_tc_bn(ctx, bn, L.cg_fwd[l], ABS_KC_FWD, amap, ctx->tcl[l].fwd_b, ctx->tcl[l].fwd_out, p, tiles);
     } else if (L.path[l] == PATH_NARROW) {
       NarrowArgs a = narrow_args(l);
@@ -820,9 +791,12 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
   // per-chunk sums that a fixed-order reduction adds up into partial 0 of the gradient vector
   for (int b = 1; b >= 0 && phase == PH_BACKWARD && L.cnn; --b) {
     const conv::Args c = conv_args(b);
-    launch_ex(ctx, ABS_KC_WGRAD, conv::conv_block_bwd_kernel<T>, dim3(L.rows_cap / conv::CHUNK), dim3(conv::THREADS),
-              conv::bwd_smem_bytes(c.Hi, c.Wi, c.Ci, c.k, c.Co), c);
-    launch_ex(ctx, ABS_KC_WGRAD, chunk_reduce_kernel, dim3(((int)L.c_len[b] + 31) / 32), dim3(256), 0, st, ri, c.part, (int)L.c_len[b],
+    if (b == 1)      // delta of the first block's pooled maps (one CTA per row)
+      launch_ex(ctx, ABS_KC_CONV, conv::conv_block_dgrad_kernel<T>, dim3(L.rows_cap), dim3(conv::THREADS),
+                conv::dgrad_smem_bytes(c.Hi, c.Wi, c.Ci, c.k, c.Co), c);
+    launch_ex(ctx, ABS_KC_CONV, conv::conv_block_wgrad_kernel<T>, dim3(L.rows_cap / conv::CHUNK), dim3(conv::THREADS),
+              conv::wgrad_smem_bytes(c.Hi, c.Wi, c.Ci, c.k, c.Co), c);
+    launch_ex(ctx, ABS_KC_CONV, chunk_reduce_kernel, dim3(((int)L.c_len[b] + 31) / 32), dim3(256), 0, st, ri, c.part, (int)L.c_len[b],
               ctx->at<float>(L.G) + L.c_off[b], conv::CHUNK);
   }
 }
@@ -850,9 +824,6 @@ void enqueue_update(abs_ctx* ctx, int par) {
   // durations (its first warps); tensor-core networks keep a small kernel of their own for that
   const bool look = !L.any_tc;
   u.job = ctx->ctl.job; u.next_dur = ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
-  u.zero_words = nullptr; u.n_zero = 0;
-  for (int l = 0; l < ctx->m.n_layers; ++l)
-    if (L.pair_fwd[l]) { u.zero_words = ctx->at<int>(L.done); u.n_zero = L.n_tiles_cap; }
   // one wave of resident blocks striding over the vector (a partly filled second wave would only add a tail)
   const size_t n4 = L.d_pad / 4;
   int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * ctx->upd_blocks_per_sm), (size_t)(ctx->W + 31) / 32);
@@ -1124,8 +1095,10 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
                                      conv::bwd_smem_bytes(L.cHi[b], L.cWi[b], L.cCi[b], L.ck, L.cCo[b])));
     cudaError_t ec = cudaFuncSetAttribute(conv::conv_block_fwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
     if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_fwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
-    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
-    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_bwd_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_wgrad_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_wgrad_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_dgrad_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (ec == cudaSuccess) ec = cudaFuncSetAttribute(conv::conv_block_dgrad_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
     if (ec != cudaSuccess) return bail(cuda_fail(nullptr, ec, "cudaFuncSetAttribute(conv_block kernels)"));
   }
   if (!(model->flags & ABS_FLAG_NO_OVERLAP) && L.any_tc && !L.local_net && !L.cnn) {

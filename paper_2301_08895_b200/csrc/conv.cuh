@@ -12,8 +12,8 @@
 // over all rows.)  Maps are stored [row][y][x][channel] in the storage type; the images of the
 // first block are dataset rows fetched by sample index.  The channel counts of this model class
 // are far below a tensor-core tile (3 -> 6 -> 16 in the benchmark network), so these are FP32-FMA
-// kernels: one CTA per gradient row forward, one CTA per 16 rows backward, everything the CTA
-// needs staged in shared memory, fixed summation orders.
+// kernels: one CTA per gradient row (forward, input delta) or per 16 rows (weight gradient),
+// everything the CTA needs staged in shared memory, fixed summation orders.
 #pragma once
 #include "common.cuh"
 #include "simt.cuh"
@@ -37,17 +37,24 @@ struct Args {
   void* pooled;             // [rows][Ph][Pw][Co] pooled ReLU outputs (storage type)
   unsigned char* arg;       // [rows][Ph][Pw][Co] window position (0..3 = (wy, wx) row-major) of the first maximum
   const void* d_pooled;     // backward: [rows][Ph][Pw][Co] delta of the pooled maps
-  void* d_in;               // backward: [rows][Hi][Wi][Ci] delta of the input maps, or null (first block)
+  void* d_in;               // backward: [rows][Hi][Wi][Ci] delta of the input maps (second block)
   float* part;              // backward: [chunks][k k Ci Co + Co] per-chunk sums of the weight and bias gradient
 };
 
 inline size_t fwd_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
   return sizeof(float) * ((size_t)Hi * Wi * Ci + (size_t)k * k * Ci * Co + Co);
 }
-inline size_t bwd_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
+inline size_t wgrad_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
   const int Ho = Hi - k + 1, Wo = Wi - k + 1;
-  return sizeof(float) * ((size_t)Hi * Wi * Ci + (size_t)k * k * Ci * Co + (size_t)Ho * Wo * Co +
-                          (size_t)(Ho / 2) * (Wo / 2) * Co) + (size_t)(Ho / 2) * (Wo / 2) * Co + 16;
+  return sizeof(float) * ((size_t)Hi * Wi * Ci + (size_t)(Ho / 2) * (Wo / 2) * Co) + (size_t)(Ho / 2) * (Wo / 2) * Co + 16;
+}
+inline size_t dgrad_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
+  const int Ho = Hi - k + 1, Wo = Wi - k + 1;
+  return sizeof(float) * ((size_t)k * k * Ci * Co + (size_t)Ho * Wo * Co);
+}
+inline size_t bwd_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
+  return wgrad_smem_bytes(Hi, Wi, Ci, k, Co) > dgrad_smem_bytes(Hi, Wi, Ci, k, Co) ? wgrad_smem_bytes(Hi, Wi, Ci, k, Co)
+                                                                                   : dgrad_smem_bytes(Hi, Wi, Ci, k, Co);
 }
 
 template <typename T>
@@ -106,10 +113,11 @@ __global__ void __launch_bounds__(THREADS) conv_block_fwd_kernel(Args a) {
   }
 }
 
-// One block backward for CHUNK consecutive gradient rows (they share a model version): this CTA's
-// share of the weight and bias gradient, and (second block) the delta of the block's input maps.
+// Weight and bias gradient of one block over CHUNK consecutive gradient rows: this CTA's share of
+// the sum of Eq. 3 (a fixed-order reduction over the CTAs follows).  Only the window position that
+// supplied a pooled maximum carries a delta, so the sum runs over pooled pixels.
 template <typename T>
-__global__ void __launch_bounds__(THREADS) conv_block_bwd_kernel(Args a) {
+__global__ void __launch_bounds__(THREADS) conv_block_wgrad_kernel(Args a) {
   grid_dependency_sync();
   extern __shared__ __align__(16) float csm[];
   DevState* st = a.st;
@@ -119,16 +127,10 @@ __global__ void __launch_bounds__(THREADS) conv_block_bwd_kernel(Args a) {
   if (r0 >= ri->n_rows) return;
   const int Hi = a.Hi, Wi = a.Wi, Ci = a.Ci, k = a.k, Co = a.Co;
   const int Ho = Hi - k + 1, Wo = Wi - k + 1, Ph = Ho >> 1, Pw = Wo >> 1;
-  const int n_in = Hi * Wi * Ci, n_w = k * k * Ci * Co, n_out = Ph * Pw * Co, n_z = Ho * Wo * Co;
+  const int n_in = Hi * Wi * Ci, n_w = k * k * Ci * Co, n_out = Ph * Pw * Co;
   float* img = csm;                          // [Hi][Wi][Ci] input maps of the current row
-  float* wk = img + n_in;                    // [k][k][Ci][Co]
-  float* dz = wk + n_w;                      // [Ho][Wo][Co] delta before the pool, dense (second block only)
-  float* dp = dz + n_z;                      // [Ph][Pw][Co] delta of the pooled maps
+  float* dp = img + n_in;                    // [Ph][Pw][Co] delta of the pooled maps
   unsigned char* ag = reinterpret_cast<unsigned char*>(dp + n_out);   // [Ph][Pw][Co]
-  const bool dgrad = a.d_in != nullptr;
-  const int slot = a.tile_slot[r0 / st->RB];
-  const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
-  if (dgrad) for (int i = threadIdx.x; i < n_w; i += THREADS) wk[i] = ldf(Wm, i);
   // weight-gradient elements this thread owns: e = tid, tid + THREADS, ... (at most MAXE);
   // elements n_w .. n_w + Co - 1 are the bias sums
   constexpr int MAXE = 16;
@@ -139,30 +141,14 @@ __global__ void __launch_bounds__(THREADS) conv_block_bwd_kernel(Args a) {
   for (int rr = 0; rr < CHUNK && r0 + rr < n_rows; ++rr) {
     const int r = r0 + rr;
     const int s = a.row_idx[r];
+    if (s < 0) continue;                     // padding row: zero deltas (same decision in every thread)
     __syncthreads();                         // the previous row's maps are no longer read
-    if (s < 0) {                             // padding row: zero deltas, nothing to add
-      if (dgrad) {
-        T* din = (T*)a.d_in + (size_t)r * n_in;
-        for (int i = threadIdx.x; i < n_in; i += THREADS) stf(din, i, 0.f);
-      }
-      continue;
-    }
     const T* src = (const T*)a.in + (size_t)(a.from_dataset ? s : r) * n_in;
     const T* dps = (const T*)a.d_pooled + (size_t)r * n_out;
     const unsigned char* args = a.arg + (size_t)r * n_out;
     for (int i = threadIdx.x; i < n_in; i += THREADS) img[i] = ldf(src, i);
     for (int i = threadIdx.x; i < n_out; i += THREADS) { dp[i] = ldf(dps, i); ag[i] = args[i]; }
-    if (dgrad) for (int i = threadIdx.x; i < n_z; i += THREADS) dz[i] = 0.f;
     __syncthreads();
-    if (dgrad) {
-      for (int e = threadIdx.x; e < n_out; e += THREADS) {
-        const int co = e % Co, px = (e / Co) % Pw, py = e / (Co * Pw);
-        const int q = ag[e];
-        dz[((2 * py + (q >> 1)) * Wo + 2 * px + (q & 1)) * Co + co] = dp[e];
-      }
-      __syncthreads();
-    }
-    // weight gradient: only the window position that supplied the maximum carries a delta
 #pragma unroll
     for (int j = 0; j < MAXE; ++j) {
       const int e = threadIdx.x + j * THREADS;
@@ -183,33 +169,68 @@ __global__ void __launch_bounds__(THREADS) conv_block_bwd_kernel(Args a) {
         acc[j] += sum;
       }
     }
-    if (dgrad) {
-      // delta of the input maps: every tap of every output pixel that covers (y, x), masked by the
-      // ReLU that produced the input (it is a pooled ReLU output: positive where active)
-      T* din = (T*)a.d_in + (size_t)r * n_in;
-      for (int e = threadIdx.x; e < n_in; e += THREADS) {
-        const int ci = e % Ci, x = (e / Ci) % Wi, y = e / (Ci * Wi);
-        float sum = 0.f;
-        for (int dy = 0; dy < k; ++dy) {
-          const int oy = y - dy;
-          if (oy < 0 || oy >= Ho) continue;
-          for (int dx = 0; dx < k; ++dx) {
-            const int ox = x - dx;
-            if (ox < 0 || ox >= Wo) continue;
-            const float* zp = dz + (oy * Wo + ox) * Co;
-            const float* wp = wk + ((dy * k + dx) * Ci + ci) * Co;
-            for (int co = 0; co < Co; ++co) sum = fmaf(zp[co], wp[co], sum);
-          }
-        }
-        stf(din, e, img[e] > 0.f ? sum : 0.f);
-      }
-    }
   }
   float* dst = a.part + (size_t)blockIdx.x * (size_t)(n_w + Co);
 #pragma unroll
   for (int j = 0; j < MAXE; ++j) {
     const int e = threadIdx.x + j * THREADS;
     if (e < n_w + Co) dst[e] = acc[j];
+  }
+}
+
+// Delta of a block's input maps (second block only), CTA = gradient row: the pooled delta is put
+// back at the window positions that supplied the maxima (dense map in shared memory), then every
+// input element adds up the taps of the output pixels that cover it, masked by the ReLU that
+// produced the input (it is a pooled ReLU output: positive where active).
+template <typename T>
+__global__ void __launch_bounds__(THREADS) conv_block_dgrad_kernel(Args a) {
+  grid_dependency_sync();
+  extern __shared__ __align__(16) float csm[];
+  DevState* st = a.st;
+  RoundInfo* ri = a.ri;
+  if (st->status != ST_OK) return;
+  const int r = blockIdx.x;
+  if (r >= ri->n_rows) return;
+  const int Hi = a.Hi, Wi = a.Wi, Ci = a.Ci, k = a.k, Co = a.Co;
+  const int Ho = Hi - k + 1, Wo = Wi - k + 1, Ph = Ho >> 1, Pw = Wo >> 1;
+  const int n_in = Hi * Wi * Ci, n_w = k * k * Ci * Co, n_out = Ph * Pw * Co, n_z = Ho * Wo * Co;
+  T* din = (T*)a.d_in + (size_t)r * n_in;
+  const int s = a.row_idx[r];
+  if (s < 0) {                               // padding row: zero deltas
+    for (int i = threadIdx.x; i < n_in; i += THREADS) stf(din, i, 0.f);
+    return;
+  }
+  float* wk = csm;                           // [k][k][Ci][Co]
+  float* dz = wk + n_w;                      // [Ho][Wo][Co] delta before the pool, dense
+  const int slot = a.tile_slot[r / st->RB];
+  const T* Wm = (const T*)a.ring + (size_t)slot * a.slot_stride + a.w_off;
+  const T* dps = (const T*)a.d_pooled + (size_t)r * n_out;
+  const unsigned char* args = a.arg + (size_t)r * n_out;
+  const T* src = (const T*)a.in + (size_t)r * n_in;
+  for (int i = threadIdx.x; i < n_w; i += THREADS) wk[i] = ldf(Wm, i);
+  for (int i = threadIdx.x; i < n_z; i += THREADS) dz[i] = 0.f;
+  __syncthreads();
+  for (int e = threadIdx.x; e < n_out; e += THREADS) {
+    const int co = e % Co, px = (e / Co) % Pw, py = e / (Co * Pw);
+    const int q = args[e];
+    dz[((2 * py + (q >> 1)) * Wo + 2 * px + (q & 1)) * Co + co] = ldf(dps, e);
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < n_in; e += THREADS) {
+    const int ci = e % Ci, x = (e / Ci) % Wi, y = e / (Ci * Wi);
+    float sum = 0.f;
+    for (int dy = 0; dy < k; ++dy) {
+      const int oy = y - dy;
+      if (oy < 0 || oy >= Ho) continue;
+      for (int dx = 0; dx < k; ++dx) {
+        const int ox = x - dx;
+        if (ox < 0 || ox >= Wo) continue;
+        const float* zp = dz + (oy * Wo + ox) * Co;
+        const float* wp = wk + ((dy * k + dx) * Ci + ci) * Co;
+        for (int co = 0; co < Co; ++co) sum = fmaf(zp[co], wp[co], sum);
+      }
+    }
+    stf(din, e, ldf(src, e) > 0.f ? sum : 0.f);
   }
 }
 

@@ -337,7 +337,6 @@ struct UpdateArgs {
   const int* sel_tau;     // [K^t] staleness of each selected worker's upload (read when the staleness-aware
                           // step size is applied to whole uploads: DevState::sa_penalty == 2, P == 0)
   float lr;
-  int* zero_words; int n_zero;   // counters of the round's kernels to clear for the next round (or null)
   // Output-layer gradient still in per-chunk partial sums (or null): blocks [n_main_blocks, gridDim.x)
   // add the chunks of 32 outputs each in a fixed order and apply Eq. 3 to those parameters; the
   // streaming blocks skip the range.
@@ -361,8 +360,6 @@ __global__ void __launch_bounds__(256, 4) update_kernel(UpdateArgs a) {
   // duration look-ahead for the workers whose job index moved (first warp of the first ceil(N/32) blocks)
   if (LOOK && threadIdx.x < 32 && (int)blockIdx.x * 32 < st->W)
     refresh_next_durations(st, a.job, a.next_dur, a.dur_job, (int)blockIdx.x * 32 + (int)threadIdx.x);
-  if (a.zero_words != nullptr && blockIdx.x == gridDim.x - 1)
-    for (int i = threadIdx.x; i < a.n_zero; i += blockDim.x) a.zero_words[i] = 0;
   if (ri->diverged) return;
   const int K = ri->K;
   const int P = a.P > 0 ? a.P : K;

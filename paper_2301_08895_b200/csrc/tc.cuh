@@ -43,13 +43,6 @@ struct Params {
                                    // the word at bit (j >> 1) + 16 * (j & 1) (even columns low half, odd high)
   uint32_t* relu_bits;             // FWD: the same bits for this layer's output (may be null)
   int mask_words;                  // words per row of mask_bits / relu_bits = ceil(N_total / 32)
-  // Two forward problems in one launch: the second reads what the first writes.  Every epilogue
-  // warp of the first adds 1 to done[row tile] once its stores of a tile have completed; the
-  // producer of the second waits until done[row tile] reaches done_target before it loads rows
-  // of that tile.  The counters are zeroed between rounds by the Eq. 3 kernel.
-  int* done_signal;                // FWD (first problem): counters to add to, or null
-  const int* done_wait;            // FWD (second problem): counters to wait on, or null
-  int done_target;
   __nv_bfloat16* out_bf16;         // FWD/DGRAD result [rows][N_total]
   float* out_f32;                  // WGRAD: G + w_off, partial p at + p*slot_stride, row pitch N_total
 };
@@ -212,12 +205,10 @@ struct TileCoord { int which, rt, a_row, b_col, slot, k_begin, n_kb, split, bias
 // Tiling of one problem of a launch.
 struct Prob { int mode, n_ct, n_mt_w, n_mt, n_tiles, chunk; };
 
-// A launch serves one problem (p0), or two (p1.mode >= 0): either two independent ones, a layer's
-// weight gradient (p0) next to its delta back-propagation (p1), or two consecutive forward layers,
-// where the second reads the first's output tile by tile behind completion counters (the tail of
-// the first layer's last, partly empty wave is filled with tiles of the second).  Both are short (one or two tiles per CTA),
-// so sharing one launch halves their fixed costs; the weight gradient's few long tiles go to the
-// first CTAs, the remaining CTAs split the many short tiles of the back-propagation.
+// A launch serves one problem (p0), or two independent ones (p1.mode >= 0): a layer's weight
+// gradient (p0) next to its delta back-propagation (p1).  Both are short (one or two tiles per
+// CTA), so sharing one launch halves their fixed costs; the weight gradient's few long tiles go to
+// the first CTAs, the remaining CTAs split the many short tiles of the back-propagation.
 // CG = 1: one CTA per tile of 128 x BN.  CG = 2: a cluster of two CTAs per tile of 256 x BN; the
 // leader (cluster rank 0) issues the MMAs for both, every CTA loads its own A rows and its half of
 // B and drains its own half of the accumulator.
@@ -318,34 +309,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     lead = max(1, (int)(long_t / short_t + 0.5f));
   }
   const int n_lead = split_units ? min(T1, lead * R_units) : 0;      // short tiles handed out before the long-tile units join
-  // Second problem reading the first's output (two forward layers) when the first has between one
-  // and two waves of tiles: the units left idle by its second wave take the tiles of the second
-  // problem whose inputs the FIRST wave produced (row tiles [0, n_units / n_ct0)), and whatever is
-  // left of the second problem is strided over all units afterwards.
-  const bool chain = T1 > 0 && p1.done_wait != nullptr && T0 > n_units && T0 < 2 * n_units;
-  const int ch_idle = 2 * n_units - T0;                                   // units without a second-wave tile
-  const int ch_early = min(T1, (n_units / P0.n_ct) * P1.n_ct);            // tiles of problem 1 fed by wave one
-  const int ch_per = chain ? (ch_early + ch_idle - 1) / ch_idle : 0;      // early tiles per idle unit
   auto tile_at = [&](int i) -> int {
-    if (chain) {
-      const int first_idle = T0 - n_units;                               // units [first_idle, n_units) are idle in wave two
-      if (i == 0) return unit;
-      if (unit < first_idle) {
-        if (i == 1) return unit + n_units;
-        const int t = T0 + ch_early + unit + (i - 2) * n_units;
-        return t < T0 + T1 ? t : -1;
-      }
-      if (i <= ch_per) {
-        const int e = (unit - first_idle) + (i - 1) * ch_idle;
-        if (e < ch_early) return T0 + e;
-      }
-      // after its early tiles (a unit may have one fewer than ch_per) the unit joins the late tiles
-      const int n_early_mine = (ch_early - (unit - first_idle) + ch_idle - 1) / ch_idle;
-      const int k = i - 1 - max(0, n_early_mine);
-      if (k < 0) return -1;
-      const int t = T0 + ch_early + unit + k * n_units;
-      return t < T0 + T1 ? t : -1;
-    }
     if (split_units) {
       if (unit < T0) {
         if (i == 0) return unit;
@@ -430,23 +394,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const CUtensorMap& map_a = c.which ? map_a1 : map_a0;
         const CUtensorMap& map_b = c.which ? map_b1 : map_b0;
         const int b0 = c.b_col + rank * BH;
-        {
-          // rows written by the other problem of this launch: wait (bounded) until all of their
-          // stores are complete, then order the tensor loads below after what was observed
-          const int* dw = c.which ? p1.done_wait : p0.done_wait;
-          if (dw != nullptr) {
-            const int target = c.which ? p1.done_target : p0.done_target;
-            const unsigned long long t0 = global_ns();
-            int seen;
-            for (uint32_t spin = 0;; ++spin) {
-              asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(dw + c.rt) : "memory");
-              if (seen >= target) break;
-              if ((spin & 63u) == 63u && (*abort || global_ns() - t0 > WAIT_LIMIT_NS)) { *abort = 1; ok = false; break; }
-            }
-            if (!ok) break;
-            asm volatile("fence.proxy.async;" ::: "memory");
-          }
-        }
         for (int kb = 0; kb < c.n_kb; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1u, abort)) { ok = false; break; }
           uint8_t* sa = smem + (size_t)stage * C::STAGE_BYTES;
@@ -708,15 +655,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
-      }
-      if (p.done_signal != nullptr) {
-        // this warp's stores of the tile are complete and ordered before the count that publishes them
-        if (issuer) {
-          asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-          asm volatile("fence.proxy.async;" ::: "memory");
-          __threadfence();
-          asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.done_signal + c.rt) : "memory");
-        }
       }
     }
     // shared memory may be released once the stores have read it; their global writes complete

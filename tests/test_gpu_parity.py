@@ -353,21 +353,6 @@ def test_merged_backward_launch_matches_separate_launches(dims, W, B):
     compare_with_oracle(cfg, X, y, w0, 25, TOL_BF16, forced=True, loss_tol=5e-2)
 
 
-@pytest.mark.parametrize("dims,W,B", [((3072, 1024, 512, 10), 128, 64), ((3072, 1024, 512, 10), 20, 64),
-                                      ((256, 512, 512, 256, 10), 24, 32), ((320, 520, 264, 10), 13, 40)])
-def test_paired_forward_launch_matches_separate_launches(dims, W, B):
-    """With the flag two consecutive hidden layers run their forward GEMMs in one launch; tiles of the
-    second wait on completion counters of the first's row tiles.  Every tile is computed the same way
-    either way, so the bits must be identical, and both match the oracle."""
-    cfg = _small_cfg(inputs.MLP, dims, inputs.BF16, W, B, max(3, W // 8), 5, PARETO, n=6000)
-    X, y, w0 = _problem(cfg)
-    rows_a, params_a = gpu_run(cfg, X, y, w0, 30)
-    rows_b, params_b = gpu_run(cfg, X, y, w0, 30, flags=gpu.FLAG_FUSED_FORWARD)
-    assert rows_a == rows_b
-    assert np.array_equal(params_a, params_b)
-    compare_with_oracle(cfg, X, y, w0, 12, TOL_BF16, forced=True, loss_tol=5e-2, flags=gpu.FLAG_FUSED_FORWARD)
-
-
 def test_bf16_network_without_tensor_cores():
     """ABS_FLAG_NO_TENSOR_CORES: the hidden layers of a bf16 network on the FP32-FMA tile kernels
     (same storage points, other summation order)."""
