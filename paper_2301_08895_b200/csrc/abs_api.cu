@@ -79,6 +79,7 @@ struct Layout {
   size_t c_off[2] = {}, c_src[2] = {}, c_len[2] = {};               // W[k][k][Ci][Co] + b[Co]: padded / caller offset, length
   size_t x_len = 0;                       // elements of one dataset row
   size_t pool1 = 0, dpool1 = 0, arg1 = 0, arg2 = 0, cpart[2] = {};  // pooled maps of block 1, their delta, pool positions, chunk sums
+  int cchunk = 1;                         // gradient rows per CTA of the convolution weight-gradient kernel
   size_t bits[ABS_MAX_LAYERS + 1];      // ReLU sign bits of act[l] (tensor-core layers)
   size_t act[ABS_MAX_LAYERS + 1], delta[ABS_MAX_LAYERS + 1];
   size_t tr_K, tr_R, tr_theta, tr_T, tr_loss, tr_comm, tr_sel_off, tr_rst_off;
@@ -319,7 +320,10 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       L->dpool1 = cv.take(L->esz * (size_t)L->rows_cap * n_p1);
       L->arg1 = cv.take((size_t)L->rows_cap * n_p1);
       L->arg2 = cv.take((size_t)L->rows_cap * m->dims[0]);
-      for (int b = 0; b < 2; ++b) L->cpart[b] = cv.take(4 * L->c_len[b] * (size_t)(L->rows_cap / conv::CHUNK));
+      // rows per weight-gradient CTA: about two CTAs per SM when every worker is selected
+      L->cchunk = 1;
+      while (L->cchunk < conv::MAX_CHUNK && L->rows_cap / (2 * L->cchunk) >= 2 * 148) L->cchunk *= 2;
+      for (int b = 0; b < 2; ++b) L->cpart[b] = cv.take(4 * L->c_len[b] * (size_t)(L->rows_cap / L->cchunk));
     }
   }
   const size_t R = (size_t)m->max_rounds;
@@ -629,6 +633,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     c.d_pooled = b == 0 ? ctx->at<void>(L.dpool1) : ctx->at<void>(L.delta[0]);
     c.d_in = b == 0 ? nullptr : ctx->at<void>(L.dpool1);
     c.part = ctx->at<float>(L.cpart[b]);
+    c.chunk = L.cchunk;
     return c;
   };
   auto tc_params = [&](int l, int mode) {
@@ -794,10 +799,10 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     if (b == 1)      // delta of the first block's pooled maps (one CTA per row)
       launch_ex(ctx, ABS_KC_CONV, conv::conv_block_dgrad_kernel<T>, dim3(L.rows_cap), dim3(conv::THREADS),
                 conv::dgrad_smem_bytes(c.Hi, c.Wi, c.Ci, c.k, c.Co), c);
-    launch_ex(ctx, ABS_KC_CONV, conv::conv_block_wgrad_kernel<T>, dim3(L.rows_cap / conv::CHUNK), dim3(conv::THREADS),
+    launch_ex(ctx, ABS_KC_CONV, conv::conv_block_wgrad_kernel<T>, dim3(L.rows_cap / L.cchunk), dim3(conv::THREADS),
               conv::wgrad_smem_bytes(c.Hi, c.Wi, c.Ci, c.k, c.Co), c);
     launch_ex(ctx, ABS_KC_CONV, chunk_reduce_kernel, dim3(((int)L.c_len[b] + 31) / 32), dim3(256), 0, st, ri, c.part, (int)L.c_len[b],
-              ctx->at<float>(L.G) + L.c_off[b], conv::CHUNK);
+              ctx->at<float>(L.G) + L.c_off[b], L.cchunk);
   }
 }
 

@@ -12,7 +12,7 @@
 // over all rows.)  Maps are stored [row][y][x][channel] in the storage type; the images of the
 // first block are dataset rows fetched by sample index.  The channel counts of this model class
 // are far below a tensor-core tile (3 -> 6 -> 16 in the benchmark network), so these are FP32-FMA
-// kernels: one CTA per gradient row (forward, input delta) or per 16 rows (weight gradient),
+// kernels: one CTA per gradient row (forward, input delta) or per small chunk of rows (weight gradient),
 // everything the CTA needs staged in shared memory, fixed summation orders.
 #pragma once
 #include "common.cuh"
@@ -22,7 +22,7 @@ namespace absb {
 namespace conv {
 
 constexpr int THREADS = 256;
-constexpr int CHUNK = 16;        // gradient rows per CTA of the backward kernel (divides the row padding unit)
+constexpr int MAX_CHUNK = 16;    // most gradient rows per CTA of the weight-gradient kernel
 
 struct Args {
   DevState* st;
@@ -39,6 +39,9 @@ struct Args {
   const void* d_pooled;     // backward: [rows][Ph][Pw][Co] delta of the pooled maps
   void* d_in;               // backward: [rows][Hi][Wi][Ci] delta of the input maps (second block)
   float* part;              // backward: [chunks][k k Ci Co + Co] per-chunk sums of the weight and bias gradient
+  int chunk;                // gradient rows per CTA of the weight-gradient kernel: a power of two (divides the row
+                            // padding unit, so a chunk never straddles two model versions), chosen by the host so
+                            // that the worst-case round gives every SM about two CTAs
 };
 
 inline size_t fwd_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
@@ -113,7 +116,7 @@ __global__ void __launch_bounds__(THREADS) conv_block_fwd_kernel(Args a) {
   }
 }
 
-// Weight and bias gradient of one block over CHUNK consecutive gradient rows: this CTA's share of
+// Weight and bias gradient of one block over `chunk` consecutive gradient rows: this CTA's share of
 // the sum of Eq. 3 (a fixed-order reduction over the CTAs follows).  Only the window position that
 // supplied a pooled maximum carries a delta, so the sum runs over pooled pixels.
 template <typename T>
@@ -123,6 +126,7 @@ __global__ void __launch_bounds__(THREADS) conv_block_wgrad_kernel(Args a) {
   DevState* st = a.st;
   RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
+  const int CHUNK = a.chunk;
   const int r0 = blockIdx.x * CHUNK;
   if (r0 >= ri->n_rows) return;
   const int Hi = a.Hi, Wi = a.Wi, Ci = a.Ci, k = a.k, Co = a.Co;

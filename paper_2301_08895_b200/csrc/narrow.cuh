@@ -651,9 +651,11 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
     wf[(size_t)c * wld + k] = ldf(wraw, i);
   }
   __syncthreads();
-  // ---- logits, loss, delta: a warp takes four rows at a time
+  // ---- logits, loss, delta: a warp takes four rows at a time (two, one when the block has fewer
+  // rows than that keeps all eight warps busy; a row's sum is formed in the same order either way)
   bool bad = false;
-  for (int rb = warp * 4; rb < R; rb += 32) {
+  const int rpw = R >= 32 ? 4 : (R >= 16 ? 2 : 1);
+  for (int rb = warp * rpw; rb < R; rb += 8 * rpw) {
     float acc[4][CC];
 #pragma unroll
     for (int q = 0; q < 4; ++q)
@@ -662,25 +664,31 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
     for (int v = lane; v < nvec; v += 32) {
       float xv[4][8];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) load8(hs + (size_t)(rb + q) * in + v * 8, xv[q]);
+      for (int q = 0; q < 4; ++q)
+        if (q < rpw) load8(hs + (size_t)(rb + q) * in + v * 8, xv[q]);
 #pragma unroll
       for (int c = 0; c < CC; ++c) {
         float wv[8];
         load8(wf + (size_t)c * wld + v * 8, wv);
 #pragma unroll
         for (int q = 0; q < 4; ++q)
+          if (q < rpw) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) acc[q][c] = fmaf(xv[q][j], wv[j], acc[q][c]);
+            for (int j = 0; j < 8; ++j) acc[q][c] = fmaf(xv[q][j], wv[j], acc[q][c]);
+          }
       }
     }
 #pragma unroll
     for (int q = 0; q < 4; ++q)
+      if (q < rpw) {
 #pragma unroll
-      for (int c = 0; c < CC; ++c)
+        for (int c = 0; c < CC; ++c)
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc[q][c] += __shfl_xor_sync(0xffffffffu, acc[q][c], o);
+          for (int o = 16; o > 0; o >>= 1) acc[q][c] += __shfl_xor_sync(0xffffffffu, acc[q][c], o);
+      }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
+      if (q >= rpw) break;
       const int rr = rb + q, r = r0 + rr;
       const int s = a.row_idx[r];
       if (s < 0) {                              // padding row: contributes nothing to Eq. 3
@@ -744,8 +752,11 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
       }
     }
   }
-  // ---- this block's share of the weight and bias gradient
+  // ---- this block's share of the weight and bias gradient, staged in the (no longer needed)
+  // transposed-weight area in the layout of the result and then copied out with coalesced stores
   float* dst = part + (size_t)blockIdx.x * (size_t)(in + 1) * CC;
+  __syncthreads();                              // all reads of the transposed weights are done
+  float* stg = wf;                              // [(in + 1)][CC]
   for (int it = tid; it < in / 2; it += 256) {
     const int m = 2 * it;
     float acc0[CC], acc1[CC];
@@ -763,13 +774,15 @@ __global__ void __launch_bounds__(256) narrow_fused_cc_kernel(NarrowArgs a, floa
       }
     }
 #pragma unroll
-    for (int c = 0; c < CC; ++c) { dst[(size_t)m * CC + c] = acc0[c]; dst[(size_t)(m + 1) * CC + c] = acc1[c]; }
+    for (int c = 0; c < CC; ++c) { stg[m * CC + c] = acc0[c]; stg[(m + 1) * CC + c] = acc1[c]; }
   }
   if (tid < CC) {
     float tot = 0.f;
     for (int rr = 0; rr < R; ++rr) tot += d3[rr * CC + tid];
-    dst[(size_t)in * CC + tid] = tot;
+    stg[in * CC + tid] = tot;
   }
+  __syncthreads();
+  for (int i = tid; i < (in + 1) * CC; i += 256) dst[i] = stg[i];
 }
 
 // ---------------------------------------------------------------------------------------------
