@@ -232,7 +232,10 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     // sums the Eq. 3 step then has to read
     double best = 1e30;
     int bestP = 1;
-    const int maxP = std::max(1, std::min(4, W * m->batch / 512));   // more partials cost the Eq. 3 step too much
+    // splits of at least 512 rows: up to 4, because each split is one more partial vector for the Eq. 3 step to
+    // read (measured on configuration 4: 7 splits cost it 12 us and win the weight gradient nothing); up to 8 for
+    // small models, whose single-wave weight gradient halves its k loop and whose partials stay in L2
+    const int maxP = std::max(1, std::min(L->d_pad < ((size_t)1 << 20) ? 8 : 4, W * m->batch / 512));
     for (int P = 1; P <= maxP; ++P) {
       double t = 4.0 * (double)L->d_pad * P / 5e12;
       for (int l = 0; l < m->n_layers; ++l) {
@@ -812,7 +815,7 @@ void enqueue_update(abs_ctx* ctx, int par) {
   RoundInfo* ri = ctx->at<RoundInfo>(L.ri) + par;
   if (ctx->lsq_v2) {
     LsqUpdateArgs q;
-    q.st = ctx->at<DevState>(L.st); q.ri = ri; q.job = ctx->ctl.job; q.next_dur = ctx->overlap ? nullptr : ctx->ctl.next_dur; q.dur_job = ctx->ctl.dur_job;
+    q.st = ctx->at<DevState>(L.st); q.ri = ri; q.job = ctx->ctl.job; q.next_dur = nullptr; q.dur_job = ctx->ctl.dur_job;   // durations: control kernel
     q.master = ctx->at<float>(L.master); q.ring = ctx->at<void>(L.ring); q.G = ctx->at<float>(L.G);
     q.d_pad = L.d_pad; q.d = ctx->m.dims[0]; q.P = ctx->lsq_grid; q.lr = ctx->m.lr;
     q.loss_part = ctx->lsq_pipe ? ctx->at<float>(L.row_loss) : nullptr;
@@ -827,7 +830,8 @@ void enqueue_update(abs_ctx* ctx, int par) {
   u.sel_tau = ctx->ctl.sel_tau[par];
   // for the latency-bound models (always one stream) the Eq. 3 kernel also prepares the next job
   // durations (its first warps); tensor-core networks keep a small kernel of their own for that
-  const bool look = !L.any_tc;
+  // job durations are prepared by the control kernel, except on the local-step paths
+  const bool look = ctx->local_sgd || (L.local_net && !L.any_tc);
   u.job = ctx->ctl.job; u.next_dur = ctx->ctl.next_dur; u.dur_job = ctx->ctl.dur_job;
   // one wave of resident blocks striding over the vector (a partly filled second wave would only add a tail)
   const size_t n4 = L.d_pad / 4;
@@ -1001,6 +1005,7 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     c.row_idx[q] = ctx->at<int>(L.row_idx[q]); c.tile_slot[q] = ctx->at<int>(L.tile_slot[q]);
   }
   c.loss = ctx->at<float>(L.loss);
+  c.loss_part = nullptr; c.loss_groups = 0;
   // with local steps a worker's loss is uploaded whole (no per-row losses, no row layout)
   c.row_loss = (model->kind == ABS_LSQ || model->local_steps > 1) ? nullptr : ctx->at<float>(L.row_loss);
   c.tr_K = ctx->at<int>(L.tr_K); c.tr_R = ctx->at<int>(L.tr_R); c.tr_theta = ctx->at<int>(L.tr_theta);
@@ -1077,6 +1082,12 @@ int abs_init(abs_ctx** out, const abs_model_desc* model, int W, int K0, int stal
     if (er != cudaSuccess) return bail(cuda_fail(nullptr, er, "cudaFuncSetAttribute(abs_lsq_rounds_kernel)"));
     ctx->lsq_rounds = true;
   }
+  if (ctx->lsq_pipe && !ctx->lsq_rounds) {
+    // the pipeline kernel leaves per-group loss sums: the control step finishes the uploaded losses
+    // itself (it runs next to the Eq. 3 kernel, which finishes them too, for its own divergence check)
+    ctx->ctl.loss_part = ctx->at<float>(L.row_loss);
+    ctx->ctl.loss_groups = (model->batch + lsqp::GROUP - 1) / lsqp::GROUP;
+  }
   rc = setup_tc(ctx);
   if (rc != ABS_OK) return bail(rc);
   {
@@ -1137,7 +1148,7 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     return fail(ABS_ENOSPACE, "%d rounds requested, %d of capacity %d already used", n, ctx->rounds_enqueued, ctx->m.max_rounds);
   const bool f32 = ctx->m.dtype == ABS_FP32;
   const size_t csm = sizeof(CtlShared);
-  void (*ctl_kernel)(CtlArgs, int, int, int) = ctx->W <= 256 ? abs_ctl_small_kernel : abs_ctl_kernel;
+  void (*ctl_kernel)(CtlArgs, int, int, int, int, int) = ctx->W <= 256 ? abs_ctl_small_kernel : abs_ctl_kernel;
   const int ctl_threads = ctx->W <= 256 ? 256 : 1024;
   const int times_blocks = (ctx->W + 31) / 32;
   const DevState* stc = ctx->at<DevState>(ctx->L.st);
@@ -1162,14 +1173,14 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     const int nt = local::threads_for(q.lsq ? q.in : q.in * q.C + q.C);
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
-      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
+      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t, 0, 0);
       q.ri = ctx->at<RoundInfo>(ctx->L.ri) + par;
       q.sel = ctx->ctl.sel[par]; q.sel_tau = ctx->ctl.sel_tau[par];
       if (f32) launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<float>, dim3(ctx->W), dim3(nt), sm, q);
       else launch_ex(ctx, ABS_KC_LSQ, local::local_sgd_kernel<__nv_bfloat16>, dim3(ctx->W), dim3(nt), sm, q);
       update(par);
     }
-    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n, 0, 0);
   } else if (n > 0 && ctx->L.local_net) {
     // U > 1 on a multi-layer network: per round, the workers' copies are set up, then every local
     // step is one pass of the gradient kernels over the private copies (which add each worker's
@@ -1186,7 +1197,7 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     const int bx = (int)std::max<size_t>(1, std::min<size_t>((L.d_pad / 4 + 1023) / 1024, 64));
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
-      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
+      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t, 0, 0);
       if (L.any_tc)
         launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
       q.ri = ctx->at<RoundInfo>(L.ri) + par;
@@ -1203,7 +1214,7 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
       }
       update(par);
     }
-    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n, 0, 0);
   } else if (n > 0 && ctx->lsq_rounds) {
     LsqRoundsArgs q;
     q.X = ctx->X; q.y = (const float*)ctx->y;
@@ -1213,18 +1224,22 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     if (f32) launch_ex(ctx, ABS_KC_ROUNDS, abs_lsq_rounds_kernel<float>, dim3(1), dim3(LSQ_ROUNDS_NT), sm, ctx->ctl, q, ctx->rounds_enqueued, n);
     else launch_ex(ctx, ABS_KC_ROUNDS, abs_lsq_rounds_kernel<__nv_bfloat16>, dim3(1), dim3(LSQ_ROUNDS_NT), sm, ctx->ctl, q, ctx->rounds_enqueued, n);
   } else if (n > 0 && !ctx->overlap) {
+    // One stream.  The control step of round t+1 does not depend on the Eq. 3 step of round t, which
+    // is the kernel in front of it: it is launched without waiting for it (programmatic dependent
+    // launch: it starts once every block of the Eq. 3 kernel has passed its own wait, i.e. once the
+    // gradient kernels of round t are complete), runs next to it, prepares the next job durations
+    // itself and waits for the Eq. 3 kernel at its end.  The first control step of a call follows
+    // something else and waits at its start.
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
       // the control kernel completes the previous round (if any) and selects this round's arrivals
-      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
-      if (ctx->L.any_tc)    // the other models prepare the next durations inside their Eq. 3 kernel
-        launch_ex(ctx, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
+      launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t, r > 0 ? 1 : 0, 1);
       gradient(par, PH_GATHER);
       gradient(par, PH_FORWARD);
       gradient(par, PH_BACKWARD);
       update(par);
     }
-    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+    launch_ex(ctx, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n, 1, 1);
   } else if (n > 0) {
     // Two streams.  Side stream per round t: control kernel (finish t-1, select t), row gather,
     // [event ctl], duration look-ahead.  Main stream: wait ctl, forward kernels, [event loss],
@@ -1235,7 +1250,7 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
     CU(cudaStreamWaitEvent(B, ctx->ev_loss, 0));
     for (int r = 0; r < n; ++r) {
       const int t = ctx->rounds_enqueued + r, par = t & 1;
-      launch_on(ctx, B, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t);
+      launch_on(ctx, B, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 1, t, 0, 0);
       gradient(par, PH_GATHER);
       CU(cudaEventRecord(ctx->ev_ctl, B));
       launch_on(ctx, B, ABS_KC_CTL, abs_times_kernel, dim3(times_blocks), dim3(32), 0, stc, ctx->ctl.job, ctx->ctl.next_dur, ctx->ctl.dur_job);
@@ -1246,7 +1261,7 @@ int abs_enqueue_rounds(abs_ctx* ctx, int n) {
       gradient(par, PH_BACKWARD);
       update(par);
     }
-    launch_on(ctx, B, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n);
+    launch_on(ctx, B, ABS_KC_CTL, ctl_kernel, dim3(1), dim3(ctl_threads), csm, ctx->ctl, 1, 0, ctx->rounds_enqueued + n, 0, 0);
     CU(cudaEventRecord(ctx->ev_ctl, B));
     CU(cudaStreamWaitEvent(A, ctx->ev_ctl, 0));       // the caller's stream covers all of it
   }

@@ -94,6 +94,8 @@ struct CtlArgs {
   int* tile_slot[2];   // [rows_cap / RB] ring slot of each row tile
   u64* next_dur;       // [W] duration of the job each worker starts next, computed ahead of time
   int* dur_job;        // [W] job index next_dur[n] belongs to
+  const float* loss_part;  // least-squares pipeline: per (selected worker, row group) sums of 1/2 r^2, or null;
+  int loss_groups;         // the upload's loss is their sum over the groups divided by B
   // trace
   int* tr_K; int* tr_R; int* tr_theta; u64* tr_T; float* tr_loss; u64* tr_comm;
   i64* tr_sel_off; i64* tr_rst_off;

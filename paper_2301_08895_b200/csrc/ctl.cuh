@@ -32,11 +32,14 @@ __device__ __forceinline__ double ln_series(double u) {
   if (m >= 1.4142135623730951) { m = __dmul_rn(m, 0.5); e += 1; }
   const double s = __ddiv_rn(__dadd_rn(m, -1.0), __dadd_rn(m, 1.0));
   const double s2 = __dmul_rn(s, s);
-  double p = __ddiv_rn(1.0, 23.0);
+  // the coefficients 1 / (2k + 1) are correctly rounded quotients of constants: compile-time values
+  constexpr double INV_ODD[12] = {1.0 / 1.0,  1.0 / 3.0,  1.0 / 5.0,  1.0 / 7.0,  1.0 / 9.0,  1.0 / 11.0,
+                                  1.0 / 13.0, 1.0 / 15.0, 1.0 / 17.0, 1.0 / 19.0, 1.0 / 21.0, 1.0 / 23.0};
+  double p = INV_ODD[11];
 #pragma unroll
   for (int k = 10; k >= 0; --k) {
     p = __dmul_rn(p, s2);
-    p = __dadd_rn(p, __ddiv_rn(1.0, (double)(2 * k + 1)));
+    p = __dadd_rn(p, INV_ODD[k]);
   }
   const double head = __dmul_rn((double)e, 0.6931471805599453);
   const double tail = __dmul_rn(__dmul_rn(2.0, s), p);
@@ -153,10 +156,21 @@ struct CtlShared {
 // needs is loaded up front in one wave and later phases work from registers and shared memory.
 //   t_sel:     index of the round that follows the open one (the host counts rounds; parity of
 //              t_sel - 1 / t_sel picks the layout copy of the open / the new round)
+//   look_here: the workers that were renewed also get the duration of the job AFTER the one they
+//              start now prepared here, at the end of the step (see refresh_next_durations), for
+//              callers that have no other kernel between two control steps to do it
+//   late_status: when the step runs next to the Eq. 3 kernel of the round it finishes, a status it
+//              raises must not be seen by that kernel's blocks (they would skip a valid step):
+//              the status is left in *late_status (shared memory) for the caller to publish later
 template <int NT>
-__device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do_finish, int do_select, int t_sel) {
+__device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do_finish, int do_select, int t_sel,
+                                         int look_here = 0, int* late_status = nullptr) {
   DevState* st = a.st;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  auto raise = [&](int code) {
+    if (late_status != nullptr) *late_status = code;
+    else st->status = code;
+  };
   // ---- one wave of loads
   const int W = st->W, S = st->S, B = st->B, RB = st->RB, K0 = st->K0;
   const int po = (t_sel - 1) & 1, pn = t_sel & 1;     // layout copy of the open / of the new round
@@ -184,10 +198,17 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
   float my_loss = 0.f;
   if (fin && tid < K) {
     my_sel = a.sel[po][tid]; my_tau = a.sel_tau[po][tid]; my_row0 = a.sel_row0[po][tid];
-    if (!net) my_loss = a.loss[tid];
+    if (!net && a.loss_part == nullptr) my_loss = a.loss[tid];
+    if (!net && a.loss_part != nullptr) {
+      // the least-squares pipeline leaves per-group sums; same order and rounding as its Eq. 3 kernel
+      float s = 0.f;
+      for (int g = 0; g < a.loss_groups; ++g) s += a.loss_part[(size_t)tid * a.loss_groups + g];
+      my_loss = __fdiv_rn(s, (float)B);
+    }
   }
   if (status0 != ST_OK) return 1;
 
+  int renewed = 0;          // this thread's worker started a new job in the finish step
   // ------------------------------------------------------------------ finish round t
   if (fin) {
     const u64 T_end = T_end0;
@@ -214,7 +235,7 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
     }
     const int bad = __syncthreads_or((tid < K) && !isfinite(my_loss)) || diverged0;
     if (bad) {
-      if (tid == 0) { st->status = ST_DIVERGED; st->open = 0; }
+      if (tid == 0) { raise(ST_DIVERGED); st->open = 0; }
       return 1;
     }
     // loss estimate: adjacent-pair tree sum in binary32 over 1024 leaves, /K in binary32
@@ -287,6 +308,7 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
       const u64 cn = T_end + dt;
       if (dt == 0ull || cn >= (1ull << 53)) range_err = 1;
       my_job = j; my_version = t + 1; my_c = cn;
+      renewed = 1;
       a.job[tid] = j;
       a.version[tid] = t + 1;
       a.c[tid] = cn;
@@ -311,7 +333,7 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
       a.tr_sel_off[t + 1] = sel_off + K; a.tr_rst_off[t + 1] = rst_off + R;
       st->sel_total = sel_off + K; st->rst_total = rst_off + R; st->comm = comm;
       st->L0 = L0; st->theta = theta; st->K = K_next; st->t = t + 1; st->open = 0;
-      if (range_err) st->status = ST_RANGE;
+      if (range_err) raise(ST_RANGE);
     }
     if (range_err) return 1;
     t = t + 1;
@@ -319,14 +341,19 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
     __syncthreads();
   }
 
+  // duration of the job after the one just started, for the next control step to look up
+  if (look_here && renewed) {
+    a.next_dur[tid] = job_ticks(st->dist, key0, key1, tid, my_job + 1);
+    a.dur_job[tid] = my_job + 1;
+  }
   // ------------------------------------------------------------------ select round t
   if (!do_select) return 1;
   if (t != t_sel) {                      // host and device disagree on the round index
-    if (tid == 0) st->status = ST_INTERNAL;
+    if (tid == 0) raise(ST_INTERNAL);
     return 1;
   }
   if (t >= max_rounds) {
-    if (tid == 0) st->status = ST_NOSPACE;
+    if (tid == 0) raise(ST_NOSPACE);
     return 1;
   }
   {
@@ -350,7 +377,7 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
       // with forced restarts this cannot happen (consumed staleness <= threshold <= S); without
       // them the arrival's model version may have left the ring: the run ends here, before any
       // kernel reads the slot that was overwritten
-      if (tid == 0) st->status = no_restart ? ST_STALE : ST_INTERNAL;
+      if (tid == 0) raise(no_restart ? ST_STALE : ST_INTERNAL);
       return 1;
     }
     // network models: group the arrivals by staleness (all members of a group read the same
@@ -444,20 +471,40 @@ __device__ __forceinline__ int ctl_round(const CtlArgs& a, CtlShared& sh, int do
   return 0;
 }
 
-__global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select, int t_sel) {
-  grid_dependency_sync();
+// pdl = 0: the step waits for the kernel in front of it before it starts.  pdl = 1: the kernel in
+// front is the Eq. 3 step of the round being finished, which this step does not depend on (it reads
+// the uploaded losses, which were complete before the Eq. 3 kernel passed its own wait, and it
+// prepares the job durations itself): the two run side by side, and this kernel waits for the
+// Eq. 3 kernel only at its end, so that whatever follows in the stream sees both complete.
+// look: see ctl_round (the Eq. 3 kernel then does not touch the prepared durations).
+__global__ void __launch_bounds__(1024, 1) abs_ctl_kernel(CtlArgs a, int do_finish, int do_select, int t_sel, int pdl, int look) {
+  if (pdl) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  else grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char ctl_smem[];
   CtlShared& sh = *reinterpret_cast<CtlShared*>(ctl_smem);
-  ctl_round<1024>(a, sh, do_finish, do_select, t_sel);
+  __shared__ int late;
+  if (threadIdx.x == 0) late = ST_OK;
+  ctl_round<1024>(a, sh, do_finish, do_select, t_sel, look, pdl ? &late : nullptr);
+  if (pdl) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (threadIdx.x == 0 && late != ST_OK) a.st->status = late;      // the Eq. 3 kernel is done: publish
+  }
 }
 
 // The same step with 256 threads for runs of at most 256 workers (one thread per worker is all the
 // step needs; its block-wide barriers are cheaper with 8 warps than with 32).
-__global__ void __launch_bounds__(256, 1) abs_ctl_small_kernel(CtlArgs a, int do_finish, int do_select, int t_sel) {
-  grid_dependency_sync();
+__global__ void __launch_bounds__(256, 1) abs_ctl_small_kernel(CtlArgs a, int do_finish, int do_select, int t_sel, int pdl, int look) {
+  if (pdl) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  else grid_dependency_sync();
   extern __shared__ __align__(16) unsigned char ctl_smem[];
   CtlShared& sh = *reinterpret_cast<CtlShared*>(ctl_smem);
-  ctl_round<256>(a, sh, do_finish, do_select, t_sel);
+  __shared__ int late;
+  if (threadIdx.x == 0) late = ST_OK;
+  ctl_round<256>(a, sh, do_finish, do_select, t_sel, look, pdl ? &late : nullptr);
+  if (pdl) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (threadIdx.x == 0 && late != ST_OK) a.st->status = late;      // the Eq. 3 kernel is done: publish
+  }
 }
 
 // Duration look-ahead (see refresh_next_durations): one warp per 32 workers.
