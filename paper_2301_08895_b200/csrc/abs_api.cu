@@ -232,10 +232,11 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     // sums the Eq. 3 step then has to read
     double best = 1e30;
     int bestP = 1;
-    // splits of at least 512 rows: up to 4, because each split is one more partial vector for the Eq. 3 step to
-    // read (measured on configuration 4: 7 splits cost it 12 us and win the weight gradient nothing); up to 8 for
-    // small models, whose single-wave weight gradient halves its k loop and whose partials stay in L2
-    const int maxP = std::max(1, std::min(L->d_pad < ((size_t)1 << 20) ? 8 : 4, W * m->batch / 512));
+    // splits of at least 512 rows, at most 4: each split is one more partial vector for the Eq. 3 step (7 splits cost
+    // it 12 us on configuration 4 and win the weight gradient nothing), and on small models a weight gradient spread
+    // over more CTAs takes the SMs the side-stream kernels of the next round run on (configuration 3: 8 splits make
+    // the kernel 4 us shorter and the round 5 us longer)
+    const int maxP = std::max(1, std::min(4, W * m->batch / 512));
     for (int P = 1; P <= maxP; ++P) {
       double t = 4.0 * (double)L->d_pad * P / 5e12;
       for (int l = 0; l < m->n_layers; ++l) {
