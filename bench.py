@@ -210,6 +210,9 @@ def main():
     ap.add_argument("--samples", type=int, default=None,
                     help="dataset rows (default: the configuration's; smaller for profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work")
+    ap.add_argument("--timeline", type=int, default=0,
+                    help="instead of the benchmark: print the event-bracketed launches (class, start us, end us; both "
+                         "streams) of this many rounds after 50 warm rounds, in the configured launch mode")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -332,6 +335,25 @@ def main():
         d2h = params.nbytes + sum(v.nbytes for v in tr.values())
         ctx.close()
         return dt, wg, d2h
+
+    if args.timeline:
+        # measurement aid: every launch between two CUDA events (about 2.6 us each on their stream, and the
+        # events break the back-to-back chaining of the kernels, so periods are longer than in the timed runs)
+        ctx = new_ctx()
+        warm = min(50, max(0, rounds - args.timeline))
+        ctx.run_rounds(warm)
+        ctx.profile_start(args.timeline * 40)
+        ctx.run_rounds(args.timeline)
+        tl = ctx.profile_timeline(args.timeline * 40)
+        ctx.profile_read()
+        ctx.close()
+        upd = [i for i, (c, _, _) in enumerate(tl) if c == "update"]
+        t0 = tl[0][1]
+        for c, a, b in tl:
+            print("%-8s start %8.1f  end %8.1f  dur %6.1f" % (c, 1e3 * (a - t0), 1e3 * (b - t0), 1e3 * (b - a)))
+        if len(upd) >= 3:
+            print("round period us: %.1f" % (1e3 * (tl[upd[-1]][2] - tl[upd[0]][2]) / (len(upd) - 1)))
+        return
 
     for _ in range(args.warmup):
         device_step()

@@ -73,3 +73,14 @@ def test_restore_rejects_an_image_of_another_run():
         c.restore_state(image)
     assert e.value.code == gpu.EINVAL
     c.close()
+    # same sizes, other hyper-parameters: the image carries the model description and the modes
+    for kw_other, cfg_other in (({}, dataclasses.replace(cfg, lr=0.03)),               # step size
+                                ({"local_steps": 3}, cfg),                               # U (the upload block keeps its size)
+                                ({"sa_penalty": 1}, cfg),                                # staleness-aware step size
+                                ({"restart_rule": gpu.RESTART_NONE}, cfg),               # no forced restarts
+                                ({"flags": gpu.FLAG_NO_PERSISTENT}, cfg)):               # another kernel path
+        d, keep_d = _ctx(cfg_other, X, y, w0, 20, **kw_other)
+        with pytest.raises(gpu.AbsError) as e:
+            d.restore_state(image)
+        assert e.value.code == gpu.EINVAL, kw_other
+        d.close()
