@@ -4,13 +4,17 @@
 // Work item = (selected worker i, group g of 8 minibatch rows).  Items are dealt round-robin to one
 // persistent CTA per SM.  A producer warp copies an item's rows X[idx_b][:] (8 KB each at d = 4096)
 // and the model vector of the worker's version into a ring of shared-memory stages with
-// cp.async.bulk + mbarrier; 256 consumer threads take a stage, each reading ITS columns of all
+// cp.async.bulk + mbarrier; 512 consumer threads take a stage, each reading ITS columns of all
 // rows once into registers (column slice = the 16-byte vector tid of every row), and from those
 // registers form the partial dot products (block-reduced in a fixed order to the residuals
 // r_b = x_b . w_v - y_b) and then the gradient contribution sum_b r_b x_b into accumulators that
 // persist over all items of the CTA.  Every sample row is read from HBM exactly once and from
-// shared memory exactly once.  Eq. 3 only needs the sum over workers: a CTA writes one partial sum,
-// and one partial loss sum per item; the Eq. 3 kernel adds both up in a fixed order.
+// shared memory exactly once.  The copies keep up easily (the producer waits for free stages a third
+// of the time); what bounds a CTA is the consumers' instruction issue and the shared-memory /
+// shuffle pipe, so their inner loops are packed FMAs on operands kept in 64-bit registers and the
+// block reduction costs each warp one store, one 16-byte load and 19 shuffles per item.  Eq. 3 only
+// needs the sum over workers: a CTA writes one partial sum, and one partial loss sum per item; the
+// Eq. 3 kernel adds both up in a fixed order.
 #pragma once
 #include "common.cuh"
 #include "ctl.cuh"
@@ -25,6 +29,8 @@ constexpr int NWARPS = CONSUMERS / 32;
 constexpr int THREADS = CONSUMERS + 32;  // + producer warp
 constexpr int MAX_ITEMS = 64;            // items whose sample indices and targets are staged at once
 constexpr int MAX_STAGES = 6;
+constexpr int RS = 20;                   // floats between rows of the partial-dot table [GROUP][RS]: 16-byte reads of a row's
+                                         // quarters by 8 lanes fall into different banks
 
 struct Args {
   DevState* st;
@@ -41,16 +47,32 @@ struct Args {
 
 inline size_t stage_bytes(int d) { return (size_t)(GROUP + 1) * d * 2; }
 inline size_t smem_bytes(int d, int stages) {
-  return (size_t)stages * stage_bytes(d) + (size_t)MAX_ITEMS * GROUP * 8 + MAX_ITEMS * 8 + 2 * NWARPS * GROUP * 4 +
+  return (size_t)stages * stage_bytes(d) + (size_t)MAX_ITEMS * GROUP * 8 + MAX_ITEMS * 8 + 2 * GROUP * RS * 4 +
          2 * MAX_STAGES * 8 + 64;
 }
 
-// (d0, d1) += (a0, a1) * (b0, b1): two binary32 FMAs in one instruction (each lane rounds like a
-// scalar fma); the consumers are bound by instruction issue, so this halves their FMA count.
-__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
-  asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%0, %1};\n\t"
-      "fma.rn.f32x2 rc, ra, rb, rc;\n\tmov.b64 {%0, %1}, rc;\n\t}"
-      : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+// Two binary32 values in one 64-bit register (first value in the low word).  The consumers are bound
+// by instruction issue: a packed FMA (each half rounds like a scalar fma) halves their FMA count, and
+// operands that are created, kept and consumed as 64-bit registers need no moves around it.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// the two bf16 values of a 32-bit word as binary32 values (exact): element 0 (low half) first; a byte
+// permute and a mask, both on the integer pipe, so that the FMA pipe is left to the packed FMAs
+__device__ __forceinline__ f32x2 bf16x2_to_f32x2(uint32_t u) {
+  f32x2 r;
+  asm("{\n\t.reg .b32 lo, hi;\n\tprmt.b32 lo, %1, 0, 0x1044;\n\tand.b32 hi, %1, 0xffff0000;\n\tmov.b64 %0, {lo, hi};\n\t}"
+      : "=l"(r) : "r"(u));
+  return r;
+}
+__device__ __forceinline__ void ffma2(f32x2& d, f32x2 a, f32x2 b) {      // d += a * b, per half
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
 }
 
 __device__ __forceinline__ void bulk_row(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -76,8 +98,8 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
   float* m_y = reinterpret_cast<float*>(m_idx + MAX_ITEMS * GROUP);        // [MAX_ITEMS][GROUP] target
   int* m_slot = reinterpret_cast<int*>(m_y + MAX_ITEMS * GROUP);           // [MAX_ITEMS] ring slot of the worker
   float* m_sa = reinterpret_cast<float*>(m_slot + MAX_ITEMS);              // [MAX_ITEMS] weight of the worker's gradient in Eq. 3
-  float* red = m_sa + MAX_ITEMS;                                           // [2][NWARPS][GROUP] partial dots
-  uint64_t* full = reinterpret_cast<uint64_t*>(red + 2 * NWARPS * GROUP);  // [STAGES]
+  float* red = m_sa + MAX_ITEMS;                                           // [2][GROUP][RS] partial dots, [row][warp]
+  uint64_t* full = reinterpret_cast<uint64_t*>(red + 2 * GROUP * RS);      // [STAGES]
   uint64_t* empty = full + MAX_STAGES;                                     // [STAGES]
   volatile int* abort = reinterpret_cast<volatile int*>(empty + MAX_STAGES);
   volatile int* okflag = abort + 1;
@@ -91,9 +113,9 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
   // items of this CTA: it = blockIdx.x + q * gridDim.x, q = 0 .. my_items - 1
   const int my_items = n_items > (int)blockIdx.x ? (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
-  float acc[8];
+  f32x2 acc[4];                     // gradient sums of this thread's 8 columns (all-zero bits = two zeros)
 #pragma unroll
-  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  for (int j = 0; j < 4; ++j) acc[j] = 0ull;
   int stage = 0, buf = 0;
   uint32_t phase = 0;
   bool ok = true;
@@ -157,33 +179,37 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
         const int it = (int)blockIdx.x + (q0 + q) * (int)gridDim.x;
         const int g = it % groups;
         const int rows = min(GROUP, B - g * GROUP);
-        uint4 xr[GROUP];
-        const uint4 wr = in ? *reinterpret_cast<const uint4*>(sb + (size_t)GROUP * row_bytes + (size_t)vec * 16) : make_uint4(0u, 0u, 0u, 0u);
+        uint4 xr[GROUP], wr;
+        if (rows == GROUP && nvec == CONSUMERS) {      // the usual case (uniform in the CTA): no predicates
+          wr = *reinterpret_cast<const uint4*>(sb + (size_t)GROUP * row_bytes + (size_t)vec * 16);
 #pragma unroll
-        for (int r = 0; r < GROUP; ++r)
-          xr[r] = (in && r < rows) ? *reinterpret_cast<const uint4*>(sb + (size_t)r * row_bytes + (size_t)vec * 16)
-                                   : make_uint4(0u, 0u, 0u, 0u);
+          for (int r = 0; r < GROUP; ++r) xr[r] = *reinterpret_cast<const uint4*>(sb + (size_t)r * row_bytes + (size_t)vec * 16);
+        } else {
+          wr = in ? *reinterpret_cast<const uint4*>(sb + (size_t)GROUP * row_bytes + (size_t)vec * 16) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+          for (int r = 0; r < GROUP; ++r)
+            xr[r] = (in && r < rows) ? *reinterpret_cast<const uint4*>(sb + (size_t)r * row_bytes + (size_t)vec * 16)
+                                     : make_uint4(0u, 0u, 0u, 0u);
+        }
         // the stage is in registers now: hand it back to the producer
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(&empty[stage]);
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         // partial dot products of the 8 rows over this thread's 8 columns
-        float wf[8], pd[GROUP];
+        float pd[GROUP];
         {
-          const __nv_bfloat162* wh = reinterpret_cast<const __nv_bfloat162*>(&wr);
+          const f32x2 w2[4] = {bf16x2_to_f32x2(wr.x), bf16x2_to_f32x2(wr.y), bf16x2_to_f32x2(wr.z), bf16x2_to_f32x2(wr.w)};
 #pragma unroll
-          for (int j = 0; j < 4; ++j) { const float2 f = __bfloat1622float2(wh[j]); wf[2 * j] = f.x; wf[2 * j + 1] = f.y; }
-        }
-#pragma unroll
-        for (int r = 0; r < GROUP; ++r) {
-          const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xr[r]);
-          float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float2 f = __bfloat1622float2(xh[j]);
-            ffma2(s0, s1, f.x, f.y, wf[2 * j], wf[2 * j + 1]);
+          for (int r = 0; r < GROUP; ++r) {
+            f32x2 s2 = 0ull;               // (sum over even columns, sum over odd columns)
+            ffma2(s2, bf16x2_to_f32x2(xr[r].x), w2[0]);
+            ffma2(s2, bf16x2_to_f32x2(xr[r].y), w2[1]);
+            ffma2(s2, bf16x2_to_f32x2(xr[r].z), w2[2]);
+            ffma2(s2, bf16x2_to_f32x2(xr[r].w), w2[3]);
+            float s0, s1;
+            unpack2(s2, s0, s1);
+            pd[r] = s0 + s1;
           }
-          pd[r] = s0 + s1;
         }
         // warp sum of the 8 values with 9 shuffles: each exchange halves the rows a lane still carries;
         // afterwards lane l holds the warp's sum for row (l >> 2) & 7
@@ -207,16 +233,17 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
           k1 += __shfl_xor_sync(0xffffffffu, k1, 2);
           k1 += __shfl_xor_sync(0xffffffffu, k1, 1);
         }
-        float* rb = red + buf * (NWARPS * GROUP);
-        if ((lane & 3) == 0) rb[warp * GROUP + (lane >> 2)] = k1;
+        float* rb = red + buf * (GROUP * RS);
+        if ((lane & 3) == 0) rb[(lane >> 2) * RS + warp] = k1;
         asm volatile("bar.sync 1, %0;" ::"n"(CONSUMERS) : "memory");
-        // every warp adds the warps' sums up in the same order; lane r < 8 takes row r
-        float mine = 0.f;
-        if (lane < GROUP) {
-#pragma unroll
-          for (int w8 = 0; w8 < NWARPS; ++w8) mine += rb[w8 * GROUP + lane];
-          mine = lane < rows ? mine - m_y[q * GROUP + lane] : 0.f;
-        }
+        // every warp adds the 16 warps' sums of a row up in the same order: lane l takes row l & 7 and
+        // the four warps of quarter l >> 3 (one 16-byte load), then the quarters are added across lanes
+        const int row = lane & 7;
+        const float4 four = *reinterpret_cast<const float4*>(rb + row * RS + 4 * (lane >> 3));
+        float mine = (four.x + four.y) + (four.z + four.w);
+        mine += __shfl_xor_sync(0xffffffffu, mine, 8);
+        mine += __shfl_xor_sync(0xffffffffu, mine, 16);
+        mine = row < rows ? mine - m_y[q * GROUP + row] : 0.f;
         float res[GROUP], lsum = 0.f;
 #pragma unroll
         for (int r = 0; r < GROUP; ++r) {
@@ -227,13 +254,12 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
         const float sa = m_sa[q];
 #pragma unroll
         for (int r = 0; r < GROUP; ++r) {
-          res[r] *= sa;
-          const __nv_bfloat162* xh = reinterpret_cast<const __nv_bfloat162*>(&xr[r]);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float2 f = __bfloat1622float2(xh[j]);
-            ffma2(acc[2 * j], acc[2 * j + 1], f.x, f.y, res[r], res[r]);
-          }
+          const float rr = res[r] * sa;
+          const f32x2 r2 = pack2(rr, rr);
+          ffma2(acc[0], bf16x2_to_f32x2(xr[r].x), r2);
+          ffma2(acc[1], bf16x2_to_f32x2(xr[r].y), r2);
+          ffma2(acc[2], bf16x2_to_f32x2(xr[r].z), r2);
+          ffma2(acc[3], bf16x2_to_f32x2(xr[r].w), r2);
         }
         buf ^= 1;
       }
@@ -251,8 +277,11 @@ __global__ void __launch_bounds__(THREADS, 1) lsq_pipe_kernel(Args a) {
   if (tid < CONSUMERS) {
     float* gout = a.G + (size_t)blockIdx.x * a.slot_stride;
     if (tid < nvec) {
-      reinterpret_cast<float4*>(gout + (size_t)tid * 8)[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-      reinterpret_cast<float4*>(gout + (size_t)tid * 8)[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+      float g[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) unpack2(acc[j], g[2 * j], g[2 * j + 1]);
+      reinterpret_cast<float4*>(gout + (size_t)tid * 8)[0] = make_float4(g[0], g[1], g[2], g[3]);
+      reinterpret_cast<float4*>(gout + (size_t)tid * 8)[1] = make_float4(g[4], g[5], g[6], g[7]);
     }
   }
 }
