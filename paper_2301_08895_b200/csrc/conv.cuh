@@ -96,19 +96,31 @@ __global__ void __launch_bounds__(THREADS) conv_block_fwd_kernel(Args a) {
   __syncthreads();
   for (int e = threadIdx.x; e < n_out; e += THREADS) {
     const int co = e % Co, px = (e / Co) % Pw, py = e / (Co * Pw);
+    // the four window positions share their taps: per (dy, ci) the two image rows slide along dx,
+    // so a weight is read once for four FMAs and an image value once for two
+    float acc4[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int dy = 0; dy < k; ++dy)
+      for (int ci = 0; ci < Ci; ++ci) {
+        const float* r0 = img + ((2 * py + dy) * Wi + 2 * px) * Ci + ci;
+        const float* r1 = r0 + Wi * Ci;
+        const float* wp = wk + ((dy * k) * Ci + ci) * Co + co;
+        float p0 = r0[0], p1 = r1[0];
+        for (int dx = 0; dx < k; ++dx) {
+          const float n0 = r0[(dx + 1) * Ci], n1 = r1[(dx + 1) * Ci];
+          const float w = wp[dx * Ci * Co];
+          acc4[0] = fmaf(p0, w, acc4[0]);
+          acc4[1] = fmaf(n0, w, acc4[1]);
+          acc4[2] = fmaf(p1, w, acc4[2]);
+          acc4[3] = fmaf(n1, w, acc4[3]);
+          p0 = n0;
+          p1 = n1;
+        }
+      }
     float best = 0.f;
     int where = 0;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const int y = 2 * py + (q >> 1), x = 2 * px + (q & 1);
-      float acc = 0.f;
-      for (int dy = 0; dy < k; ++dy)
-        for (int dx = 0; dx < k; ++dx) {
-          const float* ip = img + ((y + dy) * Wi + (x + dx)) * Ci;
-          const float* wp = wk + ((dy * k + dx) * Ci) * Co + co;
-          for (int ci = 0; ci < Ci; ++ci) acc = fmaf(ip[ci], wp[ci * Co], acc);
-        }
-      const float v = as_stored_value<T>(fmaxf(acc + bias[co], 0.f));      // the stored ReLU output
+      const float v = as_stored_value<T>(fmaxf(acc4[q] + bias[co], 0.f));  // the stored ReLU output
       if (q == 0 || v > best) { best = v; where = q; }                      // first maximum wins a tie
     }
     stf(out, e, best);
