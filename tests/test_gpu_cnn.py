@@ -40,6 +40,7 @@ def _cnn_cfg(conv, fc, dtype, W, B, K0, S, time, n=3000, lr=0.01, seed=11):
     ((14, 14, 2, 3, 3, 4), (7, 6, 5), inputs.BF16, 9, 12, 30, TOL_BF16),
     ((32, 32, 3, 5, 6, 16), (120, 84, 10), inputs.BF16, 8, 32, 20, TOL_BF16),       # first affine layer on tensor cores (400 -> 120)
     ((22, 22, 3, 3, 8, 16), (128, 64, 10), inputs.BF16, 20, 24, 30, TOL_BF16),      # 256 features -> 128 -> 64 on tensor cores
+    ((14, 14, 2, 3, 16, 24), (12, 5), inputs.FP32, 6, 10, 10, TOL_FP32),            # wide blocks: 16 and 24 channels, 3480 parameters in the second one
 ])
 def test_cnn_matches_oracle(conv, fc, dtype, W, B, rounds, tol):
     cfg = _cnn_cfg(conv, fc, dtype, W, B, 3, 5, GAMMA3)
