@@ -236,7 +236,9 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
     // it 12 us on configuration 4 and win the weight gradient nothing), and on small models a weight gradient spread
     // over more CTAs takes the SMs the side-stream kernels of the next round run on (configuration 3: 8 splits make
     // the kernel 4 us shorter and the round 5 us longer)
-    const int maxP = std::max(1, std::min(4, W * m->batch / 512));
+    // (the CNN's affine layers see at most a few hundred rows per round and run on one stream: splits of 128 rows,
+    // so that its FP32 weight-gradient kernels, whose grid is tiles x splits, are more than a handful of CTAs)
+    const int maxP = std::max(1, std::min(4, W * m->batch / (L->cnn ? 128 : 512)));
     for (int P = 1; P <= maxP; ++P) {
       double t = 4.0 * (double)L->d_pad * P / 5e12;
       for (int l = 0; l < m->n_layers; ++l) {
