@@ -41,7 +41,7 @@ struct Args {
   float* part;              // backward: [chunks][k k Ci Co + Co] per-chunk sums of the weight and bias gradient
   int chunk;                // gradient rows per CTA of the weight-gradient kernel: a power of two (divides the row
                             // padding unit, so a chunk never straddles two model versions), chosen by the host so
-                            // that the worst-case round gives every SM about two CTAs
+                            // that a round with every worker selected gives every SM at least four CTAs
 };
 
 inline size_t fwd_smem_bytes(int Hi, int Wi, int Ci, int k, int Co) {
