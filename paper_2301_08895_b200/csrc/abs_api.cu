@@ -63,6 +63,8 @@ struct Layout {
   bool any_tc = false;
   int cg_fwd[ABS_MAX_LAYERS] = {}, cg_dg[ABS_MAX_LAYERS] = {}, cg_wg[ABS_MAX_LAYERS] = {};
   bool pair_bwd[ABS_MAX_LAYERS] = {};   // delta back-propagation and weight gradient of the layer share a launch
+  bool bias_colsum[ABS_MAX_LAYERS] = {}; // the layer's bias gradient = column sums of the delta the layer above back-propagates
+  size_t colsum[ABS_MAX_LAYERS] = {};   // [rows_cap / 32][out] those sums per group of 32 rows
   int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
   bool out_mma = false;                 // output layer through the mma.sync kernel (bf16, 64 rows per CTA)
   size_t esz = 4;                       // bytes per stored element (4 or 2)
@@ -227,6 +229,14 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       const long wg_tiles_min = (long)((in + 127) / 128 + 1) * ((out + bn - 1) / bn);   // at P = 1
       if (wg_tiles_min * 4 < 148) { L->pair_bwd[l] = true; L->bn_wg[l] = bn; }
     }
+    // A layer whose output delta is produced by the tensor-core back-propagation of the layer above gets its bias
+    // gradient from column sums taken in that kernel's epilogue; its weight gradient then needs no row tile of ones.
+    // (for at most as many layers as the Eq. 3 kernel takes partial-sum regions besides the output layer's)
+    for (int l = 0, n = 0; l + 1 < m->n_layers; ++l) {
+      L->bias_colsum[l] = L->path[l] == PATH_TC && L->path[l + 1] == PATH_TC && !L->local_net && m->local_steps <= 1 &&
+                          n < UpdateArgs::MAX_REGIONS - 1;
+      n += L->bias_colsum[l] ? 1 : 0;
+    }
     // split count P of the row reduction: the one that minimises the modelled time of all weight
     // gradients (whole waves of 148 CTAs, one tile = 128 x BN x rows/P) plus the extra partial
     // sums the Eq. 3 step then has to read
@@ -245,7 +255,7 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
         if (L->path[l] != PATH_TC) continue;
         const int in = m->dims[l], out = m->dims[l + 1], bn = L->bn_wg[l];
         const int cg = L->cg_wg[l], tm = 128 * cg, units = 148 / cg;
-        const long tiles = (long)((in + tm - 1) / tm + 1) * ((out + bn - 1) / bn) * P;
+        const long tiles = (long)((in + tm - 1) / tm + (L->bias_colsum[l] ? 0 : 1)) * ((out + bn - 1) / bn) * P;
         const long waves = (tiles + units - 1) / units;
         t += (double)waves * 2.0 * 128.0 * bn * ((double)L->rows_cap / P) / 9e12;
       }
@@ -309,6 +319,8 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
       L->red = cv.take(4 * len * (size_t)(L->rows_cap / (L->fused_R ? L->fused_R : 64)));
     }
     L->ones = L->any_tc ? cv.take(2 * 64 * (size_t)L->rows_cap) : 0;
+    for (int l = 0; l < m->n_layers; ++l)
+      if (L->bias_colsum[l]) L->colsum[l] = cv.take(4 * (size_t)(L->rows_cap / 32) * m->dims[l + 1]);
     for (int l = 0; l <= m->n_layers; ++l) L->bits[l] = 0;
     for (int l = 0; l + 1 < m->n_layers; ++l)
       if (L->path[l] == PATH_TC) L->bits[l + 1] = cv.take(4 * (size_t)L->rows_cap * ((m->dims[l + 1] + 31) / 32));
@@ -749,16 +761,19 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       pd.mask_bits = L.bits[l] ? ctx->at<uint32_t>(L.bits[l]) : nullptr;
       pd.mask_words = (la[l].in + 31) / 32;
       pd.out_bf16 = (__nv_bfloat16*)la[l].delta_in;
+      if (l > 0 && L.bias_colsum[l - 1]) pd.colsum = ctx->at<float>(L.colsum[l - 1]);   // bias gradient of the layer below
       const int bnd = L.bn_dg[l];
       const int dg_tiles = (row_tiles128 / std::max(1, L.cg_dg[l])) * ((la[l].in + std::max(1, bnd) - 1) / std::max(1, bnd));
       tc::Params p = tc_params(l, tc::WGRAD);
       p.M_total = la[l].in + 1; p.N_total = la[l].out;     // row `in` of the result is the bias gradient
       p.out_f32 = ctx->at<float>(L.G) + L.w_off[l];
+      p.no_bias_tile = L.bias_colsum[l] ? 1 : 0;
+      const int bias_tiles = L.bias_colsum[l] ? 0 : 1;
       if (l > 0 && L.pair_bwd[l]) {
         // the layer's delta back-propagation shares the weight gradient's launch (same tile width)
         const TcProblem second = {&ctx->tcl[l].dg_a, &ctx->tcl[l].dg_b, &ctx->tcl[l].dg_out, &pd, dg_tiles};
         launch_tc_bn(ctx, bnd, 1, ABS_KC_WGRAD, ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
-                     ((la[l].in + 127) / 128 + 1) * ((la[l].out + bnd - 1) / bnd) * n_splits, &second);
+                     ((la[l].in + 127) / 128 + bias_tiles) * ((la[l].out + bnd - 1) / bnd) * n_splits, &second);
         continue;
       }
       if (l > 0 || L.cnn)
@@ -766,7 +781,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
       const int bn = L.bn_wg[l];
       const int tmw = 128 * L.cg_wg[l];
       launch_tc_bn(ctx, bn, L.cg_wg[l], ABS_KC_WGRAD, (l == 0 && par) ? ctx->tcl[l].wg_a_odd : ctx->tcl[l].wg_a, ctx->tcl[l].wg_b, ctx->tcl[l].wg_out, p,
-                   ((la[l].in + tmw - 1) / tmw + 1) * ((la[l].out + bn - 1) / bn) * n_splits);
+                   ((la[l].in + tmw - 1) / tmw + bias_tiles) * ((la[l].out + bn - 1) / bn) * n_splits);
     } else if (L.path[l] == PATH_NARROW && L.fused_R) {
       // forward, loss, delta of the layer below and the gradient were all done by the fused kernel
     } else if (L.path[l] == PATH_NARROW) {
@@ -841,16 +856,20 @@ void enqueue_update(abs_ctx* ctx, int par) {
   // one wave of resident blocks striding over the vector (a partly filled second wave would only add a tail)
   const size_t n4 = L.d_pad / 4;
   int blocks = (int)std::max<size_t>(std::min<size_t>((n4 + 255) / 256, (size_t)ctx->sm_count * ctx->upd_blocks_per_sm), (size_t)(ctx->W + 31) / 32);
-  u.part = nullptr; u.part_len = 0; u.part_chunk_rows = 1; u.part_off = 0; u.n_main_blocks = blocks;
+  u.n_regions = 0; u.n_main_blocks = blocks;
+  memset(u.region, 0, sizeof u.region);
+  auto add_region = [&](const float* part, int len, int chunk_rows, size_t off) {
+    UpdateArgs::Region& R = u.region[u.n_regions++];
+    R.part = part; R.len = len; R.chunk_rows = chunk_rows; R.off = off; R.first_block = blocks - u.n_main_blocks;
+    blocks += (len + 31) / 32;
+  };
   const int last = ctx->m.n_layers - 1;
-  if (ctx->m.kind != ABS_LSQ && L.fused_R && L.path[last] == PATH_NARROW && !L.local_net && !ctx->local_sgd) {
+  if (ctx->m.kind != ABS_LSQ && L.fused_R && L.path[last] == PATH_NARROW && !L.local_net && !ctx->local_sgd)
     // the fused output-layer kernel left its gradient as per-chunk partial sums
-    u.part = ctx->at<float>(L.red);
-    u.part_len = (ctx->m.dims[last] + 1) * ctx->m.dims[last + 1];
-    u.part_chunk_rows = L.out_mma ? outl::ROWS : L.fused_R;
-    u.part_off = L.w_off[last];
-    blocks += (u.part_len + 31) / 32;
-  }
+    add_region(ctx->at<float>(L.red), (ctx->m.dims[last] + 1) * ctx->m.dims[last + 1], L.out_mma ? outl::ROWS : L.fused_R, L.w_off[last]);
+  for (int l = 0; l < ctx->m.n_layers && u.n_regions < UpdateArgs::MAX_REGIONS; ++l)
+    if (L.bias_colsum[l])     // bias gradient as column sums per 32 rows, left by the back-propagation of the layer above
+      add_region(ctx->at<float>(L.colsum[l]), ctx->m.dims[l + 1], 32, L.w_off[l] + (size_t)ctx->m.dims[l] * ctx->m.dims[l + 1]);
   if (look) launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T, true>, dim3(blocks), dim3(256), 0, u);
   else launch_ex(ctx, ABS_KC_UPDATE, update_kernel<T, false>, dim3(blocks), dim3(256), 0, u);
 }

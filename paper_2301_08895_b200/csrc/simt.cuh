@@ -337,13 +337,20 @@ struct UpdateArgs {
   const int* sel_tau;     // [K^t] staleness of each selected worker's upload (read when the staleness-aware
                           // step size is applied to whole uploads: DevState::sa_penalty == 2, P == 0)
   float lr;
-  // Output-layer gradient still in per-chunk partial sums (or null): blocks [n_main_blocks, gridDim.x)
-  // add the chunks of 32 outputs each in a fixed order and apply Eq. 3 to those parameters; the
-  // streaming blocks skip the range.
-  const float* part;      // [chunks][part_len]
-  int part_len;           // (in + 1) * C parameters of the output layer
-  int part_chunk_rows;    // gradient rows per chunk
-  size_t part_off;        // element offset of the output layer inside the parameter vector (multiple of 4)
+  // Parts of the gradient that are still per-chunk partial sums (the output layer's block left by the fused
+  // output kernels; bias gradients left as column sums per 32 rows by the back-propagation GEMM): blocks
+  // [n_main_blocks, gridDim.x) add the chunks of 32 parameters each in a fixed order and apply Eq. 3 to those
+  // parameters; the streaming blocks skip the ranges.
+  struct Region {
+    const float* part;    // [chunks][len]
+    int len;              // parameters
+    int chunk_rows;       // gradient rows per chunk
+    size_t off;           // element offset inside the parameter vector (multiple of 4; len too, unless it ends a layer)
+    int first_block;      // first of its (len + 31) / 32 blocks, counted from n_main_blocks
+  };
+  static constexpr int MAX_REGIONS = 3;
+  Region region[MAX_REGIONS];
+  int n_regions;
   int n_main_blocks;
 };
 
@@ -366,24 +373,30 @@ __global__ void __launch_bounds__(256, 4) update_kernel(UpdateArgs a) {
   const float step = __fdiv_rn(a.lr, (float)(K * st->B));
   const int slot = (ri->t + 1) % (st->S + 1);
   T* dst = (T*)a.ring + (size_t)slot * a.d_pad;
-  if (a.part != nullptr && (int)blockIdx.x >= a.n_main_blocks) {
+  if ((int)blockIdx.x >= a.n_main_blocks) {
     // lane w adds chunks w, w + 8, ... in order, then the 8 lanes are added in order
     __shared__ float red[8][33];
-    const int n_chunks = ri->n_rows / a.part_chunk_rows;
+    const int rb = (int)blockIdx.x - a.n_main_blocks;
+    int ri_ = 0;
+#pragma unroll
+    for (int q = 1; q < UpdateArgs::MAX_REGIONS; ++q)
+      if (q < a.n_regions && rb >= a.region[q].first_block) ri_ = q;
+    const UpdateArgs::Region& R = a.region[ri_];
+    const int n_chunks = ri->n_rows / R.chunk_rows;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int j = ((int)blockIdx.x - a.n_main_blocks) * 32 + lane;
+    const int j = (rb - R.first_block) * 32 + lane;
     float acc = 0.f;
-    if (j < a.part_len) {
+    if (j < R.len) {
 #pragma unroll 8
-      for (int q = w; q < n_chunks; q += 8) acc += a.part[(size_t)q * a.part_len + j];
+      for (int q = w; q < n_chunks; q += 8) acc += R.part[(size_t)q * R.len + j];
     }
     red[w][lane] = acc;
     __syncthreads();
-    if (w == 0 && j < a.part_len) {
+    if (w == 0 && j < R.len) {
       float tot = 0.f;
 #pragma unroll
       for (int q = 0; q < 8; ++q) tot += red[q][lane];
-      const size_t e = a.part_off + (size_t)j;
+      const size_t e = R.off + (size_t)j;
       const float m = fmaf(-step, tot, a.master[e]);
       a.master[e] = m;
       stf(dst, e, m);
@@ -391,13 +404,21 @@ __global__ void __launch_bounds__(256, 4) update_kernel(UpdateArgs a) {
     return;
   }
   const size_t n4 = a.d_pad / 4;
-  const size_t part_lo4 = a.part != nullptr ? a.part_off / 4 : n4;
-  const size_t part_hi4 = a.part != nullptr ? (a.part_off + (size_t)a.part_len + 3) / 4 : n4;
-  const int n_blocks = a.part != nullptr ? a.n_main_blocks : (int)gridDim.x;
+  // float4 ranges done by the reduce blocks (32-bit: the vector has fewer than 2^34 parameters)
+  unsigned lo4[UpdateArgs::MAX_REGIONS], hi4[UpdateArgs::MAX_REGIONS];
+#pragma unroll
+  for (int q = 0; q < UpdateArgs::MAX_REGIONS; ++q) {
+    lo4[q] = q < a.n_regions ? (unsigned)(a.region[q].off / 4) : 0xffffffffu;
+    hi4[q] = q < a.n_regions ? (unsigned)((a.region[q].off + (size_t)a.region[q].len + 3) / 4) : 0xffffffffu;
+  }
+  const int n_blocks = a.n_main_blocks;
   const size_t stride = (size_t)n_blocks * blockDim.x;
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   auto finish = [&](size_t i, float4 g, float4 m) {
-    if (i >= part_lo4 && i < part_hi4) return;     // the output layer is done by the reduce blocks
+    bool skip = false;
+#pragma unroll
+    for (int q = 0; q < UpdateArgs::MAX_REGIONS; ++q) skip |= (unsigned)i - lo4[q] < hi4[q] - lo4[q];
+    if (skip) return;                              // done by the reduce blocks
     m.x = fmaf(-step, g.x, m.x); m.y = fmaf(-step, g.y, m.y);
     m.z = fmaf(-step, g.z, m.z); m.w = fmaf(-step, g.w, m.w);
     reinterpret_cast<float4*>(a.master)[i] = m;

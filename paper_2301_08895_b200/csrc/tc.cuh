@@ -45,6 +45,9 @@ struct Params {
   int mask_words;                  // words per row of mask_bits / relu_bits = ceil(N_total / 32)
   __nv_bfloat16* out_bf16;         // FWD/DGRAD result [rows][N_total]
   float* out_f32;                  // WGRAD: G + w_off, partial p at + p*slot_stride, row pitch N_total
+  float* colsum;                   // DGRAD: [rows / 32][N_total] column sums of the stored result over each group of 32
+                                   // rows (they add up to the bias gradient of the layer below), or null
+  int no_bias_tile;                // WGRAD: the bias gradient comes from such column sums: no extra row tile
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -284,7 +287,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     // WGRAD: one extra row tile multiplies a column of ones with the deltas, which yields the bias
     // gradient (row `in` of the [in + 1][out] gradient block) on the tensor cores for free
     r.n_mt_w = (q.M_total - 1 + TM_ROWS - 1) / TM_ROWS;
-    r.n_mt = (q.mode == WGRAD) ? r.n_mt_w + 1 : n_row_tiles;
+    r.n_mt = (q.mode == WGRAD) ? r.n_mt_w + (q.no_bias_tile ? 0 : 1) : n_row_tiles;
     const int n_splits = max(1, q.P > 0 ? q.P : ri->K);   // P = 0: one split per selected worker (its own rows)
     r.n_tiles = (q.mode == WGRAD) ? r.n_mt * r.n_ct * n_splits : n_row_tiles * r.n_ct;
     r.chunk = (q.mode == WGRAD) ? round_up((n_rows + n_splits - 1) / n_splits, BK) : 0;
@@ -630,6 +633,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
+        if (mode == DGRAD && p.colsum != nullptr) {
+          // column sums of the warp's 32 x 64 box of stored (rounded, masked) deltas: lane l adds columns
+          // 2l, 2l + 1 over the 32 rows in order, reading the swizzled staging box row by row
+          float s0 = 0.f, s1 = 0.f;
+#pragma unroll 8
+          for (int rr = 0; rr < 32; ++rr) {
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(my_box + rr * 128 + ((((lane >> 2) ^ (rr & 7))) << 4) + ((lane & 3) << 2));
+            s0 += __uint_as_float(w << 16);
+            s1 += __uint_as_float(w & 0xffff0000u);
+          }
+          const int n = n0 + 2 * lane;
+          if (n < p.N_total)
+            *reinterpret_cast<float2*>(p.colsum + (size_t)((c.a_row + q * 32) >> 5) * p.N_total + n) = make_float2(s0, s1);
+        }
         if (issuer && !(mode == WGRAD && c.bias_tile)) {
           if (mode == WGRAD && p.P == 0)       // one split per worker: the tile adds to that worker's upload
             asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
