@@ -30,7 +30,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) per launch at K = N on configuration 4, from ncu captures of the GEMM and the
 # Eq. 3 kernel (summaries under profiles/); each figure is valid only for the kernel source it was taken
 # from (first 16 hex digits of the file's sha256).
-TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 44.2e6, "file": "tc.cuh", "sha256_16": "e0087777156b55f6",
+TRAFFIC = {"gemm": {"config": 4, "bytes_per_launch": 44.2e6, "file": "tc.cuh", "sha256_16": "041b65e9b34f49da",
                     "source": "ncu capture of the four GEMM launches of one round, profiles/tc_gemm_kernel_cfg4.md"},
            "update": {"config": 4, "bytes_per_launch": 63.7e6, "file": "simt.cuh", "sha256_16": "c178f6ac2b11a58b",
                       "source": "ncu capture of two launches, profiles/update_kernel_cfg4.md"}}

@@ -5,6 +5,8 @@
 //   FWD    H[r][n]  = relu( sum_k A[r][k] W_s[k][n] + b_s[n] )          rows grouped by model version
 //   DGRAD  D[r][m]  = ( sum_n Dl[r][n] W_s[m][n] ) * [H[r][m] > 0]
 //   WGRAD  G_p[m][n] = sum_{r in chunk p} A[r][m] Dl[r][n]               summed over ALL selected workers
+// (DGRAD can also leave the column sums of D over each group of 32 rows: they add up to the bias gradient of the
+// layer below, whose WGRAD then needs no row of ones.)
 // "s" is the ring slot of the row tile's model version (all rows of a 128-row tile share it).
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns the tensor-memory allocation),
