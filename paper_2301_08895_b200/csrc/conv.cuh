@@ -232,9 +232,17 @@ __global__ void __launch_bounds__(THREADS) conv_block_dgrad_kernel(Args a) {
     dz[((2 * py + (q >> 1)) * Wo + 2 * px + (q & 1)) * Co + co] = ldf(dps, e);
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < n_in; e += THREADS) {
-    const int ci = e % Ci, x = (e / Ci) % Wi, y = e / (Ci * Wi);
-    float sum = 0.f;
+  // a thread takes one input pixel and up to DG of its channels: a delta read from shared memory is used for
+  // DG FMAs (the weights of the DG channels for one tap and output channel are DG reads)
+  constexpr int DG = 8;
+  const int n_groups = (Ci + DG - 1) / DG;
+  for (int item = threadIdx.x; item < Hi * Wi * n_groups; item += THREADS) {
+    const int grp = item % n_groups, pix = item / n_groups;
+    const int x = pix % Wi, y = pix / Wi;
+    const int ci0 = grp * DG, nch = min(DG, Ci - ci0);
+    float sum[DG];
+#pragma unroll
+    for (int j = 0; j < DG; ++j) sum[j] = 0.f;
     for (int dy = 0; dy < k; ++dy) {
       const int oy = y - dy;
       if (oy < 0 || oy >= Ho) continue;
@@ -242,11 +250,19 @@ __global__ void __launch_bounds__(THREADS) conv_block_dgrad_kernel(Args a) {
         const int ox = x - dx;
         if (ox < 0 || ox >= Wo) continue;
         const float* zp = dz + (oy * Wo + ox) * Co;
-        const float* wp = wk + ((dy * k + dx) * Ci + ci) * Co;
-        for (int co = 0; co < Co; ++co) sum = fmaf(zp[co], wp[co], sum);
+        const float* wp = wk + ((dy * k + dx) * Ci + ci0) * Co;
+        for (int co = 0; co < Co; ++co) {
+          const float z = zp[co];
+#pragma unroll
+          for (int j = 0; j < DG; ++j)
+            if (j < nch) sum[j] = fmaf(z, wp[j * Co + co], sum[j]);
+        }
       }
     }
-    stf(din, e, ldf(src, e) > 0.f ? sum : 0.f);
+    const int e0 = pix * Ci + ci0;
+#pragma unroll
+    for (int j = 0; j < DG; ++j)
+      if (j < nch) stf(din, e0 + j, ldf(src, e0 + j) > 0.f ? sum[j] : 0.f);
   }
 }
 
