@@ -147,12 +147,13 @@ __global__ void __launch_bounds__(THREADS) conv_block_wgrad_kernel(Args a) {
   float* img = csm;                          // [Hi][Wi][Ci] input maps of the current row
   float* dp = img + n_in;                    // [Ph][Pw][Co] delta of the pooled maps
   unsigned char* ag = reinterpret_cast<unsigned char*>(dp + n_out);   // [Ph][Pw][Co]
-  // weight-gradient elements this thread owns: e = tid, tid + THREADS, ... (at most MAXE);
-  // elements n_w .. n_w + Co - 1 are the bias sums
-  constexpr int MAXE = 16;
-  float acc[MAXE];
-#pragma unroll
-  for (int j = 0; j < MAXE; ++j) acc[j] = 0.f;
+  // A thread takes a unit (tap (dy, dx), output channel co) and up to DG input channels of it: per pooled pixel
+  // the pool position and the delta are read once and feed DG FMAs on neighbouring image values.  The sums of a
+  // row are added to this CTA's block of `part` by the thread that owns the elements (same thread every row).
+  constexpr int DG = 8;
+  const int n_units = k * k * Co, n_groups = (Ci + DG - 1) / DG;
+  float* dst = a.part + (size_t)blockIdx.x * (size_t)(n_w + Co);
+  bool first = true;
   const int n_rows = ri->n_rows;
   for (int rr = 0; rr < CHUNK && r0 + rr < n_rows; ++rr) {
     const int r = r0 + rr;
@@ -165,33 +166,39 @@ __global__ void __launch_bounds__(THREADS) conv_block_wgrad_kernel(Args a) {
     for (int i = threadIdx.x; i < n_in; i += THREADS) img[i] = ldf(src, i);
     for (int i = threadIdx.x; i < n_out; i += THREADS) { dp[i] = ldf(dps, i); ag[i] = args[i]; }
     __syncthreads();
+    for (int item = threadIdx.x; item < n_units * n_groups; item += THREADS) {
+      const int u = item % n_units, grp = item / n_units;
+      const int co = u % Co, tap = u / Co, dx = tap % k, dy = tap / k;
+      const int ci0 = grp * DG, nch = min(DG, Ci - ci0);
+      float sum[DG];
 #pragma unroll
-    for (int j = 0; j < MAXE; ++j) {
-      const int e = threadIdx.x + j * THREADS;
-      if (e < n_w) {
-        const int co = e % Co, ci = (e / Co) % Ci, dx = (e / (Co * Ci)) % k, dy = e / (Co * Ci * k);
-        float sum = 0.f;
-        for (int py = 0; py < Ph; ++py)
-          for (int px = 0; px < Pw; ++px) {
-            const int o = (py * Pw + px) * Co + co;
-            const int q = ag[o];
-            sum = fmaf(img[((2 * py + (q >> 1) + dy) * Wi + 2 * px + (q & 1) + dx) * Ci + ci], dp[o], sum);
-          }
-        acc[j] += sum;
-      } else if (e < n_w + Co) {
-        const int co = e - n_w;
-        float sum = 0.f;
-        for (int o = co; o < n_out; o += Co) sum += dp[o];
-        acc[j] += sum;
-      }
+      for (int j = 0; j < DG; ++j) sum[j] = 0.f;
+      for (int py = 0; py < Ph; ++py)
+        for (int px = 0; px < Pw; ++px) {
+          const int o = (py * Pw + px) * Co + co;
+          const int q = ag[o];
+          const float d = dp[o];
+          const float* ip = img + ((2 * py + (q >> 1) + dy) * Wi + 2 * px + (q & 1) + dx) * Ci + ci0;
+#pragma unroll
+          for (int j = 0; j < DG; ++j)
+            if (j < nch) sum[j] = fmaf(ip[j], d, sum[j]);
+        }
+#pragma unroll
+      for (int j = 0; j < DG; ++j)
+        if (j < nch) {
+          const int e = (tap * Ci + ci0 + j) * Co + co;
+          dst[e] = first ? sum[j] : dst[e] + sum[j];
+        }
     }
+    if (threadIdx.x < Co) {                  // bias sums
+      float sum = 0.f;
+      for (int o = threadIdx.x; o < n_out; o += Co) sum += dp[o];
+      dst[n_w + threadIdx.x] = first ? sum : dst[n_w + threadIdx.x] + sum;
+    }
+    first = false;
   }
-  float* dst = a.part + (size_t)blockIdx.x * (size_t)(n_w + Co);
-#pragma unroll
-  for (int j = 0; j < MAXE; ++j) {
-    const int e = threadIdx.x + j * THREADS;
-    if (e < n_w + Co) dst[e] = acc[j];
-  }
+  if (first)                                 // no row with a gradient in this chunk
+    for (int e = threadIdx.x; e < n_w + Co; e += THREADS) dst[e] = 0.f;
 }
 
 // Delta of a block's input maps (second block only), CTA = gradient row: the pooled delta is put
