@@ -94,37 +94,53 @@ __global__ void __launch_bounds__(THREADS) conv_block_fwd_kernel(Args a) {
   for (int i = threadIdx.x; i < n_in; i += THREADS) img[i] = ldf(src, i);
   for (int i = threadIdx.x; i < n_w + Co; i += THREADS) wk[i] = ldf(Wm, i);     // the bias follows the weights
   __syncthreads();
-  for (int e = threadIdx.x; e < n_out; e += THREADS) {
-    const int co = e % Co, px = (e / Co) % Pw, py = e / (Co * Pw);
-    // the four window positions share their taps: per (dy, ci) the two image rows slide along dx,
-    // so a weight is read once for four FMAs and an image value once for two
-    float acc4[4] = {0.f, 0.f, 0.f, 0.f};
+  // A thread computes the four window positions of CT neighbouring output channels of one pooled pixel: per
+  // (dy, ci) the two image rows slide along dx, so an image value is read once for 2 CT FMAs and a weight once
+  // for four.
+  constexpr int CT = 2;
+  const int cgs = (Co + CT - 1) / CT;
+  for (int item = threadIdx.x; item < Ph * Pw * cgs; item += THREADS) {
+    const int co0 = (item % cgs) * CT, px = (item / cgs) % Pw, py = item / (cgs * Pw);
+    const int nco = min(CT, Co - co0);
+    float acc4[CT][4];
+#pragma unroll
+    for (int c = 0; c < CT; ++c)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc4[c][q] = 0.f;
     for (int dy = 0; dy < k; ++dy)
       for (int ci = 0; ci < Ci; ++ci) {
         const float* r0 = img + ((2 * py + dy) * Wi + 2 * px) * Ci + ci;
         const float* r1 = r0 + Wi * Ci;
-        const float* wp = wk + ((dy * k) * Ci + ci) * Co + co;
+        const float* wp = wk + ((dy * k) * Ci + ci) * Co + co0;
         float p0 = r0[0], p1 = r1[0];
         for (int dx = 0; dx < k; ++dx) {
           const float n0 = r0[(dx + 1) * Ci], n1 = r1[(dx + 1) * Ci];
-          const float w = wp[dx * Ci * Co];
-          acc4[0] = fmaf(p0, w, acc4[0]);
-          acc4[1] = fmaf(n0, w, acc4[1]);
-          acc4[2] = fmaf(p1, w, acc4[2]);
-          acc4[3] = fmaf(n1, w, acc4[3]);
+#pragma unroll
+          for (int c = 0; c < CT; ++c) {
+            const float w = c < nco ? wp[dx * Ci * Co + c] : 0.f;
+            acc4[c][0] = fmaf(p0, w, acc4[c][0]);
+            acc4[c][1] = fmaf(n0, w, acc4[c][1]);
+            acc4[c][2] = fmaf(p1, w, acc4[c][2]);
+            acc4[c][3] = fmaf(n1, w, acc4[c][3]);
+          }
           p0 = n0;
           p1 = n1;
         }
       }
-    float best = 0.f;
-    int where = 0;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const float v = as_stored_value<T>(fmaxf(acc4[q] + bias[co], 0.f));  // the stored ReLU output
-      if (q == 0 || v > best) { best = v; where = q; }                      // first maximum wins a tie
+    for (int c = 0; c < CT; ++c) {
+      if (c >= nco) break;
+      const int co = co0 + c, e = (py * Pw + px) * Co + co;
+      float best = 0.f;
+      int where = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float v = as_stored_value<T>(fmaxf(acc4[c][q] + bias[co], 0.f));  // the stored ReLU output
+        if (q == 0 || v > best) { best = v; where = q; }                         // first maximum wins a tie
+      }
+      stf(out, e, best);
+      arg[e] = (unsigned char)where;
     }
-    stf(out, e, best);
-    arg[e] = (unsigned char)where;
   }
 }
 
