@@ -66,6 +66,7 @@ struct Layout {
   bool bias_colsum[ABS_MAX_LAYERS] = {}; // the layer's bias gradient = column sums of the delta the layer above back-propagates
   size_t colsum[ABS_MAX_LAYERS] = {};   // [rows_cap / 32][out] those sums per group of 32 rows
   int fused_R = 0;                      // rows per block of the fused output-layer kernel (0: not used)
+  int narrow_rpb = 64;                  // rows per block of the row-tiled output-layer kernels that are not fused
   bool out_mma = false;                 // output layer through the mma.sync kernel (bf16, 64 rows per CTA)
   size_t esz = 4;                       // bytes per stored element (4 or 2)
   size_t d = 0, d_pad = 0;
@@ -316,7 +317,12 @@ void make_layout(const abs_model_desc* m, int W, int S, Layout* L) {
                   (size_t)R * 64 <= 100 * 1024) { L->fused_R = R; break; }
       L->out_mma = L->fused_R && tc_ok && m->n_layers > 1 &&
                    (inl == 128 || inl == 256 || inl == 512 || inl == 1024);
-      L->red = cv.take(4 * len * (size_t)(L->rows_cap / (L->fused_R ? L->fused_R : 64)));
+      // the non-fused output-layer kernels: fewer rows per block when a round has few rows, so that the grid is
+      // more than a handful of blocks (each is a chain of dependent loads)
+      L->narrow_rpb = 64;
+      if (!L->local_net)
+        while (L->narrow_rpb > 8 && (long long)W * m->batch / L->narrow_rpb < 2 * 148) L->narrow_rpb /= 2;
+      L->red = cv.take(4 * len * (size_t)(L->rows_cap / (L->fused_R ? L->fused_R : L->narrow_rpb)));
     }
     L->ones = L->any_tc ? cv.take(2 * 64 * (size_t)L->rows_cap) : 0;
     for (int l = 0; l < m->n_layers; ++l)
@@ -673,6 +679,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
     a.delta_out = ctx->at<void>(L.delta[l + 1]);
     a.delta_in = (l == 0) ? nullptr : ctx->at<void>(L.delta[l]);
     a.row_loss = L.local_net ? ctx->at<float>(L.row_loss) : ctx->ctl.row_loss; a.G = ctx->at<float>(L.G); a.P = L.P;
+    a.rpb = L.narrow_rpb;
     return a;
   };
   if (phase == PH_GATHER && L.cnn) {
@@ -736,7 +743,7 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
         launch_ex(ctx, ABS_KC_OUTPUT, narrow_fwd_loss_v8_kernel<T>, dim3(L.rows_cap / NARROW_ROWS), dim3(256), sm, a);
       } else {
         const size_t sm = sizeof(float) * ((size_t)a.in * a.C + a.C);
-        launch_ex(ctx, ABS_KC_OUTPUT, narrow_fwd_loss_kernel<T>, dim3(row_tiles), dim3(256), sm, a);
+        launch_ex(ctx, ABS_KC_OUTPUT, narrow_fwd_loss_kernel<T>, dim3(L.rows_cap / L.narrow_rpb), dim3(256), sm, a);
       }
     } else {
       dim3 grid((la[l].out + TN - 1) / TN, row_tiles);
@@ -792,19 +799,19 @@ void enqueue_gradient(abs_ctx* ctx, int par, int phase) {
           launch_ex(ctx, ABS_KC_OUTPUT, narrow_dgrad_v8_kernel<T>, dim3(L.rows_cap / NARROW_ROWS), dim3(256), sm, a);
         } else {
           const size_t sm = sizeof(float) * ((size_t)a.in * a.C + 64 * a.C);
-          launch_ex(ctx, ABS_KC_OUTPUT, narrow_dgrad_kernel<T>, dim3(row_tiles), dim3(256), sm, a);
+          launch_ex(ctx, ABS_KC_OUTPUT, narrow_dgrad_kernel<T>, dim3(L.rows_cap / L.narrow_rpb), dim3(256), sm, a);
         }
       }
       // weight gradient: per-chunk partial sums, then one ordered sum over the chunks into partial 0
       float* part = ctx->at<float>(L.red);
       float* dstw = ctx->at<float>(L.G) + L.w_off[l];
       const int len = (a.in + 1) * a.C;
-      launch_ex(ctx, ABS_KC_OUTPUT, narrow_wgrad_chunk_kernel<T>, dim3(L.rows_cap / 64), dim3(256), 0, a, part);
+      launch_ex(ctx, ABS_KC_OUTPUT, narrow_wgrad_chunk_kernel<T>, dim3(L.rows_cap / L.narrow_rpb), dim3(256), 0, a, part);
       if (L.local_net)
         launch_ex(ctx, ABS_KC_OUTPUT, lnet::chunk_reduce_worker_kernel, dim3((len + 255) / 256, ctx->W), dim3(256), 0, st, ri, part, len,
                   dstw, L.d_pad, 64, L.RBp);
       else
-        launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, 64);
+        launch_ex(ctx, ABS_KC_OUTPUT, chunk_reduce_kernel, dim3((len + 31) / 32), dim3(256), 0, st, ri, part, len, dstw, L.narrow_rpb);
     } else {
       const bool last = l == nl - 1;
       if (l > 0 || L.cnn) {

@@ -53,6 +53,7 @@ struct NarrowArgs {
   void* delta_in;          // [rows][in] storage type (dgrad result)
   float* row_loss;         // [rows]
   float* G; int P;
+  int rpb;                 // gradient rows per block of the row-tiled kernels below (8..64, a multiple of 8; 0 = 64)
 };
 
 // Output layer forward + soft-max cross-entropy + delta for 64 rows per block (one ring slot).
@@ -64,7 +65,8 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_kernel(NarrowArgs a) {
   DevState* st = a.st;
   RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
-  const int r0 = blockIdx.x * 64;
+  const int RPB = a.rpb ? a.rpb : 64;
+  const int r0 = blockIdx.x * RPB;
   if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   const int slot = a.tile_slot[r0 / st->RB];
@@ -76,7 +78,7 @@ __global__ void __launch_bounds__(256) narrow_fwd_loss_kernel(NarrowArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const T* src = (const T*)a.act_in;
   bool bad = false;
-  for (int rr = warp; rr < 64; rr += 8) {
+  for (int rr = warp; rr < RPB; rr += 8) {
     const int r = r0 + rr;
     const int s = a.row_idx[r];
     T* d = (T*)a.delta_out + (size_t)r * C;
@@ -134,7 +136,8 @@ __global__ void __launch_bounds__(256) narrow_dgrad_kernel(NarrowArgs a) {
   DevState* st = a.st;
   RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
-  const int r0 = blockIdx.x * 64;
+  const int RPB = a.rpb ? a.rpb : 64;
+  const int r0 = blockIdx.x * RPB;
   if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   const int slot = a.tile_slot[r0 / st->RB];
@@ -142,7 +145,7 @@ __global__ void __launch_bounds__(256) narrow_dgrad_kernel(NarrowArgs a) {
   float* dsm = wsm + (size_t)in * C;
   for (int i = threadIdx.x; i < in * C; i += 256) wsm[i] = ldf(Wm, i);
   const T* dl = (const T*)a.delta_out + (size_t)r0 * C;
-  for (int i = threadIdx.x; i < 64 * C; i += 256) dsm[i] = ldf(dl, i);
+  for (int i = threadIdx.x; i < RPB * C; i += 256) dsm[i] = ldf(dl, i);
   __syncthreads();
   const T* h = (const T*)a.act_in;
   T* out = (T*)a.delta_in;
@@ -150,7 +153,7 @@ __global__ void __launch_bounds__(256) narrow_dgrad_kernel(NarrowArgs a) {
     float w[NARROW_MAX_C];
 #pragma unroll
     for (int c = 0; c < NARROW_MAX_C; ++c) w[c] = (c < C) ? wsm[(size_t)m * C + c] : 0.f;
-    for (int rr = 0; rr < 64; ++rr) {
+    for (int rr = 0; rr < RPB; ++rr) {
       float acc = 0.f;
 #pragma unroll
       for (int c = 0; c < NARROW_MAX_C; ++c)
@@ -343,12 +346,13 @@ __global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, f
   DevState* st = a.st;
   RoundInfo* ri = a.ri;
   if (st->status != ST_OK) return;
-  const int r0 = blockIdx.x * 64;
+  const int RPB = a.rpb ? a.rpb : 64;
+  const int r0 = blockIdx.x * RPB;
   if (r0 >= ri->n_rows) return;
   const int in = a.in, C = a.C;
   const T* dl = (const T*)a.delta_out + (size_t)r0 * C;
-  for (int i = threadIdx.x; i < 64 * C; i += 256) dsm[i / C][i % C] = ldf(dl, i);
-  if (threadIdx.x < 64) {
+  for (int i = threadIdx.x; i < RPB * C; i += 256) dsm[i / C][i % C] = ldf(dl, i);
+  if (threadIdx.x < RPB) {
     const int r = r0 + threadIdx.x;
     long long off = (long long)r * in;
     if (a.gather) { const int s = a.row_idx[r]; off = s < 0 ? 0 : (long long)s * in; }
@@ -364,7 +368,7 @@ __global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, f
     float acc0[NARROW_MAX_C], acc1[NARROW_MAX_C];
 #pragma unroll
     for (int c = 0; c < NARROW_MAX_C; ++c) { acc0[c] = 0.f; acc1[c] = 0.f; }
-    for (int rb = 0; rb < 64; rb += 8) {
+    for (int rb = 0; rb < RPB; rb += 8) {
       float x0[8], x1[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -391,7 +395,7 @@ __global__ void __launch_bounds__(256) narrow_wgrad_chunk_kernel(NarrowArgs a, f
   }
   if (threadIdx.x < C) {                       // bias row: column sums of the deltas
     float tot = 0.f;
-    for (int rr = 0; rr < 64; ++rr) tot += dsm[rr][threadIdx.x];
+    for (int rr = 0; rr < RPB; ++rr) tot += dsm[rr][threadIdx.x];
     dst[(size_t)in * C + threadIdx.x] = tot;
   }
 }
